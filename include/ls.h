@@ -1,0 +1,224 @@
+/*
+ * ls.h -- C ABI of the B200 (sm_100a) library for batch-1 self-speculative greedy
+ * decoding on a Llama-style decoder (LayerSkip, arXiv 2404.16710, Sec. 4.3 and
+ * Appendix A.4).
+ *
+ * Conventions for every entry point
+ *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers
+ *     are ordinary host memory.  The library BORROWS every device pointer it is given
+ *     (weights, workspace, operands): the caller allocates them, keeps them alive and
+ *     frees them.  The library itself allocates no device memory.
+ *   - bf16 matrices are row-major [out_features, in_features] and 16-byte aligned;
+ *     in_features must be a multiple of 8.
+ *   - Return value: LS_OK (0) or a negative ls_status.  No exception crosses the ABI,
+ *     nothing aborts the process.  ls_strerror() names a status; after LS_ERR_CUDA,
+ *     ls_last_cuda_error() returns the cudaError_t value seen.
+ *   - A model handle is bound to one device and one stream; calls on one handle must
+ *     not overlap.  Compute capability 10.x is required (LS_ERR_UNSUPPORTED otherwise);
+ *     there is no CPU fallback.
+ *   - Numerics: bf16 weights, bf16 KV cache, bf16 inputs of every linear layer, fp32
+ *     residual stream and fp32 accumulation.  A row's result never depends on how many
+ *     rows share the pass, so the verification pass (Sec. 4.3.2) reproduces
+ *     single-token decoding bit for bit and ls_generate returns exactly the ids of
+ *     ls_generate_full.
+ */
+#ifndef LS_B200_H
+#define LS_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum ls_status {
+    LS_OK = 0,
+    LS_ERR_INVALID_ARG = -1,   /* null / misaligned pointer, value out of range            */
+    LS_ERR_CAPACITY = -2,      /* KV capacity, workspace size or max_draft exceeded         */
+    LS_ERR_CUDA = -3,          /* a CUDA runtime call failed; see ls_last_cuda_error()      */
+    LS_ERR_DEVICE_STATUS = -4, /* a kernel's own bounds check refused an access             */
+    LS_ERR_UNSUPPORTED = -5    /* not an sm_100 device, or a shape the kernels do not cover */
+} ls_status;
+
+#define LS_MAX_ROWS 16 /* rows (tokens) per pass: num_draft + 1 <= LS_MAX_ROWS */
+
+/* Which kernel family runs every linear layer of a model.  The choice is per model,
+ * never per call: results are bit-identical across M only within one family. */
+enum { LS_LINEAR_AUTO = 0, LS_LINEAR_FMA = 1, LS_LINEAR_MMA = 2 };
+
+/* Decoder shape (Sec. 4.1: L residual layers and the shared LM head g). */
+typedef struct ls_config {
+    int32_t n_layers;    /* L                                                            */
+    int32_t d_model;     /* D, multiple of 8                                             */
+    int32_t n_heads;     /* query heads Hq                                               */
+    int32_t n_kv_heads;  /* KV heads Hkv, divides Hq, Hq/Hkv <= 8                        */
+    int32_t head_dim;    /* 64 or 128                                                    */
+    int32_t d_ffn;       /* F, multiple of 8                                             */
+    int32_t vocab;       /* V                                                            */
+    float rms_eps;
+    float rope_theta;
+    int32_t max_seq;     /* KV capacity in tokens: n_prompt + max_new + num_draft + 1    */
+    int32_t page_size;   /* tokens per KV page: power of two, 16..1024                   */
+    int32_t max_draft;   /* largest num_draft this model will be asked for (<= 15)       */
+    int32_t eos_id;      /* -1: never stop early                                         */
+    int32_t linear_path; /* LS_LINEAR_*                                                  */
+} ls_config;
+
+/* Device pointers to the bf16 weights.  The per-layer members are HOST arrays of
+ * n_layers device pointers.  Matrices [out, in]: wq [Hq*hd, D], wk/wv [Hkv*hd, D],
+ * wo [D, Hq*hd], w_gate/w_up [F, D], w_down [D, F], tok_embed/lm_head [V, D];
+ * norm gains are [D]. */
+typedef struct ls_weights {
+    const void *tok_embed, *final_norm, *lm_head;
+    const void *const *attn_norm, *const *wq, *const *wk, *const *wv, *const *wo;
+    const void *const *ffn_norm, *const *w_gate, *const *w_up, *const *w_down;
+} ls_weights;
+
+typedef struct ls_model ls_model; /* opaque, owned by the library (host memory only) */
+
+/* Counters of the most recent prefill / decode on a handle. */
+typedef struct ls_stats {
+    double prefill_ms;       /* device time of the prompt pass                              */
+    double decode_ms;        /* device time of the decode loop (CUDA events on the stream)  */
+    int64_t weight_bytes;    /* weight bytes the schedule had to read during decode         */
+    int64_t kv_bytes;        /* KV-cache bytes the schedule had to read during decode       */
+    int64_t kernel_launches; /* kernels launched by the decode loop                         */
+    int32_t n_generated;
+    int32_t n_steps;         /* speculative steps (== n_generated for plain greedy)         */
+    int32_t n_accepted;      /* sum of accepted drafts over the steps                       */
+    int32_t host_syncs;      /* host<->device synchronisations inside the decode loop       */
+} ls_stats;
+
+const char *ls_strerror(int status);
+int ls_last_cuda_error(void);
+
+/* Bytes of device workspace a model of this shape needs (KV pages, page table,
+ * activations, exit-layer activation cache, control words).  0 if cfg is invalid. */
+size_t ls_workspace_bytes(const ls_config *cfg);
+
+/* Create a model over borrowed weights and workspace (256-byte aligned, at least
+ * ls_workspace_bytes(cfg)).  cuda_stream is a cudaStream_t (NULL = default stream).
+ * The workspace is cleared; the page table starts as the identity. */
+int ls_model_create(const ls_config *cfg, const ls_weights *w, void *workspace_dev,
+                    size_t workspace_bytes, void *cuda_stream, ls_model **out);
+int ls_model_destroy(ls_model *m);
+
+/* Replace the logical->physical KV page table: host array of
+ * ceil(max_seq/page_size) distinct physical page numbers in [0, n_pages). */
+int ls_set_page_table(ls_model *m, const int32_t *table_host, int32_t n_pages);
+
+/* Self-speculative greedy decoding (Sec. 4.3, Appendix A.4).
+ * The prompt except its last token is run through all L layers; then every step
+ *   drafts num_draft tokens with layers 0..E-1 and the shared LM head (Sec. 4.3.1),
+ *   verifies them with layers E..L-1 in one pass of num_draft+1 rows that starts from
+ *   the cached exit-layer activations and shares the KV cache (Sec. 4.3.2, 4.3.3),
+ *   accepts the longest agreeing prefix plus the verified token after it and rolls the
+ *   cache back to "every emitted token but the last" (Appendix A.4: match, crop).
+ * prompt_ids_host [n_prompt]; exit_layer E in [1, L-1]; num_draft in [1, max_draft];
+ * out_ids_host [max_new] receives *out_n <= max_new ids (fewer only after an EOS);
+ * accepted_per_step_host [max_new] receives the accepted-draft count of each of the
+ * *out_n_steps steps (the last one counted before truncation at max_new).
+ * LS_ERR_CAPACITY if n_prompt + max_new + num_draft + 1 > max_seq. */
+int ls_generate(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt,
+                int32_t exit_layer, int32_t num_draft, int32_t max_new,
+                int32_t *out_ids_host, int32_t *out_n,
+                int32_t *accepted_per_step_host, int32_t *out_n_steps);
+
+/* Autoregressive greedy decoding with all L layers: the baseline of Sec. 6.2 and,
+ * by construction of the method, the exact result ls_generate must reproduce. */
+int ls_generate_full(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt,
+                     int32_t max_new, int32_t *out_ids_host, int32_t *out_n);
+
+/* Early-exit greedy decoding (Sec. 4.2): every token is argmax g(x_E). */
+int ls_generate_early(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt,
+                      int32_t exit_layer, int32_t max_new, int32_t *out_ids_host, int32_t *out_n);
+
+/* The two halves of a generate call, for callers that keep everything on the device
+ * (and for timing the decode loop alone).  ls_prefill copies the prompt, runs
+ * prompt[0..n-2] through the first `layers` layers (0 = all L; early-exit decoding
+ * needs only E) and leaves the loop state at cache length n-1.  ls_decode runs the
+ * loop from that state: exit_layer == 0 selects plain greedy with all layers,
+ * num_draft == 0 with exit_layer > 0 selects early-exit greedy.  ls_decode may be
+ * repeated after one ls_prefill: it restarts from the prefilled state every time.
+ * Results stay on the device until ls_read_output. */
+int ls_prefill(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt, int32_t layers);
+int ls_decode(ls_model *m, int32_t exit_layer, int32_t num_draft, int32_t max_new);
+int ls_read_output(ls_model *m, int32_t *out_ids_host, int32_t *out_n,
+                   int32_t *accepted_per_step_host, int32_t *out_n_steps);
+
+/* Teacher-forced logits for parity checks: feed ids_host[0..n-1] at positions 0..n-1
+ * and return g(x_E) and g(x_L) for every position (host fp32 [n, V]; either may be
+ * NULL).  g is the shared head of Sec. 2.1 / 4.2.  n <= max_seq. */
+int ls_debug_logits(ls_model *m, const int32_t *ids_host, int32_t n, int32_t exit_layer,
+                    float *exit_logits_host, float *final_logits_host);
+
+int ls_get_stats(const ls_model *m, ls_stats *out);
+
+/* ------------------------------------------------------------------------------
+ * Single operations of the path (each is one kernel family of the loop), exposed so
+ * that each can be checked against its definition and profiled alone.  All pointers
+ * are device pointers; M <= LS_MAX_ROWS rows; the call is enqueued on cuda_stream and
+ * returns without synchronising.  linear_path is LS_LINEAR_FMA or LS_LINEAR_MMA.
+ * ------------------------------------------------------------------------------ */
+
+/* x[m,:] = float(Emb[tok[m],:]) -- the embedding lookup x_0 of Sec. 4.1. */
+int ls_op_embed(const void *emb_bf16_dev, const int32_t *tok_dev, int32_t M, int32_t D, int32_t V,
+                float *x_dev, void *cuda_stream);
+
+/* RMSNorm of each row: out[m,i] = bf16( x[m,i] / sqrt(mean_j x[m,j]^2 + eps) * g[i] ). */
+int ls_op_rmsnorm(const float *x_dev, const void *gain_dev, int32_t M, int32_t D, float eps,
+                  void *out_bf16_dev, void *cuda_stream);
+
+/* out[m,n] = sum_k W[n,k] h[m,k]; W bf16 [N,K], h bf16 [M,K], out fp32 [M,N].
+ * If residual != 0 the product is ADDED to out (the x <- x + f(x) update of Sec. 4.1). */
+int ls_op_linear(int32_t linear_path, const void *w_dev, const void *h_bf16_dev, int32_t M,
+                 int32_t N, int32_t K, float *out_dev, int32_t residual, void *cuda_stream);
+
+/* SwiGLU feed-forward input: out[m,f] = bf16( silu(Wg h)[f] * (Wu h)[f] ). */
+int ls_op_gate_up_swiglu(int32_t linear_path, const void *w_gate_dev, const void *w_up_dev,
+                         const void *h_bf16_dev, int32_t M, int32_t F, int32_t K,
+                         void *out_bf16_dev, void *cuda_stream);
+
+/* Shared LM head fused with argmax (Sec. 2.1, Sec. 4.2): tok[m] = argmax_v (W h[m])_v,
+ * the lowest index wins a tie.  scratch_dev: ls_op_lm_head_scratch_bytes(V) bytes.
+ * logits_dev (fp32 [M,V]) may be NULL. */
+size_t ls_op_lm_head_scratch_bytes(int32_t V);
+int ls_op_lm_head_argmax(int32_t linear_path, const void *w_dev, const void *h_bf16_dev,
+                         int32_t M, int32_t V, int32_t K, void *scratch_dev, int32_t *tok_dev,
+                         float *logits_dev, void *cuda_stream);
+
+/* Rotary embedding + KV append: rows m = 0..M-1 sit at positions pos0+m.  qkv fp32
+ * [M, (Hq+2Hkv)*hd] (q heads, then k heads, then v heads).  Writes q_out bf16
+ * [M, Hq*hd] and k, v (bf16) into the paged cache: k_pages / v_pages hold physical
+ * pages of [Hkv][page_size][hd]; page_table_dev maps logical page -> physical page. */
+int ls_op_rope_append(const float *qkv_dev, int32_t M, int32_t pos0, int32_t Hq, int32_t Hkv,
+                      int32_t hd, float rope_theta, int32_t page_size, const int32_t *page_table_dev,
+                      int32_t max_seq, void *q_out_bf16_dev, void *k_pages_dev, void *v_pages_dev,
+                      void *cuda_stream);
+
+/* Causal attention of rows m at positions pos0+m over cache positions 0..pos0+m, with
+ * grouped KV heads (query head i reads KV head i / (Hq/Hkv)).  q bf16 [M, Hq*hd];
+ * out bf16 [M, Hq*hd].  The cache is split into fixed chunks of absolute positions
+ * whose partial (max, sum, weighted values) are merged in chunk order.
+ * scratch_dev: ls_op_attention_scratch_bytes(...) bytes. */
+size_t ls_op_attention_scratch_bytes(int32_t Hq, int32_t hd, int32_t max_seq);
+int ls_op_attention(const void *q_bf16_dev, int32_t M, int32_t pos0, int32_t Hq, int32_t Hkv,
+                    int32_t hd, int32_t page_size, const int32_t *page_table_dev, int32_t max_seq,
+                    const void *k_pages_dev, const void *v_pages_dev, void *scratch_dev,
+                    void *out_bf16_dev, void *cuda_stream);
+
+/* match + crop of Appendix A.4 on device arrays: n = number of leading i < d with
+ * draft[i] == verified[i]; appends draft[0..n-1], verified[n] to out_ids (truncated at
+ * max_new, and after the first eos_id if eos_id >= 0).
+ * state_dev int32[8]: {cache_len, cur_token, n_out, n_steps, done, max_new, eos_id, status};
+ * updated in place: cache_len += n+1, cur_token = verified[n], accepted[n_steps++] = n,
+ * done = (n_out == max_new || EOS emitted). */
+int ls_op_accept(const int32_t *draft_dev, const int32_t *verified_dev, int32_t d,
+                 int32_t *state_dev, int32_t *out_ids_dev, int32_t *accepted_dev,
+                 void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LS_B200_H */

@@ -1,0 +1,70 @@
+// Shared device-side definitions of the decode kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ls {
+
+// Control words of the decode loop, int32 in device memory.  Every kernel of the loop
+// reads its positions from here, so one captured CUDA graph serves every step.
+enum Ctl : int {
+    CTL_CACHE_LEN = 0,  // tokens whose k, v are valid in the cache
+    CTL_CUR_TOK = 1,    // input token of the next step (emitted, not yet cached)
+    CTL_N_OUT = 2,      // ids emitted so far
+    CTL_N_STEPS = 3,    // steps taken so far
+    CTL_DONE = 4,       // loop finished: later kernels return at once
+    CTL_MAX_NEW = 5,
+    CTL_EOS = 6,
+    CTL_STATUS = 7,     // non-zero: a kernel's bounds check refused an access
+    CTL_WORDS = 8
+};
+
+enum DevStatus : int { DEV_OK = 0, DEV_BAD_TOKEN = 1, DEV_POS_OVERFLOW = 2 };
+
+constexpr int kMaxRows = 16;    // rows per pass
+constexpr int kAttnChunk = 64;  // keys per attention chunk (absolute positions)
+
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+__device__ __forceinline__ float bf16f(uint16_t u) { return __uint_as_float(((uint32_t)u) << 16); }
+__device__ __forceinline__ uint16_t f2bf(float f)
+{
+    return __bfloat16_as_ushort(__float2bfloat16_rn(f));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    return (uint32_t)f2bf(lo) | ((uint32_t)f2bf(hi) << 16);
+}
+
+// 16-byte read of streamed-once data (weights): do not allocate in L1, so that the
+// activations, which every CTA re-reads, stay there.
+__device__ __forceinline__ uint4 ld_stream16(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+// 16-byte read of small, heavily re-used data (activations): keep in L1.
+__device__ __forceinline__ uint4 ld_reuse16(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::evict_last.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+struct ValIdx {
+    float v;
+    int i;
+};
+// total order: larger value first, then lower index (ties go to the lowest index)
+__device__ __forceinline__ bool better(float v, int i, float bv, int bi)
+{
+    return v > bv || (v == bv && i < bi);
+}
+
+}  // namespace ls

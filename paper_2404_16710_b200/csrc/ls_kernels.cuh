@@ -1,0 +1,416 @@
+// Non-GEMV kernels of the decode loop: embedding, RMSNorm, rotary embedding + KV append,
+// chunked causal attention over the paged cache, chunk merge, argmax finish, accept/rollback.
+//
+// Invariant kept by every kernel here: the instructions that produce row m's result do
+// not depend on how many rows the pass has.  The verification pass of num_draft+1 rows
+// (LayerSkip Sec. 4.3.2) therefore reproduces single-token decoding bit for bit.
+#pragma once
+#include "ls_common.cuh"
+
+namespace ls {
+
+// position of row 0 of this pass: the loop's cache length plus a per-launch offset
+__device__ __forceinline__ bool pass_begin(const int32_t* ctl, int pos_off, int& pos0)
+{
+    if (ctl) {
+        if (ctl[CTL_DONE]) return false;
+        pos0 = ctl[CTL_CACHE_LEN] + pos_off;
+    } else {
+        pos0 = pos_off;
+    }
+    return true;
+}
+
+// ------------------------------------------------------------------ embedding (x_0 = Emb[id])
+// grid M, block 256.  tok[m] is read from device memory.
+__global__ void __launch_bounds__(256)
+embed_kernel(const uint16_t* __restrict__ emb, const int32_t* __restrict__ tok, int D, int V,
+             float* __restrict__ x, int32_t* ctl)
+{
+    if (ctl && ctl[CTL_DONE]) return;
+    int m = blockIdx.x;
+    int id = tok[m];
+    if (id < 0 || id >= V) {
+        if (ctl && threadIdx.x == 0) ctl[CTL_STATUS] = DEV_BAD_TOKEN;
+        id = 0;
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(emb + (size_t)id * D);
+    float4* dst = reinterpret_cast<float4*>(x + (size_t)m * D);
+    for (int c = threadIdx.x; c < D / 8; c += blockDim.x) {
+        uint4 v = src[c];
+        dst[2 * c] = make_float4(bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y));
+        dst[2 * c + 1] = make_float4(bf16lo(v.z), bf16hi(v.z), bf16lo(v.w), bf16hi(v.w));
+    }
+}
+
+// ------------------------------------------------------------------ RMSNorm
+// grid M, block 256.  out = bf16(x / sqrt(mean x^2 + eps) * g).
+__device__ __forceinline__ float block_sum_256(float v, float* red)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) s += red[w];
+    return s;
+}
+
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(const float* __restrict__ x, const uint16_t* __restrict__ g, int D, float eps,
+               uint16_t* __restrict__ out, const int32_t* ctl)
+{
+    __shared__ float red[8];
+    if (ctl && ctl[CTL_DONE]) return;
+    int m = blockIdx.x;
+    const float4* xr = reinterpret_cast<const float4*>(x + (size_t)m * D);
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < D / 4; c += 256) {
+        float4 v = xr[c];
+        ss = fmaf(v.x, v.x, ss);
+        ss = fmaf(v.y, v.y, ss);
+        ss = fmaf(v.z, v.z, ss);
+        ss = fmaf(v.w, v.w, ss);
+    }
+    float tot = block_sum_256(ss, red);
+    float r = 1.0f / sqrtf(tot / (float)D + eps);
+    const uint2* gr = reinterpret_cast<const uint2*>(g);
+    uint2* o = reinterpret_cast<uint2*>(out + (size_t)m * D);
+    for (int c = threadIdx.x; c < D / 4; c += 256) {
+        float4 v = xr[c];
+        uint2 gg = gr[c];
+        uint2 w;
+        w.x = pack_bf16(v.x * r * bf16lo(gg.x), v.y * r * bf16hi(gg.x));
+        w.y = pack_bf16(v.z * r * bf16lo(gg.y), v.w * r * bf16hi(gg.y));
+        o[c] = w;
+    }
+}
+
+// fp32 row copy (exit-layer activation cache <-> residual stream, Sec. 4.3.3); grid M, block 256
+__global__ void __launch_bounds__(256)
+copy_rows_kernel(const float* __restrict__ src, float* __restrict__ dst, int D, const int32_t* ctl)
+{
+    if (ctl && ctl[CTL_DONE]) return;
+    const float4* s = reinterpret_cast<const float4*>(src + (size_t)blockIdx.x * D);
+    float4* d = reinterpret_cast<float4*>(dst + (size_t)blockIdx.x * D);
+    for (int c = threadIdx.x; c < D / 4; c += 256) d[c] = s[c];
+}
+
+// ------------------------------------------------------------------ paged KV addressing
+// Physical page p of a layer holds [Hkv][page_size][hd] bf16 for K (and the same for V).
+__device__ __forceinline__ size_t kv_row_offset(const int32_t* __restrict__ page_table, int pos,
+                                                int page_shift, int Hkv, int kh, int hd)
+{
+    int page = pos >> page_shift;
+    int off = pos & ((1 << page_shift) - 1);
+    int phys = page_table[page];
+    return (((size_t)phys * Hkv + kh) * ((size_t)1 << page_shift) + off) * (size_t)hd;
+}
+
+// ------------------------------------------------------------------ RoPE + KV append
+// grid (M, Hq + 2 Hkv), block hd/2.  Row m sits at position pos0 + m.  Pairs (j, j + hd/2)
+// are rotated by pos * theta^(-2j/hd).  q -> bf16 [M, Hq*hd]; k, v -> bf16 cache rows.
+__global__ void rope_append_kernel(const float* __restrict__ qkv, int Hq, int Hkv, int hd,
+                                   const float* __restrict__ inv_freq, float theta, int page_shift,
+                                   const int32_t* __restrict__ page_table, int max_seq,
+                                   uint16_t* __restrict__ q_out, uint16_t* __restrict__ kpages,
+                                   uint16_t* __restrict__ vpages, int32_t* ctl, int pos_off)
+{
+    int pos0;
+    if (!pass_begin(ctl, pos_off, pos0)) return;
+    int m = blockIdx.x, h = blockIdx.y, j = threadIdx.x, half = hd >> 1;
+    int pos = pos0 + m;
+    if (pos < 0 || pos >= max_seq) {
+        if (ctl && j == 0) ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
+        return;
+    }
+    int width = (Hq + 2 * Hkv) * hd;
+    const float* src = qkv + (size_t)m * width + (size_t)h * hd;
+    float a = src[j], b = src[j + half];
+    if (h < Hq + Hkv) {
+        float f = inv_freq ? inv_freq[j] : (float)pow((double)theta, -2.0 * (double)j / (double)hd);
+        float s, c;
+        sincosf((float)pos * f, &s, &c);
+        float ra = a * c - b * s;
+        float rb = a * s + b * c;
+        a = ra;
+        b = rb;
+    }
+    uint16_t* dst;
+    if (h < Hq) {
+        dst = q_out + (size_t)m * Hq * hd + (size_t)h * hd;
+    } else if (h < Hq + Hkv) {
+        dst = kpages + kv_row_offset(page_table, pos, page_shift, Hkv, h - Hq, hd);
+    } else {
+        dst = vpages + kv_row_offset(page_table, pos, page_shift, Hkv, h - Hq - Hkv, hd);
+    }
+    dst[j] = f2bf(a);
+    dst[j + half] = f2bf(b);
+}
+
+// ------------------------------------------------------------------ attention, one chunk of keys
+// grid (chunks, Hkv), block 128.  CTA = keys [64*ch, 64*ch + 64) of KV head kh, all
+// G = Hq/Hkv query heads of the group, all M rows.  Writes, per (row, head, chunk),
+// the un-normalised partial (o[HD], max, sum).  Row m at position pos0+m sees keys <= pos0+m.
+//
+// shared memory: Ks [64][HD*2+16 B] | Vs [64][HD*2 B] | Qs f32 [Q][HD] | Sp f32 [2][Q][64]
+//                | P f32 [Q][64] | Ored f32 [NKS][4][HD]
+template <int HD>
+__host__ __device__ constexpr size_t attn_smem_bytes(int Q)
+{
+    return (size_t)kAttnChunk * (HD * 2 + 16) + (size_t)kAttnChunk * HD * 2 +
+           sizeof(float) * ((size_t)Q * HD + 3 * (size_t)Q * kAttnChunk + (size_t)(128 / (HD / 2)) * 4 * HD);
+}
+
+template <int HD>
+__global__ void __launch_bounds__(128)
+attn_chunk_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
+                  const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table,
+                  int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift,
+                  int max_seq, int chunk_cap, float* __restrict__ part)
+{
+    constexpr int C = kAttnChunk;
+    constexpr int KROW = HD * 2 + 16;        // padded K row, bytes
+    constexpr int NKS = 128 / (HD / 2);      // key slices in the P.V phase
+    constexpr int HALF = HD / 2;
+    int pos0;
+    if (!pass_begin(ctl, pos_off, pos0)) return;
+    const int ch = blockIdx.x, kh = blockIdx.y, tid = threadIdx.x;
+    const int last_pos = pos0 + M - 1;
+    const int key0 = ch * C;
+    if (key0 > last_pos) return;
+    if (last_pos >= max_seq || pos0 < 0 || ch >= chunk_cap) {
+        if (ctl && tid == 0) ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
+        return;
+    }
+    const int G = Hq / Hkv, Q = G * M;  // query qi = m * G + g
+
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned char* Ks = smem;
+    unsigned char* Vs = Ks + C * KROW;
+    float* Qs = reinterpret_cast<float*>(Vs + C * HD * 2);
+    float* Sp = Qs + (size_t)Q * HD;
+    float* P = Sp + 2 * (size_t)Q * C;
+    float* Ored = P + (size_t)Q * C;
+
+    // stage K and V rows of the chunk (zero beyond the last visible key)
+    constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
+    for (int idx = tid; idx < C * SEGS; idx += 128) {
+        int r = idx / SEGS, sg = idx % SEGS;
+        int p = key0 + r;
+        uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
+        if (p <= last_pos) {
+            size_t off = kv_row_offset(page_table, p, page_shift, Hkv, kh, HD) + (size_t)sg * 8;
+            kv = *reinterpret_cast<const uint4*>(kpages + off);
+            vv = *reinterpret_cast<const uint4*>(vpages + off);
+        }
+        *reinterpret_cast<uint4*>(Ks + r * KROW + sg * 16) = kv;
+        *reinterpret_cast<uint4*>(Vs + r * HD * 2 + sg * 16) = vv;
+    }
+    // queries of this group -> fp32
+    for (int idx = tid; idx < Q * HALF; idx += 128) {
+        int qi = idx / HALF, dp = idx % HALF;
+        int m = qi / G, g = qi % G;
+        uint32_t u = *reinterpret_cast<const uint32_t*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + 2 * dp);
+        Qs[qi * HD + 2 * dp] = bf16lo(u);
+        Qs[qi * HD + 2 * dp + 1] = bf16hi(u);
+    }
+    __syncthreads();
+
+    // phase 1: thread = (key j, half of the dims); partial dot products in groups of 4 queries
+    {
+        const int j = tid & 63, hf = tid >> 6;
+        const unsigned char* krow = Ks + j * KROW + hf * HALF * 2;
+        for (int q0 = 0; q0 < Q; q0 += 4) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
+            for (int b = 0; b < HALF / 8; ++b) {
+                uint4 kk = *reinterpret_cast<const uint4*>(krow + b * 16);
+                float kf[8] = {bf16lo(kk.x), bf16hi(kk.x), bf16lo(kk.y), bf16hi(kk.y),
+                               bf16lo(kk.z), bf16hi(kk.z), bf16lo(kk.w), bf16hi(kk.w)};
+#pragma unroll
+                for (int qq = 0; qq < 4; ++qq) {
+                    int qi = min(q0 + qq, Q - 1);
+                    const float4* qv = reinterpret_cast<const float4*>(Qs + qi * HD + hf * HALF + b * 8);
+                    float4 a = qv[0], c = qv[1];
+                    float s = acc[qq];
+                    s = fmaf(kf[0], a.x, s);
+                    s = fmaf(kf[1], a.y, s);
+                    s = fmaf(kf[2], a.z, s);
+                    s = fmaf(kf[3], a.w, s);
+                    s = fmaf(kf[4], c.x, s);
+                    s = fmaf(kf[5], c.y, s);
+                    s = fmaf(kf[6], c.z, s);
+                    s = fmaf(kf[7], c.w, s);
+                    acc[qq] = s;
+                }
+            }
+#pragma unroll
+            for (int qq = 0; qq < 4; ++qq)
+                if (q0 + qq < Q) Sp[((size_t)hf * Q + q0 + qq) * C + j] = acc[qq];
+        }
+    }
+    __syncthreads();
+
+    // phase 2: one warp per query: mask, max, exp, sum over the 64 keys of the chunk
+    {
+        const int warp = tid >> 5, lane = tid & 31;
+        const float scale = rsqrtf((float)HD);
+        for (int qi = warp; qi < Q; qi += 4) {
+            int m = qi / G, g = qi % G;
+            int pos = pos0 + m;
+            float s0 = (Sp[(size_t)qi * C + lane] + Sp[((size_t)Q + qi) * C + lane]) * scale;
+            float s1 = (Sp[(size_t)qi * C + lane + 32] + Sp[((size_t)Q + qi) * C + lane + 32]) * scale;
+            if (key0 + lane > pos) s0 = -INFINITY;
+            if (key0 + lane + 32 > pos) s1 = -INFINITY;
+            float mx = fmaxf(s0, s1);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            float p0 = (s0 == -INFINITY) ? 0.f : expf(s0 - mx);
+            float p1 = (s1 == -INFINITY) ? 0.f : expf(s1 - mx);
+            float l = p0 + p1;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+            P[(size_t)qi * C + lane] = p0;
+            P[(size_t)qi * C + lane + 32] = p1;
+            if (lane == 0) {
+                float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * (HD + 2);
+                dst[HD] = mx;
+                dst[HD + 1] = l;
+            }
+        }
+    }
+    __syncthreads();
+
+    // phase 3: thread = (dim pair dp, key slice ks); o[q][dims] = sum_j P[q][j] V[j][dims]
+    {
+        const int dp = tid % HALF, ks = tid / HALF;
+        for (int q0 = 0; q0 < Q; q0 += 4) {
+            float acc[4][2] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll 4
+            for (int j = ks; j < C; j += NKS) {
+                uint32_t u = *reinterpret_cast<const uint32_t*>(Vs + j * HD * 2 + dp * 4);
+                float v0 = bf16lo(u), v1 = bf16hi(u);
+#pragma unroll
+                for (int qq = 0; qq < 4; ++qq) {
+                    int qi = min(q0 + qq, Q - 1);
+                    float p = P[(size_t)qi * C + j];
+                    acc[qq][0] = fmaf(p, v0, acc[qq][0]);
+                    acc[qq][1] = fmaf(p, v1, acc[qq][1]);
+                }
+            }
+#pragma unroll
+            for (int qq = 0; qq < 4; ++qq) {
+                Ored[((size_t)ks * 4 + qq) * HD + 2 * dp] = acc[qq][0];
+                Ored[((size_t)ks * 4 + qq) * HD + 2 * dp + 1] = acc[qq][1];
+            }
+            __syncthreads();
+            for (int idx = tid; idx < 4 * HD; idx += 128) {
+                int qq = idx / HD, dd = idx % HD;
+                if (q0 + qq < Q) {
+                    float s = 0.f;
+#pragma unroll
+                    for (int k2 = 0; k2 < NKS; ++k2) s += Ored[((size_t)k2 * 4 + qq) * HD + dd];
+                    int qi = q0 + qq, m = qi / G, g = qi % G;
+                    part[(((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * (HD + 2) + dd] = s;
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// merge the chunk partials of one (row, head) in chunk order; grid (M, Hq), block HD
+template <int HD>
+__global__ void __launch_bounds__(HD)
+attn_merge_kernel(const float* __restrict__ part, int32_t* ctl, int pos_off, int Hq, int chunk_cap,
+                  uint16_t* __restrict__ out)
+{
+    int pos0;
+    if (!pass_begin(ctl, pos_off, pos0)) return;
+    int m = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
+    int pos = pos0 + m;
+    int nch = pos / kAttnChunk + 1;
+    if (pos < 0 || nch > chunk_cap) return;  // refused by the chunk kernel (status word set)
+    const float* base = part + ((size_t)m * Hq + h) * chunk_cap * (HD + 2);
+    float mx = -INFINITY;
+    for (int c = 0; c < nch; ++c) mx = fmaxf(mx, base[(size_t)c * (HD + 2) + HD]);
+    float l = 0.f, o = 0.f;
+    for (int c = 0; c < nch; ++c) {
+        const float* pc = base + (size_t)c * (HD + 2);
+        float w = expf(pc[HD] - mx);
+        l = fmaf(pc[HD + 1], w, l);
+        o = fmaf(pc[d], w, o);
+    }
+    out[((size_t)m * Hq + h) * HD + d] = f2bf(o / l);
+}
+
+// ------------------------------------------------------------------ argmax finish
+// grid M, block 256: reduce the per-CTA (value, index) candidates of the LM-head kernel.
+// (value desc, index asc) is a total order, so the result does not depend on the
+// reduction tree; the lowest index wins a tie.
+__global__ void __launch_bounds__(256)
+argmax_finish_kernel(const ValIdx* __restrict__ cand, int n_cand, int cand_stride,
+                     int32_t* __restrict__ tok_out, const int32_t* ctl)
+{
+    __shared__ float sv[256];
+    __shared__ int si[256];
+    if (ctl && ctl[CTL_DONE]) return;
+    int m = blockIdx.x;
+    const ValIdx* c = cand + (size_t)m * cand_stride;
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int k = threadIdx.x; k < n_cand; k += 256) {
+        ValIdx e = c[k];
+        if (better(e.v, e.i, bv, bi)) {
+            bv = e.v;
+            bi = e.i;
+        }
+    }
+    sv[threadIdx.x] = bv;
+    si[threadIdx.x] = bi;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) {
+        if (threadIdx.x < s) {
+            float v = sv[threadIdx.x + s];
+            int i = si[threadIdx.x + s];
+            if (better(v, i, sv[threadIdx.x], si[threadIdx.x])) {
+                sv[threadIdx.x] = v;
+                si[threadIdx.x] = i;
+            }
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) tok_out[m] = si[0];
+}
+
+// ------------------------------------------------------------------ accept / rollback
+// match + crop of the paper's loop (Appendix A.4), one thread.  With d == 0 it is the
+// bookkeeping of plain greedy decoding (emit verified[0]).
+__global__ void accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ verified,
+                              int d, int32_t* ctl, int32_t* __restrict__ out_ids,
+                              int32_t* __restrict__ accepted)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (ctl[CTL_DONE]) return;
+    int n = 0;
+    while (n < d && draft[n] == verified[n]) ++n;
+    int n_out = ctl[CTL_N_OUT];
+    const int max_new = ctl[CTL_MAX_NEW], eos = ctl[CTL_EOS];
+    bool stop = false;
+    for (int i = 0; i <= n && n_out < max_new && !stop; ++i) {
+        int t = (i < n) ? draft[i] : verified[n];
+        out_ids[n_out++] = t;
+        if (eos >= 0 && t == eos) stop = true;
+    }
+    int steps = ctl[CTL_N_STEPS];
+    accepted[steps] = n;
+    ctl[CTL_N_STEPS] = steps + 1;
+    ctl[CTL_N_OUT] = n_out;
+    ctl[CTL_CUR_TOK] = verified[n];
+    ctl[CTL_CACHE_LEN] += n + 1;
+    if (stop || n_out >= max_new) ctl[CTL_DONE] = 1;
+}
+
+}  // namespace ls

@@ -1,0 +1,361 @@
+// Weight-streaming linear layers for M <= 16 rows: y[m, n] = sum_k W[n, k] h[m, k].
+//
+// Batch-1 decoding reads every weight byte once per pass and does 2*M flops per weight
+// element, so these kernels are HBM-bound; their job is to keep enough 16-byte loads in
+// flight and to spend few issue slots per byte.  Two families, chosen per model:
+//
+//   FMA  one warp per 4 weight rows, lanes stride over K with 128-bit loads, fp32 FMA
+//        chains per (row, token), butterfly reduction.  Cheap for M <= 4.
+//   MMA  one CTA per 16 weight rows, its 8 warps interleave over K; weights go from
+//        global memory straight into mma.sync.m16n8k16 A fragments (the contraction
+//        index may be permuted freely as long as A and B agree, so a thread's 16-byte
+//        load IS its fragment), tokens are the n8 dimension.  Issue cost per weight byte
+//        does not grow with M up to 8 (16 with a second n-tile).
+//
+// In both, the sequence of operations that produces (row n, token m) is the same for
+// every M, so results are bit-identical across pass sizes within a family.
+//
+// Epilogues: plain store, residual add (x <- x + W h, Sec. 4.1 of the paper), SwiGLU
+// (gate and up rows of one feature meet in one thread), and LM head + argmax candidates
+// (Sec. 2.1 / 4.2: the shared head g; greedy decoding needs only the index).
+#pragma once
+#include "ls_kernels.cuh"
+
+namespace ls {
+
+enum Epi : int { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_ARGMAX = 3 };
+
+struct LinArgs {
+    const uint16_t* w0;  // row segments: rows [0, n0) of w0, then n1 rows of w1, the rest of w2
+    const uint16_t* w1;  // (QKV as one launch); SwiGLU: w0 = gate, w1 = up
+    const uint16_t* w2;
+    int n0, n1;
+    const uint16_t* h;   // [M][K] bf16
+    int M, N, K;         // N: output rows (SwiGLU: features F)
+    float* out;          // fp32 [M][ldo]: store / residual / optional logits
+    int ldo;
+    uint16_t* out_bf16;  // SwiGLU result [M][N]
+    ValIdx* cand;        // argmax candidates [M][cand_stride], one per CTA
+    int cand_stride;
+    const int32_t* ctl;
+};
+
+__device__ __forceinline__ const uint16_t* weight_row(const LinArgs& a, int n)
+{
+    n = min(n, a.N - 1);
+    if (n < a.n0) return a.w0 + (size_t)n * a.K;
+    n -= a.n0;
+    if (n < a.n1) return a.w1 + (size_t)n * a.K;
+    n -= a.n1;
+    return a.w2 + (size_t)n * a.K;
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.0f + expf(-g)) * u; }
+
+// =============================================================================== FMA family
+// grid ceil(N/16) (SwiGLU: ceil(F/8)), block 128 = 4 warps x 4 weight rows.
+template <int MT, int EPI>
+__global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
+{
+    if (a.ctl && a.ctl[CTL_DONE]) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint16_t* rp[4];
+    int nrow[4];  // output index of each of the warp's rows
+    if (EPI == EPI_SWIGLU) {
+        int f = blockIdx.x * 8 + warp * 2;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            nrow[r] = f + (r & 1);
+            int fc = min(nrow[r], a.N - 1);
+            rp[r] = ((r < 2) ? a.w0 : a.w1) + (size_t)fc * a.K;
+        }
+    } else {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            nrow[r] = blockIdx.x * 16 + warp * 4 + r;
+            rp[r] = weight_row(a, nrow[r]);
+        }
+    }
+    float acc[4][MT];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int m = 0; m < MT; ++m) acc[r][m] = 0.f;
+
+    const int nchunks = a.K >> 3;
+#pragma unroll 2
+    for (int c = lane; c < nchunks; c += 32) {
+        float wf[4][8];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            uint4 v = ld_stream16(rp[r] + 8 * c);
+            wf[r][0] = bf16lo(v.x); wf[r][1] = bf16hi(v.x);
+            wf[r][2] = bf16lo(v.y); wf[r][3] = bf16hi(v.y);
+            wf[r][4] = bf16lo(v.z); wf[r][5] = bf16hi(v.z);
+            wf[r][6] = bf16lo(v.w); wf[r][7] = bf16hi(v.w);
+        }
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            uint4 v = ld_reuse16(a.h + (size_t)min(m, a.M - 1) * a.K + 8 * c);
+            float xf[8] = {bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y),
+                           bf16lo(v.z), bf16hi(v.z), bf16lo(v.w), bf16hi(v.w)};
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                float s = acc[r][m];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) s = fmaf(wf[r][e], xf[e], s);
+                acc[r][m] = s;
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            float v = acc[r][m];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            acc[r][m] = v;
+        }
+
+    if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (lane == m && m < a.M) {
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    if (nrow[r] < a.N) {
+                        float* o = a.out + (size_t)m * a.ldo + nrow[r];
+                        *o = (EPI == EPI_RESIDUAL) ? (*o + acc[r][m]) : acc[r][m];
+                    }
+            }
+    } else if (EPI == EPI_SWIGLU) {
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (lane == m && m < a.M) {
+#pragma unroll
+                for (int r = 0; r < 2; ++r)
+                    if (nrow[r] < a.N)
+                        a.out_bf16[(size_t)m * a.N + nrow[r]] = f2bf(silu_mul(acc[r][m], acc[r + 2][m]));
+            }
+    } else {  // EPI_ARGMAX
+        __shared__ float bv[4][MT];
+        __shared__ int bi[4][MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (lane == m) {
+                float v = -INFINITY;
+                int idx = 0x7fffffff;
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    if (nrow[r] < a.N) {
+                        if (a.out && m < a.M) a.out[(size_t)m * a.ldo + nrow[r]] = acc[r][m];
+                        if (better(acc[r][m], nrow[r], v, idx)) {
+                            v = acc[r][m];
+                            idx = nrow[r];
+                        }
+                    }
+                bv[warp][m] = v;
+                bi[warp][m] = idx;
+            }
+        __syncthreads();
+        if (threadIdx.x < MT && threadIdx.x < a.M) {
+            int m = threadIdx.x;
+            float v = bv[0][m];
+            int idx = bi[0][m];
+#pragma unroll
+            for (int w = 1; w < 4; ++w)
+                if (better(bv[w][m], bi[w][m], v, idx)) {
+                    v = bv[w][m];
+                    idx = bi[w][m];
+                }
+            ValIdx e;
+            e.v = v;
+            e.i = idx;
+            a.cand[(size_t)m * a.cand_stride + blockIdx.x] = e;
+        }
+    }
+}
+
+// =============================================================================== MMA family
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// grid ceil(N/16) (SwiGLU: ceil(F/8)), block 256 = 8 warps that interleave over K in steps
+// of 32.  Fragment roles (g = lane/4, t = lane%4): the thread's 16 bytes of row g (and of
+// row g+8) at k = 32 s + 8 t feed two MMAs; contraction slots {2t, 2t+1, 2t+8, 2t+9} of
+// the first take elements k..k+3, of the second k+4..k+7, for A and for B alike.
+// SwiGLU: row g is the gate row of feature f, row g+8 its up row.
+template <int NT, int EPI>
+__global__ void __launch_bounds__(256) linear_mma_kernel(const LinArgs a)
+{
+    constexpr int U = 4;  // k-steps in flight per warp
+    if (a.ctl && a.ctl[CTL_DONE]) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const uint16_t *pa, *pb;
+    if (EPI == EPI_SWIGLU) {
+        int f = min(blockIdx.x * 8 + g, a.N - 1);
+        pa = a.w0 + (size_t)f * a.K;
+        pb = a.w1 + (size_t)f * a.K;
+    } else {
+        pa = weight_row(a, blockIdx.x * 16 + g);
+        pb = weight_row(a, blockIdx.x * 16 + g + 8);
+    }
+    const uint16_t* hb[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) hb[nt] = a.h + (size_t)min(nt * 8 + g, a.M - 1) * a.K;
+
+    float c[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c[nt][i] = 0.f;
+
+    const int nsteps = (a.K + 31) >> 5;
+    for (int s0 = warp; s0 < nsteps; s0 += 8 * U) {
+        uint4 A0[U], A1[U], B[U][NT];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            int k = (s0 + 8 * u) * 32 + 8 * t;
+            bool ok = (s0 + 8 * u < nsteps) && (k < a.K);
+            A0[u] = A1[u] = make_uint4(0, 0, 0, 0);
+            if (ok) {
+                A0[u] = ld_stream16(pa + k);
+                A1[u] = ld_stream16(pb + k);
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                B[u][nt] = make_uint4(0, 0, 0, 0);
+                if (ok) B[u][nt] = ld_reuse16(hb[nt] + k);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                mma_bf16_16816(c[nt], A0[u].x, A1[u].x, A0[u].y, A1[u].y, B[u][nt].x, B[u][nt].y);
+                mma_bf16_16816(c[nt], A0[u].z, A1[u].z, A0[u].w, A1[u].w, B[u][nt].z, B[u][nt].w);
+            }
+        }
+    }
+
+    // cross-warp reduction in warp order (fixed), then the epilogue on 32*NT threads
+    __shared__ float red[8][NT * 4][32];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) red[warp][nt * 4 + i][lane] = c[nt][i];
+    __syncthreads();
+    __shared__ float vals[16][NT * 8 + 1];
+    if (threadIdx.x < 32 * NT) {
+        const int nt = threadIdx.x >> 5;
+        const int gg = lane >> 2, tt = lane & 3;
+        float r[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float s = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) s += red[w][nt * 4 + i][lane];
+            r[i] = s;
+        }
+        const int m0 = nt * 8 + 2 * tt;  // tokens m0, m0+1
+        if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+            const int nlo = blockIdx.x * 16 + gg, nhi = nlo + 8;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                int m = m0 + (i & 1), n = (i < 2) ? nlo : nhi;
+                if (m < a.M && n < a.N) {
+                    float* o = a.out + (size_t)m * a.ldo + n;
+                    *o = (EPI == EPI_RESIDUAL) ? (*o + r[i]) : r[i];
+                }
+            }
+        } else if (EPI == EPI_SWIGLU) {
+            const int f = blockIdx.x * 8 + gg;
+            if (f < a.N) {
+                if (m0 < a.M) a.out_bf16[(size_t)m0 * a.N + f] = f2bf(silu_mul(r[0], r[2]));
+                if (m0 + 1 < a.M) a.out_bf16[(size_t)(m0 + 1) * a.N + f] = f2bf(silu_mul(r[1], r[3]));
+            }
+        } else {
+            vals[gg][m0] = r[0];
+            vals[gg][m0 + 1] = r[1];
+            vals[gg + 8][m0] = r[2];
+            vals[gg + 8][m0 + 1] = r[3];
+        }
+    }
+    if (EPI == EPI_ARGMAX) {
+        __syncthreads();
+        if (threadIdx.x < a.M) {
+            const int m = threadIdx.x;
+            float v = -INFINITY;
+            int idx = 0x7fffffff;
+#pragma unroll
+            for (int rr = 0; rr < 16; ++rr) {
+                int n = blockIdx.x * 16 + rr;
+                if (n < a.N) {
+                    float x = vals[rr][m];
+                    if (a.out) a.out[(size_t)m * a.ldo + n] = x;
+                    if (better(x, n, v, idx)) {
+                        v = x;
+                        idx = n;
+                    }
+                }
+            }
+            ValIdx e;
+            e.v = v;
+            e.i = idx;
+            a.cand[(size_t)m * a.cand_stride + blockIdx.x] = e;
+        }
+    }
+}
+
+// =============================================================================== launchers
+inline int lin_grid(int epi, int N) { return epi == EPI_SWIGLU ? (N + 7) / 8 : (N + 15) / 16; }
+
+template <int EPI>
+inline cudaError_t launch_linear_fma(const LinArgs& a, cudaStream_t st)
+{
+    dim3 grid(lin_grid(EPI, a.N)), block(128);
+    if (a.M <= 1) linear_fma_kernel<1, EPI><<<grid, block, 0, st>>>(a);
+    else if (a.M <= 2) linear_fma_kernel<2, EPI><<<grid, block, 0, st>>>(a);
+    else if (a.M <= 4) linear_fma_kernel<4, EPI><<<grid, block, 0, st>>>(a);
+    else if (a.M <= 8) linear_fma_kernel<8, EPI><<<grid, block, 0, st>>>(a);
+    else linear_fma_kernel<16, EPI><<<grid, block, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+template <int EPI>
+inline cudaError_t launch_linear_mma(const LinArgs& a, cudaStream_t st)
+{
+    dim3 grid(lin_grid(EPI, a.N)), block(256);
+    if (a.M <= 8) linear_mma_kernel<1, EPI><<<grid, block, 0, st>>>(a);
+    else linear_mma_kernel<2, EPI><<<grid, block, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+// path: 1 = FMA, 2 = MMA
+inline cudaError_t launch_linear(int path, int epi, const LinArgs& a, cudaStream_t st)
+{
+    if (path == 1) {
+        switch (epi) {
+            case EPI_STORE: return launch_linear_fma<EPI_STORE>(a, st);
+            case EPI_RESIDUAL: return launch_linear_fma<EPI_RESIDUAL>(a, st);
+            case EPI_SWIGLU: return launch_linear_fma<EPI_SWIGLU>(a, st);
+            default: return launch_linear_fma<EPI_ARGMAX>(a, st);
+        }
+    }
+    switch (epi) {
+        case EPI_STORE: return launch_linear_mma<EPI_STORE>(a, st);
+        case EPI_RESIDUAL: return launch_linear_mma<EPI_RESIDUAL>(a, st);
+        case EPI_SWIGLU: return launch_linear_mma<EPI_SWIGLU>(a, st);
+        default: return launch_linear_mma<EPI_ARGMAX>(a, st);
+    }
+}
+
+}  // namespace ls
