@@ -1,0 +1,856 @@
+// Host side of the library: model handle, workspace carve-up, the draft / verify /
+// accept schedule of LayerSkip's self-speculative decoding (Sec. 4.3, Appendix A.4)
+// as CUDA graphs, and the C ABI declared in ls.h.
+//
+// Schedule of one speculative step (E early layers, d drafts), all on one stream, all
+// positions read by the kernels from the control words in device memory:
+//   for j = 0..d:   embed(input_j) -> layers 0..E-1 on residual row j at position c+j
+//                   (j < d: final norm + LM head + argmax -> draft[j] = input_{j+1})
+//   verify:         layers E..L-1 on residual rows 0..d (they ARE the exit-layer
+//                   activations: nothing is copied), final norm + LM head + argmax
+//   accept:         match, emit, crop (one tiny kernel); sets the done flag
+// The host launches a batch of step graphs sized to the tokens still missing and only
+// then looks at the control words, so there is no host sync per token; steps launched
+// past the end see the done flag and return at once.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <new>
+#include <vector>
+
+#include "ls.h"
+#include "ls_linear.cuh"
+
+using namespace ls;
+
+namespace {
+
+thread_local int g_last_cuda = 0;
+
+#define LS_CK(expr)                         \
+    do {                                    \
+        cudaError_t e_ = (expr);            \
+        if (e_ != cudaSuccess) {            \
+            g_last_cuda = (int)e_;          \
+            return LS_ERR_CUDA;             \
+        }                                   \
+    } while (0)
+
+#define LS_TRY(expr)            \
+    do {                        \
+        int rc_ = (expr);       \
+        if (rc_ != LS_OK) return rc_; \
+    } while (0)
+
+struct LayerW {
+    const uint16_t *attn_norm, *wq, *wk, *wv, *wo, *ffn_norm, *wg, *wu, *wd;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return p && ((uintptr_t)p & 15u) == 0; }
+
+int log2_exact(int v)
+{
+    int s = 0;
+    while ((1 << s) < v) ++s;
+    return ((1 << s) == v) ? s : -1;
+}
+
+bool config_ok(const ls_config* c)
+{
+    if (!c) return false;
+    if (c->n_layers < 1 || c->d_model < 8 || c->d_model % 8 || c->d_ffn < 8 || c->d_ffn % 8) return false;
+    if (c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->n_heads < 1 || c->n_kv_heads < 1 || c->n_heads % c->n_kv_heads) return false;
+    if (c->n_heads / c->n_kv_heads > 8) return false;
+    if (c->vocab < 1 || c->max_seq < 2) return false;
+    if (c->page_size < 16 || c->page_size > 1024 || log2_exact(c->page_size) < 0) return false;
+    if (c->max_draft < 0 || c->max_draft + 1 > LS_MAX_ROWS) return false;
+    if (c->linear_path < 0 || c->linear_path > 2) return false;
+    if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return false;
+    return true;
+}
+
+}  // namespace
+
+struct ls_model {
+    ls_config c;
+    int path;
+    cudaStream_t st;
+    std::vector<LayerW> lw;
+    const uint16_t *emb, *fnorm, *lm;
+    // workspace
+    uint16_t *kpages, *vpages;
+    size_t layer_kv_elems;
+    int32_t *page_table, *ctl, *draft, *verified, *out_ids, *accepted, *ids;
+    float *inv_freq, *x, *qkv, *part, *logits;
+    uint16_t *h, *q, *o, *a;
+    ValIdx* cand;
+    int page_shift, n_pages, chunk_cap, cand_stride;
+    // loop state
+    int n_prompt, last_tok, prefilled_layers, grid_chunks;
+    bool use_graphs, capturing;
+    int64_t launches;  // kernels enqueued (counted while building a step)
+    struct G {
+        cudaGraphExec_t exec;
+        int64_t nodes;
+    };
+    std::map<uint64_t, G> graphs;
+    cudaEvent_t ev0, ev1;
+    ls_stats stats;
+    std::vector<int32_t> h_out, h_acc;
+    int h_n_out, h_n_steps;
+};
+
+namespace {
+
+// carve the workspace; with base == nullptr only sizes are computed
+size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
+{
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        unsigned char* p = base ? base + off : nullptr;
+        off = align_up(off + bytes, 256);
+        return p;
+    };
+    const int n_pages = (c.max_seq + c.page_size - 1) / c.page_size;
+    const int chunk_cap = (c.max_seq + kAttnChunk - 1) / kAttnChunk;
+    const int cand_stride = (c.vocab + 15) / 16;
+    const size_t layer_kv = (size_t)n_pages * c.n_kv_heads * c.page_size * c.head_dim;
+    const size_t qw = (size_t)c.n_heads * c.head_dim, kvw = (size_t)c.n_kv_heads * c.head_dim;
+    unsigned char* kp = take(layer_kv * c.n_layers * 2);
+    unsigned char* vp = take(layer_kv * c.n_layers * 2);
+    unsigned char* pt = take(sizeof(int32_t) * n_pages);
+    unsigned char* fr = take(sizeof(float) * (c.head_dim / 2));
+    unsigned char* ctl = take(sizeof(int32_t) * CTL_WORDS);
+    unsigned char* dr = take(sizeof(int32_t) * kMaxRows);
+    unsigned char* ve = take(sizeof(int32_t) * kMaxRows);
+    unsigned char* oi = take(sizeof(int32_t) * c.max_seq);
+    unsigned char* ac = take(sizeof(int32_t) * c.max_seq);
+    unsigned char* ids = take(sizeof(int32_t) * c.max_seq);
+    unsigned char* x = take(sizeof(float) * kMaxRows * c.d_model);
+    unsigned char* qkv = take(sizeof(float) * kMaxRows * (qw + 2 * kvw));
+    unsigned char* part = take(sizeof(float) * kMaxRows * c.n_heads * chunk_cap * (c.head_dim + 2));
+    unsigned char* logits = take(sizeof(float) * kMaxRows * c.vocab);
+    unsigned char* h = take(2 * (size_t)kMaxRows * c.d_model);
+    unsigned char* q = take(2 * (size_t)kMaxRows * qw);
+    unsigned char* o = take(2 * (size_t)kMaxRows * qw);
+    unsigned char* a = take(2 * (size_t)kMaxRows * c.d_ffn);
+    unsigned char* cand = take(sizeof(ValIdx) * kMaxRows * cand_stride);
+    if (m) {
+        m->kpages = (uint16_t*)kp;
+        m->vpages = (uint16_t*)vp;
+        m->layer_kv_elems = layer_kv;
+        m->page_table = (int32_t*)pt;
+        m->inv_freq = (float*)fr;
+        m->ctl = (int32_t*)ctl;
+        m->draft = (int32_t*)dr;
+        m->verified = (int32_t*)ve;
+        m->out_ids = (int32_t*)oi;
+        m->accepted = (int32_t*)ac;
+        m->ids = (int32_t*)ids;
+        m->x = (float*)x;
+        m->qkv = (float*)qkv;
+        m->part = (float*)part;
+        m->logits = (float*)logits;
+        m->h = (uint16_t*)h;
+        m->q = (uint16_t*)q;
+        m->o = (uint16_t*)o;
+        m->a = (uint16_t*)a;
+        m->cand = (ValIdx*)cand;
+        m->n_pages = n_pages;
+        m->chunk_cap = chunk_cap;
+        m->cand_stride = cand_stride;
+        m->page_shift = log2_exact(c.page_size);
+    }
+    return off;
+}
+
+// ------------------------------------------------------------------ kernel launch helpers
+int attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
+                int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int hd, int page_shift,
+                int max_seq, int chunk_cap, int grid_chunks, float* part, uint16_t* out,
+                cudaStream_t st)
+{
+    const int Q = Hq / Hkv * M;
+    dim3 grid(grid_chunks, Hkv), mgrid(M, Hq);
+    if (hd == 128) {
+        size_t sm = attn_smem_bytes<128>(Q);
+        attn_chunk_kernel<128><<<grid, 128, sm, st>>>(q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv,
+                                                        page_shift, max_seq, chunk_cap, part);
+        attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(part, ctl, pos_off, Hq, chunk_cap, out);
+    } else {
+        size_t sm = attn_smem_bytes<64>(Q);
+        attn_chunk_kernel<64><<<grid, 128, sm, st>>>(q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv,
+                                                       page_shift, max_seq, chunk_cap, part);
+        attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(part, ctl, pos_off, Hq, chunk_cap, out);
+    }
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+int attn_allow_smem(int hd, int group)
+{
+    const int Q = group * kMaxRows;
+    if (hd == 128) {
+        LS_CK(cudaFuncSetAttribute(attn_chunk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)attn_smem_bytes<128>(Q)));
+    } else {
+        LS_CK(cudaFuncSetAttribute(attn_chunk_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)attn_smem_bytes<64>(Q)));
+    }
+    return LS_OK;
+}
+
+LinArgs lin_args(const uint16_t* w, const uint16_t* h, int M, int N, int K)
+{
+    LinArgs a;
+    memset(&a, 0, sizeof(a));
+    a.w0 = a.w1 = a.w2 = w;
+    a.n0 = N;
+    a.n1 = 0;
+    a.h = h;
+    a.M = M;
+    a.N = N;
+    a.K = K;
+    return a;
+}
+
+// layers [l0, l1) on M residual rows starting at xrow; row r sits at ctl.cache_len + pos_off + r
+int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
+{
+    const ls_config& c = m->c;
+    const int D = c.d_model, Hq = c.n_heads, Hkv = c.n_kv_heads, hd = c.head_dim, F = c.d_ffn;
+    const int qw = Hq * hd, kvw = Hkv * hd;
+    cudaStream_t st = m->st;
+    for (int l = l0; l < l1; ++l) {
+        const LayerW& w = m->lw[l];
+        uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
+        uint16_t* vp = m->vpages + (size_t)l * m->layer_kv_elems;
+        rmsnorm_kernel<<<M, 256, 0, st>>>(xrow, w.attn_norm, D, c.rms_eps, m->h, m->ctl);
+        LinArgs a = lin_args(w.wq, m->h, M, qw + 2 * kvw, D);
+        a.w1 = w.wk;
+        a.w2 = w.wv;
+        a.n0 = qw;
+        a.n1 = kvw;
+        a.out = m->qkv;
+        a.ldo = qw + 2 * kvw;
+        a.ctl = m->ctl;
+        LS_CK(launch_linear(m->path, EPI_STORE, a, st));
+        rope_append_kernel<<<dim3(M, Hq + 2 * Hkv), hd / 2, 0, st>>>(
+            m->qkv, Hq, Hkv, hd, m->inv_freq, c.rope_theta, m->page_shift, m->page_table, c.max_seq,
+            m->q, kp, vp, m->ctl, pos_off);
+        LS_TRY(attn_launch(m->q, kp, vp, m->page_table, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift,
+                           c.max_seq, m->chunk_cap, m->grid_chunks, m->part, m->o, st));
+        a = lin_args(w.wo, m->o, M, D, qw);
+        a.out = xrow;
+        a.ldo = D;
+        a.ctl = m->ctl;
+        LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
+        rmsnorm_kernel<<<M, 256, 0, st>>>(xrow, w.ffn_norm, D, c.rms_eps, m->h, m->ctl);
+        a = lin_args(w.wg, m->h, M, F, D);
+        a.w1 = w.wu;
+        a.out_bf16 = m->a;
+        a.ctl = m->ctl;
+        LS_CK(launch_linear(m->path, EPI_SWIGLU, a, st));
+        a = lin_args(w.wd, m->a, M, D, F);
+        a.out = xrow;
+        a.ldo = D;
+        a.ctl = m->ctl;
+        LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
+        m->launches += 9;
+    }
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+// shared head g(.) = final norm + LM head (+ argmax) on M residual rows
+int run_head(ls_model* m, int M, const float* xrow, int32_t* tok_out, float* logits)
+{
+    const ls_config& c = m->c;
+    rmsnorm_kernel<<<M, 256, 0, m->st>>>(xrow, m->fnorm, c.d_model, c.rms_eps, m->h, m->ctl);
+    LinArgs a = lin_args(m->lm, m->h, M, c.vocab, c.d_model);
+    a.cand = m->cand;
+    a.cand_stride = m->cand_stride;
+    a.out = logits;
+    a.ldo = c.vocab;
+    a.ctl = m->ctl;
+    LS_CK(launch_linear(m->path, EPI_ARGMAX, a, m->st));
+    argmax_finish_kernel<<<M, 256, 0, m->st>>>(m->cand, lin_grid(EPI_ARGMAX, c.vocab), m->cand_stride,
+                                               tok_out, m->ctl);
+    m->launches += 3;
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+int run_embed(ls_model* m, const int32_t* tok_dev, int M, float* xrow)
+{
+    embed_kernel<<<M, 256, 0, m->st>>>(m->emb, tok_dev, m->c.d_model, m->c.vocab, xrow, m->ctl);
+    m->launches += 1;
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+// one step of the loop.  E == L with d == 0: plain greedy; E < L with d == 0: early exit.
+int enqueue_step(ls_model* m, int E, int d)
+{
+    const int D = m->c.d_model, L = m->c.n_layers;
+    if (d == 0) {
+        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x));
+        LS_TRY(run_layers(m, 0, E, 1, m->x, 0));
+        LS_TRY(run_head(m, 1, m->x, m->verified, nullptr));
+    } else {
+        for (int j = 0; j <= d; ++j) {  // self-drafting (Sec. 4.3.1) + the extra early pass
+            float* xr = m->x + (size_t)j * D;
+            LS_TRY(run_embed(m, j == 0 ? m->ctl + CTL_CUR_TOK : m->draft + (j - 1), 1, xr));
+            LS_TRY(run_layers(m, 0, E, 1, xr, j));
+            if (j < d) LS_TRY(run_head(m, 1, xr, m->draft + j, nullptr));
+        }
+        // self-verification (Sec. 4.3.2) from the exit-layer activations (Sec. 4.3.3)
+        LS_TRY(run_layers(m, E, L, d + 1, m->x, 0));
+        LS_TRY(run_head(m, d + 1, m->x, m->verified, nullptr));
+    }
+    accept_kernel<<<1, 32, 0, m->st>>>(m->draft, m->verified, d, m->ctl, m->out_ids, m->accepted);
+    m->launches += 1;
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+void drop_graphs(ls_model* m)
+{
+    for (auto& kv : m->graphs) cudaGraphExecDestroy(kv.second.exec);
+    m->graphs.clear();
+}
+
+int get_graph(ls_model* m, int E, int d, ls_model::G** out)
+{
+    uint64_t key = ((uint64_t)E << 32) | ((uint64_t)d << 16) | (uint64_t)m->grid_chunks;
+    auto it = m->graphs.find(key);
+    if (it == m->graphs.end()) {
+        cudaGraph_t graph = nullptr;
+        int64_t before = m->launches;
+        LS_CK(cudaStreamBeginCapture(m->st, cudaStreamCaptureModeRelaxed));
+        int rc = enqueue_step(m, E, d);
+        cudaError_t e = cudaStreamEndCapture(m->st, &graph);
+        if (rc != LS_OK) {
+            if (graph) cudaGraphDestroy(graph);
+            return rc;
+        }
+        LS_CK(e);
+        ls_model::G g;
+        g.nodes = m->launches - before;
+        e = cudaGraphInstantiate(&g.exec, graph, 0);
+        cudaGraphDestroy(graph);
+        LS_CK(e);
+        it = m->graphs.emplace(key, g).first;
+    }
+    *out = &it->second;
+    return LS_OK;
+}
+
+int write_ctl(ls_model* m, int cache_len, int cur, int max_new)
+{
+    int32_t w[CTL_WORDS] = {cache_len, cur, 0, 0, 0, max_new, m->c.eos_id, 0};
+    LS_CK(cudaMemcpyAsync(m->ctl, w, sizeof(w), cudaMemcpyHostToDevice, m->st));
+    LS_CK(cudaStreamSynchronize(m->st));  // w is a stack array
+    return LS_OK;
+}
+
+int read_ctl(ls_model* m, int32_t* w)
+{
+    LS_CK(cudaMemcpyAsync(w, m->ctl, sizeof(int32_t) * CTL_WORDS, cudaMemcpyDeviceToHost, m->st));
+    LS_CK(cudaStreamSynchronize(m->st));
+    return LS_OK;
+}
+
+int check_ids(const ls_model* m, const int32_t* ids, int n)
+{
+    if (!ids || n < 1) return LS_ERR_INVALID_ARG;
+    for (int i = 0; i < n; ++i)
+        if (ids[i] < 0 || ids[i] >= m->c.vocab) return LS_ERR_INVALID_ARG;
+    return LS_OK;
+}
+
+void set_grid_chunks(ls_model* m, int max_pos_exclusive)
+{
+    int g = (max_pos_exclusive + kAttnChunk - 1) / kAttnChunk;
+    if (g > m->chunk_cap) g = m->chunk_cap;
+    if (g < 1) g = 1;
+    if (g != m->grid_chunks) {
+        m->grid_chunks = g;
+        drop_graphs(m);
+    }
+}
+
+}  // namespace
+
+// =============================================================================== C ABI
+extern "C" {
+
+const char* ls_strerror(int s)
+{
+    switch (s) {
+        case LS_OK: return "ok";
+        case LS_ERR_INVALID_ARG: return "invalid argument";
+        case LS_ERR_CAPACITY: return "capacity exceeded (KV cache, workspace or max_draft)";
+        case LS_ERR_CUDA: return "CUDA runtime error (see ls_last_cuda_error)";
+        case LS_ERR_DEVICE_STATUS: return "a kernel's bounds check refused an access";
+        case LS_ERR_UNSUPPORTED: return "unsupported device or shape";
+        default: return "unknown status";
+    }
+}
+
+int ls_last_cuda_error(void) { return g_last_cuda; }
+
+size_t ls_workspace_bytes(const ls_config* cfg)
+{
+    if (!config_ok(cfg)) return 0;
+    return carve(*cfg, nullptr, nullptr);
+}
+
+int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, size_t workspace_bytes,
+                    void* cuda_stream, ls_model** out)
+{
+    if (!out) return LS_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!config_ok(cfg) || !w || !workspace) return LS_ERR_INVALID_ARG;
+    if (((uintptr_t)workspace & 255u) != 0) return LS_ERR_INVALID_ARG;
+    if (workspace_bytes < carve(*cfg, nullptr, nullptr)) return LS_ERR_CAPACITY;
+    int dev = 0;
+    cudaDeviceProp prop;
+    LS_CK(cudaGetDevice(&dev));
+    LS_CK(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return LS_ERR_UNSUPPORTED;
+    if (!aligned16(w->tok_embed) || !aligned16(w->final_norm) || !aligned16(w->lm_head)) return LS_ERR_INVALID_ARG;
+    const void* const* per[9] = {w->attn_norm, w->wq, w->wk, w->wv, w->wo, w->ffn_norm, w->w_gate, w->w_up, w->w_down};
+    for (int i = 0; i < 9; ++i) {
+        if (!per[i]) return LS_ERR_INVALID_ARG;
+        for (int l = 0; l < cfg->n_layers; ++l)
+            if (!aligned16(per[i][l])) return LS_ERR_INVALID_ARG;
+    }
+    ls_model* m = new (std::nothrow) ls_model();
+    if (!m) return LS_ERR_CAPACITY;
+    m->c = *cfg;
+    m->path = cfg->linear_path == LS_LINEAR_AUTO ? (cfg->max_draft + 1 > 4 ? LS_LINEAR_MMA : LS_LINEAR_FMA)
+                                                 : cfg->linear_path;
+    if (const char* e = getenv("LS_LINEAR_PATH")) {
+        if (!strcmp(e, "fma")) m->path = LS_LINEAR_FMA;
+        if (!strcmp(e, "mma")) m->path = LS_LINEAR_MMA;
+    }
+    m->st = (cudaStream_t)cuda_stream;
+    m->emb = (const uint16_t*)w->tok_embed;
+    m->fnorm = (const uint16_t*)w->final_norm;
+    m->lm = (const uint16_t*)w->lm_head;
+    m->lw.resize(cfg->n_layers);
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        LayerW& x = m->lw[l];
+        x.attn_norm = (const uint16_t*)w->attn_norm[l];
+        x.wq = (const uint16_t*)w->wq[l];
+        x.wk = (const uint16_t*)w->wk[l];
+        x.wv = (const uint16_t*)w->wv[l];
+        x.wo = (const uint16_t*)w->wo[l];
+        x.ffn_norm = (const uint16_t*)w->ffn_norm[l];
+        x.wg = (const uint16_t*)w->w_gate[l];
+        x.wu = (const uint16_t*)w->w_up[l];
+        x.wd = (const uint16_t*)w->w_down[l];
+    }
+    size_t used = carve(*cfg, (unsigned char*)workspace, m);
+    m->n_prompt = 0;
+    m->prefilled_layers = 0;
+    m->grid_chunks = m->chunk_cap;
+    m->use_graphs = getenv("LS_NO_GRAPH") == nullptr;
+    m->launches = 0;
+    memset(&m->stats, 0, sizeof(m->stats));
+    m->h_n_out = m->h_n_steps = 0;
+    m->ev0 = m->ev1 = nullptr;
+    auto fail = [&](int rc) {
+        if (m->ev0) cudaEventDestroy(m->ev0);
+        if (m->ev1) cudaEventDestroy(m->ev1);
+        delete m;
+        return rc;
+    };
+    cudaError_t e = cudaMemsetAsync(workspace, 0, used, m->st);
+    if (e == cudaSuccess) {
+        std::vector<int32_t> pt(m->n_pages);
+        for (int i = 0; i < m->n_pages; ++i) pt[i] = i;
+        std::vector<float> fr(cfg->head_dim / 2);
+        for (int j = 0; j < cfg->head_dim / 2; ++j)
+            fr[j] = (float)pow((double)cfg->rope_theta, -2.0 * (double)j / (double)cfg->head_dim);
+        e = cudaMemcpyAsync(m->page_table, pt.data(), sizeof(int32_t) * pt.size(), cudaMemcpyHostToDevice, m->st);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(m->inv_freq, fr.data(), sizeof(float) * fr.size(), cudaMemcpyHostToDevice, m->st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(m->st);
+    }
+    if (e == cudaSuccess) e = cudaEventCreate(&m->ev0);
+    if (e == cudaSuccess) e = cudaEventCreate(&m->ev1);
+    if (e != cudaSuccess) {
+        g_last_cuda = (int)e;
+        return fail(LS_ERR_CUDA);
+    }
+    int rc = attn_allow_smem(cfg->head_dim, cfg->n_heads / cfg->n_kv_heads);
+    if (rc != LS_OK) return fail(rc);
+    *out = m;
+    return LS_OK;
+}
+
+int ls_model_destroy(ls_model* m)
+{
+    if (!m) return LS_ERR_INVALID_ARG;
+    cudaStreamSynchronize(m->st);
+    drop_graphs(m);
+    cudaEventDestroy(m->ev0);
+    cudaEventDestroy(m->ev1);
+    delete m;
+    return LS_OK;
+}
+
+int ls_set_page_table(ls_model* m, const int32_t* table, int32_t n_pages)
+{
+    if (!m || !table || n_pages != m->n_pages) return LS_ERR_INVALID_ARG;
+    std::vector<char> seen(n_pages, 0);
+    for (int i = 0; i < n_pages; ++i) {
+        if (table[i] < 0 || table[i] >= n_pages || seen[table[i]]) return LS_ERR_INVALID_ARG;
+        seen[table[i]] = 1;
+    }
+    LS_CK(cudaMemcpyAsync(m->page_table, table, sizeof(int32_t) * n_pages, cudaMemcpyHostToDevice, m->st));
+    LS_CK(cudaStreamSynchronize(m->st));
+    m->n_prompt = 0;  // cached positions moved
+    return LS_OK;
+}
+
+int ls_prefill(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t layers)
+{
+    if (!m) return LS_ERR_INVALID_ARG;
+    LS_TRY(check_ids(m, prompt, n_prompt));
+    const int L = m->c.n_layers;
+    if (layers == 0) layers = L;
+    if (layers < 1 || layers > L) return LS_ERR_INVALID_ARG;
+    if (n_prompt > m->c.max_seq) return LS_ERR_CAPACITY;
+    m->n_prompt = 0;
+    set_grid_chunks(m, n_prompt);
+    LS_CK(cudaMemcpyAsync(m->ids, prompt, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, m->st));
+    LS_TRY(write_ctl(m, 0, 0, 0));
+    LS_CK(cudaEventRecord(m->ev0, m->st));
+    for (int r0 = 0; r0 < n_prompt - 1; r0 += kMaxRows) {
+        int M = n_prompt - 1 - r0;
+        if (M > kMaxRows) M = kMaxRows;
+        LS_TRY(run_embed(m, m->ids + r0, M, m->x));
+        LS_TRY(run_layers(m, 0, layers, M, m->x, r0));
+    }
+    LS_CK(cudaEventRecord(m->ev1, m->st));
+    int32_t w[CTL_WORDS];
+    LS_TRY(read_ctl(m, w));
+    if (w[CTL_STATUS]) return LS_ERR_DEVICE_STATUS;
+    float ms = 0.f;
+    LS_CK(cudaEventElapsedTime(&ms, m->ev0, m->ev1));
+    m->stats.prefill_ms = ms;
+    m->n_prompt = n_prompt;
+    m->last_tok = prompt[n_prompt - 1];
+    m->prefilled_layers = layers;
+    return LS_OK;
+}
+
+int ls_decode(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new)
+{
+    if (!m || m->n_prompt < 1) return LS_ERR_INVALID_ARG;
+    const ls_config& c = m->c;
+    const int L = c.n_layers;
+    int E = exit_layer, d = num_draft;
+    if (max_new < 1 || d < 0 || E < 0) return LS_ERR_INVALID_ARG;
+    if (E == 0) {
+        if (d != 0) return LS_ERR_INVALID_ARG;
+        E = L;  // plain greedy
+    } else if (d == 0) {
+        if (E > L) return LS_ERR_INVALID_ARG;  // early exit
+    } else {
+        if (E > L - 1) return LS_ERR_INVALID_ARG;
+        if (d > c.max_draft) return LS_ERR_CAPACITY;
+    }
+    const int need_layers = (d > 0) ? L : E;
+    if (m->prefilled_layers < need_layers) return LS_ERR_INVALID_ARG;
+    if ((int64_t)m->n_prompt + max_new + d + 1 > c.max_seq) return LS_ERR_CAPACITY;
+    set_grid_chunks(m, m->n_prompt + max_new + d + 1);
+
+    ls_model::G* g = nullptr;
+    if (m->use_graphs) LS_TRY(get_graph(m, E, d, &g));
+    LS_TRY(write_ctl(m, m->n_prompt - 1, m->last_tok, max_new));
+    int64_t launched = 0;
+    int syncs = 0, n_out = 0;
+    int32_t w[CTL_WORDS];
+    LS_CK(cudaEventRecord(m->ev0, m->st));
+    for (;;) {
+        int remaining = max_new - n_out;
+        int steps = (remaining + d) / (d + 1);
+        for (int i = 0; i < steps; ++i) {
+            if (g) {
+                LS_CK(cudaGraphLaunch(g->exec, m->st));
+                launched += g->nodes;
+            } else {
+                int64_t before = m->launches;
+                LS_TRY(enqueue_step(m, E, d));
+                launched += m->launches - before;
+            }
+        }
+        LS_TRY(read_ctl(m, w));
+        ++syncs;
+        if (w[CTL_STATUS]) return LS_ERR_DEVICE_STATUS;
+        n_out = w[CTL_N_OUT];
+        if (w[CTL_DONE]) break;
+    }
+    LS_CK(cudaEventRecord(m->ev1, m->st));
+    LS_CK(cudaEventSynchronize(m->ev1));
+    float ms = 0.f;
+    LS_CK(cudaEventElapsedTime(&ms, m->ev0, m->ev1));
+
+    m->h_n_out = w[CTL_N_OUT];
+    m->h_n_steps = w[CTL_N_STEPS];
+    m->h_out.resize(m->h_n_out);
+    m->h_acc.resize(m->h_n_steps);
+    LS_CK(cudaMemcpyAsync(m->h_out.data(), m->out_ids, sizeof(int32_t) * m->h_n_out, cudaMemcpyDeviceToHost, m->st));
+    LS_CK(cudaMemcpyAsync(m->h_acc.data(), m->accepted, sizeof(int32_t) * m->h_n_steps, cudaMemcpyDeviceToHost, m->st));
+    LS_CK(cudaStreamSynchronize(m->st));
+
+    // algorithmic bytes of the schedule (matrices only; norm gains and activations are noise)
+    const int64_t qw = (int64_t)c.n_heads * c.head_dim, kvw = (int64_t)c.n_kv_heads * c.head_dim;
+    const int64_t w_layer = 2 * ((qw + 2 * kvw) * c.d_model + qw * c.d_model + 3 * (int64_t)c.d_model * c.d_ffn);
+    const int64_t w_lm = 2 * (int64_t)c.vocab * c.d_model;
+    const int64_t kvb = 2 * 2 * kvw;
+    int64_t wb = 0, kb = 0, cl = m->n_prompt - 1, acc_sum = 0;
+    for (int s = 0; s < m->h_n_steps; ++s) {
+        int n = m->h_acc[s];
+        if (d == 0) {
+            wb += E * w_layer + w_lm;
+            kb += (int64_t)E * kvb * (cl + 1);
+        } else {
+            wb += (int64_t)(d + 1) * E * w_layer + (int64_t)d * w_lm + (int64_t)(L - E) * w_layer + w_lm;
+            for (int j = 0; j <= d; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
+            kb += (int64_t)(L - E) * kvb * (cl + d + 1);
+        }
+        cl += n + 1;
+        acc_sum += n;
+    }
+    m->stats.decode_ms = ms;
+    m->stats.weight_bytes = wb;
+    m->stats.kv_bytes = kb;
+    m->stats.kernel_launches = launched;
+    m->stats.n_generated = m->h_n_out;
+    m->stats.n_steps = m->h_n_steps;
+    m->stats.n_accepted = (int32_t)acc_sum;
+    m->stats.host_syncs = syncs;
+    return LS_OK;
+}
+
+int ls_read_output(ls_model* m, int32_t* out_ids, int32_t* out_n, int32_t* accepted, int32_t* out_steps)
+{
+    if (!m) return LS_ERR_INVALID_ARG;
+    if (out_ids && m->h_n_out) memcpy(out_ids, m->h_out.data(), sizeof(int32_t) * m->h_n_out);
+    if (out_n) *out_n = m->h_n_out;
+    if (accepted && m->h_n_steps) memcpy(accepted, m->h_acc.data(), sizeof(int32_t) * m->h_n_steps);
+    if (out_steps) *out_steps = m->h_n_steps;
+    return LS_OK;
+}
+
+int ls_generate(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t exit_layer, int32_t num_draft,
+                int32_t max_new, int32_t* out_ids, int32_t* out_n, int32_t* accepted, int32_t* out_steps)
+{
+    if (!m || !out_ids || !out_n || !accepted || !out_steps) return LS_ERR_INVALID_ARG;
+    if (exit_layer < 1 || exit_layer > m->c.n_layers - 1 || num_draft < 1 || max_new < 1) return LS_ERR_INVALID_ARG;
+    if (num_draft > m->c.max_draft) return LS_ERR_CAPACITY;
+    if (n_prompt < 1) return LS_ERR_INVALID_ARG;
+    if ((int64_t)n_prompt + max_new + num_draft + 1 > m->c.max_seq) return LS_ERR_CAPACITY;
+    LS_TRY(ls_prefill(m, prompt, n_prompt, 0));
+    LS_TRY(ls_decode(m, exit_layer, num_draft, max_new));
+    return ls_read_output(m, out_ids, out_n, accepted, out_steps);
+}
+
+int ls_generate_full(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t max_new, int32_t* out_ids,
+                     int32_t* out_n)
+{
+    if (!m || !out_ids || !out_n || max_new < 1 || n_prompt < 1) return LS_ERR_INVALID_ARG;
+    if ((int64_t)n_prompt + max_new + 1 > m->c.max_seq) return LS_ERR_CAPACITY;
+    LS_TRY(ls_prefill(m, prompt, n_prompt, 0));
+    LS_TRY(ls_decode(m, 0, 0, max_new));
+    return ls_read_output(m, out_ids, out_n, nullptr, nullptr);
+}
+
+int ls_generate_early(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t exit_layer, int32_t max_new,
+                      int32_t* out_ids, int32_t* out_n)
+{
+    if (!m || !out_ids || !out_n || max_new < 1 || n_prompt < 1) return LS_ERR_INVALID_ARG;
+    if (exit_layer < 1 || exit_layer > m->c.n_layers) return LS_ERR_INVALID_ARG;
+    if ((int64_t)n_prompt + max_new + 1 > m->c.max_seq) return LS_ERR_CAPACITY;
+    LS_TRY(ls_prefill(m, prompt, n_prompt, exit_layer));
+    LS_TRY(ls_decode(m, exit_layer, 0, max_new));
+    return ls_read_output(m, out_ids, out_n, nullptr, nullptr);
+}
+
+int ls_debug_logits(ls_model* m, const int32_t* ids, int32_t n, int32_t exit_layer, float* exit_logits,
+                    float* final_logits)
+{
+    if (!m) return LS_ERR_INVALID_ARG;
+    LS_TRY(check_ids(m, ids, n));
+    const int L = m->c.n_layers, V = m->c.vocab;
+    if (exit_layer < 1 || exit_layer > L) return LS_ERR_INVALID_ARG;
+    if (n > m->c.max_seq) return LS_ERR_CAPACITY;
+    m->n_prompt = 0;
+    set_grid_chunks(m, n);
+    LS_CK(cudaMemcpyAsync(m->ids, ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, m->st));
+    LS_TRY(write_ctl(m, 0, 0, 0));
+    for (int r0 = 0; r0 < n; r0 += kMaxRows) {
+        int M = n - r0 < kMaxRows ? n - r0 : kMaxRows;
+        LS_TRY(run_embed(m, m->ids + r0, M, m->x));
+        LS_TRY(run_layers(m, 0, exit_layer, M, m->x, r0));
+        if (exit_logits) {
+            LS_TRY(run_head(m, M, m->x, m->verified, m->logits));
+            LS_CK(cudaMemcpyAsync(exit_logits + (size_t)r0 * V, m->logits, sizeof(float) * (size_t)M * V,
+                                  cudaMemcpyDeviceToHost, m->st));
+            LS_CK(cudaStreamSynchronize(m->st));
+        }
+        LS_TRY(run_layers(m, exit_layer, L, M, m->x, r0));
+        if (final_logits) {
+            LS_TRY(run_head(m, M, m->x, m->verified, m->logits));
+            LS_CK(cudaMemcpyAsync(final_logits + (size_t)r0 * V, m->logits, sizeof(float) * (size_t)M * V,
+                                  cudaMemcpyDeviceToHost, m->st));
+            LS_CK(cudaStreamSynchronize(m->st));
+        }
+    }
+    int32_t w[CTL_WORDS];
+    LS_TRY(read_ctl(m, w));
+    return w[CTL_STATUS] ? LS_ERR_DEVICE_STATUS : LS_OK;
+}
+
+int ls_get_stats(const ls_model* m, ls_stats* out)
+{
+    if (!m || !out) return LS_ERR_INVALID_ARG;
+    *out = m->stats;
+    return LS_OK;
+}
+
+// ------------------------------------------------------------------ single operations
+int ls_op_embed(const void* emb, const int32_t* tok, int32_t M, int32_t D, int32_t V, float* x, void* stream)
+{
+    if (!aligned16(emb) || !tok || !aligned16(x) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8 || V < 1)
+        return LS_ERR_INVALID_ARG;
+    embed_kernel<<<M, 256, 0, (cudaStream_t)stream>>>((const uint16_t*)emb, tok, D, V, x, nullptr);
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+int ls_op_rmsnorm(const float* x, const void* gain, int32_t M, int32_t D, float eps, void* out, void* stream)
+{
+    if (!aligned16(x) || !aligned16(gain) || !aligned16(out) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8)
+        return LS_ERR_INVALID_ARG;
+    rmsnorm_kernel<<<M, 256, 0, (cudaStream_t)stream>>>(x, (const uint16_t*)gain, D, eps, (uint16_t*)out, nullptr);
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+static int lin_check(int path, const void* w, const void* h, int M, int N, int K)
+{
+    if (path != LS_LINEAR_FMA && path != LS_LINEAR_MMA) return LS_ERR_INVALID_ARG;
+    if (!aligned16(w) || !aligned16(h) || M < 1 || M > LS_MAX_ROWS || N < 1 || K < 8 || K % 8) return LS_ERR_INVALID_ARG;
+    return LS_OK;
+}
+
+int ls_op_linear(int32_t path, const void* w, const void* h, int32_t M, int32_t N, int32_t K, float* out,
+                 int32_t residual, void* stream)
+{
+    LS_TRY(lin_check(path, w, h, M, N, K));
+    if (!out) return LS_ERR_INVALID_ARG;
+    LinArgs a = lin_args((const uint16_t*)w, (const uint16_t*)h, M, N, K);
+    a.out = out;
+    a.ldo = N;
+    LS_CK(launch_linear(path, residual ? EPI_RESIDUAL : EPI_STORE, a, (cudaStream_t)stream));
+    return LS_OK;
+}
+
+int ls_op_gate_up_swiglu(int32_t path, const void* wg, const void* wu, const void* h, int32_t M, int32_t F,
+                         int32_t K, void* out, void* stream)
+{
+    LS_TRY(lin_check(path, wg, h, M, F, K));
+    if (!aligned16(wu) || !out) return LS_ERR_INVALID_ARG;
+    LinArgs a = lin_args((const uint16_t*)wg, (const uint16_t*)h, M, F, K);
+    a.w1 = (const uint16_t*)wu;
+    a.out_bf16 = (uint16_t*)out;
+    LS_CK(launch_linear(path, EPI_SWIGLU, a, (cudaStream_t)stream));
+    return LS_OK;
+}
+
+size_t ls_op_lm_head_scratch_bytes(int32_t V)
+{
+    if (V < 1) return 0;
+    return sizeof(ValIdx) * (size_t)LS_MAX_ROWS * (size_t)((V + 15) / 16);
+}
+
+int ls_op_lm_head_argmax(int32_t path, const void* w, const void* h, int32_t M, int32_t V, int32_t K,
+                         void* scratch, int32_t* tok, float* logits, void* stream)
+{
+    LS_TRY(lin_check(path, w, h, M, V, K));
+    if (!scratch || ((uintptr_t)scratch & 7u) || !tok) return LS_ERR_INVALID_ARG;
+    LinArgs a = lin_args((const uint16_t*)w, (const uint16_t*)h, M, V, K);
+    a.cand = (ValIdx*)scratch;
+    a.cand_stride = (V + 15) / 16;
+    a.out = logits;
+    a.ldo = V;
+    LS_CK(launch_linear(path, EPI_ARGMAX, a, (cudaStream_t)stream));
+    argmax_finish_kernel<<<M, 256, 0, (cudaStream_t)stream>>>(a.cand, lin_grid(EPI_ARGMAX, V), a.cand_stride, tok,
+                                                              nullptr);
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+static int kv_check(int M, int pos0, int Hq, int Hkv, int hd, int page_size, int max_seq)
+{
+    if (M < 1 || M > LS_MAX_ROWS || pos0 < 0 || Hq < 1 || Hkv < 1 || Hq % Hkv || Hq / Hkv > 8) return LS_ERR_INVALID_ARG;
+    if ((hd != 64 && hd != 128) || page_size < 16 || page_size > 1024 || log2_exact(page_size) < 0) return LS_ERR_INVALID_ARG;
+    if (max_seq < 1 || (int64_t)pos0 + M > max_seq) return LS_ERR_CAPACITY;
+    return LS_OK;
+}
+
+int ls_op_rope_append(const float* qkv, int32_t M, int32_t pos0, int32_t Hq, int32_t Hkv, int32_t hd, float theta,
+                      int32_t page_size, const int32_t* page_table, int32_t max_seq, void* q_out, void* kp, void* vp,
+                      void* stream)
+{
+    LS_TRY(kv_check(M, pos0, Hq, Hkv, hd, page_size, max_seq));
+    if (!qkv || !page_table || !q_out || !aligned16(kp) || !aligned16(vp) || !(theta > 0.f)) return LS_ERR_INVALID_ARG;
+    rope_append_kernel<<<dim3(M, Hq + 2 * Hkv), hd / 2, 0, (cudaStream_t)stream>>>(
+        qkv, Hq, Hkv, hd, nullptr, theta, log2_exact(page_size), page_table, max_seq, (uint16_t*)q_out,
+        (uint16_t*)kp, (uint16_t*)vp, nullptr, pos0);
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+size_t ls_op_attention_scratch_bytes(int32_t Hq, int32_t hd, int32_t max_seq)
+{
+    if (Hq < 1 || hd < 1 || max_seq < 1) return 0;
+    size_t cap = (size_t)(max_seq + kAttnChunk - 1) / kAttnChunk;
+    return sizeof(float) * LS_MAX_ROWS * (size_t)Hq * cap * (size_t)(hd + 2);
+}
+
+int ls_op_attention(const void* q, int32_t M, int32_t pos0, int32_t Hq, int32_t Hkv, int32_t hd, int32_t page_size,
+                    const int32_t* page_table, int32_t max_seq, const void* kp, const void* vp, void* scratch,
+                    void* out, void* stream)
+{
+    LS_TRY(kv_check(M, pos0, Hq, Hkv, hd, page_size, max_seq));
+    if (!aligned16(q) || !page_table || !aligned16(kp) || !aligned16(vp) || !aligned16(scratch) || !out)
+        return LS_ERR_INVALID_ARG;
+    LS_TRY(attn_allow_smem(hd, Hq / Hkv));
+    const int cap = (max_seq + kAttnChunk - 1) / kAttnChunk;
+    const int chunks = (pos0 + M + kAttnChunk - 1) / kAttnChunk;
+    return attn_launch((const uint16_t*)q, (const uint16_t*)kp, (const uint16_t*)vp, page_table, nullptr, pos0, M, Hq,
+                       Hkv, hd, log2_exact(page_size), max_seq, cap, chunks, (float*)scratch, (uint16_t*)out,
+                       (cudaStream_t)stream);
+}
+
+int ls_op_accept(const int32_t* draft, const int32_t* verified, int32_t d, int32_t* state, int32_t* out_ids,
+                 int32_t* accepted, void* stream)
+{
+    if (!draft || !verified || !state || !out_ids || !accepted || d < 0 || d >= LS_MAX_ROWS) return LS_ERR_INVALID_ARG;
+    accept_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(draft, verified, d, state, out_ids, accepted);
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+}  // extern "C"

@@ -72,6 +72,9 @@ LLAMA3_8B = Shape("llama3-8b-shaped", 32, 4096, 32, 8, 128, 14336, 128256, rope_
 # small shapes for unit tests: grouped KV heads, ragged K (d_ffn not a multiple of 32)
 MICRO_GQA = Shape("micro-gqa", 3, 64, 4, 2, 16, 88, 160)
 MICRO_MHA = Shape("micro-mha", 3, 64, 4, 4, 16, 88, 160)
+# small shape the CUDA kernels accept (head_dim 64), with grouped KV heads, a ragged K
+# (d_ffn = 2*32 + 24) and a vocabulary that is not a multiple of the 16-row tile
+GPU_MICRO = Shape("gpu-micro", 3, 96, 4, 2, 64, 88, 200)
 
 WORKLOADS = {
     "tiny": Workload(TINY, 32, 64, 2, 3, 0.1),
@@ -128,6 +131,20 @@ def make_weights(shape: Shape, seed: int, scale_from: int, late_scale: float,
                     sc *= late_scale
                 w[name].append(_normal(dims[name], sd, device, sc))
     return w
+
+
+def amplify(weights: dict, factor: float) -> dict:
+    """Scale every matrix (not the norm gains) by ``factor``: N(0, 0.02) draws on a narrow
+    model give nearly flat logits, a louder draw makes comparisons sensitive to every term."""
+    out = {}
+    for k, v in weights.items():
+        if k in ("attn_norm", "ffn_norm", "final_norm"):
+            out[k] = v
+        elif isinstance(v, list):
+            out[k] = [(t.float() * factor).to(torch.bfloat16) for t in v]
+        else:
+            out[k] = (v.float() * factor).to(torch.bfloat16)
+    return out
 
 
 def make_prompt(vocab: int, n: int, seed: int) -> np.ndarray:

@@ -1,0 +1,226 @@
+"""Parity of the whole decode path (through the C ABI) against the CPU oracle, and the
+properties that hold at any size.
+
+* teacher-forced exit-layer and final logits: max|delta| <= 3e-2 * max|logit|
+  (bf16 weights / activations / KV, fp32 accumulation, against the fp64 oracle);
+* free-running ids equal the oracle's up to the first position whose oracle top-1/top-2
+  margin is inside that tolerance;
+* ls_generate == ls_generate_full bit-exactly for every (E, d) -- the losslessness of
+  self-speculative decoding (Sec. 4.3 of the paper), which on the GPU also needs every
+  kernel to be independent of the pass size;
+* accepted-per-step bookkeeping invariants, the zero-scale case, EOS, a shuffled page
+  table, determinism, and the error codes of the boundary.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2404_16710_b200 import binding as B
+from paper_2404_16710_b200 import synth
+from tests.helpers import LOGIT_TOL, assert_logits_close, first_low_margin, make_pair
+
+pytestmark = pytest.mark.gpu
+PATHS = [B.LS_LINEAR_FMA, B.LS_LINEAR_MMA]
+TINY = synth.WORKLOADS["tiny"]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("E", [1, 2, 4])
+def test_teacher_forced_logits_tiny(path, E):
+    gm, om = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 128, linear_path=path)
+    ids = synth.make_prompt(TINY.shape.vocab, 41, 99)  # 16 + 16 + 9 rows: full tiles and a ragged tail
+    gex, gfi = gm.debug_logits(ids, E)
+    oex, ofi = om.teacher_logits(ids, E)
+    r1 = assert_logits_close(gex, oex, "exit logits")
+    r2 = assert_logits_close(gfi, ofi, "final logits")
+    print(f"path {path} E {E}: max|delta|/max|logit| exit {r1:.2e} final {r2:.2e}")
+    if E == 4:
+        assert np.array_equal(gex, gfi)
+    # argmax agrees wherever the oracle's margin is beyond the tolerance
+    for g, o in ((gex, oex), (gfi, ofi)):
+        part = np.partition(o, -2, axis=1)
+        safe = (part[:, -1] - part[:, -2]) > LOGIT_TOL * np.abs(o).max()
+        assert (g.argmax(1)[safe] == o.argmax(1)[safe]).all()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_teacher_forced_logits_grouped_kv_ragged_shapes(path):
+    shape = synth.GPU_MICRO
+    gm, om = make_pair(shape, 5, 0, 1.0, 96, page_size=16, linear_path=path, amplify=6.0)
+    ids = synth.make_prompt(shape.vocab, 37, 3)
+    gex, gfi = gm.debug_logits(ids, 1)
+    oex, ofi = om.teacher_logits(ids, 1)
+    assert np.abs(ofi).max() > 0.5
+    assert_logits_close(gex, oex, "exit logits")
+    assert_logits_close(gfi, ofi, "final logits")
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_free_running_ids_follow_the_oracle_while_margins_allow(path):
+    gm, om = make_pair(TINY.shape, TINY.weight_seed, TINY.exit_layer, TINY.late_scale, 128, linear_path=path)
+    prompt = synth.make_prompt(TINY.shape.vocab, TINY.n_prompt, TINY.prompt_seed)
+    ref, margins, maxabs = om.generate_full(prompt, TINY.max_new)
+    ids = gm.generate_full(prompt, TINY.max_new)
+    assert len(ids) == TINY.max_new
+    k = first_low_margin(margins, maxabs)
+    assert k >= 1
+    np.testing.assert_array_equal(ids[:k], ref[:k])
+    assert len(gm.generate_early(prompt, 2, 8)) == 8
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_generate_equals_generate_full_for_every_exit_and_draft(path):
+    gm, _ = make_pair(TINY.shape, TINY.weight_seed, TINY.exit_layer, TINY.late_scale, 160, max_draft=15,
+                      linear_path=path, oracle=False)
+    prompt = synth.make_prompt(TINY.shape.vocab, TINY.n_prompt, TINY.prompt_seed)
+    full = gm.generate_full(prompt, TINY.max_new)
+    again = gm.generate_full(prompt, TINY.max_new)
+    np.testing.assert_array_equal(full, again)  # deterministic
+    for E in (1, 2, 3):
+        for d in (1, 2, 3, 5, 8, 15):
+            ids, acc = gm.generate(prompt, E, d, TINY.max_new)
+            np.testing.assert_array_equal(ids, full, err_msg=f"E={E} d={d}")
+            assert ((0 <= acc) & (acc <= d)).all()
+            emitted = np.cumsum(acc + 1)
+            assert emitted[-1] >= TINY.max_new and (len(emitted) == 1 or emitted[-2] < TINY.max_new)
+            st = gm.stats()
+            assert st.n_generated == TINY.max_new and st.n_steps == len(acc) and st.n_accepted == acc.sum()
+            assert st.host_syncs <= 8 < TINY.max_new  # no host sync per token
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_accepted_per_step_matches_oracle_on_the_safe_prefix(path):
+    gm, om = make_pair(TINY.shape, TINY.weight_seed, TINY.exit_layer, TINY.late_scale, 128, linear_path=path)
+    prompt = synth.make_prompt(TINY.shape.vocab, TINY.n_prompt, TINY.prompt_seed)
+    ref_ids, ref_acc, _ = om.generate_spec(prompt, TINY.exit_layer, TINY.num_draft, TINY.max_new)
+    ids, acc = gm.generate(prompt, TINY.exit_layer, TINY.num_draft, TINY.max_new)
+    _, margins, maxabs = om.generate_full(prompt, TINY.max_new)
+    k = first_low_margin(margins, maxabs)
+    np.testing.assert_array_equal(ids[:k], ref_ids[:k])
+    print(f"path {path}: mean accepted/step gpu {acc.mean():.3f} oracle {ref_acc.mean():.3f}, safe prefix {k}")
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_zero_late_scale_accepts_every_draft(path):
+    E, d = 2, 3
+    gm, om = make_pair(TINY.shape, TINY.weight_seed, E, 0.0, 128, linear_path=path)
+    prompt = synth.make_prompt(TINY.shape.vocab, 10, TINY.prompt_seed)
+    ids, acc = gm.generate(prompt, E, d, 22)
+    assert (acc == d).all() and len(acc) == -(-22 // (d + 1))
+    np.testing.assert_array_equal(ids, gm.generate_full(prompt, 22))
+    np.testing.assert_array_equal(ids, gm.generate_early(prompt, E, 22))
+    _, oacc, _ = om.generate_spec(prompt, E, d, 22)
+    np.testing.assert_array_equal(acc, oacc)
+
+
+def test_shuffled_page_table_changes_nothing():
+    gm, _ = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 128, page_size=16, oracle=False)
+    prompt = synth.make_prompt(TINY.shape.vocab, 40, 8)
+    a_ids, a_acc = gm.generate(prompt, 2, 3, 48)
+    table = np.random.default_rng(0).permutation(128 // 16).astype(np.int32)
+    B.ls_set_page_table(gm.h, table)
+    b_ids, b_acc = gm.generate(prompt, 2, 3, 48)
+    np.testing.assert_array_equal(a_ids, b_ids)
+    np.testing.assert_array_equal(a_acc, b_acc)
+    with pytest.raises(B.LsError):
+        B.ls_set_page_table(gm.h, np.zeros(8, np.int32))  # not a permutation
+
+
+def test_eos_stops_both_loops_at_the_same_token():
+    prompt = synth.make_prompt(TINY.shape.vocab, TINY.n_prompt, TINY.prompt_seed)
+    gm, _ = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 128, oracle=False)
+    full = gm.generate_full(prompt, 40)
+    eos = int(full[17])
+    first = int(np.argmax(full == eos))
+    gm2, _ = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 128, eos_id=eos, oracle=False)
+    f2 = gm2.generate_full(prompt, 40)
+    s2, _ = gm2.generate(prompt, 2, 3, 40)
+    np.testing.assert_array_equal(f2, full[:first + 1])
+    np.testing.assert_array_equal(s2, f2)
+
+
+def test_prefill_once_decode_many():
+    gm, _ = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 128, oracle=False)
+    prompt = synth.make_prompt(TINY.shape.vocab, 20, 1)
+    B.ls_prefill(gm.h, prompt)
+    B.ls_decode(gm.h, 0, 0, 30)
+    full, _ = B.ls_read_output(gm.h, 30)
+    for _ in range(2):
+        B.ls_decode(gm.h, 2, 4, 30)
+        ids, acc = B.ls_read_output(gm.h, 30)
+        np.testing.assert_array_equal(ids, full)
+    st = gm.stats()
+    assert st.decode_ms > 0 and st.weight_bytes > 0 and st.kv_bytes > 0 and st.kernel_launches > 0
+    # algorithmic bytes of the schedule: (d+1) E W_layer + d W_lm + (L-E) W_layer + W_lm per step
+    s = TINY.shape
+    per_step = (5 * 2 + 2) * s.layer_weight_bytes + 5 * s.lm_head_bytes
+    assert st.weight_bytes == per_step * st.n_steps
+
+
+def test_boundary_error_codes():
+    gm, _ = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 64, max_draft=4, oracle=False)
+    p = synth.make_prompt(TINY.shape.vocab, 8, 0)
+
+    def status(fn, *a):
+        with pytest.raises(B.LsError) as e:
+            fn(*a)
+        return e.value.status
+
+    assert status(gm.generate, p, 4, 2, 8) == B.LS_ERR_INVALID_ARG       # E must leave a layer to verify with
+    assert status(gm.generate, p, 0, 2, 8) == B.LS_ERR_INVALID_ARG
+    assert status(gm.generate, p, 2, 5, 8) == B.LS_ERR_CAPACITY          # beyond max_draft
+    assert status(gm.generate, p, 2, 2, 60) == B.LS_ERR_CAPACITY         # KV capacity
+    assert status(gm.generate_full, p, 60) == B.LS_ERR_CAPACITY
+    bad = p.copy()
+    bad[3] = TINY.shape.vocab
+    assert status(gm.generate_full, bad, 4) == B.LS_ERR_INVALID_ARG
+    assert status(gm.generate_full, p[:0], 4) == B.LS_ERR_INVALID_ARG
+    # the handle is still usable after every refusal
+    assert len(gm.generate_full(p, 4)) == 4
+    cfg = B.make_config(TINY.shape, 64)
+    ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.LsError) as e:
+        B.ls_model_create(cfg, gm.weights, ws)
+    assert e.value.status == B.LS_ERR_CAPACITY
+
+
+# ------------------------------------------------------------------ Llama-2-7B shape
+@pytest.fixture(scope="module")
+def llama7b():
+    wl = synth.WORKLOADS["llama2-7b"]
+    max_seq = wl.n_prompt + wl.max_new + wl.num_draft + 1
+    w = synth.make_weights(wl.shape, wl.weight_seed, wl.exit_layer, wl.late_scale, device="cuda")
+    gm = B.Model(wl.shape, w, max_seq, 64, 8)
+    yield wl, gm, w
+    gm.close()
+
+
+def test_llama7b_generate_equals_generate_full_at_full_size(llama7b):
+    """The benchmark's configuration: prompt 1024, 256 new tokens, E=8, d=6."""
+    wl, gm, _ = llama7b
+    prompt = synth.make_prompt(wl.shape.vocab, wl.n_prompt, wl.prompt_seed)
+    full = gm.generate_full(prompt, wl.max_new)
+    t_full = gm.stats().decode_ms
+    ids, acc = gm.generate(prompt, wl.exit_layer, wl.num_draft, wl.max_new)
+    st = gm.stats()
+    np.testing.assert_array_equal(ids, full)
+    assert len(ids) == wl.max_new and np.cumsum(acc + 1)[-1] >= wl.max_new
+    assert ((0 <= acc) & (acc <= wl.num_draft)).all()
+    print(f"7B: full {wl.max_new / t_full * 1e3:.1f} tok/s, self-spec {wl.max_new / st.decode_ms * 1e3:.1f} tok/s, "
+          f"accepted/step {acc.mean():.2f}, syncs {st.host_syncs}")
+
+
+def test_llama7b_logits_against_oracle_on_a_short_prompt(llama7b):
+    """What the oracle can afford at this shape: a few teacher-forced positions."""
+    from oracle import ls_oracle as O
+    wl, gm, w = llama7b
+    s = wl.shape
+    cfg = O.Config(s.n_layers, s.d_model, s.n_heads, s.n_kv_heads, s.head_dim, s.d_ffn, s.vocab,
+                   s.rms_eps, s.rope_theta, 8)
+    om = O.Model(cfg, synth.as_uint16(w))
+    ids = synth.make_prompt(s.vocab, 3, 17)
+    oex, ofi = om.teacher_logits(ids, wl.exit_layer)
+    gex, gfi = gm.debug_logits(ids, wl.exit_layer)
+    r1 = assert_logits_close(gex, oex, "exit logits")
+    r2 = assert_logits_close(gfi, ofi, "final logits")
+    print(f"7B: max|delta|/max|logit| exit {r1:.2e} final {r2:.2e}; max|logit| {np.abs(ofi).max():.3f}")

@@ -1,0 +1,317 @@
+"""Parity of every kernel family against the oracle's elementary operation, through the C ABI.
+
+Sizes span several tiles and a ragged tail (rows not a multiple of 16, K not a multiple
+of 32, M from 1 to 16), plus the full Llama-2-7B projection shapes checked on sampled
+output rows.  Integer results (token ids, accept bookkeeping) must be bit-exact; floating
+point results carry the tolerance their arithmetic implies: fp32 accumulation of exact
+bf16 products against the oracle's fp64 (1e-5 relative to the row's magnitude), one bf16
+rounding (2^-8 relative) where the kernel's output is bf16.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ls_oracle as O
+from paper_2404_16710_b200 import binding as B
+from tests.helpers import bf16_cuda, bits, vals
+
+pytestmark = pytest.mark.gpu
+PATHS = [B.LS_LINEAR_FMA, B.LS_LINEAR_MMA]
+BF16_REL = 2.0 ** -8
+
+
+def rnd(shape, seed, scale=1.0):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    return (torch.randn(shape, generator=g, device="cuda") * scale)
+
+
+def assert_bf16_close(got, ref, what=""):
+    tol = BF16_REL * np.abs(ref) + 1e-6 * np.abs(ref).max()
+    bad = np.abs(got - ref) > tol
+    assert not bad.any(), f"{what}: {bad.sum()} elements off, worst {np.abs(got - ref).max():.4g}"
+
+
+# ------------------------------------------------------------------ embedding, RMSNorm
+def test_embed_is_a_row_lookup():
+    emb = rnd((50, 64), 1).bfloat16()
+    tok = torch.tensor([3, 49, 0, 3, 17], dtype=torch.int32, device="cuda")
+    x = torch.empty((5, 64), dtype=torch.float32, device="cuda")
+    B.ls_op_embed(emb, tok, x)
+    torch.cuda.synchronize()
+    assert torch.equal(x, emb[tok.long()].float())
+
+
+@pytest.mark.parametrize("M,D", [(1, 64), (3, 256), (16, 4096), (7, 5120), (2, 1000)])
+def test_rmsnorm(M, D):
+    x = rnd((M, D), 2, 3.0)
+    g = (1 + 0.1 * rnd((D,), 3)).bfloat16()
+    out = torch.empty((M, D), dtype=torch.bfloat16, device="cuda")
+    B.ls_op_rmsnorm(x, g, 1e-5, out)
+    torch.cuda.synchronize()
+    xs, gb = x.cpu().numpy().astype(np.float64), bits(g)
+    for m in range(M):
+        assert_bf16_close(vals(out[m]), O.rmsnorm(xs[m], gb, 1e-5), f"row {m}")
+
+
+# ------------------------------------------------------------------ linear families
+def linear_case(path, M, N, K, residual, seed):
+    w = rnd((N, K), seed, 0.05).bfloat16()
+    h = rnd((M, K), seed + 1).bfloat16()
+    out = rnd((M, N), seed + 2) if residual else torch.empty((M, N), dtype=torch.float32, device="cuda")
+    base = out.clone()
+    B.ls_op_linear(path, w, h, out, residual)
+    torch.cuda.synchronize()
+    return w, h, base, out
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M,N,K", [(1, 16, 32), (1, 200, 88), (3, 100, 256), (4, 256, 688), (7, 333, 1000),
+                                   (8, 64, 4096), (9, 48, 72), (16, 130, 520)])
+@pytest.mark.parametrize("residual", [False, True])
+def test_linear_small_shapes(path, M, N, K, residual):
+    w, h, base, out = linear_case(path, M, N, K, residual, 10 + M)
+    wb, hv = bits(w), vals(h)
+    got = out.cpu().numpy().astype(np.float64)
+    for m in range(M):
+        ref = O.linear(wb, hv[m]) + (base[m].cpu().numpy() if residual else 0.0)
+        np.testing.assert_allclose(got[m], ref, rtol=0, atol=1e-5 * np.abs(ref).max() + 1e-6)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("N,K", [(12288, 4096), (4096, 11008), (4096, 4096)])
+def test_linear_llama7b_shapes_sampled_rows(path, N, K):
+    M = 7
+    w, h, _, out = linear_case(path, M, N, K, False, 77)
+    rows = np.unique(np.concatenate([[0, 15, 16, N - 17, N - 1],
+                                     np.random.default_rng(0).integers(0, N, 40)]))
+    wb, hv = bits(w[torch.from_numpy(rows).cuda()]), vals(h)
+    got = out.cpu().numpy().astype(np.float64)[:, rows]
+    for m in range(M):
+        ref = O.linear(wb, hv[m])
+        np.testing.assert_allclose(got[m], ref, rtol=0, atol=1e-5 * np.abs(ref).max())
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_linear_rows_do_not_depend_on_pass_size(path):
+    """Row 0 of an M-row pass is bit-identical for every M (the verification pass must
+    reproduce single-token decoding exactly)."""
+    N, K = 304, 1384
+    w = rnd((N, K), 5, 0.05).bfloat16()
+    h = rnd((16, K), 6).bfloat16()
+    outs = {}
+    for M in (1, 2, 4, 5, 8, 9, 16):
+        out = torch.empty((M, N), dtype=torch.float32, device="cuda")
+        B.ls_op_linear(path, w, h[:M].contiguous(), out)
+        outs[M] = out
+    torch.cuda.synchronize()
+    for M, out in outs.items():
+        assert torch.equal(out[0], outs[1][0]), f"M={M}"
+        assert torch.equal(out[M - 1], outs[16][M - 1]), f"M={M}"
+    # and a row's value does not depend on which slot of the pass it occupies
+    hh = h[:9].flip(0).contiguous()
+    out = torch.empty((9, N), dtype=torch.float32, device="cuda")
+    B.ls_op_linear(path, w, hh, out)
+    torch.cuda.synchronize()
+    assert torch.equal(out.flip(0), outs[9])
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M,F,K", [(1, 8, 32), (3, 88, 96), (7, 688, 256), (16, 100, 520), (5, 11008, 4096)])
+def test_gate_up_swiglu(path, M, F, K):
+    wg, wu = rnd((F, K), 20, 0.05).bfloat16(), rnd((F, K), 21, 0.05).bfloat16()
+    h = rnd((M, K), 22).bfloat16()
+    out = torch.empty((M, F), dtype=torch.bfloat16, device="cuda")
+    B.ls_op_gate_up_swiglu(path, wg, wu, h, out)
+    torch.cuda.synchronize()
+    cols = np.arange(F) if F <= 1000 else np.unique(np.concatenate(
+        [[0, 7, 8, F - 9, F - 1], np.random.default_rng(1).integers(0, F, 48)]))
+    idx = torch.from_numpy(cols).cuda()
+    gb, ub, hv = bits(wg[idx]), bits(wu[idx]), vals(h)
+    for m in range(M):
+        g, u = O.linear(gb, hv[m]), O.linear(ub, hv[m])
+        ref = np.array([O.silu(a) for a in g]) * u
+        assert_bf16_close(vals(out[m])[cols], ref, f"row {m}")
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M,V,K", [(1, 200, 96), (4, 1024, 256), (7, 32000, 4096), (16, 1000, 520)])
+def test_lm_head_argmax(path, M, V, K):
+    w = rnd((V, K), 30, 0.05).bfloat16()
+    h = rnd((M, K), 31).bfloat16()
+    scratch = torch.empty(B.ls_op_lm_head_scratch_bytes(V), dtype=torch.uint8, device="cuda")
+    tok = torch.full((M,), -1, dtype=torch.int32, device="cuda")
+    logits = torch.empty((M, V), dtype=torch.float32, device="cuda")
+    B.ls_op_lm_head_argmax(path, w, h, scratch, tok, logits)
+    tok2 = torch.full((M,), -1, dtype=torch.int32, device="cuda")
+    B.ls_op_lm_head_argmax(path, w, h, scratch, tok2, None)
+    torch.cuda.synchronize()
+    assert torch.equal(tok, tok2)
+    wb, hv = bits(w), vals(h)
+    lg = logits.cpu().numpy().astype(np.float64)
+    for m in range(M):
+        ref = O.linear(wb, hv[m])
+        np.testing.assert_allclose(lg[m], ref, rtol=0, atol=1e-5 * np.abs(ref).max())
+        # the id is the argmax of the kernel's own fp32 logits (ties -> lowest index) ...
+        assert int(tok[m]) == int(np.argmax(logits[m].cpu().numpy()))
+        # ... and the oracle's id whenever the oracle's margin is beyond fp32 accumulation error
+        i, margin, ma = O.argmax(ref)
+        if margin > 2e-5 * ma:
+            assert int(tok[m]) == i
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_lm_head_argmax_tie_goes_to_lowest_index(path):
+    V, K = 96, 64
+    w = torch.zeros((V, K), dtype=torch.bfloat16, device="cuda")
+    w[[5, 37, 70], 0] = 2.0   # three equal maxima in different tiles
+    w[11, 0] = 1.0
+    h = torch.zeros((2, K), dtype=torch.bfloat16, device="cuda")
+    h[0, 0], h[1, 0] = 1.0, -1.0  # row 1: all of {5,37,70,11} negative, the zeros tie at 0 -> index 0
+    scratch = torch.empty(B.ls_op_lm_head_scratch_bytes(V), dtype=torch.uint8, device="cuda")
+    tok = torch.empty((2,), dtype=torch.int32, device="cuda")
+    B.ls_op_lm_head_argmax(path, w, h, scratch, tok, None)
+    torch.cuda.synchronize()
+    assert tok.tolist() == [5, 0]
+
+
+# ------------------------------------------------------------------ RoPE + append, attention
+def kv_setup(Hkv, hd, page_size, max_seq, shuffle):
+    n_pages = -(-max_seq // page_size)
+    table = np.arange(n_pages, dtype=np.int32)
+    if shuffle:
+        table = np.random.default_rng(3).permutation(n_pages).astype(np.int32)
+    kp = torch.zeros((n_pages, Hkv, page_size, hd), dtype=torch.bfloat16, device="cuda")
+    vp = torch.zeros_like(kp)
+    return table, torch.from_numpy(table).cuda(), kp, vp
+
+
+def gather_cache(pages, table, page_size, n):
+    """[n, Hkv*hd] float64 rows of logical positions 0..n-1"""
+    rows = []
+    for p in range(n):
+        phys = table[p // page_size]
+        rows.append(vals(pages[phys, :, p % page_size, :]).reshape(-1))
+    return np.stack(rows)
+
+
+@pytest.mark.parametrize("Hq,Hkv,hd,theta", [(4, 2, 64, 1e4), (8, 8, 128, 1e4), (8, 2, 128, 5e5)])
+@pytest.mark.parametrize("shuffle", [False, True])
+def test_rope_append(Hq, Hkv, hd, theta, shuffle):
+    M, pos0, page_size, max_seq = 5, 1021, 16, 1100
+    table, table_d, kp, vp = kv_setup(Hkv, hd, page_size, max_seq, shuffle)
+    qkv = rnd((M, (Hq + 2 * Hkv) * hd), 40)
+    q_out = torch.empty((M, Hq * hd), dtype=torch.bfloat16, device="cuda")
+    B.ls_op_rope_append(qkv, pos0, Hq, Hkv, hd, theta, page_size, table_d, max_seq, q_out, kp, vp)
+    torch.cuda.synchronize()
+    src = qkv.cpu().numpy().astype(np.float64)
+    kc = gather_cache(kp, table, page_size, pos0 + M)
+    vc = gather_cache(vp, table, page_size, pos0 + M)
+    assert not kc[:pos0].any() and not vc[:pos0].any()  # nothing else was touched
+    for m in range(M):
+        p = pos0 + m
+        for hh in range(Hq):
+            ref = O.rope(src[m, hh * hd:(hh + 1) * hd], p, theta)
+            # fp32 angle p * inv_freq carries ~p * 2^-24 radians of error on top of the bf16 rounding
+            np.testing.assert_allclose(vals(q_out[m, hh * hd:(hh + 1) * hd]), ref, rtol=0,
+                                       atol=BF16_REL * np.abs(ref).max() + 4e-4 * np.abs(ref).max())
+        for hh in range(Hkv):
+            o = (Hq + hh) * hd
+            ref = O.rope(src[m, o:o + hd], p, theta)
+            np.testing.assert_allclose(kc[p, hh * hd:(hh + 1) * hd], ref, rtol=0,
+                                       atol=(BF16_REL + 4e-4) * np.abs(ref).max())
+            o = (Hq + Hkv + hh) * hd
+            ref = src[m, o:o + hd]
+            assert_bf16_close(vc[p, hh * hd:(hh + 1) * hd], ref)
+
+
+@pytest.mark.parametrize("Hq,Hkv,hd", [(4, 2, 64), (4, 4, 128), (8, 2, 128)])
+@pytest.mark.parametrize("M,pos0", [(1, 0), (1, 63), (1, 64), (4, 61), (7, 130), (16, 300), (3, 1000)])
+def test_attention(Hq, Hkv, hd, M, pos0):
+    page_size, max_seq = 32, 1100
+    table, table_d, kp, vp = kv_setup(Hkv, hd, page_size, max_seq, True)
+    n = pos0 + M
+    # fill logical positions 0..n-1 (and garbage beyond, which causal masking must hide)
+    kl = rnd((n + 8, Hkv, hd), 50).bfloat16()
+    vl = rnd((n + 8, Hkv, hd), 51).bfloat16()
+    for p in range(min(n + 8, max_seq)):
+        kp[table[p // page_size], :, p % page_size, :] = kl[p]
+        vp[table[p // page_size], :, p % page_size, :] = vl[p]
+    q = rnd((M, Hq * hd), 52, 0.5).bfloat16()
+    scratch = torch.empty(B.ls_op_attention_scratch_bytes(Hq, hd, max_seq), dtype=torch.uint8, device="cuda")
+    out = torch.empty((M, Hq * hd), dtype=torch.bfloat16, device="cuda")
+    B.ls_op_attention(q, pos0, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp, scratch, out)
+    torch.cuda.synchronize()
+    kf, vf, qf = vals(kl).reshape(n + 8, -1), vals(vl).reshape(n + 8, -1), vals(q)
+    for m in range(M):
+        ref = O.attention(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd)
+        np.testing.assert_allclose(vals(out[m]), ref, rtol=0, atol=BF16_REL * np.abs(ref).max() + 1e-5)
+
+
+def test_attention_rows_do_not_depend_on_pass_size():
+    Hq, Hkv, hd, page_size, max_seq, pos0 = 8, 2, 128, 64, 512, 200
+    table, table_d, kp, vp = kv_setup(Hkv, hd, page_size, max_seq, False)
+    kp.copy_(rnd(kp.shape, 60).bfloat16())
+    vp.copy_(rnd(vp.shape, 61).bfloat16())
+    q = rnd((16, Hq * hd), 62, 0.5).bfloat16()
+    scratch = torch.empty(B.ls_op_attention_scratch_bytes(Hq, hd, max_seq), dtype=torch.uint8, device="cuda")
+    full = torch.empty((16, Hq * hd), dtype=torch.bfloat16, device="cuda")
+    B.ls_op_attention(q, pos0, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp, scratch, full)
+    for m in (0, 3, 15):
+        one = torch.empty((1, Hq * hd), dtype=torch.bfloat16, device="cuda")
+        B.ls_op_attention(q[m:m + 1].contiguous(), pos0 + m, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp,
+                          scratch, one)
+        torch.cuda.synchronize()
+        assert torch.equal(one[0], full[m]), f"row {m}"
+
+
+# ------------------------------------------------------------------ accept / rollback
+@pytest.mark.parametrize("draft,verified,max_new,eos,n_out0", [
+    ([5, 6, 7], [9, 6, 7, 1], 10, -1, 0),
+    ([5, 6, 7], [5, 6, 2, 1], 10, -1, 4),
+    ([5, 6, 7], [5, 6, 7, 1], 10, -1, 0),
+    ([5, 6, 7], [5, 6, 7, 1], 6, -1, 4),     # truncated at max_new: emits 2 of 4
+    ([5, 6, 7], [5, 6, 7, 1], 10, 6, 0),     # EOS inside the accepted prefix
+    ([], [3], 10, -1, 2),                    # d = 0: plain greedy bookkeeping
+])
+def test_accept_matches_oracle_match_and_bookkeeping(draft, verified, max_new, eos, n_out0):
+    d = len(draft)
+    dr = torch.tensor(draft + [0] * (16 - d), dtype=torch.int32, device="cuda")
+    ve = torch.tensor(verified + [0] * (16 - len(verified)), dtype=torch.int32, device="cuda")
+    state = torch.tensor([100, 42, n_out0, 3, 0, max_new, eos, 0], dtype=torch.int32, device="cuda")
+    out = torch.full((32,), -1, dtype=torch.int32, device="cuda")
+    acc = torch.full((32,), -1, dtype=torch.int32, device="cuda")
+    B.ls_op_accept(dr, ve, d, state, out, acc)
+    torch.cuda.synchronize()
+    n = O.match(draft, verified[:d]) if d else 0
+    emitted, stop = [], False
+    for t in draft[:n] + [verified[n]]:
+        if n_out0 + len(emitted) < max_new and not stop:
+            emitted.append(t)
+            stop = eos >= 0 and t == eos
+    st = state.tolist()
+    assert st[0] == 100 + n + 1 and st[1] == verified[n] and st[2] == n_out0 + len(emitted) and st[3] == 4
+    assert st[4] == int(stop or st[2] >= max_new)
+    assert out[n_out0:n_out0 + len(emitted)].tolist() == emitted and int(out[n_out0 + len(emitted)]) == -1
+    assert int(acc[3]) == n
+    # a finished loop is left alone
+    if st[4]:
+        B.ls_op_accept(dr, ve, d, state, out, acc)
+        torch.cuda.synchronize()
+        assert state.tolist() == st
+
+
+def test_argument_errors_are_reported_not_launched():
+    w = torch.zeros((16, 12), dtype=torch.bfloat16, device="cuda")  # K not a multiple of 8
+    h = torch.zeros((1, 12), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros((1, 16), dtype=torch.float32, device="cuda")
+    with pytest.raises(B.LsError) as e:
+        B.ls_op_linear(B.LS_LINEAR_MMA, w, h, out)
+    assert e.value.status == B.LS_ERR_INVALID_ARG
+    w = torch.zeros((16, 16), dtype=torch.bfloat16, device="cuda")
+    h = torch.zeros((17, 16), dtype=torch.bfloat16, device="cuda")  # too many rows
+    with pytest.raises(B.LsError):
+        B.ls_op_linear(B.LS_LINEAR_FMA, w, h, torch.zeros((17, 16), dtype=torch.float32, device="cuda"))
+    with pytest.raises(B.LsError):
+        B.ls_op_linear(3, w, h[:1].contiguous(), out)
