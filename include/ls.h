@@ -98,7 +98,9 @@ int ls_last_cuda_error(void);
 size_t ls_workspace_bytes(const ls_config *cfg);
 
 /* Create a model over borrowed weights and workspace (256-byte aligned, at least
- * ls_workspace_bytes(cfg)).  cuda_stream is a cudaStream_t (NULL = default stream).
+ * ls_workspace_bytes(cfg)).  cuda_stream is a cudaStream_t that can be captured into a
+ * CUDA graph, i.e. not the legacy default stream; with NULL the model creates a (blocking)
+ * stream of its own, which still runs after work already queued on the default stream.
  * The workspace is cleared; the page table starts as the identity. */
 int ls_model_create(const ls_config *cfg, const ls_weights *w, void *workspace_dev,
                     size_t workspace_bytes, void *cuda_stream, ls_model **out);

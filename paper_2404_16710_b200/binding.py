@@ -154,7 +154,7 @@ def ls_model_create(cfg: ls_config, weights: dict, workspace, stream=None):
         keep.append(arr)
         setattr(w, k, C.cast(arr, _VPP))
     h = C.c_void_p()
-    st = _stream() if stream is None else C.c_void_p(stream)
+    st = C.c_void_p(stream) if stream else None  # None: the model makes a stream of its own
     _ck(lib().ls_model_create(C.byref(cfg), C.byref(w), _dev(workspace), workspace.numel() * workspace.element_size(),
                               st, C.byref(h)), "ls_model_create")
     return h

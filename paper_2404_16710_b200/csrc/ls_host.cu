@@ -91,7 +91,7 @@ struct ls_model {
     int page_shift, n_pages, chunk_cap, cand_stride;
     // loop state
     int n_prompt, last_tok, prefilled_layers, grid_chunks;
-    bool use_graphs, capturing;
+    bool use_graphs, own_stream;
     int64_t launches;  // kernels enqueued (counted while building a step)
     struct G {
         cudaGraphExec_t exec;
@@ -440,6 +440,18 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
         if (!strcmp(e, "mma")) m->path = LS_LINEAR_MMA;
     }
     m->st = (cudaStream_t)cuda_stream;
+    m->own_stream = false;
+    if (!m->st) {
+        // the legacy default stream cannot be captured into a graph: use a stream of our own
+        // (a blocking one, so that it still orders after the caller's default-stream work)
+        cudaError_t se = cudaStreamCreate(&m->st);
+        if (se != cudaSuccess) {
+            g_last_cuda = (int)se;
+            delete m;
+            return LS_ERR_CUDA;
+        }
+        m->own_stream = true;
+    }
     m->emb = (const uint16_t*)w->tok_embed;
     m->fnorm = (const uint16_t*)w->final_norm;
     m->lm = (const uint16_t*)w->lm_head;
@@ -468,6 +480,7 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
     auto fail = [&](int rc) {
         if (m->ev0) cudaEventDestroy(m->ev0);
         if (m->ev1) cudaEventDestroy(m->ev1);
+        if (m->own_stream) cudaStreamDestroy(m->st);
         delete m;
         return rc;
     };
@@ -502,6 +515,7 @@ int ls_model_destroy(ls_model* m)
     drop_graphs(m);
     cudaEventDestroy(m->ev0);
     cudaEventDestroy(m->ev1);
+    if (m->own_stream) cudaStreamDestroy(m->st);
     delete m;
     return LS_OK;
 }
@@ -577,12 +591,17 @@ int ls_decode(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_ne
     if (m->use_graphs) LS_TRY(get_graph(m, E, d, &g));
     LS_TRY(write_ctl(m, m->n_prompt - 1, m->last_tok, max_new));
     int64_t launched = 0;
-    int syncs = 0, n_out = 0;
+    int syncs = 0, n_out = 0, steps_done = 0;
     int32_t w[CTL_WORDS];
     LS_CK(cudaEventRecord(m->ev0, m->st));
     for (;;) {
+        // first batch: as if every draft were accepted; afterwards at the observed rate
         int remaining = max_new - n_out;
         int steps = (remaining + d) / (d + 1);
+        if (steps_done > 0 && n_out > 0) {
+            int64_t est = ((int64_t)remaining * steps_done + n_out - 1) / n_out;
+            steps = (int)(est < 1 ? 1 : est);
+        }
         for (int i = 0; i < steps; ++i) {
             if (g) {
                 LS_CK(cudaGraphLaunch(g->exec, m->st));
@@ -597,6 +616,7 @@ int ls_decode(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_ne
         ++syncs;
         if (w[CTL_STATUS]) return LS_ERR_DEVICE_STATUS;
         n_out = w[CTL_N_OUT];
+        steps_done = w[CTL_N_STEPS];
         if (w[CTL_DONE]) break;
     }
     LS_CK(cudaEventRecord(m->ev1, m->st));
