@@ -190,6 +190,29 @@ int ls_op_lm_head_argmax(int32_t linear_path, const void *w_dev, const void *h_b
                          int32_t M, int32_t V, int32_t K, void *scratch_dev, int32_t *tok_dev,
                          float *logits_dev, void *cuda_stream);
 
+/* The same operation for callers that cannot allocate device memory at all and so have
+ * no scratch buffer to pass: code running between cudaStreamBeginCapture and EndCapture,
+ * plug-ins and callbacks that are handed a stream but no allocator, and hosts whose
+ * memory pool is sized up front and closed.  (The paper has no counterpart; this is a
+ * convenience of this library.)  The per-CTA candidates go to a buffer that is part of
+ * the library image, LS_OP_LM_HEAD_STATIC_BYTES bytes on every GPU that loads the
+ * library, held until the process exits.  The call itself performs no cudaMalloc /
+ * cudaFree and calls nothing that allocates.
+ *   - V <= LS_OP_LM_HEAD_STATIC_MAX_VOCAB, otherwise LS_ERR_CAPACITY (nothing is launched).
+ *   - The first call on each device looks up the buffer's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one buffer and it keeps the previous call's contents.  Nothing
+ *     in it has to start at zero: every candidate the finishing kernel reads is rewritten
+ *     by the same call.  Two calls that may run on the GPU at the same time (different
+ *     streams, no dependency) race on it -- order them.
+ * Inputs and the tok_dev output are the caller's, as in ls_op_lm_head_argmax; there is no
+ * logits output. */
+#define LS_OP_LM_HEAD_STATIC_MAX_VOCAB 131072
+#define LS_OP_LM_HEAD_STATIC_BYTES (8u * LS_MAX_ROWS * (LS_OP_LM_HEAD_STATIC_MAX_VOCAB / 16))
+int ls_op_lm_head_argmax_static(int32_t linear_path, const void *w_dev, const void *h_bf16_dev,
+                                int32_t M, int32_t V, int32_t K, int32_t *tok_dev,
+                                void *cuda_stream);
+
 /* Rotary embedding + KV append: rows m = 0..M-1 sit at positions pos0+m.  qkv fp32
  * [M, (Hq+2Hkv)*hd] (q heads, then k heads, then v heads).  Writes q_out bf16
  * [M, Hq*hd] and k, v (bf16) into the paged cache: k_pages / v_pages hold physical

@@ -26,7 +26,7 @@ EXPORTS = (
     "ls_set_page_table", "ls_generate", "ls_generate_full", "ls_generate_early", "ls_prefill",
     "ls_decode", "ls_read_output", "ls_debug_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
     "ls_op_linear", "ls_op_gate_up_swiglu", "ls_op_lm_head_scratch_bytes", "ls_op_lm_head_argmax",
-    "ls_op_rope_append", "ls_op_attention_scratch_bytes", "ls_op_attention", "ls_op_accept",
+    "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_attention_scratch_bytes", "ls_op_attention", "ls_op_accept",
 )
 
 
@@ -95,6 +95,7 @@ def lib():
             "ls_op_gate_up_swiglu": (C.c_int, [i32, vp, vp, vp, i32, i32, i32, vp, vp]),
             "ls_op_lm_head_scratch_bytes": (C.c_size_t, [i32]),
             "ls_op_lm_head_argmax": (C.c_int, [i32, vp, vp, i32, i32, i32, vp, vp, vp, vp]),
+            "ls_op_lm_head_argmax_static": (C.c_int, [i32, vp, vp, i32, i32, i32, vp, vp]),
             "ls_op_rope_append": (C.c_int, [vp, i32, i32, i32, i32, i32, C.c_float, i32, vp, i32, vp, vp, vp, vp]),
             "ls_op_attention_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
             "ls_op_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]),
@@ -261,6 +262,18 @@ def ls_op_lm_head_argmax(path, w, h, scratch, tok, logits=None):
     (V, K), M = w.shape, h.shape[0]
     _ck(lib().ls_op_lm_head_argmax(path, _dev(w), _dev(h), M, V, K, _dev(scratch), _dev(tok), _dev(logits),
                                    _stream()), "ls_op_lm_head_argmax")
+
+
+LS_OP_LM_HEAD_STATIC_MAX_VOCAB = 131072
+
+
+def ls_op_lm_head_argmax_static(path, w, h, tok):
+    """LM head + argmax for callers that have no scratch buffer to give (they cannot
+    allocate): the candidates go to a buffer inside the library.  Vocabulary at most
+    LS_OP_LM_HEAD_STATIC_MAX_VOCAB; calls must not overlap on the GPU."""
+    (V, K), M = w.shape, h.shape[0]
+    _ck(lib().ls_op_lm_head_argmax_static(path, _dev(w), _dev(h), M, V, K, _dev(tok), _stream()),
+        "ls_op_lm_head_argmax_static")
 
 
 def ls_op_rope_append(qkv, pos0, Hq, Hkv, hd, theta, page_size, page_table, max_seq, q_out, k_pages, v_pages):

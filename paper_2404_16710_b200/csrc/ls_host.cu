@@ -17,6 +17,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -813,6 +814,52 @@ int ls_op_lm_head_argmax(int32_t path, const void* w, const void* h, int32_t M, 
     a.cand = (ValIdx*)scratch;
     a.cand_stride = (V + 15) / 16;
     a.out = logits;
+    a.ldo = V;
+    LS_CK(launch_linear(path, EPI_ARGMAX, a, (cudaStream_t)stream));
+    argmax_finish_kernel<<<M, 256, 0, (cudaStream_t)stream>>>(a.cand, lin_grid(EPI_ARGMAX, V), a.cand_stride, tok,
+                                                              nullptr);
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+// ---- LM head + argmax without any allocation by anybody: the candidate buffer lives in
+// the library image.  Every GPU that loads the library holds these bytes until exit.
+static __device__ __align__(256) unsigned char g_lm_head_static_scratch[LS_OP_LM_HEAD_STATIC_BYTES];
+static_assert(sizeof(ValIdx) * LS_MAX_ROWS * (LS_OP_LM_HEAD_STATIC_MAX_VOCAB / 16) == LS_OP_LM_HEAD_STATIC_BYTES,
+              "one (value, index) candidate per 16 vocabulary rows and pass row");
+
+// In host code the array's name is only a handle; its device address has to be asked for,
+// once per device, with that device current.
+static int static_scratch_address(void** out)
+{
+    constexpr int kMaxDevices = 64;
+    static void* addr[kMaxDevices] = {nullptr};
+    static std::mutex mu;
+    int dev = 0;
+    LS_CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return LS_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        LS_CK(cudaGetSymbolAddress(&p, g_lm_head_static_scratch));
+        if (!p || ((uintptr_t)p & 255u)) return LS_ERR_UNSUPPORTED;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return LS_OK;
+}
+
+int ls_op_lm_head_argmax_static(int32_t path, const void* w, const void* h, int32_t M, int32_t V, int32_t K,
+                                int32_t* tok, void* stream)
+{
+    LS_TRY(lin_check(path, w, h, M, V, K));
+    if (!tok) return LS_ERR_INVALID_ARG;
+    if (V > LS_OP_LM_HEAD_STATIC_MAX_VOCAB) return LS_ERR_CAPACITY;  // vocabulary beyond the built-in buffer
+    void* scratch = nullptr;
+    LS_TRY(static_scratch_address(&scratch));
+    LinArgs a = lin_args((const uint16_t*)w, (const uint16_t*)h, M, V, K);
+    a.cand = (ValIdx*)scratch;
+    a.cand_stride = (V + 15) / 16;
     a.ldo = V;
     LS_CK(launch_linear(path, EPI_ARGMAX, a, (cudaStream_t)stream));
     argmax_finish_kernel<<<M, 256, 0, (cudaStream_t)stream>>>(a.cand, lin_grid(EPI_ARGMAX, V), a.cand_stride, tok,
