@@ -146,52 +146,6 @@ def run_reference(args):
     print(json.dumps(out), flush=True)
 
 
-def time_op(fn, n_rot, iters=40, warm=5):
-    """mean device time (ms) of fn(i % n_rot), CUDA events on the launching stream"""
-    for i in range(warm):
-        fn(i % n_rot)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(iters):
-        fn(i % n_rot)
-    e1.record()
-    torch.cuda.synchronize()
-    return e0.elapsed_time(e1) / iters
-
-
-def kernel_rooflines(B, wl, w, path, peak):
-    """Each linear kernel family of one layer, timed alone on this workload's shapes at the
-    draft (M=1) and verify (M=d+1) pass sizes, rotating over the layers' weights so that no
-    launch finds its weights in L2."""
-    s, out = wl.shape, {}
-    D, F, V = s.d_model, s.d_ffn, s.vocab
-    L = s.n_layers
-    for M in (1, wl.num_draft + 1):
-        h = torch.randn((M, D), device="cuda").bfloat16()
-        a = torch.randn((M, F), device="cuda").bfloat16()
-        o = torch.randn((M, s.n_heads * s.head_dim), device="cuda").bfloat16()
-        x = torch.zeros((M, D), dtype=torch.float32, device="cuda")
-        act = torch.empty((M, F), dtype=torch.bfloat16, device="cuda")
-        q = torch.empty((M, w["wq"][0].shape[0]), dtype=torch.float32, device="cuda")
-        tok = torch.empty((M,), dtype=torch.int32, device="cuda")
-        scratch = torch.empty(B.ls_op_lm_head_scratch_bytes(V), dtype=torch.uint8, device="cuda")
-        cases = {
-            "gate_up_swiglu": (lambda i: B.ls_op_gate_up_swiglu(path, w["w_gate"][i], w["w_up"][i], h, act),
-                               2 * 2 * F * D, L),
-            "down_residual": (lambda i: B.ls_op_linear(path, w["w_down"][i], a, x, True), 2 * F * D, L),
-            "q_proj": (lambda i: B.ls_op_linear(path, w["wq"][i], h, q, False), 2 * w["wq"][0].numel(), L),
-            "o_residual": (lambda i: B.ls_op_linear(path, w["wo"][i], o, x, True), 2 * w["wo"][0].numel(), L),
-            "lm_head_argmax": (lambda i: B.ls_op_lm_head_argmax(path, (w["lm_head"], w["tok_embed"])[i], h, scratch,
-                                                                 tok), 2 * V * D, 2),
-        }
-        for name, (fn, nbytes, rot) in cases.items():
-            ms = time_op(fn, rot)
-            out[f"{name}@M={M}"] = {"ms": round(ms, 5), "GB/s": round(nbytes / ms / 1e6, 1),
-                                    "frac": round(nbytes / ms / 1e6 / peak, 4), "bytes": nbytes}
-    return out
-
-
 def run_own(args):
     from paper_2404_16710_b200 import binding as B
     rank = int(os.environ.get("RANK", "0"))
@@ -219,6 +173,20 @@ def run_own(args):
         if dist:
             dist.barrier()
         torch.cuda.synchronize()
+
+    if args.profile_region:
+        B.ls_prefill(gm.h, prompt)
+        for _ in range(max(1, args.warmup)):
+            B.ls_decode(gm.h, E, d, args.profile_region)
+            B.ls_decode(gm.h, 0, 0, args.profile_region)
+        torch.cuda.synchronize()
+        torch.cuda.profiler.start()
+        B.ls_decode(gm.h, E, d, args.profile_region)
+        B.ls_decode(gm.h, 0, 0, args.profile_region)
+        torch.cuda.synchronize()
+        torch.cuda.profiler.stop()
+        print(json.dumps({"profile_region": args.profile_region, "launches": int(gm.stats().kernel_launches)}))
+        return
 
     # ---- device-resident timing: prompt already prefilled in HBM, decode loop only
     B.ls_prefill(gm.h, prompt)
@@ -298,7 +266,8 @@ def run_own(args):
            "prefill_ms": prefill_ms}
 
     if rank == 0 and world == 1:
-        ks = kernel_rooflines(B, wl, w, path, peak)
+        from paper_2404_16710_b200 import opbench
+        ks = opbench.kernel_rooflines(s, w, path, (1, d + 1), peak)
         dom = ks[f"gate_up_swiglu@M={d + 1}"]
         out["roofline"] = {"bound": "hbm", "kernel": f"linear_{'mma' if path == 2 else 'fma'}_kernel (gate-up + SwiGLU, "
                            f"M={d + 1}, verify pass)", "achieved": dom["GB/s"], "peak": peak, "unit": "GB/s",
@@ -324,6 +293,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--workload", default="llama2-7b", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--profile-region", type=int, default=0, metavar="NEW",
+                    help="instead of the benchmark: prefill, warm up, then run one self-speculative and one "
+                         "full-greedy decode of NEW tokens between cudaProfilerStart/Stop (for a profiler "
+                         "started with --profile-from-start off) and exit")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -6,11 +6,12 @@
 //
 //   FMA  one warp per 4 weight rows, lanes stride over K with 128-bit loads, fp32 FMA
 //        chains per (row, token), butterfly reduction.  Cheap for M <= 4.
-//   MMA  one CTA per 16 weight rows, its 8 warps interleave over K; weights go from
-//        global memory straight into mma.sync.m16n8k16 A fragments (the contraction
-//        index may be permuted freely as long as A and B agree, so a thread's 16-byte
-//        load IS its fragment), tokens are the n8 dimension.  Issue cost per weight byte
-//        does not grow with M up to 8 (16 with a second n-tile).
+//   MMA  one CTA per 16 weight rows, its 8 or 16 warps interleave over K; a thread's
+//        16-byte pieces of the weight rows ARE its mma.sync.m16n8k16 A fragments (the
+//        contraction index may be permuted freely as long as A and B agree), so they
+//        need no layout change: each thread streams its own pieces through a private
+//        cp.async ring in shared memory.  Tokens are the n8 dimension.  Issue cost per
+//        weight byte does not grow with M up to 8 (16 with a second n-tile).
 //
 // In both, the sequence of operations that produces (row n, token m) is the same for
 // every M, so results are bit-identical across pass sizes within a family.
@@ -188,17 +189,55 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// grid ceil(N/16) (SwiGLU: ceil(F/8)), block 256 = 8 warps that interleave over K in steps
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead.
+// .cg: L2 only (streamed weights); .ca: also L1 (activations, re-read by every CTA).
+__device__ __forceinline__ void cp_async16_cg(uint32_t dst, const void* src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async16_ca(uint32_t dst, const void* src, int src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds16(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+template <int NT, int WARPS, int STAGES>
+constexpr size_t mma_ring_bytes()
+{
+    return (size_t)(2 + NT) * STAGES * WARPS * 32 * 16;
+}
+
+// grid ceil(N/16) (SwiGLU: ceil(F/8)), block WARPS*32: the warps interleave over K in steps
 // of 32.  Fragment roles (g = lane/4, t = lane%4): the thread's 16 bytes of row g (and of
 // row g+8) at k = 32 s + 8 t feed two MMAs; contraction slots {2t, 2t+1, 2t+8, 2t+9} of
 // the first take elements k..k+3, of the second k+4..k+7, for A and for B alike.
 // SwiGLU: row g is the gate row of feature f, row g+8 its up row.
-template <int NT, int EPI>
-__global__ void __launch_bounds__(256) linear_mma_kernel(const LinArgs a)
+//
+// Each thread prefetches exactly the 16-byte pieces it will consume itself, STAGES k-steps
+// ahead, with cp.async into a ring of its own in shared memory: the bytes in flight per
+// SM are set by the ring depth, not by registers or occupancy, and no barrier is needed
+// (nobody else reads a thread's slots).  WARPS and STAGES are chosen from (N, K) alone --
+// never from M -- so that matrices with few row tiles (N = 4096: 256 tiles) still keep
+// enough bytes in flight.
+template <int NT, int EPI, int WARPS, int STAGES>
+__global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
 {
-    constexpr int U = 4;  // k-steps in flight per warp
+    constexpr int T = WARPS * 32;
+    extern __shared__ __align__(16) unsigned char ring[];
     if (a.ctl && a.ctl[CTL_DONE]) return;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const uint16_t *pa, *pb;
     if (EPI == EPI_SWIGLU) {
         int f = min(blockIdx.x * 8 + g, a.N - 1);
@@ -212,42 +251,50 @@ __global__ void __launch_bounds__(256) linear_mma_kernel(const LinArgs a)
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) hb[nt] = a.h + (size_t)min(nt * 8 + g, a.M - 1) * a.K;
 
+    // region r (0: row g, 1: row g+8, 2..: tokens), stage s, thread tid -> 16 bytes
+    const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(ring) + (uint32_t)tid * 16u;
+    auto slot = [&](int r, int s) { return ring0 + (uint32_t)((r * STAGES + s) * T) * 16u; };
+
+    const int nsteps = (a.K + 31) >> 5;
+    auto issue = [&](int step, int s) {
+        if (step < nsteps) {
+            const int k = step * 32 + 8 * t;
+            const int nb = (k < a.K) ? 16 : 0;
+            const int kk = (k < a.K) ? k : 0;
+            cp_async16_cg(slot(0, s), pa + kk, nb);
+            cp_async16_cg(slot(1, s), pb + kk, nb);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) cp_async16_ca(slot(2 + nt, s), hb[nt] + kk, nb);
+        }
+        cp_async_commit();
+    };
+
     float c[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int i = 0; i < 4; ++i) c[nt][i] = 0.f;
 
-    const int nsteps = (a.K + 31) >> 5;
-    for (int s0 = warp; s0 < nsteps; s0 += 8 * U) {
-        uint4 A0[U], A1[U], B[U][NT];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            int k = (s0 + 8 * u) * 32 + 8 * t;
-            bool ok = (s0 + 8 * u < nsteps) && (k < a.K);
-            A0[u] = A1[u] = make_uint4(0, 0, 0, 0);
-            if (ok) {
-                A0[u] = ld_stream16(pa + k);
-                A1[u] = ld_stream16(pb + k);
-            }
+    for (int p = 0; p < STAGES - 1; ++p) issue(warp + p * WARPS, p);
+    int rd = 0, wr = STAGES - 1;
+    for (int step = warp; step < nsteps; step += WARPS) {
+        issue(step + (STAGES - 1) * WARPS, wr);
+        cp_async_wait<STAGES - 1>();
+        const uint4 A0 = lds16(slot(0, rd)), A1 = lds16(slot(1, rd));
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                B[u][nt] = make_uint4(0, 0, 0, 0);
-                if (ok) B[u][nt] = ld_reuse16(hb[nt] + k);
-            }
+        for (int nt = 0; nt < NT; ++nt) {
+            const uint4 B = lds16(slot(2 + nt, rd));
+            mma_bf16_16816(c[nt], A0.x, A1.x, A0.y, A1.y, B.x, B.y);
+            mma_bf16_16816(c[nt], A0.z, A1.z, A0.w, A1.w, B.z, B.w);
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                mma_bf16_16816(c[nt], A0[u].x, A1[u].x, A0[u].y, A1[u].y, B[u][nt].x, B[u][nt].y);
-                mma_bf16_16816(c[nt], A0[u].z, A1[u].z, A0[u].w, A1[u].w, B[u][nt].z, B[u][nt].w);
-            }
-        }
+        rd = (rd + 1 == STAGES) ? 0 : rd + 1;
+        wr = (wr + 1 == STAGES) ? 0 : wr + 1;
     }
+    cp_async_wait<0>();
 
     // cross-warp reduction in warp order (fixed), then the epilogue on 32*NT threads
-    __shared__ float red[8][NT * 4][32];
+    __shared__ float red[WARPS][NT * 4][32];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -262,7 +309,7 @@ __global__ void __launch_bounds__(256) linear_mma_kernel(const LinArgs a)
         for (int i = 0; i < 4; ++i) {
             float s = 0.f;
 #pragma unroll
-            for (int w = 0; w < 8; ++w) s += red[w][nt * 4 + i][lane];
+            for (int w = 0; w < WARPS; ++w) s += red[w][nt * 4 + i][lane];
             r[i] = s;
         }
         const int m0 = nt * 8 + 2 * tt;  // tokens m0, m0+1
@@ -330,13 +377,39 @@ inline cudaError_t launch_linear_fma(const LinArgs& a, cudaStream_t st)
     return cudaGetLastError();
 }
 
+// Warps per 16-row tile and ring depth, from the matrix shape alone: many row tiles ->
+// 8 warps x 6 stages (3 CTAs per SM); few row tiles (N = 4096) -> 16 warps x 4 stages
+// (2 CTAs per SM, all tiles resident in one wave).
+inline bool mma_wide(int epi, int N, int K)
+{
+    const int tiles = lin_grid(epi, N), nsteps = (K + 31) / 32;
+    return tiles < 600 && nsteps >= 16;
+}
+
+template <int NT, int EPI, int WARPS, int STAGES>
+inline cudaError_t launch_linear_mma_cfg(const LinArgs& a, cudaStream_t st)
+{
+    constexpr size_t smem = mma_ring_bytes<NT, WARPS, STAGES>();
+    static bool allowed[64] = {false};  // per instantiation and device: the attribute is set once
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !allowed[dev]) {
+        e = cudaFuncSetAttribute(linear_mma_kernel<NT, EPI, WARPS, STAGES>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) allowed[dev] = true;
+    }
+    linear_mma_kernel<NT, EPI, WARPS, STAGES><<<lin_grid(EPI, a.N), WARPS * 32, smem, st>>>(a);
+    return cudaGetLastError();
+}
+
 template <int EPI>
 inline cudaError_t launch_linear_mma(const LinArgs& a, cudaStream_t st)
 {
-    dim3 grid(lin_grid(EPI, a.N)), block(256);
-    if (a.M <= 8) linear_mma_kernel<1, EPI><<<grid, block, 0, st>>>(a);
-    else linear_mma_kernel<2, EPI><<<grid, block, 0, st>>>(a);
-    return cudaGetLastError();
+    if (mma_wide(EPI, a.N, a.K))
+        return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 16, 4>(a, st) : launch_linear_mma_cfg<2, EPI, 16, 4>(a, st);
+    return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 8, 6>(a, st) : launch_linear_mma_cfg<2, EPI, 8, 6>(a, st);
 }
 
 // path: 1 = FMA, 2 = MMA

@@ -1,0 +1,113 @@
+"""Time single kernels of the decode path on a workload's shapes, through the C ABI.
+
+    python -m paper_2404_16710_b200.opbench --workload llama2-7b --layers 4 --ops gate_up_swiglu --rows 7
+
+Each op is launched ``iters`` times (as one CUDA graph) with CUDA events around the batch,
+rotating over the weights of ``layers`` layers so that no launch finds its weights in L2 (one 7B-shaped
+gate+up pair is 180 MB, the L2 126 MB).  Algorithmic bytes of a launch are its weight
+bytes (2 N K; the activations, M K 2 bytes, are noise).  Also the small driver to run
+under a profiler: few launches, a few GB on the device.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as B
+from . import synth
+
+OPS = ("gate_up_swiglu", "down_residual", "qkv_proj", "o_residual", "lm_head_argmax")
+
+
+def time_op(fn, n_rot, iters=40, warm=5):
+    """mean device time (ms) of one launch of fn: ``iters`` launches are captured into a
+    CUDA graph (so that the host's launch rate does not bound kernels of a few
+    microseconds) and the graph is replayed between two CUDA events on its stream."""
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        for i in range(warm):
+            fn(i % n_rot)
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            for i in range(iters):
+                fn((warm + i) % n_rot)
+        g.replay()
+        st.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        g.replay()
+        e1.record(st)
+        st.synchronize()
+    torch.cuda.current_stream().wait_stream(st)
+    return e0.elapsed_time(e1) / iters
+
+
+def op_cases(shape, w, path, M):
+    """name -> (callable(layer index), algorithmic bytes per launch, number of distinct weights)"""
+    D, F, V = shape.d_model, shape.d_ffn, shape.vocab
+    L = len(w["wq"])
+    qw = shape.n_heads * shape.head_dim
+    kvw = shape.n_kv_heads * shape.head_dim
+    g = torch.Generator(device="cuda").manual_seed(7)
+    h = torch.randn((M, D), device="cuda", generator=g).bfloat16()
+    a = torch.randn((M, F), device="cuda", generator=g).bfloat16()
+    o = torch.randn((M, qw), device="cuda", generator=g).bfloat16()
+    x = torch.zeros((M, D), dtype=torch.float32, device="cuda")
+    act = torch.empty((M, F), dtype=torch.bfloat16, device="cuda")
+    qkv = torch.empty((M, qw + 2 * kvw), dtype=torch.float32, device="cuda")
+    tok = torch.empty((M,), dtype=torch.int32, device="cuda")
+    scratch = torch.empty(B.ls_op_lm_head_scratch_bytes(V), dtype=torch.uint8, device="cuda")
+    # q, k and v projections as one matrix of the fused launch's size
+    wqkv = [torch.cat([w["wq"][i], w["wk"][i], w["wv"][i]]) for i in range(L)]
+    heads = [w["lm_head"], w["tok_embed"]]
+    return {
+        "gate_up_swiglu": (lambda i: B.ls_op_gate_up_swiglu(path, w["w_gate"][i % L], w["w_up"][i % L], h, act),
+                           4 * F * D, L),
+        "down_residual": (lambda i: B.ls_op_linear(path, w["w_down"][i % L], a, x, True), 2 * F * D, L),
+        "qkv_proj": (lambda i: B.ls_op_linear(path, wqkv[i % L], h, qkv, False), 2 * (qw + 2 * kvw) * D, L),
+        "o_residual": (lambda i: B.ls_op_linear(path, w["wo"][i % L], o, x, True), 2 * D * qw, L),
+        "lm_head_argmax": (lambda i: B.ls_op_lm_head_argmax(path, heads[i % 2], h, scratch, tok), 2 * V * D, 2),
+    }
+
+
+def kernel_rooflines(shape, w, path, rows, peak_gbs, ops=OPS, iters=40, warm=5):
+    out = {}
+    for M in rows:
+        cases = op_cases(shape, w, path, M)
+        for name in ops:
+            fn, nbytes, rot = cases[name]
+            ms = time_op(fn, rot, iters, warm)
+            out[f"{name}@M={M}"] = {"ms": round(ms, 5), "GB/s": round(nbytes / ms / 1e6, 1),
+                                    "frac": round(nbytes / ms / 1e6 / peak_gbs, 4), "bytes": nbytes}
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="llama2-7b", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--layers", type=int, default=4, help="layers of weights to create and rotate over")
+    ap.add_argument("--ops", default=",".join(OPS))
+    ap.add_argument("--rows", default="1,7")
+    ap.add_argument("--path", default="mma", choices=["fma", "mma"])
+    ap.add_argument("--iters", type=int, default=40)
+    ap.add_argument("--warm", type=int, default=5)
+    ap.add_argument("--peak", type=float, default=6553.9, help="GB/s the fractions are quoted against")
+    a = ap.parse_args()
+    from dataclasses import replace
+    wl = synth.WORKLOADS[a.workload]
+    shape = replace(wl.shape, n_layers=a.layers)
+    w = synth.make_weights(shape, wl.weight_seed, wl.exit_layer, wl.late_scale, device="cuda")
+    path = B.LS_LINEAR_MMA if a.path == "mma" else B.LS_LINEAR_FMA
+    res = kernel_rooflines(shape, w, path, [int(r) for r in a.rows.split(",")], a.peak,
+                           [o for o in a.ops.split(",") if o], a.iters, a.warm)
+    for k, v in res.items():
+        print(f"{k:28s} {v['ms'] * 1e3:8.2f} us  {v['GB/s']:8.1f} GB/s  {v['frac']:.3f} of {a.peak:.0f}")
+    print(json.dumps(res))
+
+
+if __name__ == "__main__":
+    main()
