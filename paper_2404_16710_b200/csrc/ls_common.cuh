@@ -57,6 +57,35 @@ __device__ __forceinline__ uint4 ld_reuse16(const void* p)
     return v;
 }
 
+// Programmatic dependent launch: a kernel launched with the attribute may start while its
+// predecessor on the stream is still running.  pdl_wait() blocks until the predecessor
+// grid has completed and its writes are visible; before it, a kernel may touch only
+// memory that no kernel of the loop writes (weights, page table).  Without the launch
+// attribute both are no-ops.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+struct LaunchCtx {
+    cudaStream_t st;
+    bool pdl;  // allow the kernel to start before the previous kernel on st has finished
+};
+
+template <typename... P, typename... A>
+inline cudaError_t launch(const LaunchCtx& lc, void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, A... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = lc.st;
+    cudaLaunchAttribute at;
+    at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &at;
+    cfg.numAttrs = lc.pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+
 struct ValIdx {
     float v;
     int i;

@@ -92,7 +92,7 @@ struct ls_model {
     int page_shift, n_pages, chunk_cap, cand_stride;
     // loop state
     int n_prompt, last_tok, prefilled_layers, grid_chunks;
-    bool use_graphs, own_stream;
+    bool use_graphs, own_stream, pdl;
     int64_t launches;  // kernels enqueued (counted while building a step)
     struct G {
         cudaGraphExec_t exec;
@@ -173,22 +173,19 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
 int attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
                 int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int hd, int page_shift,
                 int max_seq, int chunk_cap, int grid_chunks, float* part, uint16_t* out,
-                cudaStream_t st)
+                const LaunchCtx& lc)
 {
     const int Q = Hq / Hkv * M;
     dim3 grid(grid_chunks, Hkv), mgrid(M, Hq);
     if (hd == 128) {
-        size_t sm = attn_smem_bytes<128>(Q);
-        attn_chunk_kernel<128><<<grid, 128, sm, st>>>(q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv,
-                                                        page_shift, max_seq, chunk_cap, part);
-        attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(part, ctl, pos_off, Hq, chunk_cap, out);
+        LS_CK(launch(lc, attn_chunk_kernel<128>, grid, dim3(128), attn_smem_bytes<128>(Q), q, kp, vp, pt, ctl,
+                     pos_off, M, Hq, Hkv, page_shift, max_seq, chunk_cap, part));
+        LS_CK(launch(lc, attn_merge_kernel<128>, mgrid, dim3(128), 0, part, ctl, pos_off, Hq, chunk_cap, out));
     } else {
-        size_t sm = attn_smem_bytes<64>(Q);
-        attn_chunk_kernel<64><<<grid, 128, sm, st>>>(q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv,
-                                                       page_shift, max_seq, chunk_cap, part);
-        attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(part, ctl, pos_off, Hq, chunk_cap, out);
+        LS_CK(launch(lc, attn_chunk_kernel<64>, grid, dim3(128), attn_smem_bytes<64>(Q), q, kp, vp, pt, ctl,
+                     pos_off, M, Hq, Hkv, page_shift, max_seq, chunk_cap, part));
+        LS_CK(launch(lc, attn_merge_kernel<64>, mgrid, dim3(64), 0, part, ctl, pos_off, Hq, chunk_cap, out));
     }
-    LS_CK(cudaGetLastError());
     return LS_OK;
 }
 
@@ -225,12 +222,12 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
     const ls_config& c = m->c;
     const int D = c.d_model, Hq = c.n_heads, Hkv = c.n_kv_heads, hd = c.head_dim, F = c.d_ffn;
     const int qw = Hq * hd, kvw = Hkv * hd;
-    cudaStream_t st = m->st;
+    const LaunchCtx st = {m->st, m->pdl};
     for (int l = l0; l < l1; ++l) {
         const LayerW& w = m->lw[l];
         uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
         uint16_t* vp = m->vpages + (size_t)l * m->layer_kv_elems;
-        rmsnorm_kernel<<<M, 256, 0, st>>>(xrow, w.attn_norm, D, c.rms_eps, m->h, m->ctl);
+        LS_CK(launch(st, rmsnorm_kernel, dim3(M), dim3(256), 0, xrow, w.attn_norm, D, c.rms_eps, m->h, m->ctl));
         LinArgs a = lin_args(w.wq, m->h, M, qw + 2 * kvw, D);
         a.w1 = w.wk;
         a.w2 = w.wv;
@@ -240,9 +237,8 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
         a.ldo = qw + 2 * kvw;
         a.ctl = m->ctl;
         LS_CK(launch_linear(m->path, EPI_STORE, a, st));
-        rope_append_kernel<<<dim3(M, Hq + 2 * Hkv), hd / 2, 0, st>>>(
-            m->qkv, Hq, Hkv, hd, m->inv_freq, c.rope_theta, m->page_shift, m->page_table, c.max_seq,
-            m->q, kp, vp, m->ctl, pos_off);
+        LS_CK(launch(st, rope_append_kernel, dim3(M, Hq + 2 * Hkv), dim3(hd / 2), 0, m->qkv, Hq, Hkv, hd, m->inv_freq,
+                     c.rope_theta, m->page_shift, m->page_table, c.max_seq, m->q, kp, vp, m->ctl, pos_off));
         LS_TRY(attn_launch(m->q, kp, vp, m->page_table, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift,
                            c.max_seq, m->chunk_cap, m->grid_chunks, m->part, m->o, st));
         a = lin_args(w.wo, m->o, M, D, qw);
@@ -250,7 +246,7 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
         a.ldo = D;
         a.ctl = m->ctl;
         LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
-        rmsnorm_kernel<<<M, 256, 0, st>>>(xrow, w.ffn_norm, D, c.rms_eps, m->h, m->ctl);
+        LS_CK(launch(st, rmsnorm_kernel, dim3(M), dim3(256), 0, xrow, w.ffn_norm, D, c.rms_eps, m->h, m->ctl));
         a = lin_args(w.wg, m->h, M, F, D);
         a.w1 = w.wu;
         a.out_bf16 = m->a;
@@ -271,26 +267,26 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
 int run_head(ls_model* m, int M, const float* xrow, int32_t* tok_out, float* logits)
 {
     const ls_config& c = m->c;
-    rmsnorm_kernel<<<M, 256, 0, m->st>>>(xrow, m->fnorm, c.d_model, c.rms_eps, m->h, m->ctl);
+    const LaunchCtx st = {m->st, m->pdl};
+    LS_CK(launch(st, rmsnorm_kernel, dim3(M), dim3(256), 0, xrow, m->fnorm, c.d_model, c.rms_eps, m->h, m->ctl));
     LinArgs a = lin_args(m->lm, m->h, M, c.vocab, c.d_model);
     a.cand = m->cand;
     a.cand_stride = m->cand_stride;
     a.out = logits;
     a.ldo = c.vocab;
     a.ctl = m->ctl;
-    LS_CK(launch_linear(m->path, EPI_ARGMAX, a, m->st));
-    argmax_finish_kernel<<<M, 256, 0, m->st>>>(m->cand, lin_grid(EPI_ARGMAX, c.vocab), m->cand_stride,
-                                               tok_out, m->ctl);
+    LS_CK(launch_linear(m->path, EPI_ARGMAX, a, st));
+    LS_CK(launch(st, argmax_finish_kernel, dim3(M), dim3(256), 0, m->cand, lin_grid(EPI_ARGMAX, c.vocab),
+                 m->cand_stride, tok_out, m->ctl));
     m->launches += 3;
-    LS_CK(cudaGetLastError());
     return LS_OK;
 }
 
 int run_embed(ls_model* m, const int32_t* tok_dev, int M, float* xrow)
 {
-    embed_kernel<<<M, 256, 0, m->st>>>(m->emb, tok_dev, m->c.d_model, m->c.vocab, xrow, m->ctl);
+    LS_CK(launch(LaunchCtx{m->st, m->pdl}, embed_kernel, dim3(M), dim3(256), 0, m->emb, tok_dev, m->c.d_model,
+                 m->c.vocab, xrow, m->ctl));
     m->launches += 1;
-    LS_CK(cudaGetLastError());
     return LS_OK;
 }
 
@@ -313,9 +309,9 @@ int enqueue_step(ls_model* m, int E, int d)
         LS_TRY(run_layers(m, E, L, d + 1, m->x, 0));
         LS_TRY(run_head(m, d + 1, m->x, m->verified, nullptr));
     }
-    accept_kernel<<<1, 32, 0, m->st>>>(m->draft, m->verified, d, m->ctl, m->out_ids, m->accepted);
+    LS_CK(launch(LaunchCtx{m->st, m->pdl}, accept_kernel, dim3(1), dim3(32), 0, m->draft, m->verified, d, m->ctl,
+                 m->out_ids, m->accepted));
     m->launches += 1;
-    LS_CK(cudaGetLastError());
     return LS_OK;
 }
 
@@ -474,6 +470,7 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
     m->prefilled_layers = 0;
     m->grid_chunks = m->chunk_cap;
     m->use_graphs = getenv("LS_NO_GRAPH") == nullptr;
+    m->pdl = getenv("LS_NO_PDL") == nullptr;
     m->launches = 0;
     memset(&m->stats, 0, sizeof(m->stats));
     m->h_n_out = m->h_n_steps = 0;
@@ -754,8 +751,8 @@ int ls_op_embed(const void* emb, const int32_t* tok, int32_t M, int32_t D, int32
 {
     if (!aligned16(emb) || !tok || !aligned16(x) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8 || V < 1)
         return LS_ERR_INVALID_ARG;
-    embed_kernel<<<M, 256, 0, (cudaStream_t)stream>>>((const uint16_t*)emb, tok, D, V, x, nullptr);
-    LS_CK(cudaGetLastError());
+    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, embed_kernel, dim3(M), dim3(256), 0, (const uint16_t*)emb, tok,
+                 D, V, x, nullptr));
     return LS_OK;
 }
 
@@ -763,8 +760,8 @@ int ls_op_rmsnorm(const float* x, const void* gain, int32_t M, int32_t D, float 
 {
     if (!aligned16(x) || !aligned16(gain) || !aligned16(out) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8)
         return LS_ERR_INVALID_ARG;
-    rmsnorm_kernel<<<M, 256, 0, (cudaStream_t)stream>>>(x, (const uint16_t*)gain, D, eps, (uint16_t*)out, nullptr);
-    LS_CK(cudaGetLastError());
+    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, rmsnorm_kernel, dim3(M), dim3(256), 0, x,
+                 (const uint16_t*)gain, D, eps, (uint16_t*)out, nullptr));
     return LS_OK;
 }
 
@@ -783,7 +780,7 @@ int ls_op_linear(int32_t path, const void* w, const void* h, int32_t M, int32_t 
     LinArgs a = lin_args((const uint16_t*)w, (const uint16_t*)h, M, N, K);
     a.out = out;
     a.ldo = N;
-    LS_CK(launch_linear(path, residual ? EPI_RESIDUAL : EPI_STORE, a, (cudaStream_t)stream));
+    LS_CK(launch_linear(path, residual ? EPI_RESIDUAL : EPI_STORE, a, LaunchCtx{(cudaStream_t)stream, false}));
     return LS_OK;
 }
 
@@ -795,7 +792,7 @@ int ls_op_gate_up_swiglu(int32_t path, const void* wg, const void* wu, const voi
     LinArgs a = lin_args((const uint16_t*)wg, (const uint16_t*)h, M, F, K);
     a.w1 = (const uint16_t*)wu;
     a.out_bf16 = (uint16_t*)out;
-    LS_CK(launch_linear(path, EPI_SWIGLU, a, (cudaStream_t)stream));
+    LS_CK(launch_linear(path, EPI_SWIGLU, a, LaunchCtx{(cudaStream_t)stream, false}));
     return LS_OK;
 }
 
@@ -815,10 +812,10 @@ int ls_op_lm_head_argmax(int32_t path, const void* w, const void* h, int32_t M, 
     a.cand_stride = (V + 15) / 16;
     a.out = logits;
     a.ldo = V;
-    LS_CK(launch_linear(path, EPI_ARGMAX, a, (cudaStream_t)stream));
-    argmax_finish_kernel<<<M, 256, 0, (cudaStream_t)stream>>>(a.cand, lin_grid(EPI_ARGMAX, V), a.cand_stride, tok,
-                                                              nullptr);
-    LS_CK(cudaGetLastError());
+    const LaunchCtx lc = {(cudaStream_t)stream, false};
+    LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
+    LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, lin_grid(EPI_ARGMAX, V), a.cand_stride, tok,
+                 nullptr));
     return LS_OK;
 }
 
@@ -861,10 +858,10 @@ int ls_op_lm_head_argmax_static(int32_t path, const void* w, const void* h, int3
     a.cand = (ValIdx*)scratch;
     a.cand_stride = (V + 15) / 16;
     a.ldo = V;
-    LS_CK(launch_linear(path, EPI_ARGMAX, a, (cudaStream_t)stream));
-    argmax_finish_kernel<<<M, 256, 0, (cudaStream_t)stream>>>(a.cand, lin_grid(EPI_ARGMAX, V), a.cand_stride, tok,
-                                                              nullptr);
-    LS_CK(cudaGetLastError());
+    const LaunchCtx lc = {(cudaStream_t)stream, false};
+    LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
+    LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, lin_grid(EPI_ARGMAX, V), a.cand_stride, tok,
+                 nullptr));
     return LS_OK;
 }
 
@@ -882,10 +879,9 @@ int ls_op_rope_append(const float* qkv, int32_t M, int32_t pos0, int32_t Hq, int
 {
     LS_TRY(kv_check(M, pos0, Hq, Hkv, hd, page_size, max_seq));
     if (!qkv || !page_table || !q_out || !aligned16(kp) || !aligned16(vp) || !(theta > 0.f)) return LS_ERR_INVALID_ARG;
-    rope_append_kernel<<<dim3(M, Hq + 2 * Hkv), hd / 2, 0, (cudaStream_t)stream>>>(
-        qkv, Hq, Hkv, hd, nullptr, theta, log2_exact(page_size), page_table, max_seq, (uint16_t*)q_out,
-        (uint16_t*)kp, (uint16_t*)vp, nullptr, pos0);
-    LS_CK(cudaGetLastError());
+    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, rope_append_kernel, dim3(M, Hq + 2 * Hkv), dim3(hd / 2), 0, qkv,
+                 Hq, Hkv, hd, nullptr, theta, log2_exact(page_size), page_table, max_seq, (uint16_t*)q_out, (uint16_t*)kp,
+                 (uint16_t*)vp, nullptr, pos0));
     return LS_OK;
 }
 
@@ -908,15 +904,15 @@ int ls_op_attention(const void* q, int32_t M, int32_t pos0, int32_t Hq, int32_t 
     const int chunks = (pos0 + M + kAttnChunk - 1) / kAttnChunk;
     return attn_launch((const uint16_t*)q, (const uint16_t*)kp, (const uint16_t*)vp, page_table, nullptr, pos0, M, Hq,
                        Hkv, hd, log2_exact(page_size), max_seq, cap, chunks, (float*)scratch, (uint16_t*)out,
-                       (cudaStream_t)stream);
+                       LaunchCtx{(cudaStream_t)stream, false});
 }
 
 int ls_op_accept(const int32_t* draft, const int32_t* verified, int32_t d, int32_t* state, int32_t* out_ids,
                  int32_t* accepted, void* stream)
 {
     if (!draft || !verified || !state || !out_ids || !accepted || d < 0 || d >= LS_MAX_ROWS) return LS_ERR_INVALID_ARG;
-    accept_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(draft, verified, d, state, out_ids, accepted);
-    LS_CK(cudaGetLastError());
+    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, accept_kernel, dim3(1), dim3(32), 0, draft, verified, d, state,
+                 out_ids, accepted));
     return LS_OK;
 }
 

@@ -12,6 +12,8 @@ namespace ls {
 // position of row 0 of this pass: the loop's cache length plus a per-launch offset
 __device__ __forceinline__ bool pass_begin(const int32_t* ctl, int pos_off, int& pos0)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (ctl) {
         if (ctl[CTL_DONE]) return false;
         pos0 = ctl[CTL_CACHE_LEN] + pos_off;
@@ -27,6 +29,8 @@ __global__ void __launch_bounds__(256)
 embed_kernel(const uint16_t* __restrict__ emb, const int32_t* __restrict__ tok, int D, int V,
              float* __restrict__ x, int32_t* ctl)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (ctl && ctl[CTL_DONE]) return;
     int m = blockIdx.x;
     int id = tok[m];
@@ -62,6 +66,8 @@ rmsnorm_kernel(const float* __restrict__ x, const uint16_t* __restrict__ g, int 
                uint16_t* __restrict__ out, const int32_t* ctl)
 {
     __shared__ float red[8];
+    pdl_launch_dependents();
+    pdl_wait();
     if (ctl && ctl[CTL_DONE]) return;
     int m = blockIdx.x;
     const float4* xr = reinterpret_cast<const float4*>(x + (size_t)m * D);
@@ -91,6 +97,8 @@ rmsnorm_kernel(const float* __restrict__ x, const uint16_t* __restrict__ g, int 
 __global__ void __launch_bounds__(256)
 copy_rows_kernel(const float* __restrict__ src, float* __restrict__ dst, int D, const int32_t* ctl)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (ctl && ctl[CTL_DONE]) return;
     const float4* s = reinterpret_cast<const float4*>(src + (size_t)blockIdx.x * D);
     float4* d = reinterpret_cast<float4*>(dst + (size_t)blockIdx.x * D);
@@ -356,6 +364,8 @@ argmax_finish_kernel(const ValIdx* __restrict__ cand, int n_cand, int cand_strid
 {
     __shared__ float sv[256];
     __shared__ int si[256];
+    pdl_launch_dependents();
+    pdl_wait();
     if (ctl && ctl[CTL_DONE]) return;
     int m = blockIdx.x;
     const ValIdx* c = cand + (size_t)m * cand_stride;
@@ -392,6 +402,8 @@ __global__ void accept_kernel(const int32_t* __restrict__ draft, const int32_t* 
                               int d, int32_t* ctl, int32_t* __restrict__ out_ids,
                               int32_t* __restrict__ accepted)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     if (ctl[CTL_DONE]) return;
     int n = 0;

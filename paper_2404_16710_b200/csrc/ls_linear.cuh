@@ -58,6 +58,8 @@ __device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.0f +
 template <int MT, int EPI>
 __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (a.ctl && a.ctl[CTL_DONE]) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint16_t* rp[4];
@@ -235,7 +237,7 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
 {
     constexpr int T = WARPS * 32;
     extern __shared__ __align__(16) unsigned char ring[];
-    if (a.ctl && a.ctl[CTL_DONE]) return;
+    pdl_launch_dependents();
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const uint16_t *pa, *pb;
@@ -256,17 +258,23 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
     auto slot = [&](int r, int s) { return ring0 + (uint32_t)((r * STAGES + s) * T) * 16u; };
 
     const int nsteps = (a.K + 31) >> 5;
-    auto issue = [&](int step, int s) {
+    auto issue_w = [&](int step, int s) {  // weights: immutable, may be fetched before pdl_wait()
         if (step < nsteps) {
             const int k = step * 32 + 8 * t;
             const int nb = (k < a.K) ? 16 : 0;
             const int kk = (k < a.K) ? k : 0;
             cp_async16_cg(slot(0, s), pa + kk, nb);
             cp_async16_cg(slot(1, s), pb + kk, nb);
+        }
+    };
+    auto issue_h = [&](int step, int s) {  // activations: written by the previous kernel
+        if (step < nsteps) {
+            const int k = step * 32 + 8 * t;
+            const int nb = (k < a.K) ? 16 : 0;
+            const int kk = (k < a.K) ? k : 0;
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) cp_async16_ca(slot(2 + nt, s), hb[nt] + kk, nb);
         }
-        cp_async_commit();
     };
 
     float c[NT][4];
@@ -275,11 +283,25 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
 #pragma unroll
         for (int i = 0; i < 4; ++i) c[nt][i] = 0.f;
 
+    // the first STAGES-1 steps of weights are on their way while the predecessor finishes
 #pragma unroll
-    for (int p = 0; p < STAGES - 1; ++p) issue(warp + p * WARPS, p);
+    for (int p = 0; p < STAGES - 1; ++p) issue_w(warp + p * WARPS, p);
+    pdl_wait();
+    if (a.ctl && a.ctl[CTL_DONE]) {
+        cp_async_commit();
+        cp_async_wait<0>();
+        return;
+    }
+#pragma unroll
+    for (int p = 0; p < STAGES - 1; ++p) {
+        issue_h(warp + p * WARPS, p);
+        cp_async_commit();
+    }
     int rd = 0, wr = STAGES - 1;
     for (int step = warp; step < nsteps; step += WARPS) {
-        issue(step + (STAGES - 1) * WARPS, wr);
+        issue_w(step + (STAGES - 1) * WARPS, wr);
+        issue_h(step + (STAGES - 1) * WARPS, wr);
+        cp_async_commit();
         cp_async_wait<STAGES - 1>();
         const uint4 A0 = lds16(slot(0, rd)), A1 = lds16(slot(1, rd));
 #pragma unroll
@@ -366,15 +388,14 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
 inline int lin_grid(int epi, int N) { return epi == EPI_SWIGLU ? (N + 7) / 8 : (N + 15) / 16; }
 
 template <int EPI>
-inline cudaError_t launch_linear_fma(const LinArgs& a, cudaStream_t st)
+inline cudaError_t launch_linear_fma(const LinArgs& a, const LaunchCtx& lc)
 {
     dim3 grid(lin_grid(EPI, a.N)), block(128);
-    if (a.M <= 1) linear_fma_kernel<1, EPI><<<grid, block, 0, st>>>(a);
-    else if (a.M <= 2) linear_fma_kernel<2, EPI><<<grid, block, 0, st>>>(a);
-    else if (a.M <= 4) linear_fma_kernel<4, EPI><<<grid, block, 0, st>>>(a);
-    else if (a.M <= 8) linear_fma_kernel<8, EPI><<<grid, block, 0, st>>>(a);
-    else linear_fma_kernel<16, EPI><<<grid, block, 0, st>>>(a);
-    return cudaGetLastError();
+    if (a.M <= 1) return launch(lc, linear_fma_kernel<1, EPI>, grid, block, 0, a);
+    if (a.M <= 2) return launch(lc, linear_fma_kernel<2, EPI>, grid, block, 0, a);
+    if (a.M <= 4) return launch(lc, linear_fma_kernel<4, EPI>, grid, block, 0, a);
+    if (a.M <= 8) return launch(lc, linear_fma_kernel<8, EPI>, grid, block, 0, a);
+    return launch(lc, linear_fma_kernel<16, EPI>, grid, block, 0, a);
 }
 
 // Warps per 16-row tile and ring depth, from the matrix shape alone: many row tiles ->
@@ -387,7 +408,7 @@ inline bool mma_wide(int epi, int N, int K)
 }
 
 template <int NT, int EPI, int WARPS, int STAGES>
-inline cudaError_t launch_linear_mma_cfg(const LinArgs& a, cudaStream_t st)
+inline cudaError_t launch_linear_mma_cfg(const LinArgs& a, const LaunchCtx& lc)
 {
     constexpr size_t smem = mma_ring_bytes<NT, WARPS, STAGES>();
     static bool allowed[64] = {false};  // per instantiation and device: the attribute is set once
@@ -400,20 +421,19 @@ inline cudaError_t launch_linear_mma_cfg(const LinArgs& a, cudaStream_t st)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) allowed[dev] = true;
     }
-    linear_mma_kernel<NT, EPI, WARPS, STAGES><<<lin_grid(EPI, a.N), WARPS * 32, smem, st>>>(a);
-    return cudaGetLastError();
+    return launch(lc, linear_mma_kernel<NT, EPI, WARPS, STAGES>, dim3(lin_grid(EPI, a.N)), dim3(WARPS * 32), smem, a);
 }
 
 template <int EPI>
-inline cudaError_t launch_linear_mma(const LinArgs& a, cudaStream_t st)
+inline cudaError_t launch_linear_mma(const LinArgs& a, const LaunchCtx& lc)
 {
     if (mma_wide(EPI, a.N, a.K))
-        return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 16, 4>(a, st) : launch_linear_mma_cfg<2, EPI, 16, 4>(a, st);
-    return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 8, 6>(a, st) : launch_linear_mma_cfg<2, EPI, 8, 6>(a, st);
+        return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 16, 4>(a, lc) : launch_linear_mma_cfg<2, EPI, 16, 4>(a, lc);
+    return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 8, 6>(a, lc) : launch_linear_mma_cfg<2, EPI, 8, 6>(a, lc);
 }
 
 // path: 1 = FMA, 2 = MMA
-inline cudaError_t launch_linear(int path, int epi, const LinArgs& a, cudaStream_t st)
+inline cudaError_t launch_linear(int path, int epi, const LinArgs& a, const LaunchCtx& st)
 {
     if (path == 1) {
         switch (epi) {
