@@ -222,10 +222,20 @@ int ls_op_rope_append(const float *qkv_dev, int32_t M, int32_t pos0, int32_t Hq,
                       int32_t max_seq, void *q_out_bf16_dev, void *k_pages_dev, void *v_pages_dev,
                       void *cuda_stream);
 
+/* The same, fused behind the q|k|v projection (what the decode loop runs): q, k, v =
+ * W_q h, W_k h, W_v h for M rows of h (bf16 [M,K]; wq [Hq*hd,K], wk/wv [Hkv*hd,K]), then
+ * rotary embedding and cache append as in ls_op_rope_append, with no fp32 round trip. */
+int ls_op_qkv_rope_append(int32_t linear_path, const void *wq_dev, const void *wk_dev, const void *wv_dev,
+                          const void *h_bf16_dev, int32_t M, int32_t K, int32_t pos0, int32_t Hq,
+                          int32_t Hkv, int32_t hd, float rope_theta, int32_t page_size,
+                          const int32_t *page_table_dev, int32_t max_seq, void *q_out_bf16_dev,
+                          void *k_pages_dev, void *v_pages_dev, void *cuda_stream);
+
 /* Causal attention of rows m at positions pos0+m over cache positions 0..pos0+m, with
  * grouped KV heads (query head i reads KV head i / (Hq/Hkv)).  q bf16 [M, Hq*hd];
  * out bf16 [M, Hq*hd].  The cache is split into fixed chunks of absolute positions
- * whose partial (max, sum, weighted values) are merged in chunk order.
+ * whose partial (max, sum, weighted values) are merged in chunk order by the
+ * CTA that finishes last (a counter in the scratch area; nothing waits).
  * scratch_dev: ls_op_attention_scratch_bytes(...) bytes. */
 size_t ls_op_attention_scratch_bytes(int32_t Hq, int32_t hd, int32_t max_seq);
 int ls_op_attention(const void *q_bf16_dev, int32_t M, int32_t pos0, int32_t Hq, int32_t Hkv,

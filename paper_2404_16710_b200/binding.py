@@ -26,7 +26,7 @@ EXPORTS = (
     "ls_set_page_table", "ls_generate", "ls_generate_full", "ls_generate_early", "ls_prefill",
     "ls_decode", "ls_read_output", "ls_debug_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
     "ls_op_linear", "ls_op_gate_up_swiglu", "ls_op_lm_head_scratch_bytes", "ls_op_lm_head_argmax",
-    "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_attention_scratch_bytes", "ls_op_attention", "ls_op_accept",
+    "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_qkv_rope_append", "ls_op_attention_scratch_bytes", "ls_op_attention", "ls_op_accept",
 )
 
 
@@ -97,6 +97,8 @@ def lib():
             "ls_op_lm_head_argmax": (C.c_int, [i32, vp, vp, i32, i32, i32, vp, vp, vp, vp]),
             "ls_op_lm_head_argmax_static": (C.c_int, [i32, vp, vp, i32, i32, i32, vp, vp]),
             "ls_op_rope_append": (C.c_int, [vp, i32, i32, i32, i32, i32, C.c_float, i32, vp, i32, vp, vp, vp, vp]),
+            "ls_op_qkv_rope_append": (C.c_int, [i32, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, C.c_float, i32, vp, i32,
+                                                vp, vp, vp, vp]),
             "ls_op_attention_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
             "ls_op_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]),
             "ls_op_accept": (C.c_int, [vp, vp, i32, vp, vp, vp, vp]),
@@ -279,6 +281,14 @@ def ls_op_lm_head_argmax_static(path, w, h, tok):
 def ls_op_rope_append(qkv, pos0, Hq, Hkv, hd, theta, page_size, page_table, max_seq, q_out, k_pages, v_pages):
     _ck(lib().ls_op_rope_append(_dev(qkv), qkv.shape[0], pos0, Hq, Hkv, hd, theta, page_size, _dev(page_table),
                                 max_seq, _dev(q_out), _dev(k_pages), _dev(v_pages), _stream()), "ls_op_rope_append")
+
+
+def ls_op_qkv_rope_append(path, wq, wk, wv, h, pos0, Hq, Hkv, hd, theta, page_size, page_table, max_seq, q_out,
+                          k_pages, v_pages):
+    M, K = h.shape
+    _ck(lib().ls_op_qkv_rope_append(path, _dev(wq), _dev(wk), _dev(wv), _dev(h), M, K, pos0, Hq, Hkv, hd, theta,
+                                    page_size, _dev(page_table), max_seq, _dev(q_out), _dev(k_pages), _dev(v_pages),
+                                    _stream()), "ls_op_qkv_rope_append")
 
 
 def ls_op_attention_scratch_bytes(Hq, hd, max_seq):

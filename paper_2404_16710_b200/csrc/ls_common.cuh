@@ -57,6 +57,29 @@ __device__ __forceinline__ uint4 ld_reuse16(const void* p)
     return v;
 }
 
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead.
+// .cg: L2 only (streamed weights); .ca: also L1 (activations, re-read by every CTA).
+__device__ __forceinline__ void cp_async16_cg(uint32_t dst, const void* src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async16_ca(uint32_t dst, const void* src, int src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds16(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
 // Programmatic dependent launch: a kernel launched with the attribute may start while its
 // predecessor on the stream is still running.  pdl_wait() blocks until the predecessor
 // grid has completed and its writes are visible; before it, a kernel may touch only

@@ -85,7 +85,7 @@ struct ls_model {
     // workspace
     uint16_t *kpages, *vpages;
     size_t layer_kv_elems;
-    int32_t *page_table, *ctl, *draft, *verified, *out_ids, *accepted, *ids;
+    int32_t *page_table, *ctl, *draft, *verified, *out_ids, *accepted, *ids, *attn_counters;
     float *inv_freq, *x, *qkv, *part, *logits;
     uint16_t *h, *q, *o, *a;
     ValIdx* cand;
@@ -133,7 +133,8 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     unsigned char* ids = take(sizeof(int32_t) * c.max_seq);
     unsigned char* x = take(sizeof(float) * kMaxRows * c.d_model);
     unsigned char* qkv = take(sizeof(float) * kMaxRows * (qw + 2 * kvw));
-    unsigned char* part = take(sizeof(float) * kMaxRows * c.n_heads * chunk_cap * (c.head_dim + 2));
+    unsigned char* part = take(sizeof(float) * kMaxRows * c.n_heads * chunk_cap * attn_part_pitch(c.head_dim));
+    unsigned char* actr = take(sizeof(int32_t) * c.n_kv_heads);
     unsigned char* logits = take(sizeof(float) * kMaxRows * c.vocab);
     unsigned char* h = take(2 * (size_t)kMaxRows * c.d_model);
     unsigned char* q = take(2 * (size_t)kMaxRows * qw);
@@ -155,6 +156,7 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
         m->x = (float*)x;
         m->qkv = (float*)qkv;
         m->part = (float*)part;
+        m->attn_counters = (int32_t*)actr;
         m->logits = (float*)logits;
         m->h = (uint16_t*)h;
         m->q = (uint16_t*)q;
@@ -172,19 +174,17 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
 // ------------------------------------------------------------------ kernel launch helpers
 int attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
                 int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int hd, int page_shift,
-                int max_seq, int chunk_cap, int grid_chunks, float* part, uint16_t* out,
+                int max_seq, int chunk_cap, int grid_chunks, float* part, int32_t* counters, uint16_t* out,
                 const LaunchCtx& lc)
 {
     const int Q = Hq / Hkv * M;
-    dim3 grid(grid_chunks, Hkv), mgrid(M, Hq);
+    dim3 grid(grid_chunks, Hkv);
     if (hd == 128) {
-        LS_CK(launch(lc, attn_chunk_kernel<128>, grid, dim3(128), attn_smem_bytes<128>(Q), q, kp, vp, pt, ctl,
-                     pos_off, M, Hq, Hkv, page_shift, max_seq, chunk_cap, part));
-        LS_CK(launch(lc, attn_merge_kernel<128>, mgrid, dim3(128), 0, part, ctl, pos_off, Hq, chunk_cap, out));
+        LS_CK(launch(lc, attn_kernel<128>, grid, dim3(128), attn_smem_bytes<128>(Q), q, kp, vp, pt, ctl, pos_off, M,
+                     Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out));
     } else {
-        LS_CK(launch(lc, attn_chunk_kernel<64>, grid, dim3(128), attn_smem_bytes<64>(Q), q, kp, vp, pt, ctl,
-                     pos_off, M, Hq, Hkv, page_shift, max_seq, chunk_cap, part));
-        LS_CK(launch(lc, attn_merge_kernel<64>, mgrid, dim3(64), 0, part, ctl, pos_off, Hq, chunk_cap, out));
+        LS_CK(launch(lc, attn_kernel<64>, grid, dim3(128), attn_smem_bytes<64>(Q), q, kp, vp, pt, ctl, pos_off, M,
+                     Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out));
     }
     return LS_OK;
 }
@@ -193,10 +193,10 @@ int attn_allow_smem(int hd, int group)
 {
     const int Q = group * kMaxRows;
     if (hd == 128) {
-        LS_CK(cudaFuncSetAttribute(attn_chunk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        LS_CK(cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)attn_smem_bytes<128>(Q)));
     } else {
-        LS_CK(cudaFuncSetAttribute(attn_chunk_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        LS_CK(cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)attn_smem_bytes<64>(Q)));
     }
     return LS_OK;
@@ -233,14 +233,22 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
         a.w2 = w.wv;
         a.n0 = qw;
         a.n1 = kvw;
-        a.out = m->qkv;
-        a.ldo = qw + 2 * kvw;
         a.ctl = m->ctl;
-        LS_CK(launch_linear(m->path, EPI_STORE, a, st));
-        LS_CK(launch(st, rope_append_kernel, dim3(M, Hq + 2 * Hkv), dim3(hd / 2), 0, m->qkv, Hq, Hkv, hd, m->inv_freq,
-                     c.rope_theta, m->page_shift, m->page_table, c.max_seq, m->q, kp, vp, m->ctl, pos_off));
+        a.inv_freq = m->inv_freq;
+        a.page_table = m->page_table;
+        a.q_out = m->q;
+        a.kpages = kp;
+        a.vpages = vp;
+        a.Hq = Hq;
+        a.Hkv = Hkv;
+        a.hd = hd;
+        a.page_shift = m->page_shift;
+        a.max_seq = c.max_seq;
+        a.pos_off = pos_off;
+        a.theta = c.rope_theta;
+        LS_CK(launch_linear(m->path, EPI_QKV, a, st));
         LS_TRY(attn_launch(m->q, kp, vp, m->page_table, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift,
-                           c.max_seq, m->chunk_cap, m->grid_chunks, m->part, m->o, st));
+                           c.max_seq, m->chunk_cap, m->grid_chunks, m->part, m->attn_counters, m->o, st));
         a = lin_args(w.wo, m->o, M, D, qw);
         a.out = xrow;
         a.ldo = D;
@@ -257,7 +265,7 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
         a.ldo = D;
         a.ctl = m->ctl;
         LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
-        m->launches += 9;
+        m->launches += 7;
     }
     LS_CK(cudaGetLastError());
     return LS_OK;
@@ -885,11 +893,41 @@ int ls_op_rope_append(const float* qkv, int32_t M, int32_t pos0, int32_t Hq, int
     return LS_OK;
 }
 
+int ls_op_qkv_rope_append(int32_t path, const void* wq, const void* wk, const void* wv, const void* h, int32_t M,
+                          int32_t K, int32_t pos0, int32_t Hq, int32_t Hkv, int32_t hd, float theta, int32_t page_size,
+                          const int32_t* page_table, int32_t max_seq, void* q_out, void* kp, void* vp, void* stream)
+{
+    LS_TRY(kv_check(M, pos0, Hq, Hkv, hd, page_size, max_seq));
+    LS_TRY(lin_check(path, wq, h, M, (Hq + 2 * Hkv) * hd, K));
+    if (!aligned16(wk) || !aligned16(wv) || !page_table || !q_out || !aligned16(kp) || !aligned16(vp) || !(theta > 0.f))
+        return LS_ERR_INVALID_ARG;
+    LinArgs a = lin_args((const uint16_t*)wq, (const uint16_t*)h, M, (Hq + 2 * Hkv) * hd, K);
+    a.w1 = (const uint16_t*)wk;
+    a.w2 = (const uint16_t*)wv;
+    a.n0 = Hq * hd;
+    a.n1 = Hkv * hd;
+    a.page_table = page_table;
+    a.q_out = (uint16_t*)q_out;
+    a.kpages = (uint16_t*)kp;
+    a.vpages = (uint16_t*)vp;
+    a.Hq = Hq;
+    a.Hkv = Hkv;
+    a.hd = hd;
+    a.page_shift = log2_exact(page_size);
+    a.max_seq = max_seq;
+    a.pos_off = pos0;
+    a.theta = theta;
+    LS_CK(launch_linear(path, EPI_QKV, a, LaunchCtx{(cudaStream_t)stream, false}));
+    return LS_OK;
+}
+
 size_t ls_op_attention_scratch_bytes(int32_t Hq, int32_t hd, int32_t max_seq)
 {
     if (Hq < 1 || hd < 1 || max_seq < 1) return 0;
     size_t cap = (size_t)(max_seq + kAttnChunk - 1) / kAttnChunk;
-    return sizeof(float) * LS_MAX_ROWS * (size_t)Hq * cap * (size_t)(hd + 2);
+    // chunk partials, then one counter per KV head (at most Hq of them)
+    return align_up(sizeof(float) * LS_MAX_ROWS * (size_t)Hq * cap * (size_t)attn_part_pitch(hd), 256) +
+           align_up(sizeof(int32_t) * (size_t)Hq, 256);
 }
 
 int ls_op_attention(const void* q, int32_t M, int32_t pos0, int32_t Hq, int32_t Hkv, int32_t hd, int32_t page_size,
@@ -902,8 +940,11 @@ int ls_op_attention(const void* q, int32_t M, int32_t pos0, int32_t Hq, int32_t 
     LS_TRY(attn_allow_smem(hd, Hq / Hkv));
     const int cap = (max_seq + kAttnChunk - 1) / kAttnChunk;
     const int chunks = (pos0 + M + kAttnChunk - 1) / kAttnChunk;
+    const size_t part_bytes = align_up(sizeof(float) * LS_MAX_ROWS * (size_t)Hq * cap * (size_t)attn_part_pitch(hd), 256);
+    int32_t* counters = (int32_t*)((unsigned char*)scratch + part_bytes);
+    LS_CK(cudaMemsetAsync(counters, 0, sizeof(int32_t) * Hkv, (cudaStream_t)stream));
     return attn_launch((const uint16_t*)q, (const uint16_t*)kp, (const uint16_t*)vp, page_table, nullptr, pos0, M, Hq,
-                       Hkv, hd, log2_exact(page_size), max_seq, cap, chunks, (float*)scratch, (uint16_t*)out,
+                       Hkv, hd, log2_exact(page_size), max_seq, cap, chunks, (float*)scratch, counters, (uint16_t*)out,
                        LaunchCtx{(cudaStream_t)stream, false});
 }
 

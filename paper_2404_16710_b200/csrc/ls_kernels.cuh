@@ -157,10 +157,13 @@ __global__ void rope_append_kernel(const float* __restrict__ qkv, int Hq, int Hk
     dst[j + half] = f2bf(b);
 }
 
-// ------------------------------------------------------------------ attention, one chunk of keys
+// ------------------------------------------------------------------ attention
 // grid (chunks, Hkv), block 128.  CTA = keys [64*ch, 64*ch + 64) of KV head kh, all
-// G = Hq/Hkv query heads of the group, all M rows.  Writes, per (row, head, chunk),
-// the un-normalised partial (o[HD], max, sum).  Row m at position pos0+m sees keys <= pos0+m.
+// G = Hq/Hkv query heads of the group, all M rows.  Row m at position pos0+m sees keys
+// <= pos0+m.  Every CTA writes, per (row, head, chunk), the un-normalised partial
+// (o[HD], max, sum); the CTA that finishes last for its KV head (a counter, no waiting)
+// merges the chunks of that head's queries IN CHUNK ORDER and writes the bf16 output.
+// Chunks are cut by absolute position, so a row's result depends on its position only.
 //
 // shared memory: Ks [64][HD*2+16 B] | Vs [64][HD*2 B] | Qs f32 [Q][HD] | Sp f32 [2][Q][64]
 //                | P f32 [Q][64] | Ored f32 [NKS][4][HD]
@@ -170,25 +173,29 @@ __host__ __device__ constexpr size_t attn_smem_bytes(int Q)
     return (size_t)kAttnChunk * (HD * 2 + 16) + (size_t)kAttnChunk * HD * 2 +
            sizeof(float) * ((size_t)Q * HD + 3 * (size_t)Q * kAttnChunk + (size_t)(128 / (HD / 2)) * 4 * HD);
 }
+// floats per (row, head, chunk) partial: o[HD], max, sum, 2 of padding (16-byte rows)
+__host__ __device__ constexpr int attn_part_pitch(int hd) { return hd + 4; }
 
 template <int HD>
 __global__ void __launch_bounds__(128)
-attn_chunk_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
-                  const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table,
-                  int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift,
-                  int max_seq, int chunk_cap, float* __restrict__ part)
+attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
+            const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table,
+            int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift,
+            int max_seq, int chunk_cap, float* part, int32_t* counters, uint16_t* __restrict__ out)
 {
     constexpr int C = kAttnChunk;
     constexpr int KROW = HD * 2 + 16;        // padded K row, bytes
     constexpr int NKS = 128 / (HD / 2);      // key slices in the P.V phase
     constexpr int HALF = HD / 2;
+    constexpr int PP = attn_part_pitch(HD);
     int pos0;
     if (!pass_begin(ctl, pos_off, pos0)) return;
     const int ch = blockIdx.x, kh = blockIdx.y, tid = threadIdx.x;
     const int last_pos = pos0 + M - 1;
     const int key0 = ch * C;
     if (key0 > last_pos) return;
-    if (last_pos >= max_seq || pos0 < 0 || ch >= chunk_cap) {
+    const int n_active = last_pos / C + 1;  // CTAs of this KV head that take part
+    if (last_pos >= max_seq || pos0 < 0 || n_active > chunk_cap || n_active > (int)gridDim.x) {
         if (ctl && tid == 0) ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
         return;
     }
@@ -202,19 +209,20 @@ attn_chunk_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k
     float* P = Sp + 2 * (size_t)Q * C;
     float* Ored = P + (size_t)Q * C;
 
-    // stage K and V rows of the chunk (zero beyond the last visible key)
-    constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
-    for (int idx = tid; idx < C * SEGS; idx += 128) {
-        int r = idx / SEGS, sg = idx % SEGS;
-        int p = key0 + r;
-        uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
-        if (p <= last_pos) {
-            size_t off = kv_row_offset(page_table, p, page_shift, Hkv, kh, HD) + (size_t)sg * 8;
-            kv = *reinterpret_cast<const uint4*>(kpages + off);
-            vv = *reinterpret_cast<const uint4*>(vpages + off);
+    // stage K and V rows of the chunk (zeros beyond the last visible key): asynchronous
+    // copies, all in flight at once
+    {
+        constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
+        const uint32_t ks0 = (uint32_t)__cvta_generic_to_shared(Ks), vs0 = (uint32_t)__cvta_generic_to_shared(Vs);
+        for (int idx = tid; idx < C * SEGS; idx += 128) {
+            const int r = idx / SEGS, sg = idx % SEGS;
+            const int p = key0 + r;
+            const bool ok = p <= last_pos;
+            const size_t off = kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD) + (size_t)sg * 8;
+            cp_async16_cg(ks0 + r * KROW + sg * 16, kpages + off, ok ? 16 : 0);
+            cp_async16_cg(vs0 + r * HD * 2 + sg * 16, vpages + off, ok ? 16 : 0);
         }
-        *reinterpret_cast<uint4*>(Ks + r * KROW + sg * 16) = kv;
-        *reinterpret_cast<uint4*>(Vs + r * HD * 2 + sg * 16) = vv;
+        cp_async_commit();
     }
     // queries of this group -> fp32
     for (int idx = tid; idx < Q * HALF; idx += 128) {
@@ -224,6 +232,7 @@ attn_chunk_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k
         Qs[qi * HD + 2 * dp] = bf16lo(u);
         Qs[qi * HD + 2 * dp + 1] = bf16hi(u);
     }
+    cp_async_wait<0>();
     __syncthreads();
 
     // phase 1: thread = (key j, half of the dims); partial dot products in groups of 4 queries
@@ -283,7 +292,7 @@ attn_chunk_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k
             P[(size_t)qi * C + lane] = p0;
             P[(size_t)qi * C + lane + 32] = p1;
             if (lane == 0) {
-                float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * (HD + 2);
+                float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP;
                 dst[HD] = mx;
                 dst[HD + 1] = l;
             }
@@ -321,37 +330,70 @@ attn_chunk_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k
 #pragma unroll
                     for (int k2 = 0; k2 < NKS; ++k2) s += Ored[((size_t)k2 * 4 + qq) * HD + dd];
                     int qi = q0 + qq, m = qi / G, g = qi % G;
-                    part[(((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * (HD + 2) + dd] = s;
+                    part[(((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP + dd] = s;
                 }
             }
             __syncthreads();
         }
     }
-}
 
-// merge the chunk partials of one (row, head) in chunk order; grid (M, Hq), block HD
-template <int HD>
-__global__ void __launch_bounds__(HD)
-attn_merge_kernel(const float* __restrict__ part, int32_t* ctl, int pos_off, int Hq, int chunk_cap,
-                  uint16_t* __restrict__ out)
-{
-    int pos0;
-    if (!pass_begin(ctl, pos_off, pos0)) return;
-    int m = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
-    int pos = pos0 + m;
-    int nch = pos / kAttnChunk + 1;
-    if (pos < 0 || nch > chunk_cap) return;  // refused by the chunk kernel (status word set)
-    const float* base = part + ((size_t)m * Hq + h) * chunk_cap * (HD + 2);
-    float mx = -INFINITY;
-    for (int c = 0; c < nch; ++c) mx = fmaxf(mx, base[(size_t)c * (HD + 2) + HD]);
-    float l = 0.f, o = 0.f;
-    for (int c = 0; c < nch; ++c) {
-        const float* pc = base + (size_t)c * (HD + 2);
-        float w = expf(pc[HD] - mx);
-        l = fmaf(pc[HD + 1], w, l);
-        o = fmaf(pc[d], w, o);
+    // who is last for this KV head?  (publish the partials, then count; nobody waits)
+    __shared__ int is_last;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int prev = atomicAdd(&counters[kh], 1);
+        is_last = (prev == n_active - 1);
+        if (is_last) counters[kh] = 0;  // ready for the next launch
     }
-    out[((size_t)m * Hq + h) * HD + d] = f2bf(o / l);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    // ordered merge: one warp per query, lanes over the dims; partials come from L2
+    {
+        constexpr int DPL = HD / 32;  // dims per lane: 4 or 2
+        const int warp = tid >> 5, lane = tid & 31;
+        for (int qi = warp; qi < Q; qi += 4) {
+            const int m = qi / G, h = kh * G + qi % G;
+            const int nch = (pos0 + m) / C + 1;
+            const float* base = part + ((size_t)m * Hq + h) * chunk_cap * PP;
+            float mx = -INFINITY;
+            for (int c = lane; c < nch; c += 32) mx = fmaxf(mx, __ldcg(base + (size_t)c * PP + HD));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            float l = 0.f, o[DPL];
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) o[i] = 0.f;
+#pragma unroll 4
+            for (int c = 0; c < nch; ++c) {
+                const float* pc = base + (size_t)c * PP;
+                const float2 ml = __ldcg(reinterpret_cast<const float2*>(pc + HD));
+                const float w = expf(ml.x - mx);
+                l = fmaf(ml.y, w, l);
+                if (DPL == 4) {
+                    const float4 v = __ldcg(reinterpret_cast<const float4*>(pc + lane * 4));
+                    o[0] = fmaf(v.x, w, o[0]);
+                    o[1] = fmaf(v.y, w, o[1]);
+                    o[DPL - 2] = fmaf(v.z, w, o[DPL - 2]);
+                    o[DPL - 1] = fmaf(v.w, w, o[DPL - 1]);
+                } else {
+                    const float2 v = __ldcg(reinterpret_cast<const float2*>(pc + lane * 2));
+                    o[0] = fmaf(v.x, w, o[0]);
+                    o[1] = fmaf(v.y, w, o[1]);
+                }
+            }
+            uint16_t* dst = out + ((size_t)m * Hq + h) * HD + lane * DPL;
+            if (DPL == 4) {
+                uint2 pk;
+                pk.x = pack_bf16(o[0] / l, o[1] / l);
+                pk.y = pack_bf16(o[DPL - 2] / l, o[DPL - 1] / l);
+                *reinterpret_cast<uint2*>(dst) = pk;
+            } else {
+                *reinterpret_cast<uint32_t*>(dst) = pack_bf16(o[0] / l, o[1] / l);
+            }
+        }
+    }
 }
 
 // ------------------------------------------------------------------ argmax finish

@@ -17,14 +17,15 @@
 // every M, so results are bit-identical across pass sizes within a family.
 //
 // Epilogues: plain store, residual add (x <- x + W h, Sec. 4.1 of the paper), SwiGLU
-// (gate and up rows of one feature meet in one thread), and LM head + argmax candidates
+// (gate and up rows of one feature meet in one thread), q|k|v with rotary embedding and
+// KV append (the two halves of a rotary pair meet in one thread), LM head + argmax candidates
 // (Sec. 2.1 / 4.2: the shared head g; greedy decoding needs only the index).
 #pragma once
 #include "ls_kernels.cuh"
 
 namespace ls {
 
-enum Epi : int { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_ARGMAX = 3 };
+enum Epi : int { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_ARGMAX = 3, EPI_QKV = 4 };
 
 struct LinArgs {
     const uint16_t* w0;  // row segments: rows [0, n0) of w0, then n1 rows of w1, the rest of w2
@@ -38,8 +39,47 @@ struct LinArgs {
     uint16_t* out_bf16;  // SwiGLU result [M][N]
     ValIdx* cand;        // argmax candidates [M][cand_stride], one per CTA
     int cand_stride;
-    const int32_t* ctl;
+    int32_t* ctl;
+    // EPI_QKV: rotary embedding + KV append fused behind the q|k|v projection
+    const float* inv_freq;       // [hd/2], or nullptr: theta^(-2j/hd) computed in place
+    const int32_t* page_table;
+    uint16_t *q_out, *kpages, *vpages;
+    int Hq, Hkv, hd, page_shift, max_seq, pos_off;
+    float theta;
 };
+
+// EPI_QKV tiles pair row j of a head with row j + hd/2, the two halves of one rotary pair:
+// tile b covers pairs j = 8 (b % (hd/16)) .. +7 of head b / (hd/16).
+__device__ __forceinline__ int qkv_row(const LinArgs& a, int tile, int pair, int hi)
+{
+    const int tph = a.hd >> 4;
+    return (tile / tph) * a.hd + (tile % tph) * 8 + pair + (hi ? (a.hd >> 1) : 0);
+}
+
+// rotate the pair (x_j, x_{j+hd/2}) of head `head` for token m and store it: q -> q_out,
+// k, v -> the paged cache row of position pos0 + m (v is not rotated)
+__device__ __forceinline__ void qkv_store(const LinArgs& a, int head, int j, int m, int pos0, float lo, float hi)
+{
+    const int pos = pos0 + m;
+    if (pos < 0 || pos >= a.max_seq) {
+        if (a.ctl) a.ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
+        return;
+    }
+    if (head < a.Hq + a.Hkv) {
+        const float f = a.inv_freq ? a.inv_freq[j] : (float)pow((double)a.theta, -2.0 * (double)j / (double)a.hd);
+        float sn, cs;
+        sincosf((float)pos * f, &sn, &cs);
+        const float r0 = lo * cs - hi * sn, r1 = lo * sn + hi * cs;
+        lo = r0;
+        hi = r1;
+    }
+    uint16_t* dst;
+    if (head < a.Hq) dst = a.q_out + ((size_t)m * a.Hq + head) * a.hd;
+    else if (head < a.Hq + a.Hkv) dst = a.kpages + kv_row_offset(a.page_table, pos, a.page_shift, a.Hkv, head - a.Hq, a.hd);
+    else dst = a.vpages + kv_row_offset(a.page_table, pos, a.page_shift, a.Hkv, head - a.Hq - a.Hkv, a.hd);
+    dst[j] = f2bf(lo);
+    dst[j + (a.hd >> 1)] = f2bf(hi);
+}
 
 __device__ __forceinline__ const uint16_t* weight_row(const LinArgs& a, int n)
 {
@@ -71,6 +111,12 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
             nrow[r] = f + (r & 1);
             int fc = min(nrow[r], a.N - 1);
             rp[r] = ((r < 2) ? a.w0 : a.w1) + (size_t)fc * a.K;
+        }
+    } else if (EPI == EPI_QKV) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            nrow[r] = qkv_row(a, blockIdx.x, warp * 2 + (r & 1), r >> 1);
+            rp[r] = weight_row(a, nrow[r]);
         }
     } else {
 #pragma unroll
@@ -141,6 +187,17 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
                     if (nrow[r] < a.N)
                         a.out_bf16[(size_t)m * a.N + nrow[r]] = f2bf(silu_mul(acc[r][m], acc[r + 2][m]));
             }
+    } else if (EPI == EPI_QKV) {
+        const int pos0 = (a.ctl ? a.ctl[CTL_CACHE_LEN] : 0) + a.pos_off;
+        const int tph = a.hd >> 4;
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (lane == m && m < a.M) {
+#pragma unroll
+                for (int r = 0; r < 2; ++r)
+                    qkv_store(a, blockIdx.x / tph, (blockIdx.x % tph) * 8 + warp * 2 + r, m, pos0, acc[r][m],
+                              acc[r + 2][m]);
+            }
     } else {  // EPI_ARGMAX
         __shared__ float bv[4][MT];
         __shared__ int bi[4][MT];
@@ -191,29 +248,6 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead.
-// .cg: L2 only (streamed weights); .ca: also L1 (activations, re-read by every CTA).
-__device__ __forceinline__ void cp_async16_cg(uint32_t dst, const void* src, int src_bytes)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async16_ca(uint32_t dst, const void* src, int src_bytes)
-{
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait()
-{
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ uint4 lds16(uint32_t addr)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-
 template <int NT, int WARPS, int STAGES>
 constexpr size_t mma_ring_bytes()
 {
@@ -245,6 +279,9 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
         int f = min(blockIdx.x * 8 + g, a.N - 1);
         pa = a.w0 + (size_t)f * a.K;
         pb = a.w1 + (size_t)f * a.K;
+    } else if (EPI == EPI_QKV) {
+        pa = weight_row(a, qkv_row(a, blockIdx.x, g, 0));
+        pb = weight_row(a, qkv_row(a, blockIdx.x, g, 1));
     } else {
         pa = weight_row(a, blockIdx.x * 16 + g);
         pb = weight_row(a, blockIdx.x * 16 + g + 8);
@@ -351,6 +388,12 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
                 if (m0 < a.M) a.out_bf16[(size_t)m0 * a.N + f] = f2bf(silu_mul(r[0], r[2]));
                 if (m0 + 1 < a.M) a.out_bf16[(size_t)(m0 + 1) * a.N + f] = f2bf(silu_mul(r[1], r[3]));
             }
+        } else if (EPI == EPI_QKV) {
+            const int pos0 = (a.ctl ? a.ctl[CTL_CACHE_LEN] : 0) + a.pos_off;
+            const int tph = a.hd >> 4;
+            const int head = blockIdx.x / tph, j = (blockIdx.x % tph) * 8 + gg;
+            if (m0 < a.M) qkv_store(a, head, j, m0, pos0, r[0], r[2]);
+            if (m0 + 1 < a.M) qkv_store(a, head, j, m0 + 1, pos0, r[1], r[3]);
         } else {
             vals[gg][m0] = r[0];
             vals[gg][m0 + 1] = r[1];
@@ -440,6 +483,7 @@ inline cudaError_t launch_linear(int path, int epi, const LinArgs& a, const Laun
             case EPI_STORE: return launch_linear_fma<EPI_STORE>(a, st);
             case EPI_RESIDUAL: return launch_linear_fma<EPI_RESIDUAL>(a, st);
             case EPI_SWIGLU: return launch_linear_fma<EPI_SWIGLU>(a, st);
+            case EPI_QKV: return launch_linear_fma<EPI_QKV>(a, st);
             default: return launch_linear_fma<EPI_ARGMAX>(a, st);
         }
     }
@@ -447,6 +491,7 @@ inline cudaError_t launch_linear(int path, int epi, const LinArgs& a, const Laun
         case EPI_STORE: return launch_linear_mma<EPI_STORE>(a, st);
         case EPI_RESIDUAL: return launch_linear_mma<EPI_RESIDUAL>(a, st);
         case EPI_SWIGLU: return launch_linear_mma<EPI_SWIGLU>(a, st);
+        case EPI_QKV: return launch_linear_mma<EPI_QKV>(a, st);
         default: return launch_linear_mma<EPI_ARGMAX>(a, st);
     }
 }

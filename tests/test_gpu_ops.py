@@ -226,6 +226,37 @@ def test_rope_append(Hq, Hkv, hd, theta, shuffle):
             assert_bf16_close(vc[p, hh * hd:(hh + 1) * hd], ref)
 
 
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("Hq,Hkv,hd,K,M", [(4, 2, 64, 96, 5), (8, 8, 128, 256, 1), (8, 2, 128, 520, 9)])
+def test_qkv_projection_fused_with_rope_and_append(path, Hq, Hkv, hd, K, M):
+    """What the decode loop runs: q|k|v projection, rotary embedding and cache append in one kernel."""
+    pos0, page_size, max_seq, theta = 77, 16, 160, 1e4
+    table, table_d, kp, vp = kv_setup(Hkv, hd, page_size, max_seq, True)
+    wq, wk, wv = (rnd((n, K), 70 + i, 0.05).bfloat16() for i, n in enumerate((Hq * hd, Hkv * hd, Hkv * hd)))
+    h = rnd((M, K), 73).bfloat16()
+    q_out = torch.empty((M, Hq * hd), dtype=torch.bfloat16, device="cuda")
+    B.ls_op_qkv_rope_append(path, wq, wk, wv, h, pos0, Hq, Hkv, hd, theta, page_size, table_d, max_seq, q_out, kp, vp)
+    torch.cuda.synchronize()
+    kc = gather_cache(kp, table, page_size, pos0 + M)
+    vc = gather_cache(vp, table, page_size, pos0 + M)
+    assert not kc[:pos0].any() and not vc[:pos0].any()
+    hv = vals(h)
+    for m in range(M):
+        p = pos0 + m
+        qr, kr, vr = O.linear(bits(wq), hv[m]), O.linear(bits(wk), hv[m]), O.linear(bits(wv), hv[m])
+        for hh in range(Hq):
+            ref = O.rope(qr[hh * hd:(hh + 1) * hd], p, theta)
+            np.testing.assert_allclose(vals(q_out[m, hh * hd:(hh + 1) * hd]), ref, rtol=0,
+                                       atol=(BF16_REL + 1e-4) * np.abs(ref).max())
+        for hh in range(Hkv):
+            ref = O.rope(kr[hh * hd:(hh + 1) * hd], p, theta)
+            np.testing.assert_allclose(kc[p, hh * hd:(hh + 1) * hd], ref, rtol=0,
+                                       atol=(BF16_REL + 1e-4) * np.abs(ref).max())
+            ref = vr[hh * hd:(hh + 1) * hd]
+            np.testing.assert_allclose(vc[p, hh * hd:(hh + 1) * hd], ref, rtol=0,
+                                       atol=(BF16_REL + 1e-5) * np.abs(ref).max())
+
+
 @pytest.mark.parametrize("Hq,Hkv,hd", [(4, 2, 64), (4, 4, 128), (8, 2, 128)])
 @pytest.mark.parametrize("M,pos0", [(1, 0), (1, 63), (1, 64), (4, 61), (7, 130), (16, 300), (3, 1000)])
 def test_attention(Hq, Hkv, hd, M, pos0):
