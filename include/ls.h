@@ -58,7 +58,7 @@ typedef struct ls_config {
     int32_t vocab;       /* V                                                            */
     float rms_eps;
     float rope_theta;
-    int32_t max_seq;     /* KV capacity in tokens: n_prompt + max_new + num_draft + 1    */
+    int32_t max_seq;     /* KV capacity in tokens (<= 16384): n_prompt+max_new+num_draft+1 */
     int32_t page_size;   /* tokens per KV page: power of two, 16..1024                   */
     int32_t max_draft;   /* largest num_draft this model will be asked for (<= 15)       */
     int32_t eos_id;      /* -1: never stop early                                         */

@@ -66,7 +66,7 @@ bool config_ok(const ls_config* c)
     if (c->head_dim != 64 && c->head_dim != 128) return false;
     if (c->n_heads < 1 || c->n_kv_heads < 1 || c->n_heads % c->n_kv_heads) return false;
     if (c->n_heads / c->n_kv_heads > 8) return false;
-    if (c->vocab < 1 || c->max_seq < 2) return false;
+    if (c->vocab < 1 || c->max_seq < 2 || c->max_seq > kAttnChunk * kAttnMaxChunks) return false;
     if (c->page_size < 16 || c->page_size > 1024 || log2_exact(c->page_size) < 0) return false;
     if (c->max_draft < 0 || c->max_draft + 1 > LS_MAX_ROWS) return false;
     if (c->linear_path < 0 || c->linear_path > 2) return false;
@@ -180,10 +180,10 @@ int attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const
     const int Q = Hq / Hkv * M;
     dim3 grid(grid_chunks, Hkv);
     if (hd == 128) {
-        LS_CK(launch(lc, attn_kernel<128>, grid, dim3(128), attn_smem_bytes<128>(Q), q, kp, vp, pt, ctl, pos_off, M,
+        LS_CK(launch(lc, attn_kernel<128>, grid, dim3(kAttnThreads), attn_smem_bytes<128>(Q), q, kp, vp, pt, ctl, pos_off, M,
                      Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out));
     } else {
-        LS_CK(launch(lc, attn_kernel<64>, grid, dim3(128), attn_smem_bytes<64>(Q), q, kp, vp, pt, ctl, pos_off, M,
+        LS_CK(launch(lc, attn_kernel<64>, grid, dim3(kAttnThreads), attn_smem_bytes<64>(Q), q, kp, vp, pt, ctl, pos_off, M,
                      Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out));
     }
     return LS_OK;
@@ -877,7 +877,7 @@ static int kv_check(int M, int pos0, int Hq, int Hkv, int hd, int page_size, int
 {
     if (M < 1 || M > LS_MAX_ROWS || pos0 < 0 || Hq < 1 || Hkv < 1 || Hq % Hkv || Hq / Hkv > 8) return LS_ERR_INVALID_ARG;
     if ((hd != 64 && hd != 128) || page_size < 16 || page_size > 1024 || log2_exact(page_size) < 0) return LS_ERR_INVALID_ARG;
-    if (max_seq < 1 || (int64_t)pos0 + M > max_seq) return LS_ERR_CAPACITY;
+    if (max_seq < 1 || max_seq > kAttnChunk * kAttnMaxChunks || (int64_t)pos0 + M > max_seq) return LS_ERR_CAPACITY;
     return LS_OK;
 }
 

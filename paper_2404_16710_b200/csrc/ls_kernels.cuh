@@ -158,35 +158,114 @@ __global__ void rope_append_kernel(const float* __restrict__ qkv, int Hq, int Hk
 }
 
 // ------------------------------------------------------------------ attention
-// grid (chunks, Hkv), block 128.  CTA = keys [64*ch, 64*ch + 64) of KV head kh, all
+// grid (chunks, Hkv), block 256.  CTA = keys [64*ch, 64*ch + 64) of KV head kh, all
 // G = Hq/Hkv query heads of the group, all M rows.  Row m at position pos0+m sees keys
 // <= pos0+m.  Every CTA writes, per (row, head, chunk), the un-normalised partial
 // (o[HD], max, sum); the CTA that finishes last for its KV head (a counter, no waiting)
 // merges the chunks of that head's queries IN CHUNK ORDER and writes the bf16 output.
 // Chunks are cut by absolute position, so a row's result depends on its position only.
 //
-// shared memory: Ks [64][HD*2+16 B] | Vs [64][HD*2 B] | Qs f32 [Q][HD] | Sp f32 [2][Q][64]
-//                | P f32 [Q][64] | Ored f32 [NKS][4][HD]
+// Work is spread thin on purpose (decode attention is a few MB per layer): four lanes
+// share one key in q.k (each a quarter of the dims, interleaved in 16-byte blocks), NKS
+// lanes share one pair of output dims in p.v (each a slice of the keys); both finish with
+// a fixed shuffle tree.  K and V rows are padded so that these accesses are free of bank
+// conflicts (K pitch = 16 banks mod 32, V pitch = 8 banks mod 32).
+//
+// shared memory: Ks [64][HD*2+64 B] | Vs [64][HD*2+32 B] | Qs f32 [Q][HD] | S f32 [Q][64]
+constexpr int kAttnThreads = 256;
+constexpr int kAttnMaxChunks = 256;  // chunks the merge can hold weights for: max_seq <= 16384
+constexpr int kMergeBatch = 8;       // queries merged together (one warp each)
 template <int HD>
 __host__ __device__ constexpr size_t attn_smem_bytes(int Q)
 {
-    return (size_t)kAttnChunk * (HD * 2 + 16) + (size_t)kAttnChunk * HD * 2 +
-           sizeof(float) * ((size_t)Q * HD + 3 * (size_t)Q * kAttnChunk + (size_t)(128 / (HD / 2)) * 4 * HD);
+    size_t stage = (size_t)kAttnChunk * (HD * 2 + 64) + (size_t)kAttnChunk * (HD * 2 + 32) +
+                   sizeof(float) * ((size_t)Q * HD + (size_t)Q * kAttnChunk);
+    // merge (reuses the same memory): weights and sums [8][256] each, slice sums [4][8 slices][HD]
+    size_t merge = sizeof(float) * (2 * (size_t)kMergeBatch * kAttnMaxChunks + 4 * 8 * (size_t)HD + kMergeBatch);
+    return stage > merge ? stage : merge;
 }
 // floats per (row, head, chunk) partial: o[HD], max, sum, 2 of padding (16-byte rows)
 __host__ __device__ constexpr int attn_part_pitch(int hd) { return hd + 4; }
 
+// scores of QB queries against the thread's key: its quarter of the dims
+template <int HD, int QB>
+__device__ __forceinline__ void attn_qk(const unsigned char* krow, const float* Qs, int q0, int qd, float* S,
+                                        int key, int lane_is_writer)
+{
+    constexpr int NB = HD / 32;  // 16-byte blocks of the key row per lane
+    float acc[QB];
+#pragma unroll
+    for (int qq = 0; qq < QB; ++qq) acc[qq] = 0.f;
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        const int blk = 4 * i + qd;
+        const uint4 kk = *reinterpret_cast<const uint4*>(krow + blk * 16);
+        const float kf[8] = {bf16lo(kk.x), bf16hi(kk.x), bf16lo(kk.y), bf16hi(kk.y),
+                             bf16lo(kk.z), bf16hi(kk.z), bf16lo(kk.w), bf16hi(kk.w)};
+#pragma unroll
+        for (int qq = 0; qq < QB; ++qq) {
+            const float4* qv = reinterpret_cast<const float4*>(Qs + (size_t)(q0 + qq) * HD + blk * 8);
+            const float4 a = qv[0], c = qv[1];
+            float s = acc[qq];
+            s = fmaf(kf[0], a.x, s);
+            s = fmaf(kf[1], a.y, s);
+            s = fmaf(kf[2], a.z, s);
+            s = fmaf(kf[3], a.w, s);
+            s = fmaf(kf[4], c.x, s);
+            s = fmaf(kf[5], c.y, s);
+            s = fmaf(kf[6], c.z, s);
+            s = fmaf(kf[7], c.w, s);
+            acc[qq] = s;
+        }
+    }
+#pragma unroll
+    for (int qq = 0; qq < QB; ++qq) {
+        float s = acc[qq];
+        s += __shfl_xor_sync(0xffffffffu, s, 1);
+        s += __shfl_xor_sync(0xffffffffu, s, 2);
+        if (lane_is_writer) S[(size_t)(q0 + qq) * kAttnChunk + key] = s;
+    }
+}
+
+// weighted values of QB queries for the thread's pair of dims: its slice of the keys
+template <int HD, int QB, int NKS>
+__device__ __forceinline__ void attn_pv(const unsigned char* Vs, const float* P, int q0, int dp, int ks,
+                                        float (&o)[QB][2])
+{
+    constexpr int VROW = HD * 2 + 32;
+#pragma unroll
+    for (int qq = 0; qq < QB; ++qq) o[qq][0] = o[qq][1] = 0.f;
+#pragma unroll 4
+    for (int j = ks; j < kAttnChunk; j += NKS) {
+        const uint32_t u = *reinterpret_cast<const uint32_t*>(Vs + j * VROW + dp * 4);
+        const float v0 = bf16lo(u), v1 = bf16hi(u);
+#pragma unroll
+        for (int qq = 0; qq < QB; ++qq) {
+            const float p = P[(size_t)(q0 + qq) * kAttnChunk + j];
+            o[qq][0] = fmaf(p, v0, o[qq][0]);
+            o[qq][1] = fmaf(p, v1, o[qq][1]);
+        }
+    }
+#pragma unroll
+    for (int qq = 0; qq < QB; ++qq)
+#pragma unroll
+        for (int sh = 1; sh < NKS; sh <<= 1) {
+            o[qq][0] += __shfl_xor_sync(0xffffffffu, o[qq][0], sh);
+            o[qq][1] += __shfl_xor_sync(0xffffffffu, o[qq][1], sh);
+        }
+}
+
 template <int HD>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kAttnThreads)
 attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
             const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table,
             int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift,
             int max_seq, int chunk_cap, float* part, int32_t* counters, uint16_t* __restrict__ out)
 {
-    constexpr int C = kAttnChunk;
-    constexpr int KROW = HD * 2 + 16;        // padded K row, bytes
-    constexpr int NKS = 128 / (HD / 2);      // key slices in the P.V phase
+    constexpr int C = kAttnChunk, T = kAttnThreads;
+    constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 32;
     constexpr int HALF = HD / 2;
+    constexpr int NKS = T / HALF;  // key slices in p.v: 4 (HD 128) or 8 (HD 64)
     constexpr int PP = attn_part_pitch(HD);
     int pos0;
     if (!pass_begin(ctl, pos_off, pos0)) return;
@@ -204,93 +283,93 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* Ks = smem;
     unsigned char* Vs = Ks + C * KROW;
-    float* Qs = reinterpret_cast<float*>(Vs + C * HD * 2);
-    float* Sp = Qs + (size_t)Q * HD;
-    float* P = Sp + 2 * (size_t)Q * C;
-    float* Ored = P + (size_t)Q * C;
+    float* Qs = reinterpret_cast<float*>(Vs + C * VROW);
+    float* S = Qs + (size_t)Q * HD;
 
+    // the group's queries: issue the global loads first, so that they travel together with
+    // the page-table lookup and the K/V copies (each is a round trip of its own otherwise)
+    constexpr int QPT = 4;  // query elements (bf16 pairs) a thread holds per sweep
+    const int nq = Q * HALF;
+    uint32_t qreg[QPT];
+#pragma unroll
+    for (int i = 0; i < QPT; ++i) {
+        const int idx = tid + i * T;
+        if (idx < nq) {
+            const int qi = idx / HALF, dp = idx % HALF;
+            const int m = qi / G, g = qi % G;
+            qreg[i] = *reinterpret_cast<const uint32_t*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + 2 * dp);
+        }
+    }
     // stage K and V rows of the chunk (zeros beyond the last visible key): asynchronous
-    // copies, all in flight at once
+    // copies, all in flight at once; a chunk never straddles a page of 64 tokens or more
     {
         constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
         const uint32_t ks0 = (uint32_t)__cvta_generic_to_shared(Ks), vs0 = (uint32_t)__cvta_generic_to_shared(Vs);
-        for (int idx = tid; idx < C * SEGS; idx += 128) {
+        const bool one_page = page_shift >= 6;
+        const size_t base = one_page ? kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD) : 0;
+#pragma unroll
+        for (int it = 0; it < C * SEGS / T; ++it) {
+            const int idx = tid + it * T;
             const int r = idx / SEGS, sg = idx % SEGS;
             const int p = key0 + r;
             const bool ok = p <= last_pos;
-            const size_t off = kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD) + (size_t)sg * 8;
+            const size_t off = (one_page ? base + (size_t)r * HD
+                                         : kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD)) +
+                               (size_t)sg * 8;
             cp_async16_cg(ks0 + r * KROW + sg * 16, kpages + off, ok ? 16 : 0);
-            cp_async16_cg(vs0 + r * HD * 2 + sg * 16, vpages + off, ok ? 16 : 0);
+            cp_async16_cg(vs0 + r * VROW + sg * 16, vpages + off, ok ? 16 : 0);
         }
         cp_async_commit();
     }
-    // queries of this group -> fp32
-    for (int idx = tid; idx < Q * HALF; idx += 128) {
-        int qi = idx / HALF, dp = idx % HALF;
-        int m = qi / G, g = qi % G;
-        uint32_t u = *reinterpret_cast<const uint32_t*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + 2 * dp);
-        Qs[qi * HD + 2 * dp] = bf16lo(u);
-        Qs[qi * HD + 2 * dp + 1] = bf16hi(u);
+#pragma unroll
+    for (int i = 0; i < QPT; ++i) {
+        const int idx = tid + i * T;
+        if (idx < nq) {
+            Qs[2 * idx] = bf16lo(qreg[i]);
+            Qs[2 * idx + 1] = bf16hi(qreg[i]);
+        }
+    }
+    for (int idx = tid + QPT * T; idx < nq; idx += T) {  // more than 16 queries of 128 dims
+        const int qi = idx / HALF, dp = idx % HALF;
+        const int m = qi / G, g = qi % G;
+        const uint32_t u = *reinterpret_cast<const uint32_t*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + 2 * dp);
+        Qs[2 * idx] = bf16lo(u);
+        Qs[2 * idx + 1] = bf16hi(u);
     }
     cp_async_wait<0>();
     __syncthreads();
 
-    // phase 1: thread = (key j, half of the dims); partial dot products in groups of 4 queries
+    // phase 1: q.k -- thread = (key, quarter of the dims); groups of 4 queries, then singles
     {
-        const int j = tid & 63, hf = tid >> 6;
-        const unsigned char* krow = Ks + j * KROW + hf * HALF * 2;
-        for (int q0 = 0; q0 < Q; q0 += 4) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 2
-            for (int b = 0; b < HALF / 8; ++b) {
-                uint4 kk = *reinterpret_cast<const uint4*>(krow + b * 16);
-                float kf[8] = {bf16lo(kk.x), bf16hi(kk.x), bf16lo(kk.y), bf16hi(kk.y),
-                               bf16lo(kk.z), bf16hi(kk.z), bf16lo(kk.w), bf16hi(kk.w)};
-#pragma unroll
-                for (int qq = 0; qq < 4; ++qq) {
-                    int qi = min(q0 + qq, Q - 1);
-                    const float4* qv = reinterpret_cast<const float4*>(Qs + qi * HD + hf * HALF + b * 8);
-                    float4 a = qv[0], c = qv[1];
-                    float s = acc[qq];
-                    s = fmaf(kf[0], a.x, s);
-                    s = fmaf(kf[1], a.y, s);
-                    s = fmaf(kf[2], a.z, s);
-                    s = fmaf(kf[3], a.w, s);
-                    s = fmaf(kf[4], c.x, s);
-                    s = fmaf(kf[5], c.y, s);
-                    s = fmaf(kf[6], c.z, s);
-                    s = fmaf(kf[7], c.w, s);
-                    acc[qq] = s;
-                }
-            }
-#pragma unroll
-            for (int qq = 0; qq < 4; ++qq)
-                if (q0 + qq < Q) Sp[((size_t)hf * Q + q0 + qq) * C + j] = acc[qq];
-        }
+        const int key = tid >> 2, qd = tid & 3;
+        const unsigned char* krow = Ks + key * KROW;
+        int q0 = 0;
+        for (; q0 + 4 <= Q; q0 += 4) attn_qk<HD, 4>(krow, Qs, q0, qd, S, key, qd == 0);
+        for (; q0 < Q; ++q0) attn_qk<HD, 1>(krow, Qs, q0, qd, S, key, qd == 0);
     }
     __syncthreads();
 
-    // phase 2: one warp per query: mask, max, exp, sum over the 64 keys of the chunk
+    // phase 2: one warp per query: scale, mask, max, exp, sum over the 64 keys of the chunk
     {
         const int warp = tid >> 5, lane = tid & 31;
         const float scale = rsqrtf((float)HD);
-        for (int qi = warp; qi < Q; qi += 4) {
-            int m = qi / G, g = qi % G;
-            int pos = pos0 + m;
-            float s0 = (Sp[(size_t)qi * C + lane] + Sp[((size_t)Q + qi) * C + lane]) * scale;
-            float s1 = (Sp[(size_t)qi * C + lane + 32] + Sp[((size_t)Q + qi) * C + lane + 32]) * scale;
+        for (int qi = warp; qi < Q; qi += T / 32) {
+            const int m = qi / G, g = qi % G;
+            const int pos = pos0 + m;
+            float s0 = S[(size_t)qi * C + lane] * scale;
+            float s1 = S[(size_t)qi * C + lane + 32] * scale;
             if (key0 + lane > pos) s0 = -INFINITY;
             if (key0 + lane + 32 > pos) s1 = -INFINITY;
             float mx = fmaxf(s0, s1);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            float p0 = (s0 == -INFINITY) ? 0.f : expf(s0 - mx);
-            float p1 = (s1 == -INFINITY) ? 0.f : expf(s1 - mx);
+            const float p0 = (s0 == -INFINITY) ? 0.f : expf(s0 - mx);
+            const float p1 = (s1 == -INFINITY) ? 0.f : expf(s1 - mx);
             float l = p0 + p1;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-            P[(size_t)qi * C + lane] = p0;
-            P[(size_t)qi * C + lane + 32] = p1;
+            S[(size_t)qi * C + lane] = p0;
+            S[(size_t)qi * C + lane + 32] = p1;
             if (lane == 0) {
                 float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP;
                 dst[HD] = mx;
@@ -300,40 +379,27 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
     }
     __syncthreads();
 
-    // phase 3: thread = (dim pair dp, key slice ks); o[q][dims] = sum_j P[q][j] V[j][dims]
+    // phase 3: p.v -- thread = (pair of dims, slice of the keys)
     {
-        const int dp = tid % HALF, ks = tid / HALF;
-        for (int q0 = 0; q0 < Q; q0 += 4) {
-            float acc[4][2] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
-#pragma unroll 4
-            for (int j = ks; j < C; j += NKS) {
-                uint32_t u = *reinterpret_cast<const uint32_t*>(Vs + j * HD * 2 + dp * 4);
-                float v0 = bf16lo(u), v1 = bf16hi(u);
+        const int ks = tid % NKS, dp = tid / NKS;
+        auto store = [&](int qi, float o0, float o1) {
+            const int m = qi / G, g = qi % G;
+            float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP + 2 * dp;
+            *reinterpret_cast<float2*>(dst) = make_float2(o0, o1);
+        };
+        int q0 = 0;
+        for (; q0 + 4 <= Q; q0 += 4) {
+            float o[4][2];
+            attn_pv<HD, 4, NKS>(Vs, S, q0, dp, ks, o);
+            if (ks == 0) {
 #pragma unroll
-                for (int qq = 0; qq < 4; ++qq) {
-                    int qi = min(q0 + qq, Q - 1);
-                    float p = P[(size_t)qi * C + j];
-                    acc[qq][0] = fmaf(p, v0, acc[qq][0]);
-                    acc[qq][1] = fmaf(p, v1, acc[qq][1]);
-                }
+                for (int qq = 0; qq < 4; ++qq) store(q0 + qq, o[qq][0], o[qq][1]);
             }
-#pragma unroll
-            for (int qq = 0; qq < 4; ++qq) {
-                Ored[((size_t)ks * 4 + qq) * HD + 2 * dp] = acc[qq][0];
-                Ored[((size_t)ks * 4 + qq) * HD + 2 * dp + 1] = acc[qq][1];
-            }
-            __syncthreads();
-            for (int idx = tid; idx < 4 * HD; idx += 128) {
-                int qq = idx / HD, dd = idx % HD;
-                if (q0 + qq < Q) {
-                    float s = 0.f;
-#pragma unroll
-                    for (int k2 = 0; k2 < NKS; ++k2) s += Ored[((size_t)k2 * 4 + qq) * HD + dd];
-                    int qi = q0 + qq, m = qi / G, g = qi % G;
-                    part[(((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP + dd] = s;
-                }
-            }
-            __syncthreads();
+        }
+        for (; q0 < Q; ++q0) {
+            float o[1][2];
+            attn_pv<HD, 1, NKS>(Vs, S, q0, dp, ks, o);
+            if (ks == 0) store(q0, o[0][0], o[0][1]);
         }
     }
 
@@ -350,47 +416,106 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
     if (!is_last) return;
     __threadfence();
 
-    // ordered merge: one warp per query, lanes over the dims; partials come from L2
+    // Merge in a fixed order, in two round trips to L2 per batch of 8 queries:
+    //  A  one warp per query: all chunk (max, sum) pairs at once -> global max, weights
+    //     w_c = exp(max_c - max) and the denominator (summed in chunk order by one lane);
+    //  B  four queries at a time: warp s sums the weighted o of chunks c = s, s+8, ... of each
+    //     (lanes over the dims), then one warp per query adds the 8 slice sums in slice
+    //     order, divides and stores.
+    // The order depends on the row's position only, never on M.
     {
         constexpr int DPL = HD / 32;  // dims per lane: 4 or 2
         const int warp = tid >> 5, lane = tid & 31;
-        for (int qi = warp; qi < Q; qi += 4) {
-            const int m = qi / G, h = kh * G + qi % G;
-            const int nch = (pos0 + m) / C + 1;
-            const float* base = part + ((size_t)m * Hq + h) * chunk_cap * PP;
-            float mx = -INFINITY;
-            for (int c = lane; c < nch; c += 32) mx = fmaxf(mx, __ldcg(base + (size_t)c * PP + HD));
+        float* Wt = reinterpret_cast<float*>(smem);                 // [8][kAttnMaxChunks] weights
+        float* Ls = Wt + kMergeBatch * kAttnMaxChunks;              // [8][kAttnMaxChunks] chunk sums
+        float* Ob = Ls + kMergeBatch * kAttnMaxChunks;              // [4 queries][8 slices][HD]
+        float* Lq = Ob + 4 * 8 * HD;                                // [8] denominators
+        for (int qb = 0; qb < Q; qb += kMergeBatch) {
+            __syncthreads();  // previous batch (and the phases before) are done with this memory
+            {
+                const int qi = qb + warp;
+                if (qi < Q) {
+                    const int m = qi / G, h = kh * G + qi % G;
+                    const int nch = (pos0 + m) / C + 1;
+                    const float* base = part + ((size_t)m * Hq + h) * chunk_cap * PP;
+                    float* wt = Wt + warp * kAttnMaxChunks;
+                    float* ls = Ls + warp * kAttnMaxChunks;
+                    float mx = -INFINITY;
+                    for (int c = lane; c < nch; c += 32) {
+                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(base + (size_t)c * PP + HD));
+                        wt[c] = ml.x;
+                        ls[c] = ml.y;
+                        mx = fmaxf(mx, ml.x);
+                    }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            float l = 0.f, o[DPL];
-#pragma unroll
-            for (int i = 0; i < DPL; ++i) o[i] = 0.f;
-#pragma unroll 4
-            for (int c = 0; c < nch; ++c) {
-                const float* pc = base + (size_t)c * PP;
-                const float2 ml = __ldcg(reinterpret_cast<const float2*>(pc + HD));
-                const float w = expf(ml.x - mx);
-                l = fmaf(ml.y, w, l);
-                if (DPL == 4) {
-                    const float4 v = __ldcg(reinterpret_cast<const float4*>(pc + lane * 4));
-                    o[0] = fmaf(v.x, w, o[0]);
-                    o[1] = fmaf(v.y, w, o[1]);
-                    o[DPL - 2] = fmaf(v.z, w, o[DPL - 2]);
-                    o[DPL - 1] = fmaf(v.w, w, o[DPL - 1]);
-                } else {
-                    const float2 v = __ldcg(reinterpret_cast<const float2*>(pc + lane * 2));
-                    o[0] = fmaf(v.x, w, o[0]);
-                    o[1] = fmaf(v.y, w, o[1]);
+                    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                    for (int c = lane; c < nch; c += 32) wt[c] = expf(wt[c] - mx);
+                    __syncwarp();
+                    if (lane == 0) {
+                        float l = 0.f;
+                        for (int c = 0; c < nch; ++c) l = fmaf(ls[c], wt[c], l);
+                        Lq[warp] = l;
+                    }
                 }
             }
-            uint16_t* dst = out + ((size_t)m * Hq + h) * HD + lane * DPL;
-            if (DPL == 4) {
-                uint2 pk;
-                pk.x = pack_bf16(o[0] / l, o[1] / l);
-                pk.y = pack_bf16(o[DPL - 2] / l, o[DPL - 1] / l);
-                *reinterpret_cast<uint2*>(dst) = pk;
-            } else {
-                *reinterpret_cast<uint32_t*>(dst) = pack_bf16(o[0] / l, o[1] / l);
+            __syncthreads();
+            for (int w0 = 0; w0 < kMergeBatch && qb + w0 < Q; w0 += 4) {  // four queries at a time
+                float o[4][DPL];
+#pragma unroll
+                for (int ww = 0; ww < 4; ++ww) {
+#pragma unroll
+                    for (int i = 0; i < DPL; ++i) o[ww][i] = 0.f;
+                    const int qi = qb + w0 + ww;
+                    if (qi < Q) {
+                        const int m = qi / G, h = kh * G + qi % G;
+                        const int nch = (pos0 + m) / C + 1;
+                        const float* base = part + ((size_t)m * Hq + h) * chunk_cap * PP + lane * DPL;
+                        const float* wt = Wt + (w0 + ww) * kAttnMaxChunks;
+#pragma unroll 4
+                        for (int c = warp; c < nch; c += 8) {
+                            const float wc = wt[c];
+                            if (DPL == 4) {
+                                const float4 v = __ldcg(reinterpret_cast<const float4*>(base + (size_t)c * PP));
+                                o[ww][0] = fmaf(v.x, wc, o[ww][0]);
+                                o[ww][1] = fmaf(v.y, wc, o[ww][1]);
+                                o[ww][DPL - 2] = fmaf(v.z, wc, o[ww][DPL - 2]);
+                                o[ww][DPL - 1] = fmaf(v.w, wc, o[ww][DPL - 1]);
+                            } else {
+                                const float2 v = __ldcg(reinterpret_cast<const float2*>(base + (size_t)c * PP));
+                                o[ww][0] = fmaf(v.x, wc, o[ww][0]);
+                                o[ww][1] = fmaf(v.y, wc, o[ww][1]);
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int ww = 0; ww < 4; ++ww)
+#pragma unroll
+                    for (int i = 0; i < DPL; ++i) Ob[(ww * 8 + warp) * HD + lane * DPL + i] = o[ww][i];
+                __syncthreads();
+                if (warp < 4 && qb + w0 + warp < Q) {  // warp ww finishes query w0 + ww
+                    const int qi = qb + w0 + warp;
+                    const int m = qi / G, h = kh * G + qi % G;
+                    const float l = Lq[w0 + warp];
+                    float r[DPL];
+#pragma unroll
+                    for (int i = 0; i < DPL; ++i) {
+                        float a = 0.f;
+#pragma unroll
+                        for (int sl = 0; sl < 8; ++sl) a += Ob[(warp * 8 + sl) * HD + lane * DPL + i];
+                        r[i] = a / l;
+                    }
+                    uint16_t* dst = out + ((size_t)m * Hq + h) * HD + lane * DPL;
+                    if (DPL == 4) {
+                        uint2 pk;
+                        pk.x = pack_bf16(r[0], r[1]);
+                        pk.y = pack_bf16(r[DPL - 2], r[DPL - 1]);
+                        *reinterpret_cast<uint2*>(dst) = pk;
+                    } else {
+                        *reinterpret_cast<uint32_t*>(dst) = pack_bf16(r[0], r[1]);
+                    }
+                }
+                __syncthreads();
             }
         }
     }

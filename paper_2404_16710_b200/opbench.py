@@ -18,7 +18,7 @@ import torch
 from . import binding as B
 from . import synth
 
-OPS = ("gate_up_swiglu", "down_residual", "qkv_proj", "o_residual", "lm_head_argmax")
+OPS = ("gate_up_swiglu", "down_residual", "qkv_proj", "o_residual", "lm_head_argmax", "attention", "rmsnorm")
 
 
 def time_op(fn, n_rot, iters=40, warm=5):
@@ -46,8 +46,10 @@ def time_op(fn, n_rot, iters=40, warm=5):
     return e0.elapsed_time(e1) / iters
 
 
-def op_cases(shape, w, path, M):
-    """name -> (callable(layer index), algorithmic bytes per launch, number of distinct weights)"""
+def op_cases(shape, w, path, M, n_ctx=1030):
+    """name -> (callable(layer index), algorithmic bytes per launch, number of distinct weights).
+    attention: rows at positions n_ctx .. n_ctx+M-1 over a cache of n_ctx earlier tokens; its
+    algorithmic bytes are the K and V rows it must read."""
     D, F, V = shape.d_model, shape.d_ffn, shape.vocab
     L = len(w["wq"])
     qw = shape.n_heads * shape.head_dim
@@ -64,7 +66,25 @@ def op_cases(shape, w, path, M):
     # q, k and v projections as one matrix of the fused launch's size
     wqkv = [torch.cat([w["wq"][i], w["wk"][i], w["wv"][i]]) for i in range(L)]
     heads = [w["lm_head"], w["tok_embed"]]
+    # paged KV cache of a few layers (rotated over), identity page table
+    Hq, Hkv, hd, ps = shape.n_heads, shape.n_kv_heads, shape.head_dim, 64
+    max_seq = n_ctx + M + 1
+    n_pages = -(-max_seq // ps)
+    kvl = min(L, 8)
+    kp = [torch.randn((n_pages, Hkv, ps, hd), device="cuda", generator=g).bfloat16() for _ in range(kvl)]
+    vp = [torch.randn((n_pages, Hkv, ps, hd), device="cuda", generator=g).bfloat16() for _ in range(kvl)]
+    table = torch.arange(n_pages, dtype=torch.int32, device="cuda")
+    q = (torch.randn((M, qw), device="cuda", generator=g) * 0.3).bfloat16()
+    ao = torch.empty((M, qw), dtype=torch.bfloat16, device="cuda")
+    asc = torch.empty(B.ls_op_attention_scratch_bytes(Hq, hd, max_seq), dtype=torch.uint8, device="cuda")
+    xs = torch.randn((M, D), device="cuda", generator=g)
+    hn = torch.empty((M, D), dtype=torch.bfloat16, device="cuda")
+    gain = w["attn_norm"][0]
+    kv_bytes = 2 * 2 * Hkv * hd * (n_ctx + M)
     return {
+        "attention": (lambda i: B.ls_op_attention(q, n_ctx, Hq, Hkv, hd, ps, table, max_seq, kp[i % kvl], vp[i % kvl],
+                                                  asc, ao), kv_bytes, kvl),
+        "rmsnorm": (lambda i: B.ls_op_rmsnorm(xs, gain, 1e-5, hn), 4 * M * D, 1),
         "gate_up_swiglu": (lambda i: B.ls_op_gate_up_swiglu(path, w["w_gate"][i % L], w["w_up"][i % L], h, act),
                            4 * F * D, L),
         "down_residual": (lambda i: B.ls_op_linear(path, w["w_down"][i % L], a, x, True), 2 * F * D, L),
