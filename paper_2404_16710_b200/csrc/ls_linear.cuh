@@ -249,7 +249,7 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 }
 
 template <int NT, int WARPS, int STAGES>
-constexpr size_t mma_ring_bytes()
+__host__ __device__ constexpr size_t mma_ring_bytes()
 {
     return (size_t)(2 + NT) * STAGES * WARPS * 32 * 16;
 }
@@ -352,8 +352,11 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
     }
     cp_async_wait<0>();
 
-    // cross-warp reduction in warp order (fixed), then the epilogue on 32*NT threads
-    __shared__ float red[WARPS][NT * 4][32];
+    // cross-warp reduction in warp order (fixed), then the epilogue on 32*NT threads; the
+    // ring is free by now (every thread has consumed its own slots) and is reused
+    __syncthreads();
+    float(*red)[NT * 4][32] = reinterpret_cast<float(*)[NT * 4][32]>(ring);
+    static_assert(sizeof(float) * WARPS * NT * 4 * 32 <= mma_ring_bytes<NT, WARPS, STAGES>(), "ring too small");
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
