@@ -202,6 +202,12 @@ int attn_allow_smem(int hd, int group)
     return LS_OK;
 }
 
+// per-CTA argmax candidates the LM-head kernel of this family writes per row
+int n_candidates(int path, int V, int K, int M)
+{
+    return path == LS_LINEAR_MMA ? mma_grid(EPI_ARGMAX, V, K, M) : lin_grid(EPI_ARGMAX, V);
+}
+
 LinArgs lin_args(const uint16_t* w, const uint16_t* h, int M, int N, int K)
 {
     LinArgs a;
@@ -284,7 +290,7 @@ int run_head(ls_model* m, int M, const float* xrow, int32_t* tok_out, float* log
     a.ldo = c.vocab;
     a.ctl = m->ctl;
     LS_CK(launch_linear(m->path, EPI_ARGMAX, a, st));
-    LS_CK(launch(st, argmax_finish_kernel, dim3(M), dim3(256), 0, m->cand, lin_grid(EPI_ARGMAX, c.vocab),
+    LS_CK(launch(st, argmax_finish_kernel, dim3(M), dim3(256), 0, m->cand, n_candidates(m->path, c.vocab, c.d_model, M),
                  m->cand_stride, tok_out, m->ctl));
     m->launches += 3;
     return LS_OK;
@@ -822,7 +828,7 @@ int ls_op_lm_head_argmax(int32_t path, const void* w, const void* h, int32_t M, 
     a.ldo = V;
     const LaunchCtx lc = {(cudaStream_t)stream, false};
     LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
-    LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, lin_grid(EPI_ARGMAX, V), a.cand_stride, tok,
+    LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, n_candidates(path, V, K, M), a.cand_stride, tok,
                  nullptr));
     return LS_OK;
 }
@@ -868,7 +874,7 @@ int ls_op_lm_head_argmax_static(int32_t path, const void* w, const void* h, int3
     a.ldo = V;
     const LaunchCtx lc = {(cudaStream_t)stream, false};
     LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
-    LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, lin_grid(EPI_ARGMAX, V), a.cand_stride, tok,
+    LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, n_candidates(path, V, K, M), a.cand_stride, tok,
                  nullptr));
     return LS_OK;
 }

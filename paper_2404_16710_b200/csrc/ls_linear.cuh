@@ -248,25 +248,27 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int NT, int WARPS, int STAGES>
+template <int NT, int TR, int WARPS, int STAGES>
 __host__ __device__ constexpr size_t mma_ring_bytes()
 {
-    return (size_t)(2 + NT) * STAGES * WARPS * 32 * 16;
+    return (size_t)(2 * TR + NT) * STAGES * WARPS * 32 * 16;
 }
 
-// grid ceil(N/16) (SwiGLU: ceil(F/8)), block WARPS*32: the warps interleave over K in steps
-// of 32.  Fragment roles (g = lane/4, t = lane%4): the thread's 16 bytes of row g (and of
-// row g+8) at k = 32 s + 8 t feed two MMAs; contraction slots {2t, 2t+1, 2t+8, 2t+9} of
-// the first take elements k..k+3, of the second k+4..k+7, for A and for B alike.
-// SwiGLU: row g is the gate row of feature f, row g+8 its up row.
+// grid ceil(tiles/TR) with tiles = ceil(N/16) (SwiGLU: ceil(F/8)), block WARPS*32: the warps
+// interleave over K in steps of 32.  Fragment roles (g = lane/4, t = lane%4): the thread's
+// 16 bytes of row g (and of row g+8) at k = 32 s + 8 t feed two MMAs; contraction slots
+// {2t, 2t+1, 2t+8, 2t+9} of the first take elements k..k+3, of the second k+4..k+7, for A
+// and for B alike.  SwiGLU: row g is the gate row of feature f, row g+8 its up row.
+// With TR = 2 a warp streams two 16-row tiles and uses its token fragments for both, which
+// halves the activation traffic from L2 per weight byte.
 //
 // Each thread prefetches exactly the 16-byte pieces it will consume itself, STAGES k-steps
 // ahead, with cp.async into a ring of its own in shared memory: the bytes in flight per
 // SM are set by the ring depth, not by registers or occupancy, and no barrier is needed
-// (nobody else reads a thread's slots).  WARPS and STAGES are chosen from (N, K) alone --
-// never from M -- so that matrices with few row tiles (N = 4096: 256 tiles) still keep
-// enough bytes in flight.
-template <int NT, int EPI, int WARPS, int STAGES>
+// (nobody else reads a thread's slots).  WARPS is chosen from (N, K) alone -- never from
+// M -- so that matrices with few row tiles (N = 4096: 256 tiles) still keep enough bytes
+// in flight; TR and STAGES do not touch the arithmetic of a row.
+template <int NT, int EPI, int TR, int WARPS, int STAGES>
 __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
 {
     constexpr int T = WARPS * 32;
@@ -274,23 +276,28 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
     pdl_launch_dependents();
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const uint16_t *pa, *pb;
-    if (EPI == EPI_SWIGLU) {
-        int f = min(blockIdx.x * 8 + g, a.N - 1);
-        pa = a.w0 + (size_t)f * a.K;
-        pb = a.w1 + (size_t)f * a.K;
-    } else if (EPI == EPI_QKV) {
-        pa = weight_row(a, qkv_row(a, blockIdx.x, g, 0));
-        pb = weight_row(a, qkv_row(a, blockIdx.x, g, 1));
-    } else {
-        pa = weight_row(a, blockIdx.x * 16 + g);
-        pb = weight_row(a, blockIdx.x * 16 + g + 8);
+    const uint16_t *pa[TR], *pb[TR];
+#pragma unroll
+    for (int tr = 0; tr < TR; ++tr) {
+        const int tile = blockIdx.x * TR + tr;
+        if (EPI == EPI_SWIGLU) {
+            int f = min(tile * 8 + g, a.N - 1);
+            pa[tr] = a.w0 + (size_t)f * a.K;
+            pb[tr] = a.w1 + (size_t)f * a.K;
+        } else if (EPI == EPI_QKV) {
+            const int tc = min(tile, (a.N >> 4) - 1);
+            pa[tr] = weight_row(a, qkv_row(a, tc, g, 0));
+            pb[tr] = weight_row(a, qkv_row(a, tc, g, 1));
+        } else {
+            pa[tr] = weight_row(a, tile * 16 + g);
+            pb[tr] = weight_row(a, tile * 16 + g + 8);
+        }
     }
     const uint16_t* hb[NT];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) hb[nt] = a.h + (size_t)min(nt * 8 + g, a.M - 1) * a.K;
 
-    // region r (0: row g, 1: row g+8, 2..: tokens), stage s, thread tid -> 16 bytes
+    // region r (2 tr: row g, 2 tr + 1: row g+8, 2 TR + nt: tokens), stage s, thread tid -> 16 bytes
     const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(ring) + (uint32_t)tid * 16u;
     auto slot = [&](int r, int s) { return ring0 + (uint32_t)((r * STAGES + s) * T) * 16u; };
 
@@ -300,8 +307,11 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             const int k = step * 32 + 8 * t;
             const int nb = (k < a.K) ? 16 : 0;
             const int kk = (k < a.K) ? k : 0;
-            cp_async16_cg(slot(0, s), pa + kk, nb);
-            cp_async16_cg(slot(1, s), pb + kk, nb);
+#pragma unroll
+            for (int tr = 0; tr < TR; ++tr) {
+                cp_async16_cg(slot(2 * tr, s), pa[tr] + kk, nb);
+                cp_async16_cg(slot(2 * tr + 1, s), pb[tr] + kk, nb);
+            }
         }
     };
     auto issue_h = [&](int step, int s) {  // activations: written by the previous kernel
@@ -310,15 +320,17 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             const int nb = (k < a.K) ? 16 : 0;
             const int kk = (k < a.K) ? k : 0;
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) cp_async16_ca(slot(2 + nt, s), hb[nt] + kk, nb);
+            for (int nt = 0; nt < NT; ++nt) cp_async16_ca(slot(2 * TR + nt, s), hb[nt] + kk, nb);
         }
     };
 
-    float c[NT][4];
+    float c[TR][NT][4];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
+    for (int tr = 0; tr < TR; ++tr)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) c[nt][i] = 0.f;
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) c[tr][nt][i] = 0.f;
 
     // the first STAGES-1 steps of weights are on their way while the predecessor finishes
 #pragma unroll
@@ -340,43 +352,53 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
         issue_h(step + (STAGES - 1) * WARPS, wr);
         cp_async_commit();
         cp_async_wait<STAGES - 1>();
-        const uint4 A0 = lds16(slot(0, rd)), A1 = lds16(slot(1, rd));
+        uint4 B[NT];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const uint4 B = lds16(slot(2 + nt, rd));
-            mma_bf16_16816(c[nt], A0.x, A1.x, A0.y, A1.y, B.x, B.y);
-            mma_bf16_16816(c[nt], A0.z, A1.z, A0.w, A1.w, B.z, B.w);
+        for (int nt = 0; nt < NT; ++nt) B[nt] = lds16(slot(2 * TR + nt, rd));
+#pragma unroll
+        for (int tr = 0; tr < TR; ++tr) {
+            const uint4 A0 = lds16(slot(2 * tr, rd)), A1 = lds16(slot(2 * tr + 1, rd));
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                mma_bf16_16816(c[tr][nt], A0.x, A1.x, A0.y, A1.y, B[nt].x, B[nt].y);
+                mma_bf16_16816(c[tr][nt], A0.z, A1.z, A0.w, A1.w, B[nt].z, B[nt].w);
+            }
         }
         rd = (rd + 1 == STAGES) ? 0 : rd + 1;
         wr = (wr + 1 == STAGES) ? 0 : wr + 1;
     }
     cp_async_wait<0>();
 
-    // cross-warp reduction in warp order (fixed), then the epilogue on 32*NT threads; the
+    // cross-warp reduction in warp order (fixed), then the epilogue on 32*TR*NT threads; the
     // ring is free by now (every thread has consumed its own slots) and is reused
     __syncthreads();
-    float(*red)[NT * 4][32] = reinterpret_cast<float(*)[NT * 4][32]>(ring);
-    static_assert(sizeof(float) * WARPS * NT * 4 * 32 <= mma_ring_bytes<NT, WARPS, STAGES>(), "ring too small");
+    constexpr int FR = TR * NT;  // accumulator fragments per warp
+    float(*red)[FR * 4][32] = reinterpret_cast<float(*)[FR * 4][32]>(ring);
+    static_assert(sizeof(float) * WARPS * FR * 4 * 32 <= mma_ring_bytes<NT, TR, WARPS, STAGES>(), "ring too small");
+    static_assert(32 * FR <= T, "not enough threads for the epilogue");
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
+    for (int tr = 0; tr < TR; ++tr)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) red[warp][nt * 4 + i][lane] = c[nt][i];
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) red[warp][(tr * NT + nt) * 4 + i][lane] = c[tr][nt][i];
     __syncthreads();
-    __shared__ float vals[16][NT * 8 + 1];
-    if (threadIdx.x < 32 * NT) {
-        const int nt = threadIdx.x >> 5;
+    __shared__ float vals[16 * TR][NT * 8 + 1];
+    if (threadIdx.x < 32 * FR) {
+        const int fr = threadIdx.x >> 5, tr = fr / NT, nt = fr % NT;
+        const int tile = blockIdx.x * TR + tr;
         const int gg = lane >> 2, tt = lane & 3;
         float r[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             float s = 0.f;
 #pragma unroll
-            for (int w = 0; w < WARPS; ++w) s += red[w][nt * 4 + i][lane];
+            for (int w = 0; w < WARPS; ++w) s += red[w][fr * 4 + i][lane];
             r[i] = s;
         }
         const int m0 = nt * 8 + 2 * tt;  // tokens m0, m0+1
         if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
-            const int nlo = blockIdx.x * 16 + gg, nhi = nlo + 8;
+            const int nlo = tile * 16 + gg, nhi = nlo + 8;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 int m = m0 + (i & 1), n = (i < 2) ? nlo : nhi;
@@ -386,22 +408,24 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
                 }
             }
         } else if (EPI == EPI_SWIGLU) {
-            const int f = blockIdx.x * 8 + gg;
+            const int f = tile * 8 + gg;
             if (f < a.N) {
                 if (m0 < a.M) a.out_bf16[(size_t)m0 * a.N + f] = f2bf(silu_mul(r[0], r[2]));
                 if (m0 + 1 < a.M) a.out_bf16[(size_t)(m0 + 1) * a.N + f] = f2bf(silu_mul(r[1], r[3]));
             }
         } else if (EPI == EPI_QKV) {
-            const int pos0 = (a.ctl ? a.ctl[CTL_CACHE_LEN] : 0) + a.pos_off;
-            const int tph = a.hd >> 4;
-            const int head = blockIdx.x / tph, j = (blockIdx.x % tph) * 8 + gg;
-            if (m0 < a.M) qkv_store(a, head, j, m0, pos0, r[0], r[2]);
-            if (m0 + 1 < a.M) qkv_store(a, head, j, m0 + 1, pos0, r[1], r[3]);
+            if (tile < (a.N >> 4)) {
+                const int pos0 = (a.ctl ? a.ctl[CTL_CACHE_LEN] : 0) + a.pos_off;
+                const int tph = a.hd >> 4;
+                const int head = tile / tph, j = (tile % tph) * 8 + gg;
+                if (m0 < a.M) qkv_store(a, head, j, m0, pos0, r[0], r[2]);
+                if (m0 + 1 < a.M) qkv_store(a, head, j, m0 + 1, pos0, r[1], r[3]);
+            }
         } else {
-            vals[gg][m0] = r[0];
-            vals[gg][m0 + 1] = r[1];
-            vals[gg + 8][m0] = r[2];
-            vals[gg + 8][m0 + 1] = r[3];
+            vals[tr * 16 + gg][m0] = r[0];
+            vals[tr * 16 + gg][m0 + 1] = r[1];
+            vals[tr * 16 + gg + 8][m0] = r[2];
+            vals[tr * 16 + gg + 8][m0 + 1] = r[3];
         }
     }
     if (EPI == EPI_ARGMAX) {
@@ -411,8 +435,8 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             float v = -INFINITY;
             int idx = 0x7fffffff;
 #pragma unroll
-            for (int rr = 0; rr < 16; ++rr) {
-                int n = blockIdx.x * 16 + rr;
+            for (int rr = 0; rr < 16 * TR; ++rr) {
+                int n = blockIdx.x * 16 * TR + rr;
                 if (n < a.N) {
                     float x = vals[rr][m];
                     if (a.out) a.out[(size_t)m * a.ldo + n] = x;
@@ -444,38 +468,52 @@ inline cudaError_t launch_linear_fma(const LinArgs& a, const LaunchCtx& lc)
     return launch(lc, linear_fma_kernel<16, EPI>, grid, block, 0, a);
 }
 
-// Warps per 16-row tile and ring depth, from the matrix shape alone: many row tiles ->
-// 8 warps x 6 stages (3 CTAs per SM); few row tiles (N = 4096) -> 16 warps x 4 stages
-// (2 CTAs per SM, all tiles resident in one wave).
+// A row's bits depend on how K is split over the warps of its tile, and on nothing else.
+// So the warps per tile come from the matrix shape alone (never from M):
+//   few row tiles (N = 4096)  -> 16 warps, 4 stages (2 CTAs per SM, all tiles in one wave)
+//   otherwise                 -> 8 warps, 6 stages (3 CTAs per SM)
+// while the tiles per CTA may follow the pass size: with the second token tile (M > 8) and
+// many row tiles (gate-up, LM head) a CTA takes two tiles (4 stages, 2 CTAs per SM).
 inline bool mma_wide(int epi, int N, int K)
 {
     const int tiles = lin_grid(epi, N), nsteps = (K + 31) / 32;
     return tiles < 600 && nsteps >= 16;
 }
+inline bool mma_pair(int epi, int N, int K, int M) { return M > 8 && !mma_wide(epi, N, K) && lin_grid(epi, N) >= 1200; }
+// CTAs the MMA family launches for this matrix (also the number of argmax candidates per row)
+inline int mma_grid(int epi, int N, int K, int M)
+{
+    const int tiles = lin_grid(epi, N);
+    return mma_pair(epi, N, K, M) ? (tiles + 1) / 2 : tiles;
+}
 
-template <int NT, int EPI, int WARPS, int STAGES>
+template <int NT, int EPI, int TR, int WARPS, int STAGES>
 inline cudaError_t launch_linear_mma_cfg(const LinArgs& a, const LaunchCtx& lc)
 {
-    constexpr size_t smem = mma_ring_bytes<NT, WARPS, STAGES>();
+    constexpr size_t smem = mma_ring_bytes<NT, TR, WARPS, STAGES>();
     static bool allowed[64] = {false};  // per instantiation and device: the attribute is set once
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !allowed[dev]) {
-        e = cudaFuncSetAttribute(linear_mma_kernel<NT, EPI, WARPS, STAGES>,
+        e = cudaFuncSetAttribute(linear_mma_kernel<NT, EPI, TR, WARPS, STAGES>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) allowed[dev] = true;
     }
-    return launch(lc, linear_mma_kernel<NT, EPI, WARPS, STAGES>, dim3(lin_grid(EPI, a.N)), dim3(WARPS * 32), smem, a);
+    const int tiles = lin_grid(EPI, a.N);
+    return launch(lc, linear_mma_kernel<NT, EPI, TR, WARPS, STAGES>, dim3((tiles + TR - 1) / TR), dim3(WARPS * 32), smem,
+                  a);
 }
 
 template <int EPI>
 inline cudaError_t launch_linear_mma(const LinArgs& a, const LaunchCtx& lc)
 {
     if (mma_wide(EPI, a.N, a.K))
-        return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 16, 4>(a, lc) : launch_linear_mma_cfg<2, EPI, 16, 4>(a, lc);
-    return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 8, 6>(a, lc) : launch_linear_mma_cfg<2, EPI, 8, 6>(a, lc);
+        return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 1, 16, 4>(a, lc) : launch_linear_mma_cfg<2, EPI, 1, 16, 4>(a, lc);
+    if (a.M <= 8) return launch_linear_mma_cfg<1, EPI, 1, 8, 6>(a, lc);
+    if (mma_pair(EPI, a.N, a.K, a.M)) return launch_linear_mma_cfg<2, EPI, 2, 8, 4>(a, lc);
+    return launch_linear_mma_cfg<2, EPI, 1, 8, 6>(a, lc);
 }
 
 // path: 1 = FMA, 2 = MMA
