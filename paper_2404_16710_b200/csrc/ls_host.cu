@@ -88,6 +88,9 @@ struct ls_model {
     int32_t *page_table, *ctl, *draft, *verified, *out_ids, *accepted, *ids, *attn_counters;
     float *inv_freq, *x, *qkv, *part, *logits;
     uint16_t *h, *q, *o, *a;
+    uint16_t* hE;  // exit-layer activations, already multiplied by the gain of layer E's norm (Sec. 4.3.3)
+    float* ss;     // [16][n_part] partial sums of squares of the residual rows (fused RMSNorm)
+    int n_part;
     ValIdx* cand;
     int page_shift, n_pages, chunk_cap, cand_stride;
     // loop state
@@ -141,7 +144,13 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     unsigned char* o = take(2 * (size_t)kMaxRows * qw);
     unsigned char* a = take(2 * (size_t)kMaxRows * c.d_ffn);
     unsigned char* cand = take(sizeof(ValIdx) * kMaxRows * cand_stride);
+    const int n_part = (c.d_model + 15) / 16;  // CTAs of a residual projection = partial sums per row
+    unsigned char* ss = take(sizeof(float) * kMaxRows * n_part);
+    unsigned char* he = take(2 * (size_t)kMaxRows * c.d_model);
     if (m) {
+        m->ss = (float*)ss;
+        m->hE = (uint16_t*)he;
+        m->n_part = n_part;
         m->kpages = (uint16_t*)kp;
         m->vpages = (uint16_t*)vp;
         m->layer_kv_elems = layer_kv;
@@ -223,18 +232,45 @@ LinArgs lin_args(const uint16_t* w, const uint16_t* h, int M, int N, int K)
 }
 
 // layers [l0, l1) on M residual rows starting at xrow; row r sits at ctl.cache_len + pos_off + r
-int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
+// fused-RMSNorm fields of a consumer / of a residual producer
+void norm_in(const ls_model* m, LinArgs& a, int slot)
+{
+    a.ss_in = m->ss + (size_t)slot * m->n_part;
+    a.ss_stride = m->n_part;
+    a.n_part = m->n_part;
+    a.inv_d = 1.0f / (float)m->c.d_model;
+    a.eps = m->c.rms_eps;
+}
+void norm_out(const ls_model* m, LinArgs& a, int slot, const uint16_t* gain_a, uint16_t* hout_a,
+              const uint16_t* gain_b, uint16_t* hout_b)
+{
+    a.ss_out = m->ss + (size_t)slot * m->n_part;
+    a.ss_stride = m->n_part;
+    a.gain_a = gain_a;
+    a.hout_a = gain_a ? hout_a : nullptr;
+    a.gain_b = gain_b;
+    a.hout_b = gain_b ? hout_b : nullptr;
+}
+
+// Layers [l0, l1) on M residual rows starting at xrow (row slot `slot` of the 16-row buffers);
+// row r sits at ctl.cache_len + pos_off + r.  h_first: the rows x*gain for layer l0's first
+// norm (left by the embedding, by the previous layer, or by a draft pass for the verify
+// pass).  The last layer's down-projection leaves x*gain_end_a in the h rows (for the LM
+// head or the next call) and x*gain_end_b in the exit-activation rows.
+int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off, int slot, const uint16_t* h_first,
+               const uint16_t* gain_end_a, const uint16_t* gain_end_b)
 {
     const ls_config& c = m->c;
     const int D = c.d_model, Hq = c.n_heads, Hkv = c.n_kv_heads, hd = c.head_dim, F = c.d_ffn;
     const int qw = Hq * hd, kvw = Hkv * hd;
     const LaunchCtx st = {m->st, m->pdl};
+    uint16_t* hrow = m->h + (size_t)slot * D;
+    uint16_t* herow = m->hE + (size_t)slot * D;
     for (int l = l0; l < l1; ++l) {
         const LayerW& w = m->lw[l];
         uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
         uint16_t* vp = m->vpages + (size_t)l * m->layer_kv_elems;
-        LS_CK(launch(st, rmsnorm_kernel, dim3(M), dim3(256), 0, xrow, w.attn_norm, D, c.rms_eps, m->h, m->ctl));
-        LinArgs a = lin_args(w.wq, m->h, M, qw + 2 * kvw, D);
+        LinArgs a = lin_args(w.wq, l == l0 ? h_first : hrow, M, qw + 2 * kvw, D);
         a.w1 = w.wk;
         a.w2 = w.wv;
         a.n0 = qw;
@@ -252,6 +288,7 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
         a.max_seq = c.max_seq;
         a.pos_off = pos_off;
         a.theta = c.rope_theta;
+        norm_in(m, a, slot);
         LS_CK(launch_linear(m->path, EPI_QKV, a, st));
         LS_TRY(attn_launch(m->q, kp, vp, m->page_table, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift,
                            c.max_seq, m->chunk_cap, m->grid_chunks, m->part, m->attn_counters, m->o, st));
@@ -259,47 +296,52 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off)
         a.out = xrow;
         a.ldo = D;
         a.ctl = m->ctl;
+        norm_out(m, a, slot, w.ffn_norm, hrow, nullptr, nullptr);
         LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
-        LS_CK(launch(st, rmsnorm_kernel, dim3(M), dim3(256), 0, xrow, w.ffn_norm, D, c.rms_eps, m->h, m->ctl));
-        a = lin_args(w.wg, m->h, M, F, D);
+        a = lin_args(w.wg, hrow, M, F, D);
         a.w1 = w.wu;
         a.out_bf16 = m->a;
         a.ctl = m->ctl;
+        norm_in(m, a, slot);
         LS_CK(launch_linear(m->path, EPI_SWIGLU, a, st));
         a = lin_args(w.wd, m->a, M, D, F);
         a.out = xrow;
         a.ldo = D;
         a.ctl = m->ctl;
+        if (l + 1 < l1) norm_out(m, a, slot, m->lw[l + 1].attn_norm, hrow, nullptr, nullptr);
+        else norm_out(m, a, slot, gain_end_a, hrow, gain_end_b, herow);
         LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
-        m->launches += 7;
+        m->launches += 5;
     }
     LS_CK(cudaGetLastError());
     return LS_OK;
 }
 
-// shared head g(.) = final norm + LM head (+ argmax) on M residual rows
-int run_head(ls_model* m, int M, const float* xrow, int32_t* tok_out, float* logits)
+// shared head g(.) = final norm + LM head (+ argmax) on the M rows of slot `slot`, whose
+// x*final_gain rows and partial sums the last down-projection has left
+int run_head(ls_model* m, int M, int slot, int32_t* tok_out, float* logits)
 {
     const ls_config& c = m->c;
     const LaunchCtx st = {m->st, m->pdl};
-    LS_CK(launch(st, rmsnorm_kernel, dim3(M), dim3(256), 0, xrow, m->fnorm, c.d_model, c.rms_eps, m->h, m->ctl));
-    LinArgs a = lin_args(m->lm, m->h, M, c.vocab, c.d_model);
+    LinArgs a = lin_args(m->lm, m->h + (size_t)slot * c.d_model, M, c.vocab, c.d_model);
     a.cand = m->cand;
     a.cand_stride = m->cand_stride;
     a.out = logits;
     a.ldo = c.vocab;
     a.ctl = m->ctl;
+    norm_in(m, a, slot);
     LS_CK(launch_linear(m->path, EPI_ARGMAX, a, st));
     LS_CK(launch(st, argmax_finish_kernel, dim3(M), dim3(256), 0, m->cand, n_candidates(m->path, c.vocab, c.d_model, M),
                  m->cand_stride, tok_out, m->ctl));
-    m->launches += 3;
+    m->launches += 2;
     return LS_OK;
 }
 
-int run_embed(ls_model* m, const int32_t* tok_dev, int M, float* xrow)
+int run_embed(ls_model* m, const int32_t* tok_dev, int M, float* xrow, int slot)
 {
     LS_CK(launch(LaunchCtx{m->st, m->pdl}, embed_kernel, dim3(M), dim3(256), 0, m->emb, tok_dev, m->c.d_model,
-                 m->c.vocab, xrow, m->ctl));
+                 m->c.vocab, xrow, m->ctl, m->lw[0].attn_norm, m->h + (size_t)slot * m->c.d_model,
+                 m->ss + (size_t)slot * m->n_part, m->n_part, m->n_part));
     m->launches += 1;
     return LS_OK;
 }
@@ -309,19 +351,22 @@ int enqueue_step(ls_model* m, int E, int d)
 {
     const int D = m->c.d_model, L = m->c.n_layers;
     if (d == 0) {
-        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x));
-        LS_TRY(run_layers(m, 0, E, 1, m->x, 0));
-        LS_TRY(run_head(m, 1, m->x, m->verified, nullptr));
+        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
+        LS_TRY(run_layers(m, 0, E, 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
+        LS_TRY(run_head(m, 1, 0, m->verified, nullptr));
     } else {
         for (int j = 0; j <= d; ++j) {  // self-drafting (Sec. 4.3.1) + the extra early pass
             float* xr = m->x + (size_t)j * D;
-            LS_TRY(run_embed(m, j == 0 ? m->ctl + CTL_CUR_TOK : m->draft + (j - 1), 1, xr));
-            LS_TRY(run_layers(m, 0, E, 1, xr, j));
-            if (j < d) LS_TRY(run_head(m, 1, xr, m->draft + j, nullptr));
+            LS_TRY(run_embed(m, j == 0 ? m->ctl + CTL_CUR_TOK : m->draft + (j - 1), 1, xr, j));
+            // the exit-layer row goes to the LM head (final gain) and, pre-scaled by layer E's
+            // gain, to the verify pass (the exit-layer cache of Sec. 4.3.3)
+            LS_TRY(run_layers(m, 0, E, 1, xr, j, j, m->h + (size_t)j * D, j < d ? m->fnorm : nullptr,
+                              m->lw[E].attn_norm));
+            if (j < d) LS_TRY(run_head(m, 1, j, m->draft + j, nullptr));
         }
-        // self-verification (Sec. 4.3.2) from the exit-layer activations (Sec. 4.3.3)
-        LS_TRY(run_layers(m, E, L, d + 1, m->x, 0));
-        LS_TRY(run_head(m, d + 1, m->x, m->verified, nullptr));
+        // self-verification (Sec. 4.3.2) from the exit-layer activations
+        LS_TRY(run_layers(m, E, L, d + 1, m->x, 0, 0, m->hE, m->fnorm, nullptr));
+        LS_TRY(run_head(m, d + 1, 0, m->verified, nullptr));
     }
     LS_CK(launch(LaunchCtx{m->st, m->pdl}, accept_kernel, dim3(1), dim3(32), 0, m->draft, m->verified, d, m->ctl,
                  m->out_ids, m->accepted));
@@ -562,8 +607,8 @@ int ls_prefill(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t lay
     for (int r0 = 0; r0 < n_prompt - 1; r0 += kMaxRows) {
         int M = n_prompt - 1 - r0;
         if (M > kMaxRows) M = kMaxRows;
-        LS_TRY(run_embed(m, m->ids + r0, M, m->x));
-        LS_TRY(run_layers(m, 0, layers, M, m->x, r0));
+        LS_TRY(run_embed(m, m->ids + r0, M, m->x, 0));
+        LS_TRY(run_layers(m, 0, layers, M, m->x, r0, 0, m->h, nullptr, nullptr));
     }
     LS_CK(cudaEventRecord(m->ev1, m->st));
     int32_t w[CTL_WORDS];
@@ -732,17 +777,18 @@ int ls_debug_logits(ls_model* m, const int32_t* ids, int32_t n, int32_t exit_lay
     LS_TRY(write_ctl(m, 0, 0, 0));
     for (int r0 = 0; r0 < n; r0 += kMaxRows) {
         int M = n - r0 < kMaxRows ? n - r0 : kMaxRows;
-        LS_TRY(run_embed(m, m->ids + r0, M, m->x));
-        LS_TRY(run_layers(m, 0, exit_layer, M, m->x, r0));
+        LS_TRY(run_embed(m, m->ids + r0, M, m->x, 0));
+        LS_TRY(run_layers(m, 0, exit_layer, M, m->x, r0, 0, m->h, m->fnorm,
+                          exit_layer < L ? m->lw[exit_layer].attn_norm : nullptr));
         if (exit_logits) {
-            LS_TRY(run_head(m, M, m->x, m->verified, m->logits));
+            LS_TRY(run_head(m, M, 0, m->verified, m->logits));
             LS_CK(cudaMemcpyAsync(exit_logits + (size_t)r0 * V, m->logits, sizeof(float) * (size_t)M * V,
                                   cudaMemcpyDeviceToHost, m->st));
             LS_CK(cudaStreamSynchronize(m->st));
         }
-        LS_TRY(run_layers(m, exit_layer, L, M, m->x, r0));
+        if (exit_layer < L) LS_TRY(run_layers(m, exit_layer, L, M, m->x, r0, 0, m->hE, m->fnorm, nullptr));
         if (final_logits) {
-            LS_TRY(run_head(m, M, m->x, m->verified, m->logits));
+            LS_TRY(run_head(m, M, 0, m->verified, m->logits));
             LS_CK(cudaMemcpyAsync(final_logits + (size_t)r0 * V, m->logits, sizeof(float) * (size_t)M * V,
                                   cudaMemcpyDeviceToHost, m->st));
             LS_CK(cudaStreamSynchronize(m->st));
@@ -766,7 +812,7 @@ int ls_op_embed(const void* emb, const int32_t* tok, int32_t M, int32_t D, int32
     if (!aligned16(emb) || !tok || !aligned16(x) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8 || V < 1)
         return LS_ERR_INVALID_ARG;
     LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, embed_kernel, dim3(M), dim3(256), 0, (const uint16_t*)emb, tok,
-                 D, V, x, nullptr));
+                 D, V, x, nullptr, nullptr, nullptr, nullptr, 0, 0));
     return LS_OK;
 }
 

@@ -23,32 +23,6 @@ __device__ __forceinline__ bool pass_begin(const int32_t* ctl, int pos_off, int&
     return true;
 }
 
-// ------------------------------------------------------------------ embedding (x_0 = Emb[id])
-// grid M, block 256.  tok[m] is read from device memory.
-__global__ void __launch_bounds__(256)
-embed_kernel(const uint16_t* __restrict__ emb, const int32_t* __restrict__ tok, int D, int V,
-             float* __restrict__ x, int32_t* ctl)
-{
-    pdl_launch_dependents();
-    pdl_wait();
-    if (ctl && ctl[CTL_DONE]) return;
-    int m = blockIdx.x;
-    int id = tok[m];
-    if (id < 0 || id >= V) {
-        if (ctl && threadIdx.x == 0) ctl[CTL_STATUS] = DEV_BAD_TOKEN;
-        id = 0;
-    }
-    const uint4* src = reinterpret_cast<const uint4*>(emb + (size_t)id * D);
-    float4* dst = reinterpret_cast<float4*>(x + (size_t)m * D);
-    for (int c = threadIdx.x; c < D / 8; c += blockDim.x) {
-        uint4 v = src[c];
-        dst[2 * c] = make_float4(bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y));
-        dst[2 * c + 1] = make_float4(bf16lo(v.z), bf16hi(v.z), bf16lo(v.w), bf16hi(v.w));
-    }
-}
-
-// ------------------------------------------------------------------ RMSNorm
-// grid M, block 256.  out = bf16(x / sqrt(mean x^2 + eps) * g).
 __device__ __forceinline__ float block_sum_256(float v, float* red)
 {
 #pragma unroll
@@ -61,6 +35,56 @@ __device__ __forceinline__ float block_sum_256(float v, float* red)
     return s;
 }
 
+// ------------------------------------------------------------------ embedding (x_0 = Emb[id])
+// grid M, block 256.  tok[m] is read from device memory.  With gain != nullptr the kernel
+// also leaves what the first layer's fused RMSNorm needs: hout = bf16(x * gain) and the
+// row's sum of squares in ss_out[m][0] (the other n_part - 1 partial sums are zero).
+__global__ void __launch_bounds__(256)
+embed_kernel(const uint16_t* __restrict__ emb, const int32_t* __restrict__ tok, int D, int V,
+             float* __restrict__ x, int32_t* ctl, const uint16_t* __restrict__ gain,
+             uint16_t* __restrict__ hout, float* __restrict__ ss_out, int ss_stride, int n_part)
+{
+    __shared__ float red[8];
+    pdl_launch_dependents();
+    pdl_wait();
+    if (ctl && ctl[CTL_DONE]) return;
+    int m = blockIdx.x;
+    int id = tok[m];
+    if (id < 0 || id >= V) {
+        if (ctl && threadIdx.x == 0) ctl[CTL_STATUS] = DEV_BAD_TOKEN;
+        id = 0;
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(emb + (size_t)id * D);
+    float4* dst = reinterpret_cast<float4*>(x + (size_t)m * D);
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < D / 8; c += 256) {
+        uint4 v = src[c];
+        const float f[8] = {bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y),
+                            bf16lo(v.z), bf16hi(v.z), bf16lo(v.w), bf16hi(v.w)};
+        dst[2 * c] = make_float4(f[0], f[1], f[2], f[3]);
+        dst[2 * c + 1] = make_float4(f[4], f[5], f[6], f[7]);
+        if (gain) {
+            const uint4 gv = reinterpret_cast<const uint4*>(gain)[c];
+            const float g[8] = {bf16lo(gv.x), bf16hi(gv.x), bf16lo(gv.y), bf16hi(gv.y),
+                                bf16lo(gv.z), bf16hi(gv.z), bf16lo(gv.w), bf16hi(gv.w)};
+            uint4 o;
+            o.x = pack_bf16(f[0] * g[0], f[1] * g[1]);
+            o.y = pack_bf16(f[2] * g[2], f[3] * g[3]);
+            o.z = pack_bf16(f[4] * g[4], f[5] * g[5]);
+            o.w = pack_bf16(f[6] * g[6], f[7] * g[7]);
+            reinterpret_cast<uint4*>(hout + (size_t)m * D)[c] = o;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+        }
+    }
+    if (gain) {
+        const float tot = block_sum_256(ss, red);
+        for (int i = threadIdx.x; i < n_part; i += 256) ss_out[(size_t)m * ss_stride + i] = (i == 0) ? tot : 0.f;
+    }
+}
+
+// ------------------------------------------------------------------ RMSNorm
+// grid M, block 256.  out = bf16(x / sqrt(mean x^2 + eps) * g).
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const float* __restrict__ x, const uint16_t* __restrict__ g, int D, float eps,
                uint16_t* __restrict__ out, const int32_t* ctl)

@@ -46,7 +46,28 @@ struct LinArgs {
     uint16_t *q_out, *kpages, *vpages;
     int Hq, Hkv, hd, page_shift, max_seq, pos_off;
     float theta;
+    // RMSNorm carried across kernel boundaries.  A producer (residual epilogue, embedding)
+    // leaves, beside the fp32 row x, the bf16 row x*gain of its consumer's norm and the sum
+    // of x^2 over its own columns; a consumer reads those rows as h, adds the partial sums in
+    // index order and scales its accumulators by 1/sqrt(mean x^2 + eps): W (x g) r = W (x r g).
+    const float* ss_in;      // consumer: [M][ss_stride] partial sums of squares; nullptr: no scaling
+    float* ss_out;           // EPI_RESIDUAL: ss_out[m * ss_stride + cta]
+    int ss_stride, n_part;   // n_part: partial sums per row (CTAs of the producer)
+    float inv_d, eps;
+    const uint16_t *gain_a, *gain_b;  // EPI_RESIDUAL: hout_x[m * N + n] = bf16(x_new[m][n] * gain_x[n])
+    uint16_t *hout_a, *hout_b;
 };
+
+// 1/sqrt(mean x^2 + eps) of row m from its partial sums: lanes stride over the partials,
+// then a butterfly -- a fixed order that depends on nothing but n_part
+__device__ __forceinline__ float row_rscale(const LinArgs& a, int m, int lane)
+{
+    float s = 0.f;
+    for (int i = lane; i < a.n_part; i += 32) s += __ldcg(a.ss_in + (size_t)m * a.ss_stride + i);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    return 1.0f / sqrtf(s * a.inv_d + a.eps);
+}
 
 // EPI_QKV tiles pair row j of a head with row j + hd/2, the two halves of one rotary pair:
 // tile b covers pairs j = 8 (b % (hd/16)) .. +7 of head b / (hd/16).
@@ -167,17 +188,50 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
             acc[r][m] = v;
         }
 
+    if (a.ss_in) {  // fused RMSNorm: scale row m by 1/sqrt(mean x^2 + eps)
+        __shared__ float rs[kMaxRows];
+        for (int m = warp; m < a.M; m += 4) {
+            const float v = row_rscale(a, m, lane);
+            if (lane == 0) rs[m] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            const float v = rs[min(m, a.M - 1)];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) acc[r][m] *= v;
+        }
+    }
+
     if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+        __shared__ float sq[4][MT];
 #pragma unroll
         for (int m = 0; m < MT; ++m)
-            if (lane == m && m < a.M) {
+            if (lane == m) {
+                float q = 0.f;
+                if (m < a.M) {
 #pragma unroll
-                for (int r = 0; r < 4; ++r)
-                    if (nrow[r] < a.N) {
-                        float* o = a.out + (size_t)m * a.ldo + nrow[r];
-                        *o = (EPI == EPI_RESIDUAL) ? (*o + acc[r][m]) : acc[r][m];
-                    }
+                    for (int r = 0; r < 4; ++r)
+                        if (nrow[r] < a.N) {
+                            float* o = a.out + (size_t)m * a.ldo + nrow[r];
+                            const float xn = (EPI == EPI_RESIDUAL) ? (*o + acc[r][m]) : acc[r][m];
+                            *o = xn;
+                            if (EPI == EPI_RESIDUAL) {
+                                q = fmaf(xn, xn, q);
+                                if (a.hout_a) a.hout_a[(size_t)m * a.N + nrow[r]] = f2bf(xn * bf16f(a.gain_a[nrow[r]]));
+                                if (a.hout_b) a.hout_b[(size_t)m * a.N + nrow[r]] = f2bf(xn * bf16f(a.gain_b[nrow[r]]));
+                            }
+                        }
+                }
+                sq[warp][m] = q;
             }
+        if (EPI == EPI_RESIDUAL && a.ss_out) {
+            __syncthreads();
+            if (threadIdx.x < MT && threadIdx.x < a.M) {
+                const int m = threadIdx.x;
+                a.ss_out[(size_t)m * a.ss_stride + blockIdx.x] = ((sq[0][m] + sq[1][m]) + sq[2][m]) + sq[3][m];
+            }
+        }
     } else if (EPI == EPI_SWIGLU) {
 #pragma unroll
         for (int m = 0; m < MT; ++m)
@@ -346,6 +400,13 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
         issue_h(warp + p * WARPS, p);
         cp_async_commit();
     }
+    __shared__ float rs[kMaxRows];
+    if (a.ss_in) {  // fused RMSNorm: per-row scale, computed while the first stages travel
+        for (int m = warp; m < a.M; m += WARPS) {
+            const float v = row_rscale(a, m, lane);
+            if (lane == 0) rs[m] = v;
+        }
+    }
     int rd = 0, wr = STAGES - 1;
     for (int step = warp; step < nsteps; step += WARPS) {
         issue_w(step + (STAGES - 1) * WARPS, wr);
@@ -397,14 +458,39 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             r[i] = s;
         }
         const int m0 = nt * 8 + 2 * tt;  // tokens m0, m0+1
+        if (a.ss_in) {
+            const float s0 = rs[min(m0, a.M - 1)], s1 = rs[min(m0 + 1, a.M - 1)];
+            r[0] *= s0;
+            r[1] *= s1;
+            r[2] *= s0;
+            r[3] *= s1;
+        }
         if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
             const int nlo = tile * 16 + gg, nhi = nlo + 8;
+            float q[2] = {0.f, 0.f};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 int m = m0 + (i & 1), n = (i < 2) ? nlo : nhi;
                 if (m < a.M && n < a.N) {
                     float* o = a.out + (size_t)m * a.ldo + n;
-                    *o = (EPI == EPI_RESIDUAL) ? (*o + r[i]) : r[i];
+                    const float xn = (EPI == EPI_RESIDUAL) ? (*o + r[i]) : r[i];
+                    *o = xn;
+                    if (EPI == EPI_RESIDUAL) {
+                        q[i & 1] = fmaf(xn, xn, q[i & 1]);
+                        if (a.hout_a) a.hout_a[(size_t)m * a.N + n] = f2bf(xn * bf16f(a.gain_a[n]));
+                        if (a.hout_b) a.hout_b[(size_t)m * a.N + n] = f2bf(xn * bf16f(a.gain_b[n]));
+                    }
+                }
+            }
+            if (EPI == EPI_RESIDUAL && a.ss_out) {  // sum over the tile's 16 rows: lanes of equal tt
+#pragma unroll
+                for (int sh = 4; sh < 32; sh <<= 1) {
+                    q[0] += __shfl_xor_sync(0xffffffffu, q[0], sh);
+                    q[1] += __shfl_xor_sync(0xffffffffu, q[1], sh);
+                }
+                if (gg == 0) {
+                    if (m0 < a.M) a.ss_out[(size_t)m0 * a.ss_stride + tile] = q[0];
+                    if (m0 + 1 < a.M) a.ss_out[(size_t)(m0 + 1) * a.ss_stride + tile] = q[1];
                 }
             }
         } else if (EPI == EPI_SWIGLU) {
