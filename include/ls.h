@@ -243,6 +243,22 @@ int ls_op_attention(const void *q_bf16_dev, int32_t M, int32_t pos0, int32_t Hq,
                     const void *k_pages_dev, const void *v_pages_dev, void *scratch_dev,
                     void *out_bf16_dev, void *cuda_stream);
 
+/* Kernels of the prompt pass (the rows that go through the model before the first draft,
+ * Appendix A.4), which is a dense contraction over hundreds of rows.
+ * ls_op_gemm: c[m, n] (+)= sum_k a[m, k] b[n, k] on the tcgen05 tensor cores; a bf16 [M, K],
+ * b bf16 [N, K], c fp32 with leading dimension ldc >= N; accumulate != 0 adds to c (the
+ * residual update of Sec. 4.1).  status_dev (device int32, may be NULL) receives 3 if one of
+ * the kernel's bounded waits ran out.
+ * ls_op_prefill_attention: causal attention of R rows at positions pos0 .. pos0+R-1 over the
+ * paged cache (as ls_op_attention, any R, no scratch: one CTA walks the key chunks of its 16
+ * rows in order with a running max / sum). */
+int ls_op_gemm(const void *a_bf16_dev, const void *b_bf16_dev, int32_t M, int32_t N, int32_t K,
+               float *c_dev, int32_t ldc, int32_t accumulate, int32_t *status_dev, void *cuda_stream);
+int ls_op_prefill_attention(const void *q_bf16_dev, int32_t R, int32_t pos0, int32_t Hq, int32_t Hkv,
+                            int32_t hd, int32_t page_size, const int32_t *page_table_dev,
+                            int32_t max_seq, const void *k_pages_dev, const void *v_pages_dev,
+                            void *out_bf16_dev, void *cuda_stream);
+
 /* match + crop of Appendix A.4 on device arrays: n = number of leading i < d with
  * draft[i] == verified[i]; appends draft[0..n-1], verified[n] to out_ids (truncated at
  * max_new, and after the first eos_id if eos_id >= 0).

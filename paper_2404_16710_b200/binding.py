@@ -27,6 +27,7 @@ EXPORTS = (
     "ls_decode", "ls_read_output", "ls_debug_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
     "ls_op_linear", "ls_op_gate_up_swiglu", "ls_op_lm_head_scratch_bytes", "ls_op_lm_head_argmax",
     "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_qkv_rope_append", "ls_op_attention_scratch_bytes", "ls_op_attention", "ls_op_accept",
+    "ls_op_gemm", "ls_op_prefill_attention",
 )
 
 
@@ -102,6 +103,8 @@ def lib():
             "ls_op_attention_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
             "ls_op_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]),
             "ls_op_accept": (C.c_int, [vp, vp, i32, vp, vp, vp, vp]),
+            "ls_op_gemm": (C.c_int, [vp, vp, i32, i32, i32, vp, i32, i32, vp, vp]),
+            "ls_op_prefill_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -298,6 +301,18 @@ def ls_op_attention_scratch_bytes(Hq, hd, max_seq):
 def ls_op_attention(q, pos0, Hq, Hkv, hd, page_size, page_table, max_seq, k_pages, v_pages, scratch, out):
     _ck(lib().ls_op_attention(_dev(q), q.shape[0], pos0, Hq, Hkv, hd, page_size, _dev(page_table), max_seq,
                               _dev(k_pages), _dev(v_pages), _dev(scratch), _dev(out), _stream()), "ls_op_attention")
+
+
+def ls_op_gemm(a, b, c, accumulate=False, status=None):
+    """c[M, N] (+)= a[M, K] @ b[N, K].T  (bf16 inputs, fp32 c, tcgen05 tensor cores)"""
+    (M, K), N = a.shape, b.shape[0]
+    _ck(lib().ls_op_gemm(_dev(a), _dev(b), M, N, K, _dev(c), c.stride(0), int(accumulate), _dev(status), _stream()),
+        "ls_op_gemm")
+
+
+def ls_op_prefill_attention(q, pos0, Hq, Hkv, hd, page_size, page_table, max_seq, k_pages, v_pages, out):
+    _ck(lib().ls_op_prefill_attention(_dev(q), q.shape[0], pos0, Hq, Hkv, hd, page_size, _dev(page_table), max_seq,
+                                      _dev(k_pages), _dev(v_pages), _dev(out), _stream()), "ls_op_prefill_attention")
 
 
 def ls_op_accept(draft, verified, d, state, out_ids, accepted):

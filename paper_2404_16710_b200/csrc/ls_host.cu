@@ -23,6 +23,7 @@
 
 #include "ls.h"
 #include "ls_linear.cuh"
+#include "ls_prefill.cuh"
 
 using namespace ls;
 
@@ -44,6 +45,8 @@ thread_local int g_last_cuda = 0;
         int rc_ = (expr);       \
         if (rc_ != LS_OK) return rc_; \
     } while (0)
+
+constexpr int kPrefillBlock = 512;  // rows the prompt pass handles at a time
 
 struct LayerW {
     const uint16_t *attn_norm, *wq, *wk, *wv, *wo, *ffn_norm, *wg, *wu, *wd;
@@ -89,13 +92,15 @@ struct ls_model {
     float *inv_freq, *x, *qkv, *part, *logits;
     uint16_t *h, *q, *o, *a;
     uint16_t* hE;  // exit-layer activations, already multiplied by the gain of layer E's norm (Sec. 4.3.3)
+    float *px, *py;          // prompt pass: residual rows and projection outputs of one block
+    uint16_t *ph, *pq, *po, *pa;
     float* ss;     // [16][n_part] partial sums of squares of the residual rows (fused RMSNorm)
     int n_part;
     ValIdx* cand;
     int page_shift, n_pages, chunk_cap, cand_stride;
     // loop state
     int n_prompt, last_tok, prefilled_layers, grid_chunks;
-    bool use_graphs, own_stream, pdl;
+    bool use_graphs, own_stream, pdl, big_prefill;
     int64_t launches;  // kernels enqueued (counted while building a step)
     struct G {
         cudaGraphExec_t exec;
@@ -147,7 +152,21 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     const int n_part = (c.d_model + 15) / 16;  // CTAs of a residual projection = partial sums per row
     unsigned char* ss = take(sizeof(float) * kMaxRows * n_part);
     unsigned char* he = take(2 * (size_t)kMaxRows * c.d_model);
+    const int pb = c.max_seq < kPrefillBlock ? c.max_seq : kPrefillBlock;  // rows per block of the prompt pass
+    const size_t ywide = (qw + 2 * kvw) > 2 * (size_t)c.d_ffn ? (qw + 2 * kvw) : 2 * (size_t)c.d_ffn;
+    unsigned char* px = take(sizeof(float) * (size_t)pb * c.d_model);
+    unsigned char* ph = take(2 * (size_t)pb * c.d_model);
+    unsigned char* py = take(sizeof(float) * (size_t)pb * ywide);
+    unsigned char* pq = take(2 * (size_t)pb * qw);
+    unsigned char* po = take(2 * (size_t)pb * qw);
+    unsigned char* pa = take(2 * (size_t)pb * c.d_ffn);
     if (m) {
+        m->px = (float*)px;
+        m->ph = (uint16_t*)ph;
+        m->py = (float*)py;
+        m->pq = (uint16_t*)pq;
+        m->po = (uint16_t*)po;
+        m->pa = (uint16_t*)pa;
         m->ss = (float*)ss;
         m->hE = (uint16_t*)he;
         m->n_part = n_part;
@@ -346,6 +365,114 @@ int run_embed(ls_model* m, const int32_t* tok_dev, int M, float* xrow, int slot)
     return LS_OK;
 }
 
+// ------------------------------------------------------------------ prompt pass (large M)
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TensorMapEncodeFn tensor_map_encoder()
+{
+    static TensorMapEncodeFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (TensorMapEncodeFn)p;
+    }
+    return fn;
+}
+
+// 2-D map of a row-major bf16 matrix [rows, K]: boxes of 64 columns (128 bytes) x 128 rows,
+// 128-byte swizzle, zeros outside the matrix
+int make_tile_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K)
+{
+    TensorMapEncodeFn fn = tensor_map_encoder();
+    if (!fn) return LS_ERR_UNSUPPORTED;
+    cuuint64_t dims[2] = {K, rows};
+    cuuint64_t strides[1] = {K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kGemmBK, (cuuint32_t)kGemmBM};
+    cuuint32_t es[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? LS_OK : LS_ERR_INVALID_ARG;
+}
+
+// C[M, N] (+)= A[M, K] B[N, K]^T on the tensor cores (tcgen05), A and B bf16, C fp32
+int gemm_launch(const uint16_t* A, const uint16_t* B, int M, int N, int K, float* C, int ldc, int accumulate,
+                int32_t* status, cudaStream_t st)
+{
+    static bool allowed[64] = {false};
+    int dev = 0;
+    LS_CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !allowed[dev]) {
+        LS_CK(cudaFuncSetAttribute(gemm_bf16_tn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes));
+        if (dev >= 0 && dev < 64) allowed[dev] = true;
+    }
+    CUtensorMap ma, mb;
+    LS_TRY(make_tile_map(&ma, A, (uint64_t)M, (uint64_t)K));
+    LS_TRY(make_tile_map(&mb, B, (uint64_t)N, (uint64_t)K));
+    dim3 grid((N + kGemmBN - 1) / kGemmBN, (M + kGemmBM - 1) / kGemmBM);
+    gemm_bf16_tn_kernel<<<grid, 128, kGemmSmemBytes, st>>>(ma, mb, M, N, K, C, ldc, accumulate, status);
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+int prefill_attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt, int pos0, int R,
+                        int Hq, int Hkv, int hd, int page_shift, uint16_t* out, cudaStream_t st)
+{
+    const int Q = Hq / Hkv * kMaxRows;
+    dim3 grid((R + 15) / 16, Hkv);
+    if (hd == 128) {
+        const size_t sm = prefill_attn_smem_bytes<128>(Q);
+        LS_CK(cudaFuncSetAttribute(prefill_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+        prefill_attn_kernel<128><<<grid, kAttnThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
+    } else {
+        const size_t sm = prefill_attn_smem_bytes<64>(Q);
+        LS_CK(cudaFuncSetAttribute(prefill_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+        prefill_attn_kernel<64><<<grid, kAttnThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
+    }
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
+// rows [r0, r0 + R) of the prompt (ids already on the device) through layers [0, layers):
+// fills the KV cache of those positions.  Unfused on purpose: this pass is compute-bound.
+int prefill_block(ls_model* m, int r0, int R, int layers)
+{
+    const ls_config& c = m->c;
+    const int D = c.d_model, Hq = c.n_heads, Hkv = c.n_kv_heads, hd = c.head_dim, F = c.d_ffn;
+    const int qw = Hq * hd, kvw = Hkv * hd, qkvw = qw + 2 * kvw;
+    cudaStream_t st = m->st;
+    const LaunchCtx lc = {st, false};
+    int32_t* status = m->ctl + CTL_STATUS;
+    LS_CK(launch(lc, embed_kernel, dim3(R), dim3(256), 0, m->emb, m->ids + r0, D, c.vocab, m->px, m->ctl, nullptr,
+                 nullptr, nullptr, 0, 0));
+    for (int l = 0; l < layers; ++l) {
+        const LayerW& w = m->lw[l];
+        uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
+        uint16_t* vp = m->vpages + (size_t)l * m->layer_kv_elems;
+        LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.attn_norm, D, c.rms_eps, m->ph, nullptr));
+        LS_TRY(gemm_launch(m->ph, w.wq, R, qw, D, m->py, qkvw, 0, status, st));
+        LS_TRY(gemm_launch(m->ph, w.wk, R, kvw, D, m->py + qw, qkvw, 0, status, st));
+        LS_TRY(gemm_launch(m->ph, w.wv, R, kvw, D, m->py + qw + kvw, qkvw, 0, status, st));
+        LS_CK(launch(lc, rope_append_kernel, dim3(R, Hq + 2 * Hkv), dim3(hd / 2), 0, m->py, Hq, Hkv, hd, m->inv_freq,
+                     c.rope_theta, m->page_shift, m->page_table, c.max_seq, m->pq, kp, vp, m->ctl, r0));
+        LS_TRY(prefill_attn_launch(m->pq, kp, vp, m->page_table, r0, R, Hq, Hkv, hd, m->page_shift, m->po, st));
+        LS_TRY(gemm_launch(m->po, w.wo, R, D, qw, m->px, D, 1, status, st));
+        LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.ffn_norm, D, c.rms_eps, m->ph, nullptr));
+        LS_TRY(gemm_launch(m->ph, w.wg, R, F, D, m->py, 2 * F, 0, status, st));
+        LS_TRY(gemm_launch(m->ph, w.wu, R, F, D, m->py + F, 2 * F, 0, status, st));
+        swiglu_rows_kernel<<<R, 256, 0, st>>>(m->py, F, m->pa);
+        LS_TRY(gemm_launch(m->pa, w.wd, R, D, F, m->px, D, 1, status, st));
+        m->launches += 13;
+    }
+    LS_CK(cudaGetLastError());
+    return LS_OK;
+}
+
 // one step of the loop.  E == L with d == 0: plain greedy; E < L with d == 0: early exit.
 int enqueue_step(ls_model* m, int E, int d)
 {
@@ -530,6 +657,7 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
     m->grid_chunks = m->chunk_cap;
     m->use_graphs = getenv("LS_NO_GRAPH") == nullptr;
     m->pdl = getenv("LS_NO_PDL") == nullptr;
+    m->big_prefill = getenv("LS_SMALL_PREFILL") == nullptr && tensor_map_encoder() != nullptr;
     m->launches = 0;
     memset(&m->stats, 0, sizeof(m->stats));
     m->h_n_out = m->h_n_steps = 0;
@@ -604,11 +732,18 @@ int ls_prefill(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t lay
     LS_CK(cudaMemcpyAsync(m->ids, prompt, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, m->st));
     LS_TRY(write_ctl(m, 0, 0, 0));
     LS_CK(cudaEventRecord(m->ev0, m->st));
-    for (int r0 = 0; r0 < n_prompt - 1; r0 += kMaxRows) {
-        int M = n_prompt - 1 - r0;
-        if (M > kMaxRows) M = kMaxRows;
-        LS_TRY(run_embed(m, m->ids + r0, M, m->x, 0));
-        LS_TRY(run_layers(m, 0, layers, M, m->x, r0, 0, m->h, nullptr, nullptr));
+    const int rows = n_prompt - 1;
+    if (rows > kMaxRows && m->big_prefill) {
+        // the prompt pass proper: blocks of up to 512 rows on the tensor cores
+        const int pb = m->c.max_seq < kPrefillBlock ? m->c.max_seq : kPrefillBlock;
+        for (int r0 = 0; r0 < rows; r0 += pb) LS_TRY(prefill_block(m, r0, rows - r0 < pb ? rows - r0 : pb, layers));
+    } else {
+        for (int r0 = 0; r0 < rows; r0 += kMaxRows) {
+            int M = rows - r0;
+            if (M > kMaxRows) M = kMaxRows;
+            LS_TRY(run_embed(m, m->ids + r0, M, m->x, 0));
+            LS_TRY(run_layers(m, 0, layers, M, m->x, r0, 0, m->h, nullptr, nullptr));
+        }
     }
     LS_CK(cudaEventRecord(m->ev1, m->st));
     int32_t w[CTL_WORDS];
@@ -998,6 +1133,27 @@ int ls_op_attention(const void* q, int32_t M, int32_t pos0, int32_t Hq, int32_t 
     return attn_launch((const uint16_t*)q, (const uint16_t*)kp, (const uint16_t*)vp, page_table, nullptr, pos0, M, Hq,
                        Hkv, hd, log2_exact(page_size), max_seq, cap, chunks, (float*)scratch, counters, (uint16_t*)out,
                        LaunchCtx{(cudaStream_t)stream, false});
+}
+
+int ls_op_gemm(const void* a, const void* b, int32_t M, int32_t N, int32_t K, float* c, int32_t ldc, int32_t accumulate,
+               int32_t* status_dev, void* stream)
+{
+    if (!aligned16(a) || !aligned16(b) || !c || M < 1 || N < 1 || K < 8 || K % 8 || ldc < N) return LS_ERR_INVALID_ARG;
+    return gemm_launch((const uint16_t*)a, (const uint16_t*)b, M, N, K, c, ldc, accumulate, status_dev,
+                       (cudaStream_t)stream);
+}
+
+int ls_op_prefill_attention(const void* q, int32_t R, int32_t pos0, int32_t Hq, int32_t Hkv, int32_t hd,
+                            int32_t page_size, const int32_t* page_table, int32_t max_seq, const void* kp,
+                            const void* vp, void* out, void* stream)
+{
+    if (R < 1 || pos0 < 0 || Hq < 1 || Hkv < 1 || Hq % Hkv || Hq / Hkv > 8 || (hd != 64 && hd != 128) ||
+        page_size < 16 || page_size > 1024 || log2_exact(page_size) < 0)
+        return LS_ERR_INVALID_ARG;
+    if ((int64_t)pos0 + R > max_seq) return LS_ERR_CAPACITY;
+    if (!aligned16(q) || !page_table || !aligned16(kp) || !aligned16(vp) || !out) return LS_ERR_INVALID_ARG;
+    return prefill_attn_launch((const uint16_t*)q, (const uint16_t*)kp, (const uint16_t*)vp, page_table, pos0, R, Hq,
+                               Hkv, hd, log2_exact(page_size), (uint16_t*)out, (cudaStream_t)stream);
 }
 
 int ls_op_accept(const int32_t* draft, const int32_t* verified, int32_t d, int32_t* state, int32_t* out_ids,

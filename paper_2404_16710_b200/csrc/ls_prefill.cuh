@@ -1,0 +1,380 @@
+// The prompt pass (everything before the decode loop starts): hundreds to thousands of
+// rows at once, so its projections are real dense contractions and run on the 5th-gen
+// tensor cores -- TMA tiles into 128B-swizzled shared memory, tcgen05.mma issued by one
+// thread with the fp32 accumulator in tensor memory, tcgen05.ld for the epilogue.  Both
+// ls_generate and ls_generate_full start from this same pass, so it needs no bit-for-bit
+// relation to the small-M decode kernels; it only has to fill the KV cache the way the
+// model defines it (LayerSkip Sec. 4.1 for the decoder; the appendix listing feeds the
+// prompt through the model before the first draft).
+#pragma once
+#include <cuda.h>
+
+#include "ls_kernels.cuh"
+
+namespace ls {
+
+// ------------------------------------------------------------------ small PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait: false if the phase did not complete within the poll budget (about a second).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (it > 1024) __nanosleep(200);
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, bf16 inputs, fp32 accumulate
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) and
+// 128B-swizzled as TMA wrote them: 8-row groups 1024 bytes apart (stride byte offset),
+// leading byte offset unused for swizzled K-major (1), descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// ------------------------------------------------------------------ GEMM: C[M,N] (+)= A[M,K] B[N,K]^T
+constexpr int kGemmBM = 128, kGemmBN = 128, kGemmBK = 64, kGemmStages = 6;
+constexpr int kGemmStageBytes = (kGemmBM + kGemmBN) * kGemmBK * 2;                   // 32 KB
+constexpr size_t kGemmSmemBytes = (size_t)kGemmStages * kGemmStageBytes + 1024 + 256;  // + alignment + barriers
+constexpr int DEV_TIMEOUT = 3;
+
+// grid (ceil(N/128), ceil(M/128)), block 128.  Warp 0 allocates tensor memory and its lane 0
+// feeds the ring with TMA; lane 0 of warp 1 issues the MMAs; all four warps read their 32
+// accumulator lanes back and store (accumulate != 0: add to C, the residual update).
+// Rows beyond M and columns beyond K come out of TMA as zeros.  Every wait is bounded; on a
+// time-out the kernel records DEV_TIMEOUT in *status, still frees its tensor memory, returns.
+__global__ void __launch_bounds__(128)
+gemm_bf16_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int M,
+                    int N, int K, float* __restrict__ C, int ldc, int accumulate, int32_t* status)
+{
+    extern __shared__ unsigned char gsm_raw[];
+    const uint32_t base = (smem_u32(gsm_raw) + 1023u) & ~1023u;  // swizzled tiles want 1024-byte alignment
+    const uint32_t bars = base + kGemmStages * kGemmStageBytes;  // full[S], empty[S], accum, tmem slot
+    auto full = [&](int s) { return bars + 8u * s; };
+    auto empty = [&](int s) { return bars + 8u * (kGemmStages + s); };
+    const uint32_t accum = bars + 8u * (2 * kGemmStages);
+    const uint32_t tslot = accum + 8u;
+    __shared__ int failed;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n0 = blockIdx.x * kGemmBN, m0 = blockIdx.y * kGemmBM;
+    const int nkb = (K + kGemmBK - 1) / kGemmBK;
+    if (tid == 0) {
+        for (int s = 0; s < kGemmStages; ++s) {
+            mbar_init(full(s), 1);
+            mbar_init(empty(s), 1);
+        }
+        mbar_init(accum, 1);
+        failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tslot), "r"(kGemmBN)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    uint32_t tmem;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem) : "r"(tslot));
+
+    if (warp == 0 && lane == 0) {  // TMA producer
+        for (int kb = 0; kb < nkb; ++kb) {
+            const int s = kb % kGemmStages;
+            if (kb >= kGemmStages && !mbar_wait(empty(s), ((kb / kGemmStages) - 1) & 1)) {
+                failed = 1;
+                break;
+            }
+            mbar_expect_tx(full(s), kGemmStageBytes);
+            const uint32_t sa = base + s * kGemmStageBytes, sb = sa + kGemmBM * kGemmBK * 2;
+            tma_load_2d(sa, &map_a, kb * kGemmBK, m0, full(s));
+            tma_load_2d(sb, &map_b, kb * kGemmBK, n0, full(s));
+        }
+    } else if (warp == 1 && lane == 0) {  // MMA issuer
+        // instruction descriptor: D fp32, A and B bf16, both K-major, N = 128, M = 128
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kGemmBN >> 3) << 17) |
+                               ((uint32_t)(kGemmBM >> 4) << 24);
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int s = kb % kGemmStages;
+            if (!mbar_wait(full(s), (kb / kGemmStages) & 1)) {
+                failed = 1;
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const uint32_t sa = base + s * kGemmStageBytes, sb = sa + kGemmBM * kGemmBK * 2;
+            const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sb);
+#pragma unroll
+            for (int k4 = 0; k4 < kGemmBK / 16; ++k4)  // 32 bytes (16 bf16) further along K per MMA
+                tc_mma_bf16(tmem, da + 2 * k4, db + 2 * k4, idesc, (kb | k4) != 0);
+            tc_commit(empty(s));  // arrives once these MMAs have finished reading the stage
+        }
+        tc_commit(accum);
+    }
+    __syncwarp();
+
+    // epilogue: warp w owns accumulator lanes 32w..32w+31 = rows m0 + 32w + lane
+    bool have = mbar_wait(accum, 0);
+    if (!have) failed = 1;
+    tc_fence_after();
+    __syncthreads();
+    if (!failed) {
+        const int row = m0 + warp * 32 + lane;
+#pragma unroll 1
+        for (int c = 0; c < kGemmBN / 32; ++c) {
+            uint32_t v[32];
+            tc_ld32(tmem + ((uint32_t)(warp * 32) << 16) + c * 32, v);
+            if (row < M) {
+                float* dst = C + (size_t)row * ldc + n0 + c * 32;
+                if (n0 + c * 32 + 32 <= N && (((uintptr_t)dst) & 15u) == 0) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                               __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                        if (accumulate) {
+                            const float4 p = *reinterpret_cast<const float4*>(dst + j);
+                            o.x += p.x;
+                            o.y += p.y;
+                            o.z += p.z;
+                            o.w += p.w;
+                        }
+                        *reinterpret_cast<float4*>(dst + j) = o;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (n0 + c * 32 + j < N) dst[j] = accumulate ? dst[j] + __uint_as_float(v[j]) : __uint_as_float(v[j]);
+                }
+            }
+        }
+    } else if (tid == 0 && status) {
+        *status = DEV_TIMEOUT;
+        __nanosleep(1000000);  // let copies that may still be in flight land before the CTA goes away
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kGemmBN) : "memory");
+}
+
+// ------------------------------------------------------------------ elementwise helpers of the prompt pass
+// a[m, f] = bf16(silu(gu[m, f]) * gu[m, F + f]); grid (rows), block 256
+__global__ void __launch_bounds__(256)
+swiglu_rows_kernel(const float* __restrict__ gu, int F, uint16_t* __restrict__ a)
+{
+    const float* g = gu + (size_t)blockIdx.x * 2 * F;
+    uint16_t* o = a + (size_t)blockIdx.x * F;
+    for (int f = threadIdx.x; f < F; f += 256) {
+        const float x = g[f];
+        o[f] = f2bf(x / (1.0f + expf(-x)) * g[F + f]);
+    }
+}
+
+// ------------------------------------------------------------------ causal attention of the prompt pass
+// grid (ceil(R/16), Hkv), block 256.  CTA = 16 consecutive rows (positions pos0 + 16 b ..),
+// KV head kh, its G query heads; it walks the key chunks 0 .. last visible in order with a
+// running (max, sum, o) per query in shared memory -- no partials, no merge.
+// shared memory: Ks | Vs | Qs f32 [Q][HD] | S f32 [Q][64] | O f32 [Q][HD] | mx, l, alpha f32 [Q] each
+template <int HD>
+__host__ __device__ constexpr size_t prefill_attn_smem_bytes(int Q)
+{
+    return (size_t)kAttnChunk * (HD * 2 + 64) + (size_t)kAttnChunk * (HD * 2 + 32) +
+           sizeof(float) * (2 * (size_t)Q * HD + (size_t)Q * kAttnChunk + 3 * (size_t)Q);
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kAttnThreads)
+prefill_attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
+                    const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table, int pos0, int R,
+                    int Hq, int Hkv, int page_shift, uint16_t* __restrict__ out)
+{
+    constexpr int C = kAttnChunk, T = kAttnThreads;
+    constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 32, HALF = HD / 2, NKS = T / HALF;
+    const int tid = threadIdx.x, kh = blockIdx.y;
+    const int r0 = blockIdx.x * 16;
+    const int M = min(16, R - r0);
+    const int G = Hq / Hkv, Q = G * M;
+    const int first_pos = pos0 + r0, last_pos = first_pos + M - 1;
+
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned char* Ks = smem;
+    unsigned char* Vs = Ks + C * KROW;
+    float* Qs = reinterpret_cast<float*>(Vs + C * VROW);
+    float* S = Qs + (size_t)Q * HD;
+    float* O = S + (size_t)Q * C;
+    float* mx = O + (size_t)Q * HD;
+    float* ls = mx + Q;
+    float* al = ls + Q;
+
+    for (int idx = tid; idx < Q * HALF; idx += T) {
+        const int qi = idx / HALF, dp = idx % HALF;
+        const int m = qi / G, g = qi % G;
+        const uint32_t u =
+            *reinterpret_cast<const uint32_t*>(q + ((size_t)(r0 + m) * Hq + (size_t)kh * G + g) * HD + 2 * dp);
+        Qs[2 * idx] = bf16lo(u);
+        Qs[2 * idx + 1] = bf16hi(u);
+        O[2 * idx] = 0.f;
+        O[2 * idx + 1] = 0.f;
+    }
+    for (int qi = tid; qi < Q; qi += T) {
+        mx[qi] = -INFINITY;
+        ls[qi] = 0.f;
+    }
+
+    const int nch = last_pos / C + 1;
+    const float scale = rsqrtf((float)HD);
+    for (int ch = 0; ch < nch; ++ch) {
+        const int key0 = ch * C;
+        __syncthreads();  // previous chunk's K, V, S are no longer read
+        {
+            constexpr int SEGS = HD * 2 / 16;
+            const uint32_t ks0 = smem_u32(Ks), vs0 = smem_u32(Vs);
+            for (int idx = tid; idx < C * SEGS; idx += T) {
+                const int r = idx / SEGS, sg = idx % SEGS;
+                const int p = key0 + r;
+                const bool ok = p <= last_pos;
+                const size_t off = kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD) + (size_t)sg * 8;
+                cp_async16_cg(ks0 + r * KROW + sg * 16, kpages + off, ok ? 16 : 0);
+                cp_async16_cg(vs0 + r * VROW + sg * 16, vpages + off, ok ? 16 : 0);
+            }
+            cp_async_commit();
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        {
+            const int key = tid >> 2, qd = tid & 3;
+            const unsigned char* krow = Ks + key * KROW;
+            int q0 = 0;
+            for (; q0 + 4 <= Q; q0 += 4) attn_qk<HD, 4>(krow, Qs, q0, qd, S, key, qd == 0);
+            for (; q0 < Q; ++q0) attn_qk<HD, 1>(krow, Qs, q0, qd, S, key, qd == 0);
+        }
+        __syncthreads();
+        {
+            const int warp = tid >> 5, lane = tid & 31;
+            for (int qi = warp; qi < Q; qi += T / 32) {
+                const int pos = first_pos + qi / G;
+                float s0 = S[(size_t)qi * C + lane] * scale;
+                float s1 = S[(size_t)qi * C + lane + 32] * scale;
+                if (key0 + lane > pos) s0 = -INFINITY;
+                if (key0 + lane + 32 > pos) s1 = -INFINITY;
+                float cm = fmaxf(s0, s1);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, o));
+                const float mo = mx[qi], mn = fmaxf(mo, cm);
+                const float p0 = (s0 == -INFINITY) ? 0.f : expf(s0 - mn);
+                const float p1 = (s1 == -INFINITY) ? 0.f : expf(s1 - mn);
+                float l = p0 + p1;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+                S[(size_t)qi * C + lane] = p0;
+                S[(size_t)qi * C + lane + 32] = p1;
+                if (lane == 0) {
+                    const float a = (mn == -INFINITY) ? 1.f : ((mo == -INFINITY) ? 0.f : expf(mo - mn));
+                    al[qi] = a;
+                    ls[qi] = ls[qi] * a + l;
+                    mx[qi] = mn;
+                }
+            }
+        }
+        __syncthreads();
+        {
+            const int ks = tid % NKS, dp = tid / NKS;
+            int q0 = 0;
+            for (; q0 + 4 <= Q; q0 += 4) {
+                float o[4][2];
+                attn_pv<HD, 4, NKS>(Vs, S, q0, dp, ks, o);
+                if (ks == 0) {
+#pragma unroll
+                    for (int qq = 0; qq < 4; ++qq) {
+                        float* dst = O + (size_t)(q0 + qq) * HD + 2 * dp;
+                        const float a = al[q0 + qq];
+                        dst[0] = dst[0] * a + o[qq][0];
+                        dst[1] = dst[1] * a + o[qq][1];
+                    }
+                }
+            }
+            for (; q0 < Q; ++q0) {
+                float o[1][2];
+                attn_pv<HD, 1, NKS>(Vs, S, q0, dp, ks, o);
+                if (ks == 0) {
+                    float* dst = O + (size_t)q0 * HD + 2 * dp;
+                    const float a = al[q0];
+                    dst[0] = dst[0] * a + o[0][0];
+                    dst[1] = dst[1] * a + o[0][1];
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < Q * HALF; idx += T) {
+        const int qi = idx / HALF, dp = idx % HALF;
+        const int m = qi / G, g = qi % G;
+        const float l = ls[qi];
+        *reinterpret_cast<uint32_t*>(out + ((size_t)(r0 + m) * Hq + (size_t)kh * G + g) * HD + 2 * dp) =
+            pack_bf16(O[2 * idx] / l, O[2 * idx + 1] / l);
+    }
+}
+
+}  // namespace ls

@@ -346,3 +346,47 @@ def test_argument_errors_are_reported_not_launched():
         B.ls_op_linear(B.LS_LINEAR_FMA, w, h, torch.zeros((17, 16), dtype=torch.float32, device="cuda"))
     with pytest.raises(B.LsError):
         B.ls_op_linear(3, w, h[:1].contiguous(), out)
+
+
+# ------------------------------------------------------------------ prompt pass: tcgen05 GEMM, causal attention
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (31, 256, 256), (200, 688, 256), (512, 4096, 4096), (300, 1024, 11008),
+                                   (130, 100, 72)])
+@pytest.mark.parametrize("accumulate", [False, True])
+def test_gemm_tensor_core(M, N, K, accumulate):
+    a = rnd((M, K), 90).bfloat16()
+    b = rnd((N, K), 91, 0.05).bfloat16()
+    c = rnd((M, N), 92) if accumulate else torch.full((M, N), float("nan"), device="cuda")
+    base = c.clone()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.ls_op_gemm(a, b, c, accumulate, status)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0, "a bounded wait inside the GEMM ran out"
+    rows = np.unique(np.concatenate([[0, M - 1, min(M - 1, 127), min(M - 1, 128)],
+                                     np.random.default_rng(2).integers(0, M, 6)]))
+    bb = bits(b)
+    got = c.cpu().numpy().astype(np.float64)
+    for m in rows:
+        ref = O.linear(bb, vals(a[m])) + (base[m].cpu().numpy() if accumulate else 0.0)
+        np.testing.assert_allclose(got[m], ref, rtol=0, atol=2e-5 * np.abs(ref).max() + 1e-6)
+    assert np.isfinite(got).all()
+
+
+@pytest.mark.parametrize("Hq,Hkv,hd", [(4, 2, 64), (4, 4, 128), (8, 2, 128)])
+@pytest.mark.parametrize("R,pos0", [(1, 0), (16, 0), (37, 0), (100, 0), (50, 70)])
+def test_prefill_attention(Hq, Hkv, hd, R, pos0):
+    page_size, max_seq = 32, 256
+    table, table_d, kp, vp = kv_setup(Hkv, hd, page_size, max_seq, True)
+    n = pos0 + R
+    kl = rnd((n + 8, Hkv, hd), 50).bfloat16()
+    vl = rnd((n + 8, Hkv, hd), 51).bfloat16()
+    for p in range(n + 8):
+        kp[table[p // page_size], :, p % page_size, :] = kl[p]
+        vp[table[p // page_size], :, p % page_size, :] = vl[p]
+    q = rnd((R, Hq * hd), 52, 0.5).bfloat16()
+    out = torch.empty((R, Hq * hd), dtype=torch.bfloat16, device="cuda")
+    B.ls_op_prefill_attention(q, pos0, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp, out)
+    torch.cuda.synchronize()
+    kf, vf, qf = vals(kl).reshape(n + 8, -1), vals(vl).reshape(n + 8, -1), vals(q)
+    for m in sorted({0, R // 2, R - 1, min(R - 1, 15), min(R - 1, 16)}):
+        ref = O.attention(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd)
+        np.testing.assert_allclose(vals(out[m]), ref, rtol=0, atol=BF16_REL * np.abs(ref).max() + 1e-5)
