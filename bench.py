@@ -36,6 +36,11 @@ from paper_2404_16710_b200 import synth  # noqa: E402
 METRIC = "batch-1 generated tokens/s, self-speculative greedy decode"
 UNIT = "tokens/s"
 
+# DRAM bytes (read + write) of one launch of the roofline kernel, from the ncu capture that
+# profiles/linear_mma_kernel_llama2-7b_shapes.md summarises; keyed by (workload, rows).  Set an
+# entry to None when the kernel changes until the counters have been taken again.
+ROOFLINE_TRAFFIC = {("llama2-7b", 7): 180.43e6 + 4.1e6}
+
 
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -254,7 +259,8 @@ def run_own(args):
            "config": {"workload": args.workload, "shape": s.name, "n_prompt": P, "max_new": NEW, "exit_layer": E,
                       "num_draft": d, "late_scale": wl.late_scale, "linear_path": "mma" if path == 2 else "fma",
                       "l2": "inputs (weights) larger than L2", "replicas": world,
-                      "timed_region": "decode loop from a prefilled prompt, device-resident"},
+                      "timed_region": "decode loop from a prefilled prompt, device-resident",
+                      "kernels_per_layer": 5, "prompt_pass": "tcgen05 GEMM, blocks of 512 rows"},
            "e2e": e2e, "gpu_launches": int(launches), "clocks": clk.summary,
            "accepted_per_step": float(acc.mean()), "acceptance_rate": float(acc.mean() / d),
            "emitted_per_step": float(NEW / len(acc)), "spec_steps": int(len(acc)), "host_syncs": int(st.host_syncs),
@@ -271,7 +277,8 @@ def run_own(args):
         dom = ks[f"gate_up_swiglu@M={d + 1}"]
         out["roofline"] = {"bound": "hbm", "kernel": f"linear_{'mma' if path == 2 else 'fma'}_kernel (gate-up + SwiGLU, "
                            f"M={d + 1}, verify pass)", "achieved": dom["GB/s"], "peak": peak, "unit": "GB/s",
-                           "frac": dom["frac"], "traffic": None, "peak_kind": f"of {peak_kind} (burst copy)",
+                           "frac": dom["frac"], "traffic": ROOFLINE_TRAFFIC.get((args.workload, d + 1)),
+                           "algorithmic_bytes": dom["bytes"], "peak_kind": f"of {peak_kind} (burst copy)",
                            "how": "CUDA events around 40 launches through the C ABI, rotating over the layers' weights"}
         out["kernels"] = ks
         # the CPU oracle on a bounded sample of the same workload
