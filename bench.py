@@ -96,6 +96,20 @@ class ClockSampler:
                             "samples": len(sm)}
 
 
+def max_over_ranks(value, dist, device):
+    """The slowest rank's time: replicas are independent, the job ends when the last one does."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(world, steps, new_tokens, total_ms):
+    """Whole-job throughput of `world` independent replicas timed by the slowest one."""
+    return world * steps * new_tokens / (total_ms / 1e3)
+
+
 def oracle_model(wl, weights, max_seq):
     from oracle import ls_oracle as O
     s = wl.shape
@@ -212,13 +226,9 @@ def run_own(args):
             loop_ms.append(st.decode_ms)
         e1.record()
         barrier()
-    total_ms = e0.elapsed_time(e1)
-    if dist:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
     st = gm.stats()
-    value = world * args.steps * NEW / (total_ms / 1e3)
+    value = job_tokens_per_s(world, args.steps, NEW, total_ms)
     sched_bytes = st.weight_bytes + st.kv_bytes
     loop_gbs = sched_bytes / (statistics.mean(loop_ms) / 1e3) / 1e9
 
@@ -243,11 +253,7 @@ def run_own(args):
         ids, a2 = gm.generate(prompt, E, d, NEW)
         if i:
             e2e_ms.append((time.perf_counter() - t0) * 1e3)
-    e2e_worst = max(e2e_ms)
-    if dist:
-        t = torch.tensor([e2e_worst], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_worst = float(t.item())
+    e2e_worst = max_over_ranks(max(e2e_ms), dist, "cuda")
     est = gm.stats()
     e2e = {"value": world * NEW / (e2e_worst / 1e3), "unit": UNIT, "h2d_bytes_per_step": 4 * P + 32 * 2,
            "d2h_bytes_per_step": 4 * len(ids) + 4 * len(a2) + 32 * (est.host_syncs + 1),
@@ -293,6 +299,52 @@ def run_own(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """The sweep on the Llama-2-7B shape (prompt 4096, 256 new tokens): exit layer x number of
+    drafts x late-layer scale.  One JSON line per point, full-greedy numbers of the same model
+    beside it.  Not the benchmark line: a table for the report."""
+    from paper_2404_16710_b200 import binding as B
+    assert torch.cuda.is_available()
+    torch.cuda.set_device(0)
+    peak, _ = peaks()
+    exits = [int(x) for x in args.sweep_exit.split(",")]
+    drafts = [int(x) for x in args.sweep_draft.split(",")]
+    scales = [float(x) for x in args.sweep_scale.split(",")]
+    for scale in scales:
+        for E in exits:
+            wl = synth.sweep_workload(E, max(drafts), scale)
+            s, P, NEW = wl.shape, wl.n_prompt, wl.max_new
+            w = synth.make_weights(s, wl.weight_seed, E, scale, device="cuda")
+            gm = B.Model(s, w, P + NEW + max(drafts) + 1, 64, max(drafts))
+            prompt = synth.make_prompt(s.vocab, P, wl.prompt_seed)
+            B.ls_prefill(gm.h, prompt)
+            prefill_ms = gm.stats().prefill_ms
+            for _ in range(2):
+                B.ls_decode(gm.h, 0, 0, NEW)
+            fst = gm.stats()
+            full_ids, _ = B.ls_read_output(gm.h, NEW)
+            full_tok_s = NEW / (fst.decode_ms / 1e3)
+            full_frac = (fst.weight_bytes + fst.kv_bytes) / (fst.decode_ms / 1e3) / 1e9 / peak
+            for d in drafts:
+                for _ in range(2):
+                    B.ls_decode(gm.h, E, d, NEW)
+                st = gm.stats()
+                ids, acc = B.ls_read_output(gm.h, NEW)
+                tok_s = NEW / (st.decode_ms / 1e3)
+                print(json.dumps({
+                    "sweep": "llama2-7b-shaped", "n_prompt": P, "max_new": NEW, "late_scale": scale, "exit_layer": E,
+                    "num_draft": d, "tokens_per_s": round(tok_s, 1), "full_greedy_tokens_per_s": round(full_tok_s, 1),
+                    "speedup": round(tok_s / full_tok_s, 3), "accepted_per_step": round(float(acc.mean()), 3),
+                    "acceptance_rate": round(float(acc.mean() / d), 3),
+                    "hbm_frac_measured": round((st.weight_bytes + st.kv_bytes) / (st.decode_ms / 1e3) / 1e9 / peak, 3),
+                    "full_greedy_hbm_frac_measured": round(full_frac, 3),
+                    "ids_equal_full_greedy": bool(np.array_equal(ids, full_ids)), "prefill_ms": round(prefill_ms, 1),
+                    "host_syncs": int(st.host_syncs)}), flush=True)
+            gm.close()
+            del gm, w
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -304,8 +356,14 @@ def main():
                     help="instead of the benchmark: prefill, warm up, then run one self-speculative and one "
                          "full-greedy decode of NEW tokens between cudaProfilerStart/Stop (for a profiler "
                          "started with --profile-from-start off) and exit")
+    ap.add_argument("--sweep", action="store_true", help="run the (exit layer, drafts, late scale) sweep instead")
+    ap.add_argument("--sweep-exit", default=",".join(map(str, synth.SWEEP_EXIT)))
+    ap.add_argument("--sweep-draft", default=",".join(map(str, synth.SWEEP_DRAFT)))
+    ap.add_argument("--sweep-scale", default=",".join(map(str, synth.SWEEP_SCALE)))
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_own(args)
