@@ -89,7 +89,7 @@ struct ls_model {
     uint16_t *kpages, *vpages;
     size_t layer_kv_elems;
     int32_t *page_table, *ctl, *draft, *verified, *out_ids, *accepted, *ids, *attn_counters;
-    float *inv_freq, *x, *qkv, *part, *logits;
+    float *inv_freq, *x, *part, *logits;
     uint16_t *h, *q, *o, *a;
     uint16_t* hE;  // exit-layer activations, already multiplied by the gain of layer E's norm (Sec. 4.3.3)
     float *px, *py;          // prompt pass: residual rows and projection outputs of one block
@@ -140,7 +140,6 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     unsigned char* ac = take(sizeof(int32_t) * c.max_seq);
     unsigned char* ids = take(sizeof(int32_t) * c.max_seq);
     unsigned char* x = take(sizeof(float) * kMaxRows * c.d_model);
-    unsigned char* qkv = take(sizeof(float) * kMaxRows * (qw + 2 * kvw));
     unsigned char* part = take(sizeof(float) * kMaxRows * c.n_heads * chunk_cap * attn_part_pitch(c.head_dim));
     unsigned char* actr = take(sizeof(int32_t) * c.n_kv_heads);
     unsigned char* logits = take(sizeof(float) * kMaxRows * c.vocab);
@@ -182,7 +181,6 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
         m->accepted = (int32_t*)ac;
         m->ids = (int32_t*)ids;
         m->x = (float*)x;
-        m->qkv = (float*)qkv;
         m->part = (float*)part;
         m->attn_counters = (int32_t*)actr;
         m->logits = (float*)logits;

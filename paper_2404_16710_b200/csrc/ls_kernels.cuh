@@ -1,5 +1,6 @@
 // Non-GEMV kernels of the decode loop: embedding, RMSNorm, rotary embedding + KV append,
-// chunked causal attention over the paged cache, chunk merge, argmax finish, accept/rollback.
+// chunked causal attention over the paged cache with its ordered merge, argmax finish,
+// accept/rollback.
 //
 // Invariant kept by every kernel here: the instructions that produce row m's result do
 // not depend on how many rows the pass has.  The verification pass of num_draft+1 rows
@@ -115,18 +116,6 @@ rmsnorm_kernel(const float* __restrict__ x, const uint16_t* __restrict__ g, int 
         w.y = pack_bf16(v.z * r * bf16lo(gg.y), v.w * r * bf16hi(gg.y));
         o[c] = w;
     }
-}
-
-// fp32 row copy (exit-layer activation cache <-> residual stream, Sec. 4.3.3); grid M, block 256
-__global__ void __launch_bounds__(256)
-copy_rows_kernel(const float* __restrict__ src, float* __restrict__ dst, int D, const int32_t* ctl)
-{
-    pdl_launch_dependents();
-    pdl_wait();
-    if (ctl && ctl[CTL_DONE]) return;
-    const float4* s = reinterpret_cast<const float4*>(src + (size_t)blockIdx.x * D);
-    float4* d = reinterpret_cast<float4*>(dst + (size_t)blockIdx.x * D);
-    for (int c = threadIdx.x; c < D / 4; c += 256) d[c] = s[c];
 }
 
 // ------------------------------------------------------------------ paged KV addressing
