@@ -80,6 +80,25 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr)
     return v;
 }
 
+// D (fp32, 16x8) += A (bf16, 16x16, row-major) * B (bf16, 16x8, "column-major": k contiguous per n)
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// four 8x8 b16 matrices from shared memory, transposed on the way (lane L gives the row address
+// L%8 of matrix L/8)
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+
 // Programmatic dependent launch: a kernel launched with the attribute may start while its
 // predecessor on the stream is still running.  pdl_wait() blocks until the predecessor
 // grid has completed and its writes are visible; before it, a kernel may touch only

@@ -178,21 +178,27 @@ __global__ void rope_append_kernel(const float* __restrict__ qkv, int Hq, int Hk
 // merges the chunks of that head's queries IN CHUNK ORDER and writes the bf16 output.
 // Chunks are cut by absolute position, so a row's result depends on its position only.
 //
-// Work is spread thin on purpose (decode attention is a few MB per layer): four lanes
-// share one key in q.k (each a quarter of the dims, interleaved in 16-byte blocks), NKS
-// lanes share one pair of output dims in p.v (each a slice of the keys); both finish with
-// a fixed shuffle tree.  K and V rows are padded so that these accesses are free of bank
-// conflicts (K pitch = 16 banks mod 32, V pitch = 8 banks mod 32).
+// q.k and p.v run on the tensor cores (mma.sync.m16n8k16, fp32 accumulate) at EVERY pass size,
+// one row or sixteen: queries are the 16-row operand (tiles of 16, zero-padded), so the
+// instruction sequence behind a row does not depend on M.  q.k: warp w owns keys 8w..8w+7;
+// a thread's 16-byte pieces of its query rows and of its key row are its fragments (the
+// contraction index is permuted alike on both sides).  p.v: p is rounded to bf16, warp w owns
+// 16 (HD 128) or 8 (HD 64) output dims, V fragments come transposed out of ldmatrix.
+// Row pitches keep every access pattern free of bank conflicts: K and Q rows 64 mod 128
+// bytes, V rows 16 mod 128 bytes.
 //
-// shared memory: Ks [64][HD*2+64 B] | Vs [64][HD*2+32 B] | Qs f32 [Q][HD] | S f32 [Q][64]
+// shared memory: Ks [64][HD*2+64 B] | Vs [64][HD*2+16 B] | Qb bf16 [Qpad][HD*2+64 B]
+//                | S f32 [Qpad][72] | Pb bf16 [Qpad][72]          (Qpad = Q rounded up to 16)
 constexpr int kAttnThreads = 256;
 constexpr int kAttnMaxChunks = 256;  // chunks the merge can hold weights for: max_seq <= 16384
 constexpr int kMergeBatch = 8;       // queries merged together (one warp each)
+constexpr int kAttnSP = 72;          // floats per row of S, bf16 per row of Pb
 template <int HD>
 __host__ __device__ constexpr size_t attn_smem_bytes(int Q)
 {
-    size_t stage = (size_t)kAttnChunk * (HD * 2 + 64) + (size_t)kAttnChunk * (HD * 2 + 32) +
-                   sizeof(float) * ((size_t)Q * HD + (size_t)Q * kAttnChunk);
+    const size_t qpad = ((size_t)Q + 15) / 16 * 16;
+    size_t stage = (size_t)kAttnChunk * (HD * 2 + 64) + (size_t)kAttnChunk * (HD * 2 + 16) + qpad * (HD * 2 + 64) +
+                   qpad * kAttnSP * 4 + qpad * kAttnSP * 2;
     // merge (reuses the same memory): weights and sums [8][256] each, slice sums [4][8 slices][HD]
     size_t merge = sizeof(float) * (2 * (size_t)kMergeBatch * kAttnMaxChunks + 4 * 8 * (size_t)HD + kMergeBatch);
     return stage > merge ? stage : merge;
@@ -276,13 +282,14 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
             int max_seq, int chunk_cap, float* part, int32_t* counters, uint16_t* __restrict__ out)
 {
     constexpr int C = kAttnChunk, T = kAttnThreads;
-    constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 32;
-    constexpr int HALF = HD / 2;
-    constexpr int NKS = T / HALF;  // key slices in p.v: 4 (HD 128) or 8 (HD 64)
+    constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 16;
+    constexpr int SP = kAttnSP, PBROW = kAttnSP * 2;
+    constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
     constexpr int PP = attn_part_pitch(HD);
     int pos0;
     if (!pass_begin(ctl, pos_off, pos0)) return;
     const int ch = blockIdx.x, kh = blockIdx.y, tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
     const int last_pos = pos0 + M - 1;
     const int key0 = ch * C;
     if (key0 > last_pos) return;
@@ -292,31 +299,35 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
         return;
     }
     const int G = Hq / Hkv, Q = G * M;  // query qi = m * G + g
+    const int Qpad = (Q + 15) & ~15;
 
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* Ks = smem;
     unsigned char* Vs = Ks + C * KROW;
-    float* Qs = reinterpret_cast<float*>(Vs + C * VROW);
-    float* S = Qs + (size_t)Q * HD;
+    unsigned char* Qb = Vs + C * VROW;
+    float* S = reinterpret_cast<float*>(Qb + (size_t)Qpad * KROW);
+    unsigned char* Pb = reinterpret_cast<unsigned char*>(S + (size_t)Qpad * SP);
 
-    // the group's queries: issue the global loads first, so that they travel together with
-    // the page-table lookup and the K/V copies (each is a round trip of its own otherwise)
-    constexpr int QPT = 4;  // query elements (bf16 pairs) a thread holds per sweep
-    const int nq = Q * HALF;
-    uint32_t qreg[QPT];
+    // the group's queries (bf16, 16-byte pieces): issue the global loads first, so that they
+    // travel together with the page-table lookup and the K/V copies
+    constexpr int QPT = 2;
+    const int nq = Qpad * SEGS;
+    uint4 qreg[QPT];
 #pragma unroll
     for (int i = 0; i < QPT; ++i) {
         const int idx = tid + i * T;
+        qreg[i] = make_uint4(0, 0, 0, 0);
         if (idx < nq) {
-            const int qi = idx / HALF, dp = idx % HALF;
-            const int m = qi / G, g = qi % G;
-            qreg[i] = *reinterpret_cast<const uint32_t*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + 2 * dp);
+            const int qi = idx / SEGS, sg = idx % SEGS;
+            if (qi < Q) {
+                const int m = qi / G, g = qi % G;
+                qreg[i] = *reinterpret_cast<const uint4*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + sg * 8);
+            }
         }
     }
     // stage K and V rows of the chunk (zeros beyond the last visible key): asynchronous
     // copies, all in flight at once; a chunk never straddles a page of 64 tokens or more
     {
-        constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
         const uint32_t ks0 = (uint32_t)__cvta_generic_to_shared(Ks), vs0 = (uint32_t)__cvta_generic_to_shared(Vs);
         const bool one_page = page_shift >= 6;
         const size_t base = one_page ? kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD) : 0;
@@ -337,40 +348,54 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
 #pragma unroll
     for (int i = 0; i < QPT; ++i) {
         const int idx = tid + i * T;
-        if (idx < nq) {
-            Qs[2 * idx] = bf16lo(qreg[i]);
-            Qs[2 * idx + 1] = bf16hi(qreg[i]);
-        }
+        if (idx < nq) *reinterpret_cast<uint4*>(Qb + (idx / SEGS) * KROW + (idx % SEGS) * 16) = qreg[i];
     }
-    for (int idx = tid + QPT * T; idx < nq; idx += T) {  // more than 16 queries of 128 dims
-        const int qi = idx / HALF, dp = idx % HALF;
-        const int m = qi / G, g = qi % G;
-        const uint32_t u = *reinterpret_cast<const uint32_t*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + 2 * dp);
-        Qs[2 * idx] = bf16lo(u);
-        Qs[2 * idx + 1] = bf16hi(u);
+    for (int idx = tid + QPT * T; idx < nq; idx += T) {  // more than two tiles of queries
+        const int qi = idx / SEGS, sg = idx % SEGS;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (qi < Q) {
+            const int m = qi / G, g = qi % G;
+            v = *reinterpret_cast<const uint4*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + sg * 8);
+        }
+        *reinterpret_cast<uint4*>(Qb + qi * KROW + sg * 16) = v;
     }
     cp_async_wait<0>();
     __syncthreads();
 
-    // phase 1: q.k -- thread = (key, quarter of the dims); groups of 4 queries, then singles
-    {
-        const int key = tid >> 2, qd = tid & 3;
-        const unsigned char* krow = Ks + key * KROW;
-        int q0 = 0;
-        for (; q0 + 4 <= Q; q0 += 4) attn_qk<HD, 4>(krow, Qs, q0, qd, S, key, qd == 0);
-        for (; q0 < Q; ++q0) attn_qk<HD, 1>(krow, Qs, q0, qd, S, key, qd == 0);
+    // phase 1: s = q.k -- warp w: keys 8w..8w+7 against every tile of 16 queries
+    for (int qt = 0; qt < Qpad; qt += 16) {
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        const unsigned char* qa = Qb + (qt + g8) * KROW + 16 * t4;
+        const unsigned char* kb = Ks + (8 * warp + g8) * KROW + 16 * t4;
+#pragma unroll
+        for (int j = 0; j < HD / 32; ++j) {
+            const uint4 A0 = *reinterpret_cast<const uint4*>(qa + 64 * j);
+            const uint4 A1 = *reinterpret_cast<const uint4*>(qa + 8 * KROW + 64 * j);
+            const uint4 Bk = *reinterpret_cast<const uint4*>(kb + 64 * j);
+            mma_bf16_16816(c, A0.x, A1.x, A0.y, A1.y, Bk.x, Bk.y);
+            mma_bf16_16816(c, A0.z, A1.z, A0.w, A1.w, Bk.z, Bk.w);
+        }
+        float* s = S + (size_t)(qt + g8) * SP + 8 * warp + 2 * t4;
+        *reinterpret_cast<float2*>(s) = make_float2(c[0], c[1]);
+        *reinterpret_cast<float2*>(s + 8 * SP) = make_float2(c[2], c[3]);
     }
     __syncthreads();
 
-    // phase 2: one warp per query: scale, mask, max, exp, sum over the 64 keys of the chunk
+    // phase 2: one warp per query: scale, mask, max, exp, sum over the 64 keys of the chunk;
+    // p goes to Pb as bf16 (zeros for the padding rows of the last tile)
     {
-        const int warp = tid >> 5, lane = tid & 31;
         const float scale = rsqrtf((float)HD);
-        for (int qi = warp; qi < Q; qi += T / 32) {
+        for (int qi = warp; qi < Qpad; qi += T / 32) {
+            uint16_t* pb = reinterpret_cast<uint16_t*>(Pb + (size_t)qi * PBROW);
+            if (qi >= Q) {
+                pb[lane] = 0;
+                pb[lane + 32] = 0;
+                continue;
+            }
             const int m = qi / G, g = qi % G;
             const int pos = pos0 + m;
-            float s0 = S[(size_t)qi * C + lane] * scale;
-            float s1 = S[(size_t)qi * C + lane + 32] * scale;
+            float s0 = S[(size_t)qi * SP + lane] * scale;
+            float s1 = S[(size_t)qi * SP + lane + 32] * scale;
             if (key0 + lane > pos) s0 = -INFINITY;
             if (key0 + lane + 32 > pos) s1 = -INFINITY;
             float mx = fmaxf(s0, s1);
@@ -381,8 +406,8 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
             float l = p0 + p1;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-            S[(size_t)qi * C + lane] = p0;
-            S[(size_t)qi * C + lane + 32] = p1;
+            pb[lane] = f2bf(p0);
+            pb[lane + 32] = f2bf(p1);
             if (lane == 0) {
                 float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP;
                 dst[HD] = mx;
@@ -392,27 +417,44 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
     }
     __syncthreads();
 
-    // phase 3: p.v -- thread = (pair of dims, slice of the keys)
+    // phase 3: o = p.v -- warp w: output dims NTW*8*w .. for every tile of 16 queries
     {
-        const int ks = tid % NKS, dp = tid / NKS;
-        auto store = [&](int qi, float o0, float o1) {
-            const int m = qi / G, g = qi % G;
-            float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP + 2 * dp;
-            *reinterpret_cast<float2*>(dst) = make_float2(o0, o1);
-        };
-        int q0 = 0;
-        for (; q0 + 4 <= Q; q0 += 4) {
-            float o[4][2];
-            attn_pv<HD, 4, NKS>(Vs, S, q0, dp, ks, o);
-            if (ks == 0) {
+        constexpr int NTW = HD / 64;  // n8 tiles per warp: 2 (HD 128) or 1 (HD 64)
+        const int d0 = NTW * 8 * warp;
+        const uint32_t vs0 = (uint32_t)__cvta_generic_to_shared(Vs);
+        // ldmatrix: lane L addresses row L%8 of matrix L/8; matrices 0, 1: keys 0-7, 8-15 of
+        // the 16-key block at dims d0..d0+7; matrices 2, 3: the same keys at dims d0+8..
+        const int mi = lane >> 3, mr = lane & 7;
+        const uint32_t vlane = vs0 + (uint32_t)(((mi & 1) * 8 + mr) * VROW + (d0 + ((NTW == 2) ? (mi >> 1) * 8 : 0)) * 2);
+        for (int qt = 0; qt < Qpad; qt += 16) {
+            float c[NTW][4];
 #pragma unroll
-                for (int qq = 0; qq < 4; ++qq) store(q0 + qq, o[qq][0], o[qq][1]);
+            for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) c[nt][i] = 0.f;
+            const unsigned char* pa = Pb + (size_t)(qt + g8) * PBROW + 4 * t4;
+#pragma unroll
+            for (int kk = 0; kk < C / 16; ++kk) {
+                const uint32_t a0 = *reinterpret_cast<const uint32_t*>(pa + 32 * kk);
+                const uint32_t a1 = *reinterpret_cast<const uint32_t*>(pa + 8 * PBROW + 32 * kk);
+                const uint32_t a2 = *reinterpret_cast<const uint32_t*>(pa + 32 * kk + 16);
+                const uint32_t a3 = *reinterpret_cast<const uint32_t*>(pa + 8 * PBROW + 32 * kk + 16);
+                uint32_t r0, r1, r2, r3;
+                ldmatrix_x4_trans(vlane + (uint32_t)(16 * kk * VROW), r0, r1, r2, r3);
+                mma_bf16_16816(c[0], a0, a1, a2, a3, r0, r1);
+                if (NTW == 2) mma_bf16_16816(c[NTW - 1], a0, a1, a2, a3, r2, r3);
             }
-        }
-        for (; q0 < Q; ++q0) {
-            float o[1][2];
-            attn_pv<HD, 1, NKS>(Vs, S, q0, dp, ks, o);
-            if (ks == 0) store(q0, o[0][0], o[0][1]);
+#pragma unroll
+            for (int hrow = 0; hrow < 2; ++hrow) {
+                const int qi = qt + g8 + 8 * hrow;
+                if (qi < Q) {
+                    const int m = qi / G, g = qi % G;
+                    float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP + d0 + 2 * t4;
+#pragma unroll
+                    for (int nt = 0; nt < NTW; ++nt)
+                        *reinterpret_cast<float2*>(dst + 8 * nt) = make_float2(c[nt][2 * hrow], c[nt][2 * hrow + 1]);
+                }
+            }
         }
     }
 
