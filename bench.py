@@ -245,6 +245,14 @@ def run_own(args):
     full_gbs = (fst.weight_bytes + fst.kv_bytes) / (statistics.mean(full_ms) / 1e3) / 1e9
     lossless = bool(np.array_equal(full_ids, spec_ids))
 
+    # ---- the paper's "without KVQ reuse" ablation (Table 7): verify recomputes the early layers
+    B.ls_decode_flags(gm.h, E, d, NEW, B.LS_DECODE_NO_EXIT_CACHE)
+    B.ls_decode_flags(gm.h, E, d, NEW, B.LS_DECODE_NO_EXIT_CACHE)
+    nst = gm.stats()
+    no_reuse_ids, _ = B.ls_read_output(gm.h, NEW)
+    no_reuse = {"value": NEW / (nst.decode_ms / 1e3), "unit": UNIT,
+                "ids_equal": bool(np.array_equal(no_reuse_ids, spec_ids))}
+
     # ---- end to end through the public call: host prompt in, host ids out, prefill included
     e2e_ms = []
     for i in range(1 + max(1, min(args.steps, 3))):
@@ -272,7 +280,7 @@ def run_own(args):
            "emitted_per_step": float(NEW / len(acc)), "spec_steps": int(len(acc)), "host_syncs": int(st.host_syncs),
            "full_greedy": {"value": full_tok_s, "unit": UNIT, "hbm_GB/s": round(full_gbs, 1),
                            "hbm_frac_measured": round(full_gbs / peak, 4), "hbm_frac_8TBs": round(full_gbs / 8000, 4)},
-           "speedup_vs_full_greedy": value / world / full_tok_s, "ids_equal_full_greedy": lossless,
+           "speedup_vs_full_greedy": value / world / full_tok_s, "without_exit_cache_reuse": no_reuse, "ids_equal_full_greedy": lossless,
            "loop_hbm": {"GB/s": round(loop_gbs, 1), "frac_measured": round(loop_gbs / peak, 4),
                         "frac_8TBs": round(loop_gbs / 8000, 4), "bytes_per_loop": int(sched_bytes)},
            "prefill_ms": prefill_ms}

@@ -146,6 +146,11 @@ int ls_generate_early(ls_model *m, const int32_t *prompt_ids_host, int32_t n_pro
  * Results stay on the device until ls_read_output. */
 int ls_prefill(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt, int32_t layers);
 int ls_decode(ls_model *m, int32_t exit_layer, int32_t num_draft, int32_t max_new);
+/* ls_decode with options.  LS_DECODE_NO_EXIT_CACHE is the paper's "without KVQ reuse" ablation
+ * (Sec. 6.2, Table 7): the verify pass does not continue from the cached exit-layer
+ * activations but runs all L layers on the num_draft+1 rows again.  Same ids, more bytes. */
+#define LS_DECODE_NO_EXIT_CACHE 1
+int ls_decode_flags(ls_model *m, int32_t exit_layer, int32_t num_draft, int32_t max_new, int32_t flags);
 int ls_read_output(ls_model *m, int32_t *out_ids_host, int32_t *out_n,
                    int32_t *accepted_per_step_host, int32_t *out_n_steps);
 

@@ -24,7 +24,7 @@ LS_LINEAR_AUTO, LS_LINEAR_FMA, LS_LINEAR_MMA = 0, 1, 2
 EXPORTS = (
     "ls_strerror", "ls_last_cuda_error", "ls_workspace_bytes", "ls_model_create", "ls_model_destroy",
     "ls_set_page_table", "ls_generate", "ls_generate_full", "ls_generate_early", "ls_prefill",
-    "ls_decode", "ls_read_output", "ls_debug_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
+    "ls_decode", "ls_decode_flags", "ls_read_output", "ls_debug_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
     "ls_op_linear", "ls_op_gate_up_swiglu", "ls_op_lm_head_scratch_bytes", "ls_op_lm_head_argmax",
     "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_qkv_rope_append", "ls_op_attention_scratch_bytes", "ls_op_attention", "ls_op_accept",
     "ls_op_gemm", "ls_op_prefill_attention",
@@ -87,6 +87,7 @@ def lib():
             "ls_generate_early": (C.c_int, [vp, ip, i32, i32, i32, ip, ip]),
             "ls_prefill": (C.c_int, [vp, ip, i32, i32]),
             "ls_decode": (C.c_int, [vp, i32, i32, i32]),
+            "ls_decode_flags": (C.c_int, [vp, i32, i32, i32, i32]),
             "ls_read_output": (C.c_int, [vp, ip, ip, ip, ip]),
             "ls_debug_logits": (C.c_int, [vp, ip, i32, i32, fp, fp]),
             "ls_get_stats": (C.c_int, [vp, C.POINTER(ls_stats)]),
@@ -211,6 +212,13 @@ def ls_prefill(h, prompt, layers=0):
 
 def ls_decode(h, exit_layer, num_draft, max_new):
     _ck(lib().ls_decode(h, exit_layer, num_draft, max_new), "ls_decode")
+
+
+LS_DECODE_NO_EXIT_CACHE = 1
+
+
+def ls_decode_flags(h, exit_layer, num_draft, max_new, flags):
+    _ck(lib().ls_decode_flags(h, exit_layer, num_draft, max_new, flags), "ls_decode_flags")
 
 
 def ls_read_output(h, max_new):

@@ -472,7 +472,7 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
 }
 
 // one step of the loop.  E == L with d == 0: plain greedy; E < L with d == 0: early exit.
-int enqueue_step(ls_model* m, int E, int d)
+int enqueue_step(ls_model* m, int E, int d, bool reuse)
 {
     const int D = m->c.d_model, L = m->c.n_layers;
     if (d == 0) {
@@ -480,17 +480,25 @@ int enqueue_step(ls_model* m, int E, int d)
         LS_TRY(run_layers(m, 0, E, 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
         LS_TRY(run_head(m, 1, 0, m->verified, nullptr));
     } else {
-        for (int j = 0; j <= d; ++j) {  // self-drafting (Sec. 4.3.1) + the extra early pass
+        for (int j = 0; j <= (reuse ? d : d - 1); ++j) {  // self-drafting (Sec. 4.3.1) + the extra early pass
             float* xr = m->x + (size_t)j * D;
             LS_TRY(run_embed(m, j == 0 ? m->ctl + CTL_CUR_TOK : m->draft + (j - 1), 1, xr, j));
             // the exit-layer row goes to the LM head (final gain) and, pre-scaled by layer E's
             // gain, to the verify pass (the exit-layer cache of Sec. 4.3.3)
             LS_TRY(run_layers(m, 0, E, 1, xr, j, j, m->h + (size_t)j * D, j < d ? m->fnorm : nullptr,
-                              m->lw[E].attn_norm));
+                              reuse ? m->lw[E].attn_norm : nullptr));
             if (j < d) LS_TRY(run_head(m, 1, j, m->draft + j, nullptr));
         }
-        // self-verification (Sec. 4.3.2) from the exit-layer activations
-        LS_TRY(run_layers(m, E, L, d + 1, m->x, 0, 0, m->hE, m->fnorm, nullptr));
+        if (reuse) {
+            // self-verification (Sec. 4.3.2) from the exit-layer activations
+            LS_TRY(run_layers(m, E, L, d + 1, m->x, 0, 0, m->hE, m->fnorm, nullptr));
+        } else {
+            // the ablation of Sec. 6.2 / Table 7: no exit-layer cache, verification recomputes the
+            // early layers of all d+1 rows (and rewrites their k, v with the same values)
+            LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
+            LS_TRY(run_embed(m, m->draft, d, m->x + D, 1));
+            LS_TRY(run_layers(m, 0, L, d + 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
+        }
         LS_TRY(run_head(m, d + 1, 0, m->verified, nullptr));
     }
     LS_CK(launch(LaunchCtx{m->st, m->pdl}, accept_kernel, dim3(1), dim3(32), 0, m->draft, m->verified, d, m->ctl,
@@ -505,15 +513,15 @@ void drop_graphs(ls_model* m)
     m->graphs.clear();
 }
 
-int get_graph(ls_model* m, int E, int d, ls_model::G** out)
+int get_graph(ls_model* m, int E, int d, bool reuse, ls_model::G** out)
 {
-    uint64_t key = ((uint64_t)E << 32) | ((uint64_t)d << 16) | (uint64_t)m->grid_chunks;
+    uint64_t key = ((uint64_t)(reuse ? 0 : 1) << 48) | ((uint64_t)E << 32) | ((uint64_t)d << 16) | (uint64_t)m->grid_chunks;
     auto it = m->graphs.find(key);
     if (it == m->graphs.end()) {
         cudaGraph_t graph = nullptr;
         int64_t before = m->launches;
         LS_CK(cudaStreamBeginCapture(m->st, cudaStreamCaptureModeRelaxed));
-        int rc = enqueue_step(m, E, d);
+        int rc = enqueue_step(m, E, d, reuse);
         cudaError_t e = cudaStreamEndCapture(m->st, &graph);
         if (rc != LS_OK) {
             if (graph) cudaGraphDestroy(graph);
@@ -758,7 +766,13 @@ int ls_prefill(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t lay
 
 int ls_decode(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new)
 {
-    if (!m || m->n_prompt < 1) return LS_ERR_INVALID_ARG;
+    return ls_decode_flags(m, exit_layer, num_draft, max_new, 0);
+}
+
+int ls_decode_flags(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new, int32_t flags)
+{
+    if (!m || m->n_prompt < 1 || (flags & ~LS_DECODE_NO_EXIT_CACHE)) return LS_ERR_INVALID_ARG;
+    const bool reuse = !(flags & LS_DECODE_NO_EXIT_CACHE);
     const ls_config& c = m->c;
     const int L = c.n_layers;
     int E = exit_layer, d = num_draft;
@@ -778,7 +792,7 @@ int ls_decode(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_ne
     set_grid_chunks(m, m->n_prompt + max_new + d + 1);
 
     ls_model::G* g = nullptr;
-    if (m->use_graphs) LS_TRY(get_graph(m, E, d, &g));
+    if (m->use_graphs) LS_TRY(get_graph(m, E, d, reuse, &g));
     LS_TRY(write_ctl(m, m->n_prompt - 1, m->last_tok, max_new));
     int64_t launched = 0;
     int syncs = 0, n_out = 0, steps_done = 0;
@@ -798,7 +812,7 @@ int ls_decode(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_ne
                 launched += g->nodes;
             } else {
                 int64_t before = m->launches;
-                LS_TRY(enqueue_step(m, E, d));
+                LS_TRY(enqueue_step(m, E, d, reuse));
                 launched += m->launches - before;
             }
         }
@@ -834,9 +848,15 @@ int ls_decode(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_ne
             wb += E * w_layer + w_lm;
             kb += (int64_t)E * kvb * (cl + 1);
         } else {
-            wb += (int64_t)(d + 1) * E * w_layer + (int64_t)d * w_lm + (int64_t)(L - E) * w_layer + w_lm;
-            for (int j = 0; j <= d; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
-            kb += (int64_t)(L - E) * kvb * (cl + d + 1);
+            if (reuse) {
+                wb += (int64_t)(d + 1) * E * w_layer + (int64_t)d * w_lm + (int64_t)(L - E) * w_layer + w_lm;
+                for (int j = 0; j <= d; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
+                kb += (int64_t)(L - E) * kvb * (cl + d + 1);
+            } else {
+                wb += (int64_t)d * (E * w_layer + w_lm) + (int64_t)L * w_layer + w_lm;
+                for (int j = 0; j < d; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
+                kb += (int64_t)L * kvb * (cl + d + 1);
+            }
         }
         cl += n + 1;
         acc_sum += n;

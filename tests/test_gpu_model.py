@@ -157,6 +157,26 @@ def test_prefill_once_decode_many():
     assert st.weight_bytes == per_step * st.n_steps
 
 
+def test_without_exit_cache_reuse_same_ids_more_bytes():
+    """The paper's "w/o KVQ reuse" ablation: verification recomputes the early layers."""
+    gm, _ = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 128, oracle=False)
+    prompt = synth.make_prompt(TINY.shape.vocab, 20, 1)
+    B.ls_prefill(gm.h, prompt)
+    B.ls_decode(gm.h, 2, 3, 40)
+    ids, acc = B.ls_read_output(gm.h, 40)
+    st = gm.stats()
+    B.ls_decode_flags(gm.h, 2, 3, 40, B.LS_DECODE_NO_EXIT_CACHE)
+    ids2, acc2 = B.ls_read_output(gm.h, 40)
+    st2 = gm.stats()
+    np.testing.assert_array_equal(ids2, ids)
+    np.testing.assert_array_equal(acc2, acc)
+    s = TINY.shape
+    assert st.weight_bytes == st.n_steps * ((4 * 2 + 2) * s.layer_weight_bytes + 4 * s.lm_head_bytes)
+    assert st2.weight_bytes == st2.n_steps * ((3 * 2 + 4) * s.layer_weight_bytes + 4 * s.lm_head_bytes)
+    with pytest.raises(B.LsError):
+        B.ls_decode_flags(gm.h, 2, 3, 40, 8)
+
+
 def test_boundary_error_codes():
     gm, _ = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 64, max_draft=4, oracle=False)
     p = synth.make_prompt(TINY.shape.vocab, 8, 0)
