@@ -77,9 +77,17 @@ __device__ __forceinline__ int qkv_row(const LinArgs& a, int tile, int pair, int
     return (tile / tph) * a.hd + (tile % tph) * 8 + pair + (hi ? (a.hd >> 1) : 0);
 }
 
+// rotation of pair j at position pos: (sin, cos) of pos * theta^(-2j/hd)
+__device__ __forceinline__ void qkv_rotation(const LinArgs& a, int j, int pos, float& sn, float& cs)
+{
+    const float f = a.inv_freq ? a.inv_freq[j] : (float)pow((double)a.theta, -2.0 * (double)j / (double)a.hd);
+    sincosf((float)pos * f, &sn, &cs);
+}
+
 // rotate the pair (x_j, x_{j+hd/2}) of head `head` for token m and store it: q -> q_out,
 // k, v -> the paged cache row of position pos0 + m (v is not rotated)
-__device__ __forceinline__ void qkv_store(const LinArgs& a, int head, int j, int m, int pos0, float lo, float hi)
+__device__ __forceinline__ void qkv_store(const LinArgs& a, int head, int j, int m, int pos0, float lo, float hi,
+                                          float sn, float cs)
 {
     const int pos = pos0 + m;
     if (pos < 0 || pos >= a.max_seq) {
@@ -87,9 +95,6 @@ __device__ __forceinline__ void qkv_store(const LinArgs& a, int head, int j, int
         return;
     }
     if (head < a.Hq + a.Hkv) {
-        const float f = a.inv_freq ? a.inv_freq[j] : (float)pow((double)a.theta, -2.0 * (double)j / (double)a.hd);
-        float sn, cs;
-        sincosf((float)pos * f, &sn, &cs);
         const float r0 = lo * cs - hi * sn, r1 = lo * sn + hi * cs;
         lo = r0;
         hi = r1;
@@ -248,9 +253,12 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
         for (int m = 0; m < MT; ++m)
             if (lane == m && m < a.M) {
 #pragma unroll
-                for (int r = 0; r < 2; ++r)
-                    qkv_store(a, blockIdx.x / tph, (blockIdx.x % tph) * 8 + warp * 2 + r, m, pos0, acc[r][m],
-                              acc[r + 2][m]);
+                for (int r = 0; r < 2; ++r) {
+                    const int j = (blockIdx.x % tph) * 8 + warp * 2 + r;
+                    float sn, cs;
+                    qkv_rotation(a, j, pos0 + m, sn, cs);
+                    qkv_store(a, blockIdx.x / tph, j, m, pos0, acc[r][m], acc[r + 2][m], sn, cs);
+                }
             }
     } else {  // EPI_ARGMAX
         __shared__ float bv[4][MT];
@@ -398,6 +406,38 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             if (lane == 0) rs[m] = v;
         }
     }
+    // what the epilogue will need from global memory is fetched now, while the ring fills:
+    // the residual values and gains (EPI_RESIDUAL), the rotation factors (EPI_QKV)
+    constexpr int FRAGS = TR * NT;
+    float xin[4] = {0.f, 0.f, 0.f, 0.f}, gA[2] = {0.f, 0.f}, gB[2] = {0.f, 0.f}, rsn[2] = {0.f, 0.f}, rcs[2] = {1.f, 1.f};
+    int pos0_epi = 0;
+    if (tid < 32 * FRAGS) {
+        const int efr = tid >> 5, etile = blockIdx.x * TR + efr / NT, em0 = (efr % NT) * 8 + 2 * t;
+        if (EPI == EPI_RESIDUAL) {
+            const int nlo = etile * 16 + g, nhi = nlo + 8;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int m = em0 + (i & 1), n = (i < 2) ? nlo : nhi;
+                if (m < a.M && n < a.N) xin[i] = a.out[(size_t)m * a.ldo + n];
+            }
+            if (nlo < a.N) {
+                if (a.hout_a) gA[0] = bf16f(a.gain_a[nlo]);
+                if (a.hout_b) gB[0] = bf16f(a.gain_b[nlo]);
+            }
+            if (nhi < a.N) {
+                if (a.hout_a) gA[1] = bf16f(a.gain_a[nhi]);
+                if (a.hout_b) gB[1] = bf16f(a.gain_b[nhi]);
+            }
+        } else if (EPI == EPI_QKV) {
+            pos0_epi = (a.ctl ? a.ctl[CTL_CACHE_LEN] : 0) + a.pos_off;
+            const int tph = a.hd >> 4;
+            if (etile < (a.N >> 4) && etile / tph < a.Hq + a.Hkv) {
+                const int j = (etile % tph) * 8 + g;
+                qkv_rotation(a, j, pos0_epi + em0, rsn[0], rcs[0]);
+                qkv_rotation(a, j, pos0_epi + em0 + 1, rsn[1], rcs[1]);
+            }
+        }
+    }
     int rd = 0, wr = STAGES - 1;
     for (int step = warp; step < nsteps; step += WARPS) {
         issue_w(step + (STAGES - 1) * WARPS, wr);
@@ -463,13 +503,12 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             for (int i = 0; i < 4; ++i) {
                 int m = m0 + (i & 1), n = (i < 2) ? nlo : nhi;
                 if (m < a.M && n < a.N) {
-                    float* o = a.out + (size_t)m * a.ldo + n;
-                    const float xn = (EPI == EPI_RESIDUAL) ? (*o + r[i]) : r[i];
-                    *o = xn;
+                    const float xn = (EPI == EPI_RESIDUAL) ? (xin[i] + r[i]) : r[i];
+                    a.out[(size_t)m * a.ldo + n] = xn;
                     if (EPI == EPI_RESIDUAL) {
                         q[i & 1] = fmaf(xn, xn, q[i & 1]);
-                        if (a.hout_a) a.hout_a[(size_t)m * a.N + n] = f2bf(xn * bf16f(a.gain_a[n]));
-                        if (a.hout_b) a.hout_b[(size_t)m * a.N + n] = f2bf(xn * bf16f(a.gain_b[n]));
+                        if (a.hout_a) a.hout_a[(size_t)m * a.N + n] = f2bf(xn * gA[i >> 1]);
+                        if (a.hout_b) a.hout_b[(size_t)m * a.N + n] = f2bf(xn * gB[i >> 1]);
                     }
                 }
             }
@@ -492,11 +531,10 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             }
         } else if (EPI == EPI_QKV) {
             if (tile < (a.N >> 4)) {
-                const int pos0 = (a.ctl ? a.ctl[CTL_CACHE_LEN] : 0) + a.pos_off;
                 const int tph = a.hd >> 4;
                 const int head = tile / tph, j = (tile % tph) * 8 + gg;
-                if (m0 < a.M) qkv_store(a, head, j, m0, pos0, r[0], r[2]);
-                if (m0 + 1 < a.M) qkv_store(a, head, j, m0 + 1, pos0, r[1], r[3]);
+                if (m0 < a.M) qkv_store(a, head, j, m0, pos0_epi, r[0], r[2], rsn[0], rcs[0]);
+                if (m0 + 1 < a.M) qkv_store(a, head, j, m0 + 1, pos0_epi, r[1], r[3], rsn[1], rcs[1]);
             }
         } else {
             vals[tr * 16 + gg][m0] = r[0];
