@@ -39,7 +39,7 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) of one launch of the roofline kernel, from the ncu capture that
 # profiles/linear_mma_kernel_llama2-7b_shapes.md summarises; keyed by (workload, rows).  Set an
 # entry to None when the kernel changes until the counters have been taken again.
-ROOFLINE_TRAFFIC = {("llama2-7b", 7): 180.43e6 + 4.1e6}
+ROOFLINE_TRAFFIC = {("llama2-7b", 7): 180.43e6 + 3.8e6}
 
 
 def peaks():
