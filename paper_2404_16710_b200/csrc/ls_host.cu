@@ -421,9 +421,19 @@ int gemm_launch(const uint16_t* A, const uint16_t* B, int M, int N, int K, float
 int prefill_attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt, int pos0, int R,
                         int Hq, int Hkv, int hd, int page_shift, uint16_t* out, cudaStream_t st)
 {
-    const int Q = Hq / Hkv * kMaxRows;
+    const int G = Hq / Hkv, Q = G * kMaxRows;
     dim3 grid((R + 15) / 16, Hkv);
-    if (hd == 128) {
+    if (G <= 4) {  // four query tiles fit in registers: tensor-core kernel
+        if (hd == 128) {
+            const size_t sm = prefill_attn_mma_smem_bytes<128>(Q);
+            LS_CK(cudaFuncSetAttribute(prefill_attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+            prefill_attn_mma_kernel<128><<<grid, kAttnThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
+        } else {
+            const size_t sm = prefill_attn_mma_smem_bytes<64>(Q);
+            LS_CK(cudaFuncSetAttribute(prefill_attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+            prefill_attn_mma_kernel<64><<<grid, kAttnThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
+        }
+    } else if (hd == 128) {
         const size_t sm = prefill_attn_smem_bytes<128>(Q);
         LS_CK(cudaFuncSetAttribute(prefill_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
         prefill_attn_kernel<128><<<grid, kAttnThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);

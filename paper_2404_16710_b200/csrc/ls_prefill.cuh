@@ -377,4 +377,197 @@ prefill_attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
     }
 }
 
+// The same walk on the tensor cores (used when a KV head's 16 rows x G query heads fit in four
+// query tiles, G <= 4): q.k and p.v as mma.sync.m16n8k16 exactly as in the decode attention
+// kernel (queries are the 16-row operand, V comes transposed out of ldmatrix), softmax pieces
+// per chunk in fp32, the running output of every query tile stays in registers and is rescaled
+// by exp(old max - new max) before each chunk's contribution is added.
+// shared memory: Ks [64][HD*2+64] | Vs [64][HD*2+16] | Qb bf16 [Qpad][HD*2+64] | S f32 [Qpad][72]
+//                | Pb bf16 [Qpad][72] | mx, l, alpha f32 [Qpad] each
+template <int HD>
+__host__ __device__ constexpr size_t prefill_attn_mma_smem_bytes(int Q)
+{
+    const size_t qpad = ((size_t)Q + 15) / 16 * 16;
+    return (size_t)kAttnChunk * (HD * 2 + 64) + (size_t)kAttnChunk * (HD * 2 + 16) + qpad * (HD * 2 + 64) +
+           qpad * kAttnSP * 4 + qpad * kAttnSP * 2 + 3 * qpad * sizeof(float);
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kAttnThreads)
+prefill_attn_mma_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
+                        const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table, int pos0, int R,
+                        int Hq, int Hkv, int page_shift, uint16_t* __restrict__ out)
+{
+    constexpr int C = kAttnChunk, T = kAttnThreads;
+    constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 16, SP = kAttnSP, PBROW = kAttnSP * 2;
+    constexpr int SEGS = HD * 2 / 16;
+    constexpr int NTW = HD / 64;  // n8 tiles of output dims per warp
+    constexpr int MAXQT = 4;      // query tiles held in registers
+    const int tid = threadIdx.x, kh = blockIdx.y;
+    const int warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
+    const int r0 = blockIdx.x * 16;
+    const int M = min(16, R - r0);
+    const int G = Hq / Hkv, Q = G * M, Qpad = (Q + 15) & ~15;
+    const int first_pos = pos0 + r0, last_pos = first_pos + M - 1;
+
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned char* Ks = smem;
+    unsigned char* Vs = Ks + C * KROW;
+    unsigned char* Qb = Vs + C * VROW;
+    float* S = reinterpret_cast<float*>(Qb + (size_t)Qpad * KROW);
+    unsigned char* Pb = reinterpret_cast<unsigned char*>(S + (size_t)Qpad * SP);
+    float* mx = reinterpret_cast<float*>(Pb + (size_t)Qpad * PBROW);
+    float* ls = mx + Qpad;
+    float* al = ls + Qpad;
+
+    for (int idx = tid; idx < Qpad * SEGS; idx += T) {
+        const int qi = idx / SEGS, sg = idx % SEGS;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (qi < Q) {
+            const int m = qi / G, g = qi % G;
+            v = *reinterpret_cast<const uint4*>(q + ((size_t)(r0 + m) * Hq + (size_t)kh * G + g) * HD + sg * 8);
+        }
+        *reinterpret_cast<uint4*>(Qb + qi * KROW + sg * 16) = v;
+    }
+    for (int qi = tid; qi < Qpad; qi += T) {
+        mx[qi] = -INFINITY;
+        ls[qi] = 0.f;
+        al[qi] = 1.f;
+    }
+    float o[MAXQT][NTW][4];
+#pragma unroll
+    for (int qt = 0; qt < MAXQT; ++qt)
+#pragma unroll
+        for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) o[qt][nt][i] = 0.f;
+
+    const int d0 = NTW * 8 * warp;
+    const uint32_t ks0 = smem_u32(Ks), vs0 = smem_u32(Vs);
+    const int mi = lane >> 3, mr = lane & 7;
+    const uint32_t vlane = vs0 + (uint32_t)(((mi & 1) * 8 + mr) * VROW + (d0 + ((NTW == 2) ? (mi >> 1) * 8 : 0)) * 2);
+    const float scale = rsqrtf((float)HD);
+    const int nch = last_pos / C + 1;
+    for (int ch = 0; ch < nch; ++ch) {
+        const int key0 = ch * C;
+        __syncthreads();  // the previous chunk's K, V, S, Pb are no longer read
+        {
+            const bool one_page = page_shift >= 6;
+            const size_t base = one_page ? kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD) : 0;
+#pragma unroll
+            for (int it = 0; it < C * SEGS / T; ++it) {
+                const int idx = tid + it * T;
+                const int r = idx / SEGS, sg = idx % SEGS;
+                const int p = key0 + r;
+                const bool ok = p <= last_pos;
+                const size_t off = (one_page ? base + (size_t)r * HD
+                                             : kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD)) +
+                                   (size_t)sg * 8;
+                cp_async16_cg(ks0 + r * KROW + sg * 16, kpages + off, ok ? 16 : 0);
+                cp_async16_cg(vs0 + r * VROW + sg * 16, vpages + off, ok ? 16 : 0);
+            }
+            cp_async_commit();
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        // s = q.k: warp w owns keys 8w..8w+7
+        for (int qt = 0; qt < Qpad; qt += 16) {
+            float c[4] = {0.f, 0.f, 0.f, 0.f};
+            const unsigned char* qa = Qb + (qt + g8) * KROW + 16 * t4;
+            const unsigned char* kb = Ks + (8 * warp + g8) * KROW + 16 * t4;
+#pragma unroll
+            for (int j = 0; j < HD / 32; ++j) {
+                const uint4 A0 = *reinterpret_cast<const uint4*>(qa + 64 * j);
+                const uint4 A1 = *reinterpret_cast<const uint4*>(qa + 8 * KROW + 64 * j);
+                const uint4 Bk = *reinterpret_cast<const uint4*>(kb + 64 * j);
+                mma_bf16_16816(c, A0.x, A1.x, A0.y, A1.y, Bk.x, Bk.y);
+                mma_bf16_16816(c, A0.z, A1.z, A0.w, A1.w, Bk.z, Bk.w);
+            }
+            float* sp = S + (size_t)(qt + g8) * SP + 8 * warp + 2 * t4;
+            *reinterpret_cast<float2*>(sp) = make_float2(c[0], c[1]);
+            *reinterpret_cast<float2*>(sp + 8 * SP) = make_float2(c[2], c[3]);
+        }
+        __syncthreads();
+        // per query: mask, running max and sum, p -> bf16
+        for (int qi = warp; qi < Qpad; qi += T / 32) {
+            uint16_t* pb = reinterpret_cast<uint16_t*>(Pb + (size_t)qi * PBROW);
+            if (qi >= Q) {
+                pb[lane] = 0;
+                pb[lane + 32] = 0;
+                continue;
+            }
+            const int pos = first_pos + qi / G;
+            float s0 = S[(size_t)qi * SP + lane] * scale;
+            float s1 = S[(size_t)qi * SP + lane + 32] * scale;
+            if (key0 + lane > pos) s0 = -INFINITY;
+            if (key0 + lane + 32 > pos) s1 = -INFINITY;
+            float cm = fmaxf(s0, s1);
+#pragma unroll
+            for (int sh = 16; sh > 0; sh >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, sh));
+            const float mo = mx[qi], mn = fmaxf(mo, cm);
+            const float p0 = (s0 == -INFINITY) ? 0.f : expf(s0 - mn);
+            const float p1 = (s1 == -INFINITY) ? 0.f : expf(s1 - mn);
+            float l = p0 + p1;
+#pragma unroll
+            for (int sh = 16; sh > 0; sh >>= 1) l += __shfl_xor_sync(0xffffffffu, l, sh);
+            pb[lane] = f2bf(p0);
+            pb[lane + 32] = f2bf(p1);
+            if (lane == 0) {
+                const float a = (mn == -INFINITY) ? 1.f : ((mo == -INFINITY) ? 0.f : expf(mo - mn));
+                al[qi] = a;
+                ls[qi] = ls[qi] * a + l;
+                mx[qi] = mn;
+            }
+        }
+        __syncthreads();
+        // o = o * alpha + p.v: warp w owns output dims d0 .. d0 + 8 NTW - 1
+#pragma unroll
+        for (int qt = 0; qt < MAXQT; ++qt) {
+            if (qt * 16 < Qpad) {
+                float c[NTW][4];
+#pragma unroll
+                for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) c[nt][i] = 0.f;
+                const unsigned char* pa = Pb + (size_t)(qt * 16 + g8) * PBROW + 4 * t4;
+#pragma unroll
+                for (int kk = 0; kk < C / 16; ++kk) {
+                    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(pa + 32 * kk);
+                    const uint32_t a1 = *reinterpret_cast<const uint32_t*>(pa + 8 * PBROW + 32 * kk);
+                    const uint32_t a2 = *reinterpret_cast<const uint32_t*>(pa + 32 * kk + 16);
+                    const uint32_t a3 = *reinterpret_cast<const uint32_t*>(pa + 8 * PBROW + 32 * kk + 16);
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(vlane + (uint32_t)(16 * kk * VROW), b0, b1, b2, b3);
+                    mma_bf16_16816(c[0], a0, a1, a2, a3, b0, b1);
+                    if (NTW == 2) mma_bf16_16816(c[NTW - 1], a0, a1, a2, a3, b2, b3);
+                }
+                const float alo = al[qt * 16 + g8], ahi = al[qt * 16 + g8 + 8];
+#pragma unroll
+                for (int nt = 0; nt < NTW; ++nt) {
+                    o[qt][nt][0] = o[qt][nt][0] * alo + c[nt][0];
+                    o[qt][nt][1] = o[qt][nt][1] * alo + c[nt][1];
+                    o[qt][nt][2] = o[qt][nt][2] * ahi + c[nt][2];
+                    o[qt][nt][3] = o[qt][nt][3] * ahi + c[nt][3];
+                }
+            }
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int qt = 0; qt < MAXQT; ++qt)
+#pragma unroll
+        for (int hrow = 0; hrow < 2; ++hrow) {
+            const int qi = qt * 16 + g8 + 8 * hrow;
+            if (qi < Q) {
+                const int m = qi / G, g = qi % G;
+                const float l = ls[qi];
+                uint16_t* dst = out + ((size_t)(r0 + m) * Hq + (size_t)kh * G + g) * HD + d0 + 2 * t4;
+#pragma unroll
+                for (int nt = 0; nt < NTW; ++nt)
+                    *reinterpret_cast<uint32_t*>(dst + 8 * nt) =
+                        pack_bf16(o[qt][nt][2 * hrow] / l, o[qt][nt][2 * hrow + 1] / l);
+            }
+        }
+}
+
 }  // namespace ls

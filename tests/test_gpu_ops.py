@@ -257,6 +257,16 @@ def test_qkv_projection_fused_with_rope_and_append(path, Hq, Hkv, hd, K, M):
                                        atol=(BF16_REL + 1e-5) * np.abs(ref).max())
 
 
+def attention_tol(q, k, v, Hq, Hkv, hd, ref):
+    """Elementwise bound on |kernel - oracle| for one query row.  The kernels feed the softmax
+    weights to the tensor cores as bf16 (relative error <= 2^-9 each) while the normalising
+    sum stays fp32, so output j moves by at most 2^-9 * sum_i a_i |v_ij| -- the attention
+    output of |v| -- and the bf16 result then rounds once more (BF16_REL of the largest
+    output covers that and the fp32 accumulation)."""
+    spread = O.attention(q, k, np.abs(v), Hq, Hkv, hd)
+    return BF16_REL * np.abs(ref).max() + 2.0 ** -9 * spread + 1e-5
+
+
 @pytest.mark.parametrize("Hq,Hkv,hd", [(4, 2, 64), (4, 4, 128), (8, 2, 128)])
 @pytest.mark.parametrize("M,pos0", [(1, 0), (1, 63), (1, 64), (4, 61), (7, 130), (16, 300), (3, 1000)])
 def test_attention(Hq, Hkv, hd, M, pos0):
@@ -277,7 +287,7 @@ def test_attention(Hq, Hkv, hd, M, pos0):
     kf, vf, qf = vals(kl).reshape(n + 8, -1), vals(vl).reshape(n + 8, -1), vals(q)
     for m in range(M):
         ref = O.attention(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd)
-        np.testing.assert_allclose(vals(out[m]), ref, rtol=0, atol=BF16_REL * np.abs(ref).max() + 1e-5)
+        assert (np.abs(vals(out[m]) - ref) <= attention_tol(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd, ref)).all()
 
 
 def test_attention_rows_do_not_depend_on_pass_size():
@@ -389,4 +399,4 @@ def test_prefill_attention(Hq, Hkv, hd, R, pos0):
     kf, vf, qf = vals(kl).reshape(n + 8, -1), vals(vl).reshape(n + 8, -1), vals(q)
     for m in sorted({0, R // 2, R - 1, min(R - 1, 15), min(R - 1, 16)}):
         ref = O.attention(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd)
-        np.testing.assert_allclose(vals(out[m]), ref, rtol=0, atol=BF16_REL * np.abs(ref).max() + 1e-5)
+        assert (np.abs(vals(out[m]) - ref) <= attention_tol(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd, ref)).all()
