@@ -39,6 +39,8 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) of one launch of the roofline kernel, from the ncu capture that
 # profiles/linear_mma_kernel_llama2-7b_shapes.md summarises; keyed by (workload, rows).  Set an
 # entry to None when the kernel changes until the counters have been taken again.
+# thresholds on the exit-logit margin tried by the adaptive-draft-length leg (logit units)
+ADAPTIVE_MARGINS = (0.01, 0.02, 0.04, 0.08)
 ROOFLINE_TRAFFIC = {("llama2-7b", 7): 180.43e6 + 3.8e6}
 
 
@@ -253,6 +255,23 @@ def run_own(args):
     no_reuse = {"value": NEW / (nst.decode_ms / 1e3), "unit": UNIT,
                 "ids_equal": bool(np.array_equal(no_reuse_ids, spec_ids))}
 
+    # ---- adaptive draft length (an extension beyond the paper's fixed d): drafting stops when the
+    # exit-logit top-1/top-2 margin falls below a threshold; ids must not change
+    adaptive = {"unit": UNIT, "max_draft": d, "points": []}
+    for tau in ADAPTIVE_MARGINS:
+        B.ls_decode_adaptive(gm.h, E, d, tau, NEW)
+        B.ls_decode_adaptive(gm.h, E, d, tau, NEW)
+        ast = gm.stats()
+        a_ids, a_acc = B.ls_read_output(gm.h, NEW)
+        a_dr = B.ls_read_drafted(gm.h, NEW)
+        adaptive["points"].append({"min_margin": tau, "value": round(NEW / (ast.decode_ms / 1e3), 1),
+                                   "kept_per_step": round(float(a_dr.mean()), 3),
+                                   "accepted_per_step": round(float(a_acc.mean()), 3), "steps": int(len(a_acc)),
+                                   "hbm_frac_measured": round((ast.weight_bytes + ast.kv_bytes) /
+                                                              (ast.decode_ms / 1e3) / 1e9 / peak, 4),
+                                   "ids_equal": bool(np.array_equal(a_ids, spec_ids))})
+    adaptive["best"] = max(adaptive["points"], key=lambda p: p["value"])
+
     # ---- end to end through the public call: host prompt in, host ids out, prefill included
     e2e_ms = []
     for i in range(1 + max(1, min(args.steps, 3))):
@@ -280,7 +299,8 @@ def run_own(args):
            "emitted_per_step": float(NEW / len(acc)), "spec_steps": int(len(acc)), "host_syncs": int(st.host_syncs),
            "full_greedy": {"value": full_tok_s, "unit": UNIT, "hbm_GB/s": round(full_gbs, 1),
                            "hbm_frac_measured": round(full_gbs / peak, 4), "hbm_frac_8TBs": round(full_gbs / 8000, 4)},
-           "speedup_vs_full_greedy": value / world / full_tok_s, "without_exit_cache_reuse": no_reuse, "ids_equal_full_greedy": lossless,
+           "speedup_vs_full_greedy": value / world / full_tok_s, "without_exit_cache_reuse": no_reuse, "adaptive_draft": adaptive,
+           "ids_equal_full_greedy": lossless,
            "loop_hbm": {"GB/s": round(loop_gbs, 1), "frac_measured": round(loop_gbs / peak, 4),
                         "frac_8TBs": round(loop_gbs / 8000, 4), "bytes_per_loop": int(sched_bytes)},
            "prefill_ms": prefill_ms}

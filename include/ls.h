@@ -127,6 +127,28 @@ int ls_generate(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt,
                 int32_t *out_ids_host, int32_t *out_n,
                 int32_t *accepted_per_step_host, int32_t *out_n_steps);
 
+/* Self-speculative decoding with an adaptive draft length.  The paper drafts a fixed number
+ * of tokens per step and names dynamic, per-token conditions as future work (Sec. 9); this
+ * entry point adds the simplest such condition, a confidence test on the exit logits, in the
+ * way that keeps the method exact.  Within a step, draft pass j (j = 0 .. max_draft-1)
+ * computes g(x_E) for its row; if the margin between the two largest exit logits,
+ *     margin_j = logit_(1) - logit_(2)   (fp32, 0 on a tie),
+ * is below min_margin, draft j is NOT kept and drafting stops: the step keeps k = j drafts
+ * (possibly none).  Otherwise all max_draft drafts are kept and, as in ls_generate, one more
+ * early pass prepares the last draft's row.  Verification then scores rows 0..k, accepts the
+ * longest agreeing prefix of the k kept drafts and emits the verified token after it, so the
+ * ids are still exactly those of ls_generate_full whatever min_margin is; only the number of
+ * steps and the work per step change.  The exit-layer row of the discarded draft's input is
+ * already computed, so stopping costs no extra pass.
+ * min_margin > 0 (LS_ERR_INVALID_ARG otherwise; +inf keeps no draft at all, every step then
+ * emits one token).  drafted_per_step_host [max_new] receives k of every step,
+ * accepted_per_step_host the accepted count n <= k.  Other arguments and errors as
+ * ls_generate with num_draft = max_draft. */
+int ls_generate_adaptive(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt,
+                         int32_t exit_layer, int32_t max_draft, float min_margin, int32_t max_new,
+                         int32_t *out_ids_host, int32_t *out_n, int32_t *accepted_per_step_host,
+                         int32_t *drafted_per_step_host, int32_t *out_n_steps);
+
 /* Autoregressive greedy decoding with all L layers: the baseline of Sec. 6.2 and,
  * by construction of the method, the exact result ls_generate must reproduce. */
 int ls_generate_full(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt,
@@ -147,12 +169,17 @@ int ls_generate_early(ls_model *m, const int32_t *prompt_ids_host, int32_t n_pro
 int ls_prefill(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt, int32_t layers);
 int ls_decode(ls_model *m, int32_t exit_layer, int32_t num_draft, int32_t max_new);
 /* ls_decode with options.  LS_DECODE_NO_EXIT_CACHE is the paper's "without KVQ reuse" ablation
- * (Sec. 6.2, Table 7): the verify pass does not continue from the cached exit-layer
+ * (Sec. 7, Table 7): the verify pass does not continue from the cached exit-layer
  * activations but runs all L layers on the num_draft+1 rows again.  Same ids, more bytes. */
 #define LS_DECODE_NO_EXIT_CACHE 1
 int ls_decode_flags(ls_model *m, int32_t exit_layer, int32_t num_draft, int32_t max_new, int32_t flags);
 int ls_read_output(ls_model *m, int32_t *out_ids_host, int32_t *out_n,
                    int32_t *accepted_per_step_host, int32_t *out_n_steps);
+/* The decode loop of ls_generate_adaptive from a prefilled state, and the kept-draft count of
+ * every step of the last decode call (num_draft for the non-adaptive loops). */
+int ls_decode_adaptive(ls_model *m, int32_t exit_layer, int32_t max_draft, float min_margin,
+                       int32_t max_new);
+int ls_read_drafted(ls_model *m, int32_t *drafted_per_step_host, int32_t *out_n_steps);
 
 /* Teacher-forced logits for parity checks: feed ids_host[0..n-1] at positions 0..n-1
  * and return g(x_E) and g(x_L) for every position (host fp32 [n, V]; either may be

@@ -426,6 +426,95 @@ int32_t lso_generate_spec(lso_model *m, const int32_t *prompt, int32_t P, int32_
     return 0;
 }
 
+/* Self-speculative decoding with an adaptive draft length: an extension (the paper drafts
+ * a fixed d per step and leaves dynamic per-token conditions to future work, Sec. 9), stated
+ * here so that the library's version of it has something to be compared with.
+ *
+ * One step, with at most d drafts and a confidence threshold tau > 0 on the exit logits:
+ *   draft    for j in 0..d-1: layers 0..E-1 on the current draft input at position c+j,
+ *            keep X_E[j]; z = g(X_E[j]); margin = largest - second largest entry of z
+ *            (0 on a tie).  If margin < tau: the token is not kept, drafting stops, k = j.
+ *            Otherwise draft[j] = argmax z and it becomes the next input.
+ *            If no pass stopped: k = d and, as in the fixed-length loop, layers 0..E-1 run
+ *            once more on draft[d-1] at position c+d -> X_E[d].
+ *   verify   layers E..L-1 on rows 0..k; verified[i] = argmax g(x_L[i])
+ *   match    n = leading agreements among the k kept drafts; emit draft[0..n-1], verified[n]
+ *   crop     cur = verified[n]; c += n+1
+ * Every emitted token is either a draft the full model agreed with or the full model's own
+ * token, so the ids are those of lso_generate_full for every tau.  drafted[step] = k,
+ * accepted[step] = n.  closest_gap ([max_new], may be NULL) receives, per step, the smallest
+ * |margin - tau| over the stop decisions the step took -- what a comparison with an
+ * implementation in another precision needs, to know how close to the threshold it came.
+ */
+int32_t lso_generate_adaptive(lso_model *m, const int32_t *prompt, int32_t P, int32_t exit_layer,
+                              int32_t max_draft, double tau, int32_t max_new, int32_t *out_ids,
+                              int32_t *out_n, int32_t *accepted, int32_t *drafted, int32_t *out_steps,
+                              double *closest_gap)
+{
+    const lso_config *c = &m->c;
+    int E = exit_layer, d = max_draft, L = c->n_layers, D = c->d_model;
+    if (P < 1 || E < 1 || E > L - 1 || d < 1 || !(tau > 0.0) || P + max_new + d + 1 > c->max_seq) return -1;
+    double *x = (double *)malloc(sizeof(double) * (size_t)D);
+    double *XE = (double *)malloc(sizeof(double) * (size_t)D * (size_t)(d + 1));
+    double *z = (double *)malloc(sizeof(double) * (size_t)c->vocab);
+    int32_t *draft = (int32_t *)malloc(sizeof(int32_t) * (size_t)d);
+    int32_t *verified = (int32_t *)malloc(sizeof(int32_t) * (size_t)(d + 1));
+
+    for (int t = 0; t < P - 1; ++t) {
+        embed(m, prompt[t], x);
+        layers_token(m, 0, L, x, t);
+    }
+    int32_t cur = prompt[P - 1];
+    int clen = P - 1, n_out = 0, steps = 0, stop = 0;
+    while (n_out < max_new && !stop) {
+        int32_t in = cur;
+        int k = d;
+        double gap = INFINITY; /* smallest |margin - tau| over the decisions taken this step */
+        for (int j = 0; j < d; ++j) {
+            embed(m, in, x);
+            layers_token(m, 0, E, x, clen + j);
+            memcpy(XE + (size_t)j * D, x, sizeof(double) * (size_t)D);
+            lm_head(m, x, z);
+            double margin;
+            int32_t tok = lso_argmax(z, c->vocab, &margin, NULL);
+            if (fabs(margin - tau) < gap) gap = fabs(margin - tau);
+            if (margin < tau) {
+                k = j;
+                break;
+            }
+            draft[j] = tok;
+            in = tok;
+        }
+        if (k == d) {
+            embed(m, draft[d - 1], x);
+            layers_token(m, 0, E, x, clen + d);
+            memcpy(XE + (size_t)d * D, x, sizeof(double) * (size_t)D);
+        }
+        for (int i = 0; i <= k; ++i) {
+            memcpy(x, XE + (size_t)i * D, sizeof(double) * (size_t)D);
+            layers_token(m, E, L, x, clen + i);
+            lm_head(m, x, z);
+            verified[i] = lso_argmax(z, c->vocab, NULL, NULL);
+        }
+        int n = lso_match(draft, verified, k);
+        for (int i = 0; i <= n && n_out < max_new && !stop; ++i) {
+            int32_t tok = (i < n) ? draft[i] : verified[n];
+            out_ids[n_out++] = tok;
+            if (c->eos_id >= 0 && tok == c->eos_id) stop = 1;
+        }
+        cur = verified[n];
+        clen += n + 1;
+        accepted[steps] = n;
+        drafted[steps] = k;
+        if (closest_gap) closest_gap[steps] = gap;
+        ++steps;
+    }
+    *out_n = n_out;
+    *out_steps = steps;
+    free(x); free(XE); free(z); free(draft); free(verified);
+    return 0;
+}
+
 int32_t lso_num_threads(void)
 {
 #ifdef _OPENMP

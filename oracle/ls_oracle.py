@@ -80,6 +80,9 @@ def lib():
         L.lso_generate_early.restype = i32
         L.lso_generate_spec.argtypes = [C.c_void_p, ip, i32, i32, i32, i32, ip, ip, ip, ip, ip]
         L.lso_generate_spec.restype = i32
+        L.lso_generate_adaptive.argtypes = [C.c_void_p, ip, i32, i32, i32, C.c_double, i32, ip, ip, ip, ip, ip,
+                                            C.POINTER(C.c_double)]
+        L.lso_generate_adaptive.restype = i32
         L.lso_num_threads.restype = i32
         _lib = L
     return _lib
@@ -241,6 +244,22 @@ class Model:
         if rc:
             raise ValueError("lso_generate_early: bad arguments")
         return out[:n.value]
+
+    def generate_adaptive(self, prompt, exit_layer, max_draft, min_margin, max_new):
+        """Adaptive draft length: -> ids, accepted_per_step, drafted_per_step, and per step the
+        smallest |exit-logit margin - min_margin| among the stop decisions it took."""
+        prompt = np.ascontiguousarray(prompt, dtype=np.int32)
+        out = np.zeros(max_new, dtype=np.int32)
+        acc = np.zeros(max_new, dtype=np.int32)
+        dr = np.zeros(max_new, dtype=np.int32)
+        gap = np.zeros(max_new, dtype=np.float64)
+        n, s = C.c_int32(), C.c_int32()
+        rc = lib().lso_generate_adaptive(self._h, _ip(prompt), prompt.size, exit_layer, max_draft,
+                                         float(min_margin), max_new, _ip(out), C.byref(n), _ip(acc), _ip(dr),
+                                         C.byref(s), gap.ctypes.data_as(C.POINTER(C.c_double)))
+        if rc:
+            raise ValueError("lso_generate_adaptive: bad arguments")
+        return out[:n.value], acc[:s.value], dr[:s.value], gap[:s.value]
 
     def generate_spec(self, prompt, exit_layer, num_draft, max_new):
         """-> ids, accepted_per_step, cache_len after every step"""

@@ -23,8 +23,8 @@ LS_LINEAR_AUTO, LS_LINEAR_FMA, LS_LINEAR_MMA = 0, 1, 2
 
 EXPORTS = (
     "ls_strerror", "ls_last_cuda_error", "ls_workspace_bytes", "ls_model_create", "ls_model_destroy",
-    "ls_set_page_table", "ls_generate", "ls_generate_full", "ls_generate_early", "ls_prefill",
-    "ls_decode", "ls_decode_flags", "ls_read_output", "ls_debug_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
+    "ls_set_page_table", "ls_generate", "ls_generate_adaptive", "ls_generate_full", "ls_generate_early", "ls_prefill",
+    "ls_decode", "ls_decode_flags", "ls_decode_adaptive", "ls_read_output", "ls_read_drafted", "ls_debug_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
     "ls_op_linear", "ls_op_gate_up_swiglu", "ls_op_lm_head_scratch_bytes", "ls_op_lm_head_argmax",
     "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_qkv_rope_append", "ls_op_attention_scratch_bytes", "ls_op_attention", "ls_op_accept",
     "ls_op_gemm", "ls_op_prefill_attention",
@@ -89,6 +89,9 @@ def lib():
             "ls_decode": (C.c_int, [vp, i32, i32, i32]),
             "ls_decode_flags": (C.c_int, [vp, i32, i32, i32, i32]),
             "ls_read_output": (C.c_int, [vp, ip, ip, ip, ip]),
+            "ls_generate_adaptive": (C.c_int, [vp, ip, i32, i32, i32, C.c_float, i32, ip, ip, ip, ip, ip]),
+            "ls_decode_adaptive": (C.c_int, [vp, i32, i32, C.c_float, i32]),
+            "ls_read_drafted": (C.c_int, [vp, ip, ip]),
             "ls_debug_logits": (C.c_int, [vp, ip, i32, i32, fp, fp]),
             "ls_get_stats": (C.c_int, [vp, C.POINTER(ls_stats)]),
             "ls_op_embed": (C.c_int, [vp, vp, i32, i32, i32, vp, vp]),
@@ -187,6 +190,18 @@ def ls_generate(h, prompt, exit_layer, num_draft, max_new):
     return out[:n.value], acc[:s.value]
 
 
+def ls_generate_adaptive(h, prompt, exit_layer, max_draft, min_margin, max_new):
+    """-> (ids, accepted_per_step, drafted_per_step) as numpy int32 arrays"""
+    a, p = _i32(prompt)
+    out, acc, dr = np.zeros(max_new, np.int32), np.zeros(max_new, np.int32), np.zeros(max_new, np.int32)
+    n, s = C.c_int32(), C.c_int32()
+    ip = C.POINTER(C.c_int32)
+    _ck(lib().ls_generate_adaptive(h, p, a.size, exit_layer, max_draft, float(min_margin), max_new,
+                                   out.ctypes.data_as(ip), C.byref(n), acc.ctypes.data_as(ip),
+                                   dr.ctypes.data_as(ip), C.byref(s)), "ls_generate_adaptive")
+    return out[:n.value], acc[:s.value], dr[:s.value]
+
+
 def ls_generate_full(h, prompt, max_new):
     a, p = _i32(prompt)
     out = np.zeros(max_new, np.int32)
@@ -219,6 +234,17 @@ LS_DECODE_NO_EXIT_CACHE = 1
 
 def ls_decode_flags(h, exit_layer, num_draft, max_new, flags):
     _ck(lib().ls_decode_flags(h, exit_layer, num_draft, max_new, flags), "ls_decode_flags")
+
+
+def ls_decode_adaptive(h, exit_layer, max_draft, min_margin, max_new):
+    _ck(lib().ls_decode_adaptive(h, exit_layer, max_draft, float(min_margin), max_new), "ls_decode_adaptive")
+
+
+def ls_read_drafted(h, max_new):
+    dr = np.zeros(max_new, np.int32)
+    s = C.c_int32()
+    _ck(lib().ls_read_drafted(h, dr.ctypes.data_as(C.POINTER(C.c_int32)), C.byref(s)), "ls_read_drafted")
+    return dr[:s.value]
 
 
 def ls_read_output(h, max_new):
@@ -357,6 +383,9 @@ class Model:
 
     def generate(self, prompt, exit_layer, num_draft, max_new):
         return ls_generate(self.h, prompt, exit_layer, num_draft, max_new)
+
+    def generate_adaptive(self, prompt, exit_layer, max_draft, min_margin, max_new):
+        return ls_generate_adaptive(self.h, prompt, exit_layer, max_draft, min_margin, max_new)
 
     def generate_full(self, prompt, max_new):
         return ls_generate_full(self.h, prompt, max_new)

@@ -17,8 +17,10 @@ enum Ctl : int {
     CTL_MAX_NEW = 5,
     CTL_EOS = 6,
     CTL_STATUS = 7,     // non-zero: a kernel's bounds check refused an access
-    CTL_WORDS = 8
+    CTL_D_EFF = 8,      // adaptive drafting: drafts this step keeps; kernels of draft pass j > this return at once
+    CTL_WORDS = 16
 };
+constexpr int kNoStop = 0x7fffffff;  // CTL_D_EFF while no draft pass has stopped the drafting
 
 enum DevStatus : int { DEV_OK = 0, DEV_BAD_TOKEN = 1, DEV_POS_OVERFLOW = 2 };
 
@@ -136,6 +138,35 @@ struct ValIdx {
 __device__ __forceinline__ bool better(float v, int i, float bv, int bi)
 {
     return v > bv || (v == bv && i < bi);
+}
+// best (v, idx) and second-largest value s of a growing set: one more element ...
+__device__ __forceinline__ void top2_push(float x, int n, float& v, int& idx, float& s)
+{
+    if (better(x, n, v, idx)) {
+        s = v;
+        v = x;
+        idx = n;
+    } else {
+        s = fmaxf(s, x);
+    }
+}
+// ... or the union with a disjoint set whose best is (v2, i2) and whose second value is s2
+__device__ __forceinline__ void top2_merge(float v2, int i2, float s2, float& v, int& idx, float& s)
+{
+    if (better(v2, i2, v, idx)) {
+        s = fmaxf(v, s2);
+        v = v2;
+        idx = i2;
+    } else {
+        s = fmaxf(s, v2);
+    }
+}
+
+// True when this launch has nothing to do: the loop is finished, or the launch belongs to
+// draft pass `gate` (0: not a draft pass) and the step stopped drafting before it.
+__device__ __forceinline__ bool pass_idle(const int32_t* ctl, int gate)
+{
+    return ctl && (ctl[CTL_DONE] || (gate > 0 && gate > ctl[CTL_D_EFF]));
 }
 
 }  // namespace ls

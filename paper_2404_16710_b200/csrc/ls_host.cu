@@ -97,6 +97,9 @@ struct ls_model {
     float* ss;     // [16][n_part] partial sums of squares of the residual rows (fused RMSNorm)
     int n_part;
     ValIdx* cand;
+    float* second;      // per-CTA second-largest logit beside each argmax candidate (adaptive drafting)
+    int32_t* drafted;   // drafts kept per step (adaptive drafting)
+    int gate;           // draft pass the launches being enqueued belong to (0: none)
     int page_shift, n_pages, chunk_cap, cand_stride;
     // loop state
     int n_prompt, last_tok, prefilled_layers, grid_chunks;
@@ -106,10 +109,10 @@ struct ls_model {
         cudaGraphExec_t exec;
         int64_t nodes;
     };
-    std::map<uint64_t, G> graphs;
+    std::map<std::pair<uint64_t, uint32_t>, G> graphs;
     cudaEvent_t ev0, ev1;
     ls_stats stats;
-    std::vector<int32_t> h_out, h_acc;
+    std::vector<int32_t> h_out, h_acc, h_drafted;
     int h_n_out, h_n_steps;
 };
 
@@ -148,6 +151,8 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     unsigned char* o = take(2 * (size_t)kMaxRows * qw);
     unsigned char* a = take(2 * (size_t)kMaxRows * c.d_ffn);
     unsigned char* cand = take(sizeof(ValIdx) * kMaxRows * cand_stride);
+    unsigned char* second = take(sizeof(float) * kMaxRows * cand_stride);
+    unsigned char* drafted = take(sizeof(int32_t) * c.max_seq);
     const int n_part = (c.d_model + 15) / 16;  // CTAs of a residual projection = partial sums per row
     unsigned char* ss = take(sizeof(float) * kMaxRows * n_part);
     unsigned char* he = take(2 * (size_t)kMaxRows * c.d_model);
@@ -189,6 +194,8 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
         m->o = (uint16_t*)o;
         m->a = (uint16_t*)a;
         m->cand = (ValIdx*)cand;
+        m->second = (float*)second;
+        m->drafted = (int32_t*)drafted;
         m->n_pages = n_pages;
         m->chunk_cap = chunk_cap;
         m->cand_stride = cand_stride;
@@ -201,16 +208,16 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
 int attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
                 int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int hd, int page_shift,
                 int max_seq, int chunk_cap, int grid_chunks, float* part, int32_t* counters, uint16_t* out,
-                const LaunchCtx& lc)
+                const LaunchCtx& lc, int gate = 0)
 {
     const int Q = Hq / Hkv * M;
     dim3 grid(grid_chunks, Hkv);
     if (hd == 128) {
         LS_CK(launch(lc, attn_kernel<128>, grid, dim3(kAttnThreads), attn_smem_bytes<128>(Q), q, kp, vp, pt, ctl, pos_off, M,
-                     Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out));
+                     Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out, gate));
     } else {
         LS_CK(launch(lc, attn_kernel<64>, grid, dim3(kAttnThreads), attn_smem_bytes<64>(Q), q, kp, vp, pt, ctl, pos_off, M,
-                     Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out));
+                     Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out, gate));
     }
     return LS_OK;
 }
@@ -305,26 +312,30 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off, int
         a.max_seq = c.max_seq;
         a.pos_off = pos_off;
         a.theta = c.rope_theta;
+        a.gate = m->gate;
         norm_in(m, a, slot);
         LS_CK(launch_linear(m->path, EPI_QKV, a, st));
         LS_TRY(attn_launch(m->q, kp, vp, m->page_table, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift,
-                           c.max_seq, m->chunk_cap, m->grid_chunks, m->part, m->attn_counters, m->o, st));
+                           c.max_seq, m->chunk_cap, m->grid_chunks, m->part, m->attn_counters, m->o, st, m->gate));
         a = lin_args(w.wo, m->o, M, D, qw);
         a.out = xrow;
         a.ldo = D;
         a.ctl = m->ctl;
+        a.gate = m->gate;
         norm_out(m, a, slot, w.ffn_norm, hrow, nullptr, nullptr);
         LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
         a = lin_args(w.wg, hrow, M, F, D);
         a.w1 = w.wu;
         a.out_bf16 = m->a;
         a.ctl = m->ctl;
+        a.gate = m->gate;
         norm_in(m, a, slot);
         LS_CK(launch_linear(m->path, EPI_SWIGLU, a, st));
         a = lin_args(w.wd, m->a, M, D, F);
         a.out = xrow;
         a.ldo = D;
         a.ctl = m->ctl;
+        a.gate = m->gate;
         if (l + 1 < l1) norm_out(m, a, slot, m->lw[l + 1].attn_norm, hrow, nullptr, nullptr);
         else norm_out(m, a, slot, gain_end_a, hrow, gain_end_b, herow);
         LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
@@ -336,7 +347,9 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off, int
 
 // shared head g(.) = final norm + LM head (+ argmax) on the M rows of slot `slot`, whose
 // x*final_gain rows and partial sums the last down-projection has left
-int run_head(ls_model* m, int M, int slot, int32_t* tok_out, float* logits)
+// min_margin > 0 (the head of a draft pass, adaptive drafting): also reduce the second-largest
+// logit and stop the step's drafting when the top-two margin falls below it
+int run_head(ls_model* m, int M, int slot, int32_t* tok_out, float* logits, float min_margin = 0.f)
 {
     const ls_config& c = m->c;
     const LaunchCtx st = {m->st, m->pdl};
@@ -346,10 +359,13 @@ int run_head(ls_model* m, int M, int slot, int32_t* tok_out, float* logits)
     a.out = logits;
     a.ldo = c.vocab;
     a.ctl = m->ctl;
+    a.gate = m->gate;
+    a.second = min_margin > 0.f ? m->second : nullptr;
     norm_in(m, a, slot);
     LS_CK(launch_linear(m->path, EPI_ARGMAX, a, st));
-    LS_CK(launch(st, argmax_finish_kernel, dim3(M), dim3(256), 0, m->cand, n_candidates(m->path, c.vocab, c.d_model, M),
-                 m->cand_stride, tok_out, m->ctl));
+    LS_CK(launch(st, argmax_finish_kernel, dim3(M), dim3(256), 0, (const ValIdx*)m->cand,
+                 n_candidates(m->path, c.vocab, c.d_model, M), m->cand_stride, tok_out, m->ctl,
+                 (const float*)a.second, min_margin, m->gate));
     m->launches += 2;
     return LS_OK;
 }
@@ -358,7 +374,7 @@ int run_embed(ls_model* m, const int32_t* tok_dev, int M, float* xrow, int slot)
 {
     LS_CK(launch(LaunchCtx{m->st, m->pdl}, embed_kernel, dim3(M), dim3(256), 0, m->emb, tok_dev, m->c.d_model,
                  m->c.vocab, xrow, m->ctl, m->lw[0].attn_norm, m->h + (size_t)slot * m->c.d_model,
-                 m->ss + (size_t)slot * m->n_part, m->n_part, m->n_part));
+                 m->ss + (size_t)slot * m->n_part, m->n_part, m->n_part, m->gate));
     m->launches += 1;
     return LS_OK;
 }
@@ -457,7 +473,7 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
     const LaunchCtx lc = {st, false};
     int32_t* status = m->ctl + CTL_STATUS;
     LS_CK(launch(lc, embed_kernel, dim3(R), dim3(256), 0, m->emb, m->ids + r0, D, c.vocab, m->px, m->ctl, nullptr,
-                 nullptr, nullptr, 0, 0));
+                 nullptr, nullptr, 0, 0, 0));
     for (int l = 0; l < layers; ++l) {
         const LayerW& w = m->lw[l];
         uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
@@ -482,9 +498,14 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
 }
 
 // one step of the loop.  E == L with d == 0: plain greedy; E < L with d == 0: early exit.
-int enqueue_step(ls_model* m, int E, int d, bool reuse)
+// min_margin > 0: adaptive drafting.  Draft pass j (j >= 1) is enqueued with gate j, so it idles
+// once an earlier pass's head has found its two largest exit logits closer than min_margin;
+// the verify pass always runs on d + 1 rows (the rows beyond the kept drafts are stale and
+// never read by the rows that count: causal attention, one dot product per output element).
+int enqueue_step(ls_model* m, int E, int d, bool reuse, float min_margin = 0.f)
 {
     const int D = m->c.d_model, L = m->c.n_layers;
+    const bool adaptive = min_margin > 0.f;
     if (d == 0) {
         LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
         LS_TRY(run_layers(m, 0, E, 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
@@ -492,18 +513,20 @@ int enqueue_step(ls_model* m, int E, int d, bool reuse)
     } else {
         for (int j = 0; j <= (reuse ? d : d - 1); ++j) {  // self-drafting (Sec. 4.3.1) + the extra early pass
             float* xr = m->x + (size_t)j * D;
+            m->gate = adaptive ? j : 0;
             LS_TRY(run_embed(m, j == 0 ? m->ctl + CTL_CUR_TOK : m->draft + (j - 1), 1, xr, j));
             // the exit-layer row goes to the LM head (final gain) and, pre-scaled by layer E's
             // gain, to the verify pass (the exit-layer cache of Sec. 4.3.3)
             LS_TRY(run_layers(m, 0, E, 1, xr, j, j, m->h + (size_t)j * D, j < d ? m->fnorm : nullptr,
                               reuse ? m->lw[E].attn_norm : nullptr));
-            if (j < d) LS_TRY(run_head(m, 1, j, m->draft + j, nullptr));
+            if (j < d) LS_TRY(run_head(m, 1, j, m->draft + j, nullptr, min_margin));
         }
+        m->gate = 0;
         if (reuse) {
             // self-verification (Sec. 4.3.2) from the exit-layer activations
             LS_TRY(run_layers(m, E, L, d + 1, m->x, 0, 0, m->hE, m->fnorm, nullptr));
         } else {
-            // the ablation of Sec. 6.2 / Table 7: no exit-layer cache, verification recomputes the
+            // the ablation of Sec. 7 (Table 7): no exit-layer cache, verification recomputes the
             // early layers of all d+1 rows (and rewrites their k, v with the same values)
             LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
             LS_TRY(run_embed(m, m->draft, d, m->x + D, 1));
@@ -511,8 +534,9 @@ int enqueue_step(ls_model* m, int E, int d, bool reuse)
         }
         LS_TRY(run_head(m, d + 1, 0, m->verified, nullptr));
     }
-    LS_CK(launch(LaunchCtx{m->st, m->pdl}, accept_kernel, dim3(1), dim3(32), 0, m->draft, m->verified, d, m->ctl,
-                 m->out_ids, m->accepted));
+    LS_CK(launch(LaunchCtx{m->st, m->pdl}, accept_kernel, dim3(1), dim3(32), 0, (const int32_t*)m->draft,
+                 (const int32_t*)m->verified, d, m->ctl, m->out_ids, m->accepted, adaptive ? 1 : 0,
+                 adaptive ? m->drafted : (int32_t*)nullptr));
     m->launches += 1;
     return LS_OK;
 }
@@ -523,15 +547,18 @@ void drop_graphs(ls_model* m)
     m->graphs.clear();
 }
 
-int get_graph(ls_model* m, int E, int d, bool reuse, ls_model::G** out)
+int get_graph(ls_model* m, int E, int d, bool reuse, float min_margin, ls_model::G** out)
 {
-    uint64_t key = ((uint64_t)(reuse ? 0 : 1) << 48) | ((uint64_t)E << 32) | ((uint64_t)d << 16) | (uint64_t)m->grid_chunks;
+    uint32_t mbits;
+    memcpy(&mbits, &min_margin, sizeof(mbits));
+    const std::pair<uint64_t, uint32_t> key(
+        ((uint64_t)(reuse ? 0 : 1) << 48) | ((uint64_t)E << 32) | ((uint64_t)d << 16) | (uint64_t)m->grid_chunks, mbits);
     auto it = m->graphs.find(key);
     if (it == m->graphs.end()) {
         cudaGraph_t graph = nullptr;
         int64_t before = m->launches;
         LS_CK(cudaStreamBeginCapture(m->st, cudaStreamCaptureModeRelaxed));
-        int rc = enqueue_step(m, E, d, reuse);
+        int rc = enqueue_step(m, E, d, reuse, min_margin);
         cudaError_t e = cudaStreamEndCapture(m->st, &graph);
         if (rc != LS_OK) {
             if (graph) cudaGraphDestroy(graph);
@@ -551,7 +578,7 @@ int get_graph(ls_model* m, int E, int d, bool reuse, ls_model::G** out)
 
 int write_ctl(ls_model* m, int cache_len, int cur, int max_new)
 {
-    int32_t w[CTL_WORDS] = {cache_len, cur, 0, 0, 0, max_new, m->c.eos_id, 0};
+    int32_t w[CTL_WORDS] = {cache_len, cur, 0, 0, 0, max_new, m->c.eos_id, 0, kNoStop};
     LS_CK(cudaMemcpyAsync(m->ctl, w, sizeof(w), cudaMemcpyHostToDevice, m->st));
     LS_CK(cudaStreamSynchronize(m->st));  // w is a stack array
     return LS_OK;
@@ -582,6 +609,8 @@ void set_grid_chunks(ls_model* m, int max_pos_exclusive)
         drop_graphs(m);
     }
 }
+
+int decode_loop(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new, int32_t flags, float min_margin);
 
 }  // namespace
 
@@ -781,8 +810,24 @@ int ls_decode(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_ne
 
 int ls_decode_flags(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new, int32_t flags)
 {
+    return decode_loop(m, exit_layer, num_draft, max_new, flags, 0.f);
+}
+
+int ls_decode_adaptive(ls_model* m, int32_t exit_layer, int32_t max_draft, float min_margin, int32_t max_new)
+{
+    if (!(min_margin > 0.f)) return LS_ERR_INVALID_ARG;  // also refuses NaN
+    if (exit_layer < 1 || max_draft < 1) return LS_ERR_INVALID_ARG;
+    return decode_loop(m, exit_layer, max_draft, max_new, 0, min_margin);
+}
+
+}  // extern "C"
+
+namespace {
+int decode_loop(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new, int32_t flags, float min_margin)
+{
     if (!m || m->n_prompt < 1 || (flags & ~LS_DECODE_NO_EXIT_CACHE)) return LS_ERR_INVALID_ARG;
     const bool reuse = !(flags & LS_DECODE_NO_EXIT_CACHE);
+    const bool adaptive = min_margin > 0.f;
     const ls_config& c = m->c;
     const int L = c.n_layers;
     int E = exit_layer, d = num_draft;
@@ -802,7 +847,7 @@ int ls_decode_flags(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t 
     set_grid_chunks(m, m->n_prompt + max_new + d + 1);
 
     ls_model::G* g = nullptr;
-    if (m->use_graphs) LS_TRY(get_graph(m, E, d, reuse, &g));
+    if (m->use_graphs) LS_TRY(get_graph(m, E, d, reuse, min_margin, &g));
     LS_TRY(write_ctl(m, m->n_prompt - 1, m->last_tok, max_new));
     int64_t launched = 0;
     int syncs = 0, n_out = 0, steps_done = 0;
@@ -822,7 +867,7 @@ int ls_decode_flags(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t 
                 launched += g->nodes;
             } else {
                 int64_t before = m->launches;
-                LS_TRY(enqueue_step(m, E, d, reuse));
+                LS_TRY(enqueue_step(m, E, d, reuse, min_margin));
                 launched += m->launches - before;
             }
         }
@@ -842,8 +887,12 @@ int ls_decode_flags(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t 
     m->h_n_steps = w[CTL_N_STEPS];
     m->h_out.resize(m->h_n_out);
     m->h_acc.resize(m->h_n_steps);
+    m->h_drafted.assign(m->h_n_steps, d);
     LS_CK(cudaMemcpyAsync(m->h_out.data(), m->out_ids, sizeof(int32_t) * m->h_n_out, cudaMemcpyDeviceToHost, m->st));
     LS_CK(cudaMemcpyAsync(m->h_acc.data(), m->accepted, sizeof(int32_t) * m->h_n_steps, cudaMemcpyDeviceToHost, m->st));
+    if (adaptive)
+        LS_CK(cudaMemcpyAsync(m->h_drafted.data(), m->drafted, sizeof(int32_t) * m->h_n_steps, cudaMemcpyDeviceToHost,
+                              m->st));
     LS_CK(cudaStreamSynchronize(m->st));
 
     // algorithmic bytes of the schedule (matrices only; norm gains and activations are noise)
@@ -859,9 +908,13 @@ int ls_decode_flags(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t 
             kb += (int64_t)E * kvb * (cl + 1);
         } else {
             if (reuse) {
-                wb += (int64_t)(d + 1) * E * w_layer + (int64_t)d * w_lm + (int64_t)(L - E) * w_layer + w_lm;
-                for (int j = 0; j <= d; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
-                kb += (int64_t)(L - E) * kvb * (cl + d + 1);
+                // draft passes that ran: all d + 1, or with an early stop the k + 1 up to the one
+                // whose head stopped the drafting (k drafts kept); heads: one per pass but the extra one
+                const int k = m->h_drafted[s];
+                const int heads = k < d ? k + 1 : d;
+                wb += (int64_t)(k + 1) * E * w_layer + (int64_t)heads * w_lm + (int64_t)(L - E) * w_layer + w_lm;
+                for (int j = 0; j <= k; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
+                kb += (int64_t)(L - E) * kvb * (cl + k + 1);
             } else {
                 wb += (int64_t)d * (E * w_layer + w_lm) + (int64_t)L * w_layer + w_lm;
                 for (int j = 0; j < d; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
@@ -879,6 +932,17 @@ int ls_decode_flags(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t 
     m->stats.n_steps = m->h_n_steps;
     m->stats.n_accepted = (int32_t)acc_sum;
     m->stats.host_syncs = syncs;
+    return LS_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int ls_read_drafted(ls_model* m, int32_t* drafted, int32_t* out_steps)
+{
+    if (!m) return LS_ERR_INVALID_ARG;
+    if (drafted && m->h_n_steps) memcpy(drafted, m->h_drafted.data(), sizeof(int32_t) * m->h_n_steps);
+    if (out_steps) *out_steps = m->h_n_steps;
     return LS_OK;
 }
 
@@ -902,6 +966,22 @@ int ls_generate(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t ex
     if ((int64_t)n_prompt + max_new + num_draft + 1 > m->c.max_seq) return LS_ERR_CAPACITY;
     LS_TRY(ls_prefill(m, prompt, n_prompt, 0));
     LS_TRY(ls_decode(m, exit_layer, num_draft, max_new));
+    return ls_read_output(m, out_ids, out_n, accepted, out_steps);
+}
+
+int ls_generate_adaptive(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t exit_layer, int32_t max_draft,
+                         float min_margin, int32_t max_new, int32_t* out_ids, int32_t* out_n, int32_t* accepted,
+                         int32_t* drafted, int32_t* out_steps)
+{
+    if (!m || !out_ids || !out_n || !accepted || !drafted || !out_steps) return LS_ERR_INVALID_ARG;
+    if (exit_layer < 1 || exit_layer > m->c.n_layers - 1 || max_draft < 1 || max_new < 1) return LS_ERR_INVALID_ARG;
+    if (!(min_margin > 0.f)) return LS_ERR_INVALID_ARG;
+    if (max_draft > m->c.max_draft) return LS_ERR_CAPACITY;
+    if (n_prompt < 1) return LS_ERR_INVALID_ARG;
+    if ((int64_t)n_prompt + max_new + max_draft + 1 > m->c.max_seq) return LS_ERR_CAPACITY;
+    LS_TRY(ls_prefill(m, prompt, n_prompt, 0));
+    LS_TRY(ls_decode_adaptive(m, exit_layer, max_draft, min_margin, max_new));
+    LS_TRY(ls_read_drafted(m, drafted, nullptr));
     return ls_read_output(m, out_ids, out_n, accepted, out_steps);
 }
 
@@ -975,7 +1055,7 @@ int ls_op_embed(const void* emb, const int32_t* tok, int32_t M, int32_t D, int32
     if (!aligned16(emb) || !tok || !aligned16(x) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8 || V < 1)
         return LS_ERR_INVALID_ARG;
     LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, embed_kernel, dim3(M), dim3(256), 0, (const uint16_t*)emb, tok,
-                 D, V, x, nullptr, nullptr, nullptr, nullptr, 0, 0));
+                 D, V, x, nullptr, nullptr, nullptr, nullptr, 0, 0, 0));
     return LS_OK;
 }
 
@@ -1038,7 +1118,7 @@ int ls_op_lm_head_argmax(int32_t path, const void* w, const void* h, int32_t M, 
     const LaunchCtx lc = {(cudaStream_t)stream, false};
     LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
     LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, n_candidates(path, V, K, M), a.cand_stride, tok,
-                 nullptr));
+                 nullptr, nullptr, 0.f, 0));
     return LS_OK;
 }
 
@@ -1084,7 +1164,7 @@ int ls_op_lm_head_argmax_static(int32_t path, const void* w, const void* h, int3
     const LaunchCtx lc = {(cudaStream_t)stream, false};
     LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
     LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, n_candidates(path, V, K, M), a.cand_stride, tok,
-                 nullptr));
+                 nullptr, nullptr, 0.f, 0));
     return LS_OK;
 }
 
@@ -1189,7 +1269,7 @@ int ls_op_accept(const int32_t* draft, const int32_t* verified, int32_t d, int32
 {
     if (!draft || !verified || !state || !out_ids || !accepted || d < 0 || d >= LS_MAX_ROWS) return LS_ERR_INVALID_ARG;
     LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, accept_kernel, dim3(1), dim3(32), 0, draft, verified, d, state,
-                 out_ids, accepted));
+                 out_ids, accepted, 0, nullptr));
     return LS_OK;
 }
 

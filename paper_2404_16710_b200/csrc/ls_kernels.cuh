@@ -11,12 +11,12 @@
 namespace ls {
 
 // position of row 0 of this pass: the loop's cache length plus a per-launch offset
-__device__ __forceinline__ bool pass_begin(const int32_t* ctl, int pos_off, int& pos0)
+__device__ __forceinline__ bool pass_begin(const int32_t* ctl, int pos_off, int& pos0, int gate = 0)
 {
     pdl_launch_dependents();
     pdl_wait();
     if (ctl) {
-        if (ctl[CTL_DONE]) return false;
+        if (pass_idle(ctl, gate)) return false;
         pos0 = ctl[CTL_CACHE_LEN] + pos_off;
     } else {
         pos0 = pos_off;
@@ -43,12 +43,12 @@ __device__ __forceinline__ float block_sum_256(float v, float* red)
 __global__ void __launch_bounds__(256)
 embed_kernel(const uint16_t* __restrict__ emb, const int32_t* __restrict__ tok, int D, int V,
              float* __restrict__ x, int32_t* ctl, const uint16_t* __restrict__ gain,
-             uint16_t* __restrict__ hout, float* __restrict__ ss_out, int ss_stride, int n_part)
+             uint16_t* __restrict__ hout, float* __restrict__ ss_out, int ss_stride, int n_part, int gate)
 {
     __shared__ float red[8];
     pdl_launch_dependents();
     pdl_wait();
-    if (ctl && ctl[CTL_DONE]) return;
+    if (pass_idle(ctl, gate)) return;
     int m = blockIdx.x;
     int id = tok[m];
     if (id < 0 || id >= V) {
@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(kAttnThreads)
 attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
             const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table,
             int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift,
-            int max_seq, int chunk_cap, float* part, int32_t* counters, uint16_t* __restrict__ out)
+            int max_seq, int chunk_cap, float* part, int32_t* counters, uint16_t* __restrict__ out, int gate)
 {
     constexpr int C = kAttnChunk, T = kAttnThreads;
     constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 16;
@@ -287,7 +287,7 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
     constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
     constexpr int PP = attn_part_pitch(HD);
     int pos0;
-    if (!pass_begin(ctl, pos_off, pos0)) return;
+    if (!pass_begin(ctl, pos_off, pos0, gate)) return;
     const int ch = blockIdx.x, kh = blockIdx.y, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
     const int last_pos = pos0 + M - 1;
@@ -580,54 +580,65 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
 // grid M, block 256: reduce the per-CTA (value, index) candidates of the LM-head kernel.
 // (value desc, index asc) is a total order, so the result does not depend on the
 // reduction tree; the lowest index wins a tie.
+// Adaptive drafting (second != nullptr; the launch is the head of draft pass `gate`, M = 1):
+// the per-CTA second-largest logits are reduced too, and when the margin between the two
+// largest exit logits is below min_margin this draft is not kept and drafting stops:
+// CTL_D_EFF = gate, which idles every later draft pass of the step.
 __global__ void __launch_bounds__(256)
 argmax_finish_kernel(const ValIdx* __restrict__ cand, int n_cand, int cand_stride,
-                     int32_t* __restrict__ tok_out, const int32_t* ctl)
+                     int32_t* __restrict__ tok_out, int32_t* ctl, const float* __restrict__ second,
+                     float min_margin, int gate)
 {
     __shared__ float sv[256];
+    __shared__ float s2[256];
     __shared__ int si[256];
     pdl_launch_dependents();
     pdl_wait();
-    if (ctl && ctl[CTL_DONE]) return;
+    if (pass_idle(ctl, gate)) return;
     int m = blockIdx.x;
     const ValIdx* c = cand + (size_t)m * cand_stride;
-    float bv = -INFINITY;
+    float bv = -INFINITY, bs = -INFINITY;
     int bi = 0x7fffffff;
     for (int k = threadIdx.x; k < n_cand; k += 256) {
         ValIdx e = c[k];
-        if (better(e.v, e.i, bv, bi)) {
-            bv = e.v;
-            bi = e.i;
-        }
+        top2_merge(e.v, e.i, second ? second[(size_t)m * cand_stride + k] : -INFINITY, bv, bi, bs);
     }
     sv[threadIdx.x] = bv;
+    s2[threadIdx.x] = bs;
     si[threadIdx.x] = bi;
     __syncthreads();
     for (int s = 128; s > 0; s >>= 1) {
         if (threadIdx.x < s) {
-            float v = sv[threadIdx.x + s];
-            int i = si[threadIdx.x + s];
-            if (better(v, i, sv[threadIdx.x], si[threadIdx.x])) {
-                sv[threadIdx.x] = v;
-                si[threadIdx.x] = i;
-            }
+            top2_merge(sv[threadIdx.x + s], si[threadIdx.x + s], s2[threadIdx.x + s], bv, bi, bs);
+            sv[threadIdx.x] = bv;
+            s2[threadIdx.x] = bs;
+            si[threadIdx.x] = bi;
         }
         __syncthreads();
     }
-    if (threadIdx.x == 0) tok_out[m] = si[0];
+    if (threadIdx.x == 0) {
+        tok_out[m] = bi;
+        if (second && ctl && m == 0 && bv - bs < min_margin && gate < ctl[CTL_D_EFF]) ctl[CTL_D_EFF] = gate;
+    }
 }
 
 // ------------------------------------------------------------------ accept / rollback
 // match + crop of the paper's loop (Appendix A.4), one thread.  With d == 0 it is the
-// bookkeeping of plain greedy decoding (emit verified[0]).
+// bookkeeping of plain greedy decoding (emit verified[0]).  Adaptive drafting (adaptive != 0):
+// only the drafts the step kept (CTL_D_EFF of them) can be accepted; their number goes to
+// drafted[step] and the stop mark is cleared for the next step.
 __global__ void accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ verified,
                               int d, int32_t* ctl, int32_t* __restrict__ out_ids,
-                              int32_t* __restrict__ accepted)
+                              int32_t* __restrict__ accepted, int adaptive, int32_t* __restrict__ drafted)
 {
     pdl_launch_dependents();
     pdl_wait();
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     if (ctl[CTL_DONE]) return;
+    if (adaptive) {
+        d = min(d, ctl[CTL_D_EFF]);
+        ctl[CTL_D_EFF] = kNoStop;
+    }
     int n = 0;
     while (n < d && draft[n] == verified[n]) ++n;
     int n_out = ctl[CTL_N_OUT];
@@ -640,6 +651,7 @@ __global__ void accept_kernel(const int32_t* __restrict__ draft, const int32_t* 
     }
     int steps = ctl[CTL_N_STEPS];
     accepted[steps] = n;
+    if (drafted) drafted[steps] = d;
     ctl[CTL_N_STEPS] = steps + 1;
     ctl[CTL_N_OUT] = n_out;
     ctl[CTL_CUR_TOK] = verified[n];

@@ -39,7 +39,9 @@ struct LinArgs {
     uint16_t* out_bf16;  // SwiGLU result [M][N]
     ValIdx* cand;        // argmax candidates [M][cand_stride], one per CTA
     int cand_stride;
+    float* second;       // optional [M][cand_stride]: the CTA's second-largest logit (adaptive drafting)
     int32_t* ctl;
+    int gate;            // > 0: the launch belongs to draft pass `gate` and idles once drafting has stopped
     // EPI_QKV: rotary embedding + KV append fused behind the q|k|v projection
     const float* inv_freq;       // [hd/2], or nullptr: theta^(-2j/hd) computed in place
     const int32_t* page_table;
@@ -126,7 +128,7 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
 {
     pdl_launch_dependents();
     pdl_wait();
-    if (a.ctl && a.ctl[CTL_DONE]) return;
+    if (pass_idle(a.ctl, a.gate)) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint16_t* rp[4];
     int nrow[4];  // output index of each of the warp's rows
@@ -262,39 +264,35 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
             }
     } else {  // EPI_ARGMAX
         __shared__ float bv[4][MT];
+        __shared__ float bs[4][MT];
         __shared__ int bi[4][MT];
 #pragma unroll
         for (int m = 0; m < MT; ++m)
             if (lane == m) {
-                float v = -INFINITY;
+                float v = -INFINITY, s2 = -INFINITY;
                 int idx = 0x7fffffff;
 #pragma unroll
                 for (int r = 0; r < 4; ++r)
                     if (nrow[r] < a.N) {
                         if (a.out && m < a.M) a.out[(size_t)m * a.ldo + nrow[r]] = acc[r][m];
-                        if (better(acc[r][m], nrow[r], v, idx)) {
-                            v = acc[r][m];
-                            idx = nrow[r];
-                        }
+                        top2_push(acc[r][m], nrow[r], v, idx, s2);
                     }
                 bv[warp][m] = v;
+                bs[warp][m] = s2;
                 bi[warp][m] = idx;
             }
         __syncthreads();
         if (threadIdx.x < MT && threadIdx.x < a.M) {
             int m = threadIdx.x;
-            float v = bv[0][m];
+            float v = bv[0][m], s2 = bs[0][m];
             int idx = bi[0][m];
 #pragma unroll
-            for (int w = 1; w < 4; ++w)
-                if (better(bv[w][m], bi[w][m], v, idx)) {
-                    v = bv[w][m];
-                    idx = bi[w][m];
-                }
+            for (int w = 1; w < 4; ++w) top2_merge(bv[w][m], bi[w][m], bs[w][m], v, idx, s2);
             ValIdx e;
             e.v = v;
             e.i = idx;
             a.cand[(size_t)m * a.cand_stride + blockIdx.x] = e;
+            if (a.second) a.second[(size_t)m * a.cand_stride + blockIdx.x] = s2;
         }
     }
 }
@@ -385,14 +383,24 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
 #pragma unroll
             for (int i = 0; i < 4; ++i) c[tr][nt][i] = 0.f;
 
-    // the first STAGES-1 steps of weights are on their way while the predecessor finishes
+    // the first STAGES-1 steps of weights are on their way while the predecessor finishes --
+    // unless this is a draft pass and the step's stop mark, read past L1, already says that
+    // drafting ended before it (the binding decision is the one after the wait)
+    bool early = true;
+    if (a.gate > 0 && a.ctl) early = a.gate <= __ldcg(a.ctl + CTL_D_EFF);
+    if (early) {
 #pragma unroll
-    for (int p = 0; p < STAGES - 1; ++p) issue_w(warp + p * WARPS, p);
+        for (int p = 0; p < STAGES - 1; ++p) issue_w(warp + p * WARPS, p);
+    }
     pdl_wait();
-    if (a.ctl && a.ctl[CTL_DONE]) {
+    if (pass_idle(a.ctl, a.gate)) {
         cp_async_commit();
         cp_async_wait<0>();
         return;
+    }
+    if (!early) {
+#pragma unroll
+        for (int p = 0; p < STAGES - 1; ++p) issue_w(warp + p * WARPS, p);
     }
 #pragma unroll
     for (int p = 0; p < STAGES - 1; ++p) {
@@ -547,7 +555,7 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
         __syncthreads();
         if (threadIdx.x < a.M) {
             const int m = threadIdx.x;
-            float v = -INFINITY;
+            float v = -INFINITY, s2 = -INFINITY;
             int idx = 0x7fffffff;
 #pragma unroll
             for (int rr = 0; rr < 16 * TR; ++rr) {
@@ -555,16 +563,14 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
                 if (n < a.N) {
                     float x = vals[rr][m];
                     if (a.out) a.out[(size_t)m * a.ldo + n] = x;
-                    if (better(x, n, v, idx)) {
-                        v = x;
-                        idx = n;
-                    }
+                    top2_push(x, n, v, idx, s2);
                 }
             }
             ValIdx e;
             e.v = v;
             e.i = idx;
             a.cand[(size_t)m * a.cand_stride + blockIdx.x] = e;
+            if (a.second) a.second[(size_t)m * a.cand_stride + blockIdx.x] = s2;
         }
     }
 }

@@ -177,6 +177,81 @@ def test_without_exit_cache_reuse_same_ids_more_bytes():
         B.ls_decode_flags(gm.h, 2, 3, 40, 8)
 
 
+# ------------------------------------------------------------------ adaptive draft length
+@pytest.mark.parametrize("path", PATHS)
+def test_adaptive_equals_generate_full_for_every_threshold(path):
+    gm, _ = make_pair(TINY.shape, TINY.weight_seed, TINY.exit_layer, TINY.late_scale, 160, max_draft=15,
+                      linear_path=path, oracle=False)
+    prompt = synth.make_prompt(TINY.shape.vocab, TINY.n_prompt, TINY.prompt_seed)
+    full = gm.generate_full(prompt, TINY.max_new)
+    seen = set()
+    for E in (1, 2, 3):
+        for d in (1, 3, 6, 15):
+            for tau in (0.004, 0.02, 0.05, 0.3):
+                ids, acc, drafted = gm.generate_adaptive(prompt, E, d, tau, TINY.max_new)
+                np.testing.assert_array_equal(ids, full, err_msg=f"E={E} d={d} tau={tau}")
+                assert ((0 <= acc) & (acc <= drafted) & (drafted <= d)).all()
+                emitted = np.cumsum(acc + 1)
+                assert emitted[-1] >= TINY.max_new and (len(emitted) == 1 or emitted[-2] < TINY.max_new)
+                st = gm.stats()
+                assert st.n_steps == len(acc) and st.n_accepted == acc.sum() and st.host_syncs <= 10
+                seen.update(drafted.tolist())
+    assert {0, 1, 2, 3, 6, 15} <= seen  # stops at once, in the middle, and never
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_adaptive_limits_are_the_fixed_loop_and_one_token_per_step(path):
+    E, d = TINY.exit_layer, 5
+    gm, _ = make_pair(TINY.shape, TINY.weight_seed, E, TINY.late_scale, 128, linear_path=path, oracle=False)
+    prompt = synth.make_prompt(TINY.shape.vocab, TINY.n_prompt, TINY.prompt_seed)
+    ids0, acc0 = gm.generate(prompt, E, d, 40)
+    w0 = gm.stats().weight_bytes
+    ids, acc, drafted = gm.generate_adaptive(prompt, E, d, 1e-30, 40)  # no margin is below it
+    np.testing.assert_array_equal(ids, ids0)
+    np.testing.assert_array_equal(acc, acc0)
+    assert (drafted == d).all() and gm.stats().weight_bytes == w0
+    ids, acc, drafted = gm.generate_adaptive(prompt, E, d, float("inf"), 40)  # every margin is below it
+    np.testing.assert_array_equal(ids, ids0)
+    assert len(acc) == 40 and (acc == 0).all() and (drafted == 0).all()
+    # one early pass + its head + the verify of one row per step: the bytes of plain greedy
+    s = TINY.shape
+    assert gm.stats().weight_bytes == 40 * (s.n_layers * s.layer_weight_bytes + 2 * s.lm_head_bytes)
+    np.testing.assert_array_equal(B.ls_read_drafted(gm.h, 40), drafted)
+    for bad in (0.0, -1.0, float("nan")):
+        with pytest.raises(B.LsError) as e:
+            gm.generate_adaptive(prompt, E, d, bad, 40)
+        assert e.value.status == B.LS_ERR_INVALID_ARG
+    gm.generate(prompt, E, d, 40)
+    assert (B.ls_read_drafted(gm.h, 40) == d).all()  # the fixed loop keeps d drafts every step
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("tau", [0.02, 0.05])
+def test_adaptive_steps_match_oracle_while_decisions_are_clear(path, tau):
+    """ids as far as the oracle's top-1/top-2 margins allow; kept-draft and accepted counts for
+    every step before the first one in which an exit-logit margin came within the logit
+    tolerance of the threshold (there the fp32 path may decide differently, and every later
+    step starts somewhere else)."""
+    E, d, new = TINY.exit_layer, 4, TINY.max_new
+    gm, om = make_pair(TINY.shape, TINY.weight_seed, E, TINY.late_scale, 128, linear_path=path)
+    prompt = synth.make_prompt(TINY.shape.vocab, TINY.n_prompt, TINY.prompt_seed)
+    ref_ids, ref_acc, ref_dr, gap = om.generate_adaptive(prompt, E, d, tau, new)
+    ids, acc, drafted = gm.generate_adaptive(prompt, E, d, tau, new)
+    _, margins, maxabs = om.generate_full(prompt, new)
+    k = first_low_margin(margins, maxabs)
+    np.testing.assert_array_equal(ids[:k], ref_ids[:k])
+    ex, _ = om.teacher_logits(np.concatenate([prompt, ref_ids]), E)
+    tol = 2 * LOGIT_TOL * np.abs(ex).max()  # a margin is the difference of two logits
+    emitted = np.cumsum(ref_acc + 1)
+    unclear = np.nonzero((gap <= tol) | (emitted > k))[0]
+    safe = int(unclear[0]) if unclear.size else len(ref_acc)
+    np.testing.assert_array_equal(drafted[:safe], ref_dr[:safe])
+    np.testing.assert_array_equal(acc[:safe], ref_acc[:safe])
+    print(f"path {path} tau {tau}: {safe} of {len(ref_acc)} steps compared; kept/step gpu {drafted.mean():.2f} "
+          f"oracle {ref_dr.mean():.2f}")
+    assert safe >= 1
+
+
 def test_boundary_error_codes():
     gm, _ = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 64, max_draft=4, oracle=False)
     p = synth.make_prompt(TINY.shape.vocab, 8, 0)

@@ -8,7 +8,10 @@
 * losslessness (Sec. 4.3 of the paper: verification keeps exactly the full model's
   tokens): self-speculative ids == full greedy ids for EVERY (E, d);
 * zero late-layer scale: x_L = x_E, so every draft is accepted (n == d each step);
-* bookkeeping invariants of the loop in Appendix A.4.
+* bookkeeping invariants of the loop in Appendix A.4;
+* the adaptive-draft-length extension: same ids as full greedy for every threshold, the two
+  limits (threshold -> 0: the fixed-length loop; +inf: one token per step), and every step's
+  kept-draft and accepted counts re-derived from no-cache exit logits.
 """
 from dataclasses import replace
 
@@ -149,6 +152,72 @@ def test_eos_stops_both_loops_at_the_same_token():
     s2, _, _ = m2.generate_spec(prompt, 2, 3, 24)
     np.testing.assert_array_equal(f2, full[:first + 1])
     np.testing.assert_array_equal(s2, f2)
+
+
+# ---------------------------------------------------------------- adaptive draft length
+def tiny_model(E, late_scale=None, max_seq=96):
+    wl = synth.WORKLOADS["tiny"]
+    m, cfg, w = oracle_model(wl.shape, wl.weight_seed, E, wl.late_scale if late_scale is None else late_scale,
+                             max_seq=max_seq)
+    return m, cfg, w, synth.make_prompt(wl.shape.vocab, 12, wl.prompt_seed)
+
+
+@pytest.mark.parametrize("E,d", [(1, 3), (2, 4), (3, 2)])
+@pytest.mark.parametrize("tau", [0.004, 0.02, 0.05, 0.3])
+def test_adaptive_is_lossless_for_every_threshold(E, d, tau):
+    m, _, _, prompt = tiny_model(E)
+    full, _, _ = m.generate_full(prompt, 24)
+    ids, acc, drafted, _ = m.generate_adaptive(prompt, E, d, tau, 24)
+    np.testing.assert_array_equal(ids, full)
+    assert ((0 <= acc) & (acc <= drafted) & (drafted <= d)).all()
+    emitted = np.cumsum(acc + 1)
+    assert emitted[-1] >= 24 and (len(emitted) == 1 or emitted[-2] < 24)
+
+
+def test_adaptive_limits_are_the_fixed_loop_and_one_token_per_step():
+    E, d = 2, 4
+    m, _, _, prompt = tiny_model(E)
+    ids0, acc0, _ = m.generate_spec(prompt, E, d, 24)
+    ids, acc, drafted, gap = m.generate_adaptive(prompt, E, d, 1e-300, 24)  # no margin is below it
+    np.testing.assert_array_equal(ids, ids0)
+    np.testing.assert_array_equal(acc, acc0)
+    assert (drafted == d).all() and gap.min() > 0
+    ids, acc, drafted, _ = m.generate_adaptive(prompt, E, d, np.inf, 24)  # every margin is below it
+    np.testing.assert_array_equal(ids, ids0)
+    assert len(acc) == 24 and (acc == 0).all() and (drafted == 0).all()
+    with pytest.raises(ValueError):
+        m.generate_adaptive(prompt, E, d, 0.0, 24)
+
+
+@pytest.mark.parametrize("tau", [0.02, 0.05])
+def test_adaptive_steps_rederived_from_no_cache_exit_logits(tau):
+    """Each step's kept-draft count k and accepted count n, recomputed without any cache:
+    the exit logits of the growing sequence (full [T, T] attention) give the margins and the
+    drafts; n is the agreement of those drafts with the full model's greedy continuation."""
+    E, d, new = 2, 4, 18
+    m, cfg, w, prompt = tiny_model(E)
+    ids, acc, drafted, _ = m.generate_adaptive(prompt, E, d, tau, new)
+    full = B.greedy(cfg, w, prompt, new + d + 1)
+    np.testing.assert_array_equal(ids, full[:new])
+    emitted = 0
+    for k_ref, n_ref in zip(drafted, acc):
+        seq = list(prompt) + list(full[:emitted])
+        drafts = []
+        k = d
+        for j in range(d):
+            z = B.logits_at(cfg, w, np.array(seq + drafts, dtype=np.int32), E)[-1]
+            top = np.sort(z)[-2:]
+            if top[1] - top[0] < tau:
+                k = j
+                break
+            drafts.append(int(z.argmax()))
+        n = 0
+        while n < k and drafts[n] == full[emitted + n]:
+            n += 1
+        assert (k, n) == (k_ref, n_ref)
+        emitted += n + 1
+    assert emitted >= new
+    assert 0 < drafted.mean() < d  # the threshold bites, and not always at once
 
 
 def test_argument_errors():
