@@ -40,7 +40,7 @@ UNIT = "tokens/s"
 # profiles/linear_mma_kernel_llama2-7b_shapes.md summarises; keyed by (workload, rows).  Set an
 # entry to None when the kernel changes until the counters have been taken again.
 # thresholds on the exit-logit margin tried by the adaptive-draft-length leg (logit units)
-ADAPTIVE_MARGINS = (0.01, 0.02, 0.04, 0.08)
+ADAPTIVE_MARGINS = (0.02, 0.05, 0.1, 0.2, 0.4)
 ROOFLINE_TRAFFIC = {("llama2-7b", 7): 180.43e6 + 3.8e6}
 
 
