@@ -22,7 +22,7 @@ enum Ctl : int {
 };
 constexpr int kNoStop = 0x7fffffff;  // CTL_D_EFF while no draft pass has stopped the drafting
 
-enum DevStatus : int { DEV_OK = 0, DEV_BAD_TOKEN = 1, DEV_POS_OVERFLOW = 2, DEV_BARRIER_TIMEOUT = 4 };  // 3: a bounded wait of the prompt-pass GEMM
+enum DevStatus : int { DEV_OK = 0, DEV_BAD_TOKEN = 1, DEV_POS_OVERFLOW = 2 };
 
 constexpr int kMaxRows = 16;    // rows per pass
 constexpr int kAttnChunk = 64;  // keys per attention chunk (absolute positions)

@@ -23,7 +23,6 @@
 
 #include "ls.h"
 #include "ls_linear.cuh"
-#include "ls_pass.cuh"
 #include "ls_prefill.cuh"
 
 using namespace ls;
@@ -114,13 +113,6 @@ struct ls_model {
     cudaEvent_t ev0, ev1;
     ls_stats stats;
     std::vector<int32_t> h_out, h_acc, h_drafted;
-    // one resident kernel per pass (ls_pass.cuh)
-    bool use_pass;
-    PassModel pmodel;
-    PassLayer* lwdev;
-    unsigned* bar;
-    int pass_grid[2];      // CTAs of the cooperative launch for one / two token tiles
-    size_t pass_smem[2];
     int h_n_out, h_n_steps;
 };
 
@@ -161,8 +153,6 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     unsigned char* cand = take(sizeof(ValIdx) * kMaxRows * cand_stride);
     unsigned char* second = take(sizeof(float) * kMaxRows * cand_stride);
     unsigned char* drafted = take(sizeof(int32_t) * c.max_seq);
-    unsigned char* lwdev = take(sizeof(PassLayer) * c.n_layers);
-    unsigned char* bar = take(256);
     const int n_part = (c.d_model + 15) / 16;  // CTAs of a residual projection = partial sums per row
     unsigned char* ss = take(sizeof(float) * kMaxRows * n_part);
     unsigned char* he = take(2 * (size_t)kMaxRows * c.d_model);
@@ -206,8 +196,6 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
         m->cand = (ValIdx*)cand;
         m->second = (float*)second;
         m->drafted = (int32_t*)drafted;
-        m->lwdev = (PassLayer*)lwdev;
-        m->bar = (unsigned*)bar;
         m->n_pages = n_pages;
         m->chunk_cap = chunk_cap;
         m->cand_stride = cand_stride;
@@ -510,165 +498,12 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
 }
 
 // one step of the loop.  E == L with d == 0: plain greedy; E < L with d == 0: early exit.
-// ------------------------------------------------------------------ one resident kernel per pass
-template <int NT, int HD>
-int pass_setup_one(ls_model* m, int sms)
-{
-    const size_t sm = pass_smem_bytes<HD>(NT, m->c.n_heads / m->c.n_kv_heads);
-    LS_CK(cudaFuncSetAttribute(pass_kernel<NT, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
-    int per_sm = 0;
-    LS_CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pass_kernel<NT, HD>, kPassThreads, sm));
-    if (per_sm < 1) return LS_ERR_UNSUPPORTED;
-    m->pass_smem[NT - 1] = sm;
-    m->pass_grid[NT - 1] = per_sm * sms;
-    if (getenv("LS_DEBUG"))
-        fprintf(stderr, "ls: resident pass kernel, %d token tile(s): %d CTAs per SM x %d SMs, %zu bytes shared\n", NT,
-                per_sm, sms, sm);
-    return LS_OK;
-}
-
-int pass_setup(ls_model* m, int sms)
-{
-    const ls_config& c = m->c;
-    std::vector<PassLayer> lw(c.n_layers);
-    for (int l = 0; l < c.n_layers; ++l) {
-        const LayerW& w = m->lw[l];
-        lw[l] = PassLayer{w.attn_norm, w.wq, w.wk, w.wv, w.wo, w.ffn_norm, w.wg, w.wu, w.wd};
-    }
-    LS_CK(cudaMemcpyAsync(m->lwdev, lw.data(), sizeof(PassLayer) * lw.size(), cudaMemcpyHostToDevice, m->st));
-    LS_CK(cudaStreamSynchronize(m->st));  // lw is a local
-    PassModel& p = m->pmodel;
-    memset(&p, 0, sizeof(p));
-    p.layers = m->lwdev;
-    p.emb = m->emb;
-    p.fnorm = m->fnorm;
-    p.lm = m->lm;
-    p.D = c.d_model;
-    p.Hq = c.n_heads;
-    p.Hkv = c.n_kv_heads;
-    p.hd = c.head_dim;
-    p.F = c.d_ffn;
-    p.V = c.vocab;
-    p.page_shift = m->page_shift;
-    p.max_seq = c.max_seq;
-    p.n_part = m->n_part;
-    p.chunk_cap = m->chunk_cap;
-    p.cand_stride = m->cand_stride;
-    p.eps = c.rms_eps;
-    p.theta = c.rope_theta;
-    p.inv_freq = m->inv_freq;
-    p.page_table = m->page_table;
-    p.kpages = m->kpages;
-    p.vpages = m->vpages;
-    p.layer_kv_elems = m->layer_kv_elems;
-    p.x = m->x;
-    p.ss = m->ss;
-    p.part = m->part;
-    p.h = m->h;
-    p.hE = m->hE;
-    p.q = m->q;
-    p.o = m->o;
-    p.a = m->a;
-    p.attn_counters = m->attn_counters;
-    p.ctl = m->ctl;
-    p.draft = m->draft;
-    p.verified = m->verified;
-    p.out_ids = m->out_ids;
-    p.accepted = m->accepted;
-    p.drafted = m->drafted;
-    p.cand = m->cand;
-    p.second = m->second;
-    p.bar = m->bar;
-    if (c.head_dim == 128) {
-        LS_TRY((pass_setup_one<1, 128>(m, sms)));
-        LS_TRY((pass_setup_one<2, 128>(m, sms)));
-    } else {
-        LS_TRY((pass_setup_one<1, 64>(m, sms)));
-        LS_TRY((pass_setup_one<2, 64>(m, sms)));
-    }
-    return LS_OK;
-}
-
-// a pass as one cooperative launch: every CTA is resident, so the grid barriers complete
-int run_pass(ls_model* m, const PassArgs& pa)
-{
-    const int nt = pa.M <= 8 ? 1 : 2;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(m->pass_grid[nt - 1]);
-    cfg.blockDim = dim3(kPassThreads);
-    cfg.dynamicSmemBytes = m->pass_smem[nt - 1];
-    cfg.stream = m->st;
-    cudaLaunchAttribute at;
-    at.id = cudaLaunchAttributeCooperative;
-    at.val.cooperative = 1;
-    cfg.attrs = &at;
-    cfg.numAttrs = 1;
-    if (m->c.head_dim == 128) {
-        if (nt == 1) LS_CK(cudaLaunchKernelEx(&cfg, pass_kernel<1, 128>, m->pmodel, pa));
-        else LS_CK(cudaLaunchKernelEx(&cfg, pass_kernel<2, 128>, m->pmodel, pa));
-    } else {
-        if (nt == 1) LS_CK(cudaLaunchKernelEx(&cfg, pass_kernel<1, 64>, m->pmodel, pa));
-        else LS_CK(cudaLaunchKernelEx(&cfg, pass_kernel<2, 64>, m->pmodel, pa));
-    }
-    m->launches += 1;
-    return LS_OK;
-}
-
-PassArgs pass_args(int l0, int l1, int M, int slot, int pos_off)
-{
-    PassArgs pa;
-    memset(&pa, 0, sizeof(pa));
-    pa.l0 = l0;
-    pa.l1 = l1;
-    pa.M = M;
-    pa.slot = slot;
-    pa.pos_off = pos_off;
-    pa.accept_d = -1;
-    return pa;
-}
-
-// the step of enqueue_step as d + 2 resident kernels (same schedule, same buffers)
-int enqueue_step_pass(ls_model* m, int E, int d, float min_margin)
-{
-    const int L = m->c.n_layers;
-    const bool adaptive = min_margin > 0.f;
-    if (d == 0) {
-        PassArgs pa = pass_args(0, E, 1, 0, 0);
-        pa.tok = m->ctl + CTL_CUR_TOK;
-        pa.gain_end_a = m->fnorm;
-        pa.head = 1;
-        pa.tok_out = m->verified;
-        pa.accept_d = 0;
-        return run_pass(m, pa);
-    }
-    for (int j = 0; j <= d; ++j) {
-        PassArgs pa = pass_args(0, E, 1, j, j);
-        pa.gate = adaptive ? j : 0;
-        pa.tok = j == 0 ? m->ctl + CTL_CUR_TOK : m->draft + (j - 1);
-        pa.gain_end_a = j < d ? m->fnorm : nullptr;
-        pa.gain_end_b = m->lw[E].attn_norm;
-        pa.head = j < d ? 1 : 0;
-        pa.tok_out = m->draft + j;
-        pa.min_margin = min_margin;
-        LS_TRY(run_pass(m, pa));
-    }
-    PassArgs pa = pass_args(E, L, d + 1, 0, 0);
-    pa.h_first = m->hE;
-    pa.gain_end_a = m->fnorm;
-    pa.head = 1;
-    pa.tok_out = m->verified;
-    pa.accept_d = d;
-    pa.adaptive = adaptive ? 1 : 0;
-    return run_pass(m, pa);
-}
-
 // min_margin > 0: adaptive drafting.  Draft pass j (j >= 1) is enqueued with gate j, so it idles
 // once an earlier pass's head has found its two largest exit logits closer than min_margin;
 // the verify pass always runs on d + 1 rows (the rows beyond the kept drafts are stale and
 // never read by the rows that count: causal attention, one dot product per output element).
 int enqueue_step(ls_model* m, int E, int d, bool reuse, float min_margin = 0.f)
 {
-    if (m->use_pass && reuse) return enqueue_step_pass(m, E, d, min_margin);
     const int D = m->c.d_model, L = m->c.n_layers;
     const bool adaptive = min_margin > 0.f;
     if (d == 0) {
@@ -899,12 +734,6 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
     }
     int rc = attn_allow_smem(cfg->head_dim, cfg->n_heads / cfg->n_kv_heads);
     if (rc != LS_OK) return fail(rc);
-    // the decode loop runs each pass as one resident kernel (tensor-core path only)
-    m->use_pass = m->path == LS_LINEAR_MMA && getenv("LS_PASS") != nullptr;
-    if (m->use_pass) {
-        rc = pass_setup(m, prop.multiProcessorCount);
-        if (rc != LS_OK) return fail(rc);
-    }
     *out = m;
     return LS_OK;
 }
@@ -1191,36 +1020,6 @@ int ls_debug_logits(ls_model* m, const int32_t* ids, int32_t n, int32_t exit_lay
     LS_TRY(write_ctl(m, 0, 0, 0));
     for (int r0 = 0; r0 < n; r0 += kMaxRows) {
         int M = n - r0 < kMaxRows ? n - r0 : kMaxRows;
-        if (m->use_pass) {  // the same resident kernels the decode loop runs
-            PassArgs pa = pass_args(0, exit_layer, M, 0, r0);
-            pa.tok = m->ids + r0;
-            pa.gain_end_a = m->fnorm;
-            pa.gain_end_b = exit_layer < L ? m->lw[exit_layer].attn_norm : nullptr;
-            pa.head = exit_logits ? 1 : 0;
-            pa.tok_out = m->verified;
-            pa.logits = m->logits;
-            LS_TRY(run_pass(m, pa));
-            if (exit_logits) {
-                LS_CK(cudaMemcpyAsync(exit_logits + (size_t)r0 * V, m->logits, sizeof(float) * (size_t)M * V,
-                                      cudaMemcpyDeviceToHost, m->st));
-                LS_CK(cudaStreamSynchronize(m->st));
-            }
-            if (exit_layer < L || final_logits) {
-                pa = pass_args(exit_layer, L, M, 0, r0);
-                pa.h_first = m->hE;
-                pa.gain_end_a = m->fnorm;
-                pa.head = final_logits ? 1 : 0;
-                pa.tok_out = m->verified;
-                pa.logits = m->logits;
-                LS_TRY(run_pass(m, pa));
-            }
-            if (final_logits) {
-                LS_CK(cudaMemcpyAsync(final_logits + (size_t)r0 * V, m->logits, sizeof(float) * (size_t)M * V,
-                                      cudaMemcpyDeviceToHost, m->st));
-                LS_CK(cudaStreamSynchronize(m->st));
-            }
-            continue;
-        }
         LS_TRY(run_embed(m, m->ids + r0, M, m->x, 0));
         LS_TRY(run_layers(m, 0, exit_layer, M, m->x, r0, 0, m->h, m->fnorm,
                           exit_layer < L ? m->lw[exit_layer].attn_norm : nullptr));

@@ -274,32 +274,34 @@ __device__ __forceinline__ void attn_pv(const unsigned char* Vs, const float* P,
         }
 }
 
-// One work item of the attention step: chunk `ch` (64 keys) of KV head `kh` for the M rows at
-// positions pos0 .. pos0 + M - 1.  Called by every thread of a 256-thread CTA with the same
-// arguments; n_active = chunks that hold visible keys (the caller has checked the bounds and
-// that ch is one of them).  Whoever finishes a KV head's last chunk merges the head.
-// Everything another CTA may have written (q, the partials) is read past L1, so the function
-// also serves a kernel that stays resident across the steps of a pass.
 template <int HD>
-__device__ __forceinline__ void attn_item(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
-                                          const uint16_t* __restrict__ vpages,
-                                          const int32_t* __restrict__ page_table, int pos0, int M, int Hq, int Hkv,
-                                          int page_shift, int chunk_cap, float* part, int32_t* counters,
-                                          uint16_t* __restrict__ out, int ch, int kh, int n_active,
-                                          unsigned char* smem)
+__global__ void __launch_bounds__(kAttnThreads)
+attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
+            const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table,
+            int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift,
+            int max_seq, int chunk_cap, float* part, int32_t* counters, uint16_t* __restrict__ out, int gate)
 {
     constexpr int C = kAttnChunk, T = kAttnThreads;
     constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 16;
     constexpr int SP = kAttnSP, PBROW = kAttnSP * 2;
     constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
     constexpr int PP = attn_part_pitch(HD);
-    const int tid = threadIdx.x;
+    int pos0;
+    if (!pass_begin(ctl, pos_off, pos0, gate)) return;
+    const int ch = blockIdx.x, kh = blockIdx.y, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
     const int last_pos = pos0 + M - 1;
     const int key0 = ch * C;
+    if (key0 > last_pos) return;
+    const int n_active = last_pos / C + 1;  // CTAs of this KV head that take part
+    if (last_pos >= max_seq || pos0 < 0 || n_active > chunk_cap || n_active > (int)gridDim.x) {
+        if (ctl && tid == 0) ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
+        return;
+    }
     const int G = Hq / Hkv, Q = G * M;  // query qi = m * G + g
     const int Qpad = (Q + 15) & ~15;
 
+    extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* Ks = smem;
     unsigned char* Vs = Ks + C * KROW;
     unsigned char* Qb = Vs + C * VROW;
@@ -319,7 +321,7 @@ __device__ __forceinline__ void attn_item(const uint16_t* __restrict__ q, const 
             const int qi = idx / SEGS, sg = idx % SEGS;
             if (qi < Q) {
                 const int m = qi / G, g = qi % G;
-                qreg[i] = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + sg * 8));
+                qreg[i] = *reinterpret_cast<const uint4*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + sg * 8);
             }
         }
     }
@@ -353,7 +355,7 @@ __device__ __forceinline__ void attn_item(const uint16_t* __restrict__ q, const 
         uint4 v = make_uint4(0, 0, 0, 0);
         if (qi < Q) {
             const int m = qi / G, g = qi % G;
-            v = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + sg * 8));
+            v = *reinterpret_cast<const uint4*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + sg * 8);
         }
         *reinterpret_cast<uint4*>(Qb + qi * KROW + sg * 16) = v;
     }
@@ -572,28 +574,6 @@ __device__ __forceinline__ void attn_item(const uint16_t* __restrict__ q, const 
             }
         }
     }
-}
-
-// grid (chunks, KV heads), block 256: one work item per CTA
-template <int HD>
-__global__ void __launch_bounds__(kAttnThreads)
-attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
-            const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table,
-            int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift,
-            int max_seq, int chunk_cap, float* part, int32_t* counters, uint16_t* __restrict__ out, int gate)
-{
-    extern __shared__ __align__(16) unsigned char smem[];
-    int pos0;
-    if (!pass_begin(ctl, pos_off, pos0, gate)) return;
-    const int last_pos = pos0 + M - 1;
-    if ((int)blockIdx.x * kAttnChunk > last_pos) return;
-    const int n_active = last_pos / kAttnChunk + 1;  // CTAs of this KV head that take part
-    if (last_pos >= max_seq || pos0 < 0 || n_active > chunk_cap || n_active > (int)gridDim.x) {
-        if (ctl && threadIdx.x == 0) ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
-        return;
-    }
-    attn_item<HD>(q, kpages, vpages, page_table, pos0, M, Hq, Hkv, page_shift, chunk_cap, part, counters, out,
-                  (int)blockIdx.x, (int)blockIdx.y, n_active, smem);
 }
 
 // ------------------------------------------------------------------ argmax finish
