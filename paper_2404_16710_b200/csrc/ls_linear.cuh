@@ -347,6 +347,10 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
     const uint16_t* hb[NT];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) hb[nt] = a.h + (size_t)min(nt * 8 + g, a.M - 1) * a.K;
+    // lanes whose token row does not exist copy nothing (zero fill) instead of re-reading row M-1
+    bool hrow[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) hrow[nt] = nt * 8 + g < a.M;
 
     // region r (2 tr: row g, 2 tr + 1: row g+8, 2 TR + nt: tokens), stage s, thread tid -> 16 bytes
     const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(ring) + (uint32_t)tid * 16u;
@@ -371,7 +375,7 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             const int nb = (k < a.K) ? 16 : 0;
             const int kk = (k < a.K) ? k : 0;
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) cp_async16_ca(slot(2 * TR + nt, s), hb[nt] + kk, nb);
+            for (int nt = 0; nt < NT; ++nt) cp_async16_ca(slot(2 * TR + nt, s), hb[nt] + kk, hrow[nt] ? nb : 0);
         }
     };
 
