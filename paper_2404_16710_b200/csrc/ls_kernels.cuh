@@ -286,24 +286,60 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
     constexpr int SP = kAttnSP, PBROW = kAttnSP * 2;
     constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
     constexpr int PP = attn_part_pitch(HD);
-    int pos0;
-    if (!pass_begin(ctl, pos_off, pos0, gate)) return;
-    const int ch = blockIdx.x, kh = blockIdx.y, tid = threadIdx.x;
-    const int warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
-    const int last_pos = pos0 + M - 1;
-    const int key0 = ch * C;
-    if (key0 > last_pos) return;
-    const int n_active = last_pos / C + 1;  // CTAs of this KV head that take part
-    if (last_pos >= max_seq || pos0 < 0 || n_active > chunk_cap || n_active > (int)gridDim.x) {
-        if (ctl && tid == 0) ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
-        return;
-    }
-    const int G = Hq / Hkv, Q = G * M;  // query qi = m * G + g
-    const int Qpad = (Q + 15) & ~15;
-
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* Ks = smem;
     unsigned char* Vs = Ks + C * KROW;
+    const int ch = blockIdx.x, kh = blockIdx.y, tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
+    const int key0 = ch * C;
+    const uint32_t ks0 = (uint32_t)__cvta_generic_to_shared(Ks), vs0 = (uint32_t)__cvta_generic_to_shared(Vs);
+    const bool one_page = page_shift >= 6;
+
+    // Cache rows below the loop's cache length do not change while the loop runs, so their
+    // copies start before the producer of q (and of this pass's own k, v rows) has finished.
+    // The length is read past L1 and may be an older, smaller one: then fewer rows go early.
+    pdl_launch_dependents();
+    int c_early = 0;
+    if (ctl && !(gate > 0 && gate > __ldcg(ctl + CTL_D_EFF))) c_early = min(__ldcg(ctl + CTL_CACHE_LEN), max_seq);
+    size_t base = 0;
+    auto stage_rows = [&](int p_lo, int p_hi, int p_fill) {
+        // rows p of the chunk with p_lo <= p <= p_hi are copied; rows p_hi < p <= p_fill are zeroed
+#pragma unroll
+        for (int it = 0; it < C * SEGS / T; ++it) {
+            const int idx = tid + it * T;
+            const int r = idx / SEGS, sg = idx % SEGS;
+            const int p = key0 + r;
+            if (p < p_lo || p > p_fill) continue;
+            const bool ok = p <= p_hi;
+            const size_t off = (one_page ? base + (size_t)r * HD
+                                         : kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD)) +
+                               (size_t)sg * 8;
+            cp_async16_cg(ks0 + r * KROW + sg * 16, kpages + off, ok ? 16 : 0);
+            cp_async16_cg(vs0 + r * VROW + sg * 16, vpages + off, ok ? 16 : 0);
+        }
+    };
+    if (key0 < c_early) {
+        if (one_page) base = kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD);
+        stage_rows(0, c_early - 1, c_early - 1);
+    }
+    pdl_wait();
+    auto leave = [&]() {  // nothing in flight may outlive the CTA's shared memory
+        cp_async_commit();
+        cp_async_wait<0>();
+    };
+    if (pass_idle(ctl, gate)) return leave();
+    const int pos0 = (ctl ? ctl[CTL_CACHE_LEN] : 0) + pos_off;
+    const int last_pos = pos0 + M - 1;
+    if (key0 > last_pos) return leave();
+    const int n_active = last_pos / C + 1;  // CTAs of this KV head that take part
+    if (last_pos >= max_seq || pos0 < 0 || n_active > chunk_cap || n_active > (int)gridDim.x) {
+        if (ctl && tid == 0) ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
+        return leave();
+    }
+    if (c_early > pos0) c_early = pos0;  // (cannot happen: the length only grows; rows >= pos0 are this pass's)
+    const int G = Hq / Hkv, Q = G * M;  // query qi = m * G + g
+    const int Qpad = (Q + 15) & ~15;
+
     unsigned char* Qb = Vs + C * VROW;
     float* S = reinterpret_cast<float*>(Qb + (size_t)Qpad * KROW);
     unsigned char* Pb = reinterpret_cast<unsigned char*>(S + (size_t)Qpad * SP);
@@ -325,26 +361,12 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
             }
         }
     }
-    // stage K and V rows of the chunk (zeros beyond the last visible key): asynchronous
-    // copies, all in flight at once; a chunk never straddles a page of 64 tokens or more
-    {
-        const uint32_t ks0 = (uint32_t)__cvta_generic_to_shared(Ks), vs0 = (uint32_t)__cvta_generic_to_shared(Vs);
-        const bool one_page = page_shift >= 6;
-        const size_t base = one_page ? kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD) : 0;
-#pragma unroll
-        for (int it = 0; it < C * SEGS / T; ++it) {
-            const int idx = tid + it * T;
-            const int r = idx / SEGS, sg = idx % SEGS;
-            const int p = key0 + r;
-            const bool ok = p <= last_pos;
-            const size_t off = (one_page ? base + (size_t)r * HD
-                                         : kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD)) +
-                               (size_t)sg * 8;
-            cp_async16_cg(ks0 + r * KROW + sg * 16, kpages + off, ok ? 16 : 0);
-            cp_async16_cg(vs0 + r * VROW + sg * 16, vpages + off, ok ? 16 : 0);
-        }
-        cp_async_commit();
-    }
+    // stage the remaining K and V rows of the chunk (zeros beyond the last visible key):
+    // asynchronous copies, all in flight at once; a chunk never straddles a page of 64 tokens
+    // or more
+    if (one_page) base = kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD);
+    stage_rows(c_early, last_pos, key0 + C - 1);
+    cp_async_commit();
 #pragma unroll
     for (int i = 0; i < QPT; ++i) {
         const int idx = tid + i * T;
