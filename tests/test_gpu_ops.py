@@ -381,7 +381,8 @@ def test_gemm_tensor_core(M, N, K, accumulate):
     assert np.isfinite(got).all()
 
 
-@pytest.mark.parametrize("Hq,Hkv,hd", [(4, 2, 64), (4, 4, 128), (8, 2, 128)])
+# groups of 1, 2 and 4 query heads per KV head take the tensor-core kernel, 8 the FMA walk
+@pytest.mark.parametrize("Hq,Hkv,hd", [(4, 2, 64), (4, 4, 128), (8, 2, 128), (8, 1, 64), (8, 1, 128)])
 @pytest.mark.parametrize("R,pos0", [(1, 0), (16, 0), (37, 0), (100, 0), (50, 70)])
 def test_prefill_attention(Hq, Hkv, hd, R, pos0):
     page_size, max_seq = 32, 256
