@@ -46,7 +46,7 @@ thread_local int g_last_cuda = 0;
         if (rc_ != LS_OK) return rc_; \
     } while (0)
 
-constexpr int kPrefillBlock = 512;  // rows the prompt pass handles at a time
+constexpr int kPrefillBlock = 1024;  // rows the prompt pass handles at a time
 
 struct LayerW {
     const uint16_t *attn_norm, *wq, *wk, *wv, *wo, *ffn_norm, *wg, *wu, *wd;
@@ -400,13 +400,13 @@ TensorMapEncodeFn tensor_map_encoder()
 
 // 2-D map of a row-major bf16 matrix [rows, K]: boxes of 64 columns (128 bytes) x 128 rows,
 // 128-byte swizzle, zeros outside the matrix
-int make_tile_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K)
+int make_tile_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, int box_rows)
 {
     TensorMapEncodeFn fn = tensor_map_encoder();
     if (!fn) return LS_ERR_UNSUPPORTED;
     cuuint64_t dims[2] = {K, rows};
     cuuint64_t strides[1] = {K * 2};
-    cuuint32_t box[2] = {(cuuint32_t)kGemmBK, (cuuint32_t)kGemmBM};
+    cuuint32_t box[2] = {(cuuint32_t)kGemmBK, (cuuint32_t)box_rows};
     cuuint32_t es[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -415,8 +415,10 @@ int make_tile_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K)
 }
 
 // C[M, N] (+)= A[M, K] B[N, K]^T on the tensor cores (tcgen05), A and B bf16, C fp32
-int gemm_launch(const uint16_t* A, const uint16_t* B, int M, int N, int K, float* C, int ldc, int accumulate,
-                int32_t* status, cudaStream_t st)
+// C[M, n0 + n1 + n2] (+)= A[M, K] [B0; B1; B2]^T: up to three weight matrices with the same K
+// in one launch (B1, B2 may be null)
+int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* B1, int n1, const uint16_t* B2, int n2,
+                 int M, int K, float* C, int ldc, int accumulate, int32_t* status, cudaStream_t st)
 {
     static bool allowed[64] = {false};
     int dev = 0;
@@ -425,13 +427,26 @@ int gemm_launch(const uint16_t* A, const uint16_t* B, int M, int N, int K, float
         LS_CK(cudaFuncSetAttribute(gemm_bf16_tn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes));
         if (dev >= 0 && dev < 64) allowed[dev] = true;
     }
-    CUtensorMap ma, mb;
-    LS_TRY(make_tile_map(&ma, A, (uint64_t)M, (uint64_t)K));
-    LS_TRY(make_tile_map(&mb, B, (uint64_t)N, (uint64_t)K));
-    dim3 grid((N + kGemmBN - 1) / kGemmBN, (M + kGemmBM - 1) / kGemmBM);
-    gemm_bf16_tn_kernel<<<grid, 128, kGemmSmemBytes, st>>>(ma, mb, M, N, K, C, ldc, accumulate, status);
+    CUtensorMap ma, mb[3];
+    LS_TRY(make_tile_map(&ma, A, (uint64_t)M, (uint64_t)K, kGemmBM));
+    const uint16_t* bs[3] = {B0, B1 ? B1 : B0, B2 ? B2 : B0};
+    GemmSegs segs = {{n0, B1 ? n1 : 0, B2 ? n2 : 0}};
+    int tiles = 0;
+    for (int i = 0; i < 3; ++i) {
+        const int rows = segs.n[i] > 0 ? segs.n[i] : n0;  // an unused slot still gets a valid map
+        LS_TRY(make_tile_map(&mb[i], bs[i], (uint64_t)rows, (uint64_t)K, kGemmBN));
+        tiles += (segs.n[i] + kGemmBN - 1) / kGemmBN;
+    }
+    dim3 grid(tiles, (M + kGemmBM - 1) / kGemmBM);
+    gemm_bf16_tn_kernel<<<grid, 128, kGemmSmemBytes, st>>>(ma, mb[0], mb[1], mb[2], segs, M, K, C, ldc, accumulate, status);
     LS_CK(cudaGetLastError());
     return LS_OK;
+}
+
+int gemm_launch(const uint16_t* A, const uint16_t* B, int M, int N, int K, float* C, int ldc, int accumulate,
+                int32_t* status, cudaStream_t st)
+{
+    return gemm_launch3(A, B, N, nullptr, 0, nullptr, 0, M, K, C, ldc, accumulate, status, st);
 }
 
 int prefill_attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt, int pos0, int R,
@@ -479,16 +494,13 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
         uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
         uint16_t* vp = m->vpages + (size_t)l * m->layer_kv_elems;
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.attn_norm, D, c.rms_eps, m->ph, nullptr));
-        LS_TRY(gemm_launch(m->ph, w.wq, R, qw, D, m->py, qkvw, 0, status, st));
-        LS_TRY(gemm_launch(m->ph, w.wk, R, kvw, D, m->py + qw, qkvw, 0, status, st));
-        LS_TRY(gemm_launch(m->ph, w.wv, R, kvw, D, m->py + qw + kvw, qkvw, 0, status, st));
+        LS_TRY(gemm_launch3(m->ph, w.wq, qw, w.wk, kvw, w.wv, kvw, R, D, m->py, qkvw, 0, status, st));
         LS_CK(launch(lc, rope_append_kernel, dim3(R, Hq + 2 * Hkv), dim3(hd / 2), 0, m->py, Hq, Hkv, hd, m->inv_freq,
                      c.rope_theta, m->page_shift, m->page_table, c.max_seq, m->pq, kp, vp, m->ctl, r0));
         LS_TRY(prefill_attn_launch(m->pq, kp, vp, m->page_table, r0, R, Hq, Hkv, hd, m->page_shift, m->po, st));
         LS_TRY(gemm_launch(m->po, w.wo, R, D, qw, m->px, D, 1, status, st));
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.ffn_norm, D, c.rms_eps, m->ph, nullptr));
-        LS_TRY(gemm_launch(m->ph, w.wg, R, F, D, m->py, 2 * F, 0, status, st));
-        LS_TRY(gemm_launch(m->ph, w.wu, R, F, D, m->py + F, 2 * F, 0, status, st));
+        LS_TRY(gemm_launch3(m->ph, w.wg, F, w.wu, F, nullptr, 0, R, D, m->py, 2 * F, 0, status, st));
         swiglu_rows_kernel<<<R, 256, 0, st>>>(m->py, F, m->pa);
         LS_TRY(gemm_launch(m->pa, w.wd, R, D, F, m->px, D, 1, status, st));
         m->launches += 13;
@@ -779,7 +791,7 @@ int ls_prefill(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t lay
     LS_CK(cudaEventRecord(m->ev0, m->st));
     const int rows = n_prompt - 1;
     if (rows > kMaxRows && m->big_prefill) {
-        // the prompt pass proper: blocks of up to 512 rows on the tensor cores
+        // the prompt pass proper: blocks of up to 1024 rows on the tensor cores
         const int pb = m->c.max_seq < kPrefillBlock ? m->c.max_seq : kPrefillBlock;
         for (int r0 = 0; r0 < rows; r0 += pb) LS_TRY(prefill_block(m, r0, rows - r0 < pb ? rows - r0 : pb, layers));
     } else {
