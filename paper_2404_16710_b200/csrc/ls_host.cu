@@ -495,8 +495,8 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
         uint16_t* vp = m->vpages + (size_t)l * m->layer_kv_elems;
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.attn_norm, D, c.rms_eps, m->ph, nullptr));
         LS_TRY(gemm_launch3(m->ph, w.wq, qw, w.wk, kvw, w.wv, kvw, R, D, m->py, qkvw, 0, status, st));
-        LS_CK(launch(lc, rope_append_kernel, dim3(R, Hq + 2 * Hkv), dim3(hd / 2), 0, m->py, Hq, Hkv, hd, m->inv_freq,
-                     c.rope_theta, m->page_shift, m->page_table, c.max_seq, m->pq, kp, vp, m->ctl, r0));
+        rope_append_rows_kernel<<<R, 256, 0, st>>>(m->py, Hq, Hkv, hd, m->inv_freq, m->page_shift, m->page_table, c.max_seq,
+                                                  r0, m->pq, kp, vp, status);
         LS_TRY(prefill_attn_launch(m->pq, kp, vp, m->page_table, r0, R, Hq, Hkv, hd, m->page_shift, m->po, st));
         LS_TRY(gemm_launch(m->po, w.wo, R, D, qw, m->px, D, 1, status, st));
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.ffn_norm, D, c.rms_eps, m->ph, nullptr));

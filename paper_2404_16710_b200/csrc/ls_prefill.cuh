@@ -248,15 +248,64 @@ gemm_bf16_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 }
 
 // ------------------------------------------------------------------ elementwise helpers of the prompt pass
-// a[m, f] = bf16(silu(gu[m, f]) * gu[m, F + f]); grid (rows), block 256
+// a[m, f] = bf16(silu(gu[m, f]) * gu[m, F + f]); grid (rows), block 256; four features per
+// thread and step when F allows 16-byte accesses
 __global__ void __launch_bounds__(256)
 swiglu_rows_kernel(const float* __restrict__ gu, int F, uint16_t* __restrict__ a)
 {
     const float* g = gu + (size_t)blockIdx.x * 2 * F;
     uint16_t* o = a + (size_t)blockIdx.x * F;
-    for (int f = threadIdx.x; f < F; f += 256) {
-        const float x = g[f];
-        o[f] = f2bf(x / (1.0f + expf(-x)) * g[F + f]);
+    if ((F & 3) == 0) {
+        for (int f = threadIdx.x * 4; f < F; f += 256 * 4) {
+            const float4 x = *reinterpret_cast<const float4*>(g + f);
+            const float4 u = *reinterpret_cast<const float4*>(g + F + f);
+            uint2 r;
+            r.x = pack_bf16(x.x / (1.0f + expf(-x.x)) * u.x, x.y / (1.0f + expf(-x.y)) * u.y);
+            r.y = pack_bf16(x.z / (1.0f + expf(-x.z)) * u.z, x.w / (1.0f + expf(-x.w)) * u.w);
+            *reinterpret_cast<uint2*>(o + f) = r;
+        }
+    } else {
+        for (int f = threadIdx.x; f < F; f += 256) {
+            const float x = g[f];
+            o[f] = f2bf(x / (1.0f + expf(-x)) * g[F + f]);
+        }
+    }
+}
+
+// Rotary embedding and KV append for a block of prompt rows: qkv fp32 [R][(Hq + 2 Hkv) hd] ->
+// q bf16 [R][Hq hd], k and v into the paged cache at positions pos0 + row.  grid (rows),
+// block 256: a thread keeps one rotary pair index j and walks the heads, so the sine and
+// cosine of its angle are computed once per row.  Same arithmetic as rope_append_kernel.
+__global__ void __launch_bounds__(256)
+rope_append_rows_kernel(const float* __restrict__ qkv, int Hq, int Hkv, int hd, const float* __restrict__ inv_freq,
+                        int page_shift, const int32_t* __restrict__ page_table, int max_seq, int pos0,
+                        uint16_t* __restrict__ q_out, uint16_t* __restrict__ kpages, uint16_t* __restrict__ vpages,
+                        int32_t* status)
+{
+    const int m = blockIdx.x, half = hd >> 1;
+    const int pos = pos0 + m;
+    if (pos < 0 || pos >= max_seq) {
+        if (status && threadIdx.x == 0) *status = DEV_POS_OVERFLOW;
+        return;
+    }
+    const int j = threadIdx.x % half, h0 = threadIdx.x / half, hstep = 256 / half;
+    float sn, cs;
+    sincosf((float)pos * inv_freq[j], &sn, &cs);
+    const int H = Hq + 2 * Hkv;
+    const float* src = qkv + (size_t)m * H * hd;
+    for (int h = h0; h < H; h += hstep) {
+        float a = src[(size_t)h * hd + j], b = src[(size_t)h * hd + j + half];
+        if (h < Hq + Hkv) {
+            const float ra = a * cs - b * sn, rb = a * sn + b * cs;
+            a = ra;
+            b = rb;
+        }
+        uint16_t* dst;
+        if (h < Hq) dst = q_out + ((size_t)m * Hq + h) * hd;
+        else if (h < Hq + Hkv) dst = kpages + kv_row_offset(page_table, pos, page_shift, Hkv, h - Hq, hd);
+        else dst = vpages + kv_row_offset(page_table, pos, page_shift, Hkv, h - Hq - Hkv, hd);
+        dst[j] = f2bf(a);
+        dst[j + half] = f2bf(b);
     }
 }
 
