@@ -454,15 +454,17 @@ int prefill_attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* v
 {
     const int G = Hq / Hkv, Q = G * kMaxRows;
     dim3 grid((R + 15) / 16, Hkv);
-    if (G <= 4) {  // four query tiles fit in registers: tensor-core kernel
+    if (G == 1 || G == 2 || G == 4) {  // tensor-core kernel: 64 queries per CTA, 16 per warp
+        const int rpc = 64 / G;
+        dim3 mgrid((R + rpc - 1) / rpc, Hkv);
         if (hd == 128) {
-            const size_t sm = prefill_attn_mma_smem_bytes<128>(Q);
-            LS_CK(cudaFuncSetAttribute(prefill_attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
-            prefill_attn_mma_kernel<128><<<grid, kAttnThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
+            const size_t sm = prefill_attn_fa_smem_bytes<128>();
+            LS_CK(cudaFuncSetAttribute(prefill_attn_fa_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+            prefill_attn_fa_kernel<128><<<mgrid, kFaThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
         } else {
-            const size_t sm = prefill_attn_mma_smem_bytes<64>(Q);
-            LS_CK(cudaFuncSetAttribute(prefill_attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
-            prefill_attn_mma_kernel<64><<<grid, kAttnThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
+            const size_t sm = prefill_attn_fa_smem_bytes<64>();
+            LS_CK(cudaFuncSetAttribute(prefill_attn_fa_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+            prefill_attn_fa_kernel<64><<<mgrid, kFaThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
         }
     } else if (hd == 128) {
         const size_t sm = prefill_attn_smem_bytes<128>(Q);

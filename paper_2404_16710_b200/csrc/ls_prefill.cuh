@@ -454,197 +454,190 @@ prefill_attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
     }
 }
 
-// The same walk on the tensor cores (used when a KV head's 16 rows x G query heads fit in four
-// query tiles, G <= 4): q.k and p.v as mma.sync.m16n8k16 exactly as in the decode attention
-// kernel (queries are the 16-row operand, V comes transposed out of ldmatrix), softmax pieces
-// per chunk in fp32, the running output of every query tile stays in registers and is rescaled
-// by exp(old max - new max) before each chunk's contribution is added.
-// shared memory: Ks [64][HD*2+64] | Vs [64][HD*2+16] | Qb bf16 [Qpad][HD*2+64] | S f32 [Qpad][72]
-//                | Pb bf16 [Qpad][72] | mx, l, alpha f32 [Qpad] each
+// Causal attention of a block of prompt rows on the tensor cores (G = Hq / Hkv in {1, 2, 4}),
+// in the flash-attention arrangement: a CTA of four warps takes 64 queries of one KV head
+// (64 / G rows x G query heads), each warp 16 rows of one query head.  A warp keeps its
+// queries as mma.sync A fragments, walks the 64-key chunks that all warps stage together
+// (cp.async, two buffers: the next chunk travels while this one is used), and needs nobody
+// else: s = q.k lands in accumulator registers, the running max / sum of its rows live in
+// registers (quad shuffles), p is rounded to bf16 and is, in the accumulator layout, already
+// the A fragment of p.v; the running output (16 x HD fp32) is rescaled per chunk.
+// Scores are scaled by log2(e)/sqrt(hd) so that the exponentials are exp2.
+// shared memory: 2 x (K [64][HD*2+16] | V [64][HD*2+16])
+constexpr int kFaThreads = 128;
 template <int HD>
-__host__ __device__ constexpr size_t prefill_attn_mma_smem_bytes(int Q)
+__host__ __device__ constexpr size_t prefill_attn_fa_smem_bytes()
 {
-    const size_t qpad = ((size_t)Q + 15) / 16 * 16;
-    return (size_t)kAttnChunk * (HD * 2 + 64) + (size_t)kAttnChunk * (HD * 2 + 16) + qpad * (HD * 2 + 64) +
-           qpad * kAttnSP * 4 + qpad * kAttnSP * 2 + 3 * qpad * sizeof(float);
+    return 2 * 2 * (size_t)kAttnChunk * (HD * 2 + 16);
 }
 
 template <int HD>
-__global__ void __launch_bounds__(kAttnThreads)
-prefill_attn_mma_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
-                        const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table, int pos0, int R,
-                        int Hq, int Hkv, int page_shift, uint16_t* __restrict__ out)
+__global__ void __launch_bounds__(kFaThreads)
+prefill_attn_fa_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
+                       const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table, int pos0, int R,
+                       int Hq, int Hkv, int page_shift, uint16_t* __restrict__ out)
 {
-    constexpr int C = kAttnChunk, T = kAttnThreads;
-    constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 16, SP = kAttnSP, PBROW = kAttnSP * 2;
-    constexpr int SEGS = HD * 2 / 16;
-    constexpr int NTW = HD / 64;  // n8 tiles of output dims per warp
-    constexpr int MAXQT = 4;      // query tiles held in registers
-    const int tid = threadIdx.x, kh = blockIdx.y;
-    const int warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
-    const int r0 = blockIdx.x * 16;
-    const int M = min(16, R - r0);
-    const int G = Hq / Hkv, Q = G * M, Qpad = (Q + 15) & ~15;
-    const int first_pos = pos0 + r0, last_pos = first_pos + M - 1;
-
+    constexpr int C = kAttnChunk, T = kFaThreads;
+    constexpr int ROW = HD * 2 + 16;   // bytes per staged row: conflict-free for both operand reads
+    constexpr int SEGS = HD * 2 / 16;  // 16-byte pieces per row
+    constexpr int KS = HD / 16;        // k-steps of q.k
+    constexpr int NT = HD / 8;         // n8 tiles of the output
+    constexpr int BUF = 2 * C * ROW;   // one buffer: K then V
     extern __shared__ __align__(16) unsigned char smem[];
-    unsigned char* Ks = smem;
-    unsigned char* Vs = Ks + C * KROW;
-    unsigned char* Qb = Vs + C * VROW;
-    float* S = reinterpret_cast<float*>(Qb + (size_t)Qpad * KROW);
-    unsigned char* Pb = reinterpret_cast<unsigned char*>(S + (size_t)Qpad * SP);
-    float* mx = reinterpret_cast<float*>(Pb + (size_t)Qpad * PBROW);
-    float* ls = mx + Qpad;
-    float* al = ls + Qpad;
-
-    for (int idx = tid; idx < Qpad * SEGS; idx += T) {
-        const int qi = idx / SEGS, sg = idx % SEGS;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (qi < Q) {
-            const int m = qi / G, g = qi % G;
-            v = *reinterpret_cast<const uint4*>(q + ((size_t)(r0 + m) * Hq + (size_t)kh * G + g) * HD + sg * 8);
-        }
-        *reinterpret_cast<uint4*>(Qb + qi * KROW + sg * 16) = v;
-    }
-    for (int qi = tid; qi < Qpad; qi += T) {
-        mx[qi] = -INFINITY;
-        ls[qi] = 0.f;
-        al[qi] = 1.f;
-    }
-    float o[MAXQT][NTW][4];
-#pragma unroll
-    for (int qt = 0; qt < MAXQT; ++qt)
-#pragma unroll
-        for (int nt = 0; nt < NTW; ++nt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) o[qt][nt][i] = 0.f;
-
-    const int d0 = NTW * 8 * warp;
-    const uint32_t ks0 = smem_u32(Ks), vs0 = smem_u32(Vs);
-    const int mi = lane >> 3, mr = lane & 7;
-    const uint32_t vlane = vs0 + (uint32_t)(((mi & 1) * 8 + mr) * VROW + (d0 + ((NTW == 2) ? (mi >> 1) * 8 : 0)) * 2);
-    const float scale = rsqrtf((float)HD);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int kh = blockIdx.y, G = Hq / Hkv;
+    const int rows_per_cta = 64 / G;
+    const int r0 = blockIdx.x * rows_per_cta;
+    const int M = min(rows_per_cta, R - r0);
+    const int gq = warp % G, rt = warp / G;  // the warp's query head within the group, its tile of 16 rows
+    const int head = kh * G + gq;
+    const bool active = rt * 16 < M;
+    const int last_pos = pos0 + r0 + M - 1;
     const int nch = last_pos / C + 1;
-    for (int ch = 0; ch < nch; ++ch) {
-        const int key0 = ch * C;
-        __syncthreads();  // the previous chunk's K, V, S, Pb are no longer read
-        {
-            const bool one_page = page_shift >= 6;
-            const size_t base = one_page ? kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD) : 0;
+    const int warp_nch = active ? (pos0 + r0 + min(rt * 16 + 15, M - 1)) / C + 1 : 0;
+    const int rowA = rt * 16 + g, rowB = rowA + 8;  // within the CTA's rows
+    const int posA = pos0 + r0 + rowA, posB = posA + 8;
+
+    // the warp's queries as A fragments (zeros for rows that do not exist)
+    uint32_t qf[KS][4];
+    {
+        const uint16_t* qa = q + ((size_t)(r0 + min(rowA, M - 1)) * Hq + head) * HD;
+        const uint16_t* qb = q + ((size_t)(r0 + min(rowB, M - 1)) * Hq + head) * HD;
+        const bool va = active && rowA < M, vb = active && rowB < M;
 #pragma unroll
-            for (int it = 0; it < C * SEGS / T; ++it) {
-                const int idx = tid + it * T;
-                const int r = idx / SEGS, sg = idx % SEGS;
-                const int p = key0 + r;
-                const bool ok = p <= last_pos;
-                const size_t off = (one_page ? base + (size_t)r * HD
-                                             : kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD)) +
-                                   (size_t)sg * 8;
-                cp_async16_cg(ks0 + r * KROW + sg * 16, kpages + off, ok ? 16 : 0);
-                cp_async16_cg(vs0 + r * VROW + sg * 16, vpages + off, ok ? 16 : 0);
-            }
-            cp_async_commit();
-            cp_async_wait<0>();
-        }
-        __syncthreads();
-        // s = q.k: warp w owns keys 8w..8w+7
-        for (int qt = 0; qt < Qpad; qt += 16) {
-            float c[4] = {0.f, 0.f, 0.f, 0.f};
-            const unsigned char* qa = Qb + (qt + g8) * KROW + 16 * t4;
-            const unsigned char* kb = Ks + (8 * warp + g8) * KROW + 16 * t4;
-#pragma unroll
-            for (int j = 0; j < HD / 32; ++j) {
-                const uint4 A0 = *reinterpret_cast<const uint4*>(qa + 64 * j);
-                const uint4 A1 = *reinterpret_cast<const uint4*>(qa + 8 * KROW + 64 * j);
-                const uint4 Bk = *reinterpret_cast<const uint4*>(kb + 64 * j);
-                mma_bf16_16816(c, A0.x, A1.x, A0.y, A1.y, Bk.x, Bk.y);
-                mma_bf16_16816(c, A0.z, A1.z, A0.w, A1.w, Bk.z, Bk.w);
-            }
-            float* sp = S + (size_t)(qt + g8) * SP + 8 * warp + 2 * t4;
-            *reinterpret_cast<float2*>(sp) = make_float2(c[0], c[1]);
-            *reinterpret_cast<float2*>(sp + 8 * SP) = make_float2(c[2], c[3]);
-        }
-        __syncthreads();
-        // per query: mask, running max and sum, p -> bf16
-        for (int qi = warp; qi < Qpad; qi += T / 32) {
-            uint16_t* pb = reinterpret_cast<uint16_t*>(Pb + (size_t)qi * PBROW);
-            if (qi >= Q) {
-                pb[lane] = 0;
-                pb[lane + 32] = 0;
-                continue;
-            }
-            const int pos = first_pos + qi / G;
-            float s0 = S[(size_t)qi * SP + lane] * scale;
-            float s1 = S[(size_t)qi * SP + lane + 32] * scale;
-            if (key0 + lane > pos) s0 = -INFINITY;
-            if (key0 + lane + 32 > pos) s1 = -INFINITY;
-            float cm = fmaxf(s0, s1);
-#pragma unroll
-            for (int sh = 16; sh > 0; sh >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, sh));
-            const float mo = mx[qi], mn = fmaxf(mo, cm);
-            const float p0 = (s0 == -INFINITY) ? 0.f : expf(s0 - mn);
-            const float p1 = (s1 == -INFINITY) ? 0.f : expf(s1 - mn);
-            float l = p0 + p1;
-#pragma unroll
-            for (int sh = 16; sh > 0; sh >>= 1) l += __shfl_xor_sync(0xffffffffu, l, sh);
-            pb[lane] = f2bf(p0);
-            pb[lane + 32] = f2bf(p1);
-            if (lane == 0) {
-                const float a = (mn == -INFINITY) ? 1.f : ((mo == -INFINITY) ? 0.f : expf(mo - mn));
-                al[qi] = a;
-                ls[qi] = ls[qi] * a + l;
-                mx[qi] = mn;
-            }
-        }
-        __syncthreads();
-        // o = o * alpha + p.v: warp w owns output dims d0 .. d0 + 8 NTW - 1
-#pragma unroll
-        for (int qt = 0; qt < MAXQT; ++qt) {
-            if (qt * 16 < Qpad) {
-                float c[NTW][4];
-#pragma unroll
-                for (int nt = 0; nt < NTW; ++nt)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) c[nt][i] = 0.f;
-                const unsigned char* pa = Pb + (size_t)(qt * 16 + g8) * PBROW + 4 * t4;
-#pragma unroll
-                for (int kk = 0; kk < C / 16; ++kk) {
-                    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(pa + 32 * kk);
-                    const uint32_t a1 = *reinterpret_cast<const uint32_t*>(pa + 8 * PBROW + 32 * kk);
-                    const uint32_t a2 = *reinterpret_cast<const uint32_t*>(pa + 32 * kk + 16);
-                    const uint32_t a3 = *reinterpret_cast<const uint32_t*>(pa + 8 * PBROW + 32 * kk + 16);
-                    uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4_trans(vlane + (uint32_t)(16 * kk * VROW), b0, b1, b2, b3);
-                    mma_bf16_16816(c[0], a0, a1, a2, a3, b0, b1);
-                    if (NTW == 2) mma_bf16_16816(c[NTW - 1], a0, a1, a2, a3, b2, b3);
-                }
-                const float alo = al[qt * 16 + g8], ahi = al[qt * 16 + g8 + 8];
-#pragma unroll
-                for (int nt = 0; nt < NTW; ++nt) {
-                    o[qt][nt][0] = o[qt][nt][0] * alo + c[nt][0];
-                    o[qt][nt][1] = o[qt][nt][1] * alo + c[nt][1];
-                    o[qt][nt][2] = o[qt][nt][2] * ahi + c[nt][2];
-                    o[qt][nt][3] = o[qt][nt][3] * ahi + c[nt][3];
-                }
-            }
+        for (int kk = 0; kk < KS; ++kk) {
+            qf[kk][0] = va ? *reinterpret_cast<const uint32_t*>(qa + kk * 16 + 2 * t) : 0u;
+            qf[kk][1] = vb ? *reinterpret_cast<const uint32_t*>(qb + kk * 16 + 2 * t) : 0u;
+            qf[kk][2] = va ? *reinterpret_cast<const uint32_t*>(qa + kk * 16 + 2 * t + 8) : 0u;
+            qf[kk][3] = vb ? *reinterpret_cast<const uint32_t*>(qb + kk * 16 + 2 * t + 8) : 0u;
         }
     }
-    __syncthreads();
+    const uint32_t sm0 = smem_u32(smem);
+    const bool one_page = page_shift >= 6;
+    auto stage = [&](int ch, int b) {  // rows of chunk ch -> buffer b (zeros beyond the last visible key)
+        const int key0 = ch * C;
+        const size_t base = one_page ? kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD) : 0;
+        const uint32_t kb = sm0 + b * BUF, vb = kb + C * ROW;
 #pragma unroll
-    for (int qt = 0; qt < MAXQT; ++qt)
+        for (int it = 0; it < C * SEGS / T; ++it) {
+            const int idx = tid + it * T;
+            const int r = idx / SEGS, sg = idx % SEGS;
+            const int p = key0 + r;
+            const bool ok = p <= last_pos;
+            const size_t off = (one_page ? base + (size_t)r * HD
+                                         : kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD)) +
+                               (size_t)sg * 8;
+            cp_async16_cg(kb + r * ROW + sg * 16, kpages + off, ok ? 16 : 0);
+            cp_async16_cg(vb + r * ROW + sg * 16, vpages + off, ok ? 16 : 0);
+        }
+    };
+
+    float o[NT][4];
 #pragma unroll
-        for (int hrow = 0; hrow < 2; ++hrow) {
-            const int qi = qt * 16 + g8 + 8 * hrow;
-            if (qi < Q) {
-                const int m = qi / G, g = qi % G;
-                const float l = ls[qi];
-                uint16_t* dst = out + ((size_t)(r0 + m) * Hq + (size_t)kh * G + g) * HD + d0 + 2 * t4;
+    for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int nt = 0; nt < NTW; ++nt)
-                    *reinterpret_cast<uint32_t*>(dst + 8 * nt) =
-                        pack_bf16(o[qt][nt][2 * hrow] / l, o[qt][nt][2 * hrow + 1] / l);
+        for (int i = 0; i < 4; ++i) o[nt][i] = 0.f;
+    float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;  // running max; this thread's share of the sums
+    const float sc = rsqrtf((float)HD) * 1.4426950408889634f;
+    const int mi = lane >> 3, mr = lane & 7;  // ldmatrix: lane -> row mr of matrix mi
+
+    stage(0, 0);
+    cp_async_commit();
+    for (int ch = 0; ch < nch; ++ch) {
+        if (ch + 1 < nch) stage(ch + 1, (ch + 1) & 1);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();
+        if (ch < warp_nch) {
+            const unsigned char* Kb = smem + (ch & 1) * BUF;
+            const uint32_t vb = sm0 + (ch & 1) * BUF + C * ROW;
+            float s[C / 8][4];
+#pragma unroll
+            for (int nt = 0; nt < C / 8; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) s[nt][i] = 0.f;
+#pragma unroll
+            for (int kk = 0; kk < KS; ++kk)
+#pragma unroll
+                for (int nt = 0; nt < C / 8; ++nt) {
+                    const unsigned char* kr = Kb + (nt * 8 + g) * ROW + (kk * 16 + 2 * t) * 2;
+                    mma_bf16_16816(s[nt], qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3],
+                                   *reinterpret_cast<const uint32_t*>(kr), *reinterpret_cast<const uint32_t*>(kr + 16));
+                }
+            // scale, causal mask, running max
+            float cA = -INFINITY, cB = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < C / 8; ++nt) {
+                const int key = ch * C + nt * 8 + 2 * t;
+                s[nt][0] = key <= posA ? s[nt][0] * sc : -INFINITY;
+                s[nt][1] = key + 1 <= posA ? s[nt][1] * sc : -INFINITY;
+                s[nt][2] = key <= posB ? s[nt][2] * sc : -INFINITY;
+                s[nt][3] = key + 1 <= posB ? s[nt][3] * sc : -INFINITY;
+                cA = fmaxf(cA, fmaxf(s[nt][0], s[nt][1]));
+                cB = fmaxf(cB, fmaxf(s[nt][2], s[nt][3]));
+            }
+            cA = fmaxf(cA, __shfl_xor_sync(0xffffffffu, cA, 1));
+            cA = fmaxf(cA, __shfl_xor_sync(0xffffffffu, cA, 2));
+            cB = fmaxf(cB, __shfl_xor_sync(0xffffffffu, cB, 1));
+            cB = fmaxf(cB, __shfl_xor_sync(0xffffffffu, cB, 2));
+            const float nA = fmaxf(mA, cA), nB = fmaxf(mB, cB);
+            // (a row sees key 0 in its first chunk, so nA, nB are finite from then on)
+            const float fA = nA == -INFINITY ? 0.f : nA, fB = nB == -INFINITY ? 0.f : nB;
+            const float aA = exp2f(mA - fA), aB = exp2f(mB - fB);
+            mA = nA;
+            mB = nB;
+            float pA = 0.f, pB = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < C / 8; ++nt) {
+                s[nt][0] = exp2f(s[nt][0] - fA);
+                s[nt][1] = exp2f(s[nt][1] - fA);
+                s[nt][2] = exp2f(s[nt][2] - fB);
+                s[nt][3] = exp2f(s[nt][3] - fB);
+                pA += s[nt][0] + s[nt][1];
+                pB += s[nt][2] + s[nt][3];
+            }
+            lA = lA * aA + pA;
+            lB = lB * aB + pB;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                o[nt][0] *= aA;
+                o[nt][1] *= aA;
+                o[nt][2] *= aB;
+                o[nt][3] *= aB;
+            }
+            // o += p.v: p (bf16) in the accumulator layout is the A fragment
+#pragma unroll
+            for (int k2 = 0; k2 < C / 16; ++k2) {
+                const uint32_t a0 = pack_bf16(s[2 * k2][0], s[2 * k2][1]), a1 = pack_bf16(s[2 * k2][2], s[2 * k2][3]);
+                const uint32_t a2 = pack_bf16(s[2 * k2 + 1][0], s[2 * k2 + 1][1]);
+                const uint32_t a3 = pack_bf16(s[2 * k2 + 1][2], s[2 * k2 + 1][3]);
+                const uint32_t vrow = vb + (uint32_t)((k2 * 16 + (mi & 1) * 8 + mr) * ROW + (mi >> 1) * 16);
+#pragma unroll
+                for (int np = 0; np < NT / 2; ++np) {
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(vrow + np * 32, b0, b1, b2, b3);
+                    mma_bf16_16816(o[2 * np], a0, a1, a2, a3, b0, b1);
+                    mma_bf16_16816(o[2 * np + 1], a0, a1, a2, a3, b2, b3);
+                }
             }
         }
+        __syncthreads();  // the buffer may be overwritten by the copy issued in the next round
+    }
+    if (!active) return;
+    lA += __shfl_xor_sync(0xffffffffu, lA, 1);
+    lA += __shfl_xor_sync(0xffffffffu, lA, 2);
+    lB += __shfl_xor_sync(0xffffffffu, lB, 1);
+    lB += __shfl_xor_sync(0xffffffffu, lB, 2);
+    if (rowA < M) {
+        uint16_t* dst = out + ((size_t)(r0 + rowA) * Hq + head) * HD + 2 * t;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) *reinterpret_cast<uint32_t*>(dst + nt * 8) = pack_bf16(o[nt][0] / lA, o[nt][1] / lA);
+    }
+    if (rowB < M) {
+        uint16_t* dst = out + ((size_t)(r0 + rowB) * Hq + head) * HD + 2 * t;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) *reinterpret_cast<uint32_t*>(dst + nt * 8) = pack_bf16(o[nt][2] / lB, o[nt][3] / lB);
+    }
 }
 
 }  // namespace ls
