@@ -183,6 +183,8 @@ def run_own(args):
     E, d, P, NEW = wl.exit_layer, wl.num_draft, wl.n_prompt, wl.max_new
     peak, peak_kind = peaks()
 
+    if args.profile_prompt:
+        P = args.profile_prompt
     w = synth.make_weights(s, wl.weight_seed, E, wl.late_scale, device="cuda")
     max_seq = P + NEW + d + 1
     gm = B.Model(s, w, max_seq, 64, max(d, 1))
@@ -195,6 +197,16 @@ def run_own(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.profile_prompt:
+        for _ in range(max(1, args.warmup)):
+            B.ls_prefill(gm.h, prompt)
+        torch.cuda.synchronize()
+        torch.cuda.profiler.start()
+        B.ls_prefill(gm.h, prompt)
+        torch.cuda.synchronize()
+        torch.cuda.profiler.stop()
+        print(json.dumps({"profile_prompt": P, "prefill_ms": round(gm.stats().prefill_ms, 2)}))
+        return
     if args.profile_region:
         B.ls_prefill(gm.h, prompt)
         for _ in range(max(1, args.warmup)):
@@ -384,6 +396,9 @@ def main():
                     help="instead of the benchmark: prefill, warm up, then run one self-speculative and one "
                          "full-greedy decode of NEW tokens between cudaProfilerStart/Stop (for a profiler "
                          "started with --profile-from-start off) and exit")
+    ap.add_argument("--profile-prompt", type=int, default=0, metavar="P",
+                    help="instead of the benchmark: the prompt pass of a P-token prompt, warmed up, once between "
+                         "cudaProfilerStart/Stop, then exit")
     ap.add_argument("--sweep", action="store_true", help="run the (exit layer, drafts, late scale) sweep instead")
     ap.add_argument("--sweep-exit", default=",".join(map(str, synth.SWEEP_EXIT)))
     ap.add_argument("--sweep-draft", default=",".join(map(str, synth.SWEEP_DRAFT)))
