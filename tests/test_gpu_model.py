@@ -177,6 +177,42 @@ def test_without_exit_cache_reuse_same_ids_more_bytes():
         B.ls_decode_flags(gm.h, 2, 3, 40, 8)
 
 
+# ------------------------------------------------------------------ odd shapes
+ODD_SHAPES = [
+    synth.Shape("odd-g2", 3, 104, 6, 3, 64, 200, 301),    # K = 104: ragged last k-step; 7 partial sums per row
+    synth.Shape("odd-g8", 2, 128, 8, 1, 64, 344, 1000),   # 8 query heads per KV head: FMA prompt attention
+    synth.Shape("odd-mha128", 2, 256, 2, 2, 128, 136, 77),  # vocabulary smaller than one prompt-GEMM tile
+    synth.Shape("odd-g4", 2, 64, 4, 1, 128, 72, 513),     # q width (512) != d_model (64)
+]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("shape", ODD_SHAPES, ids=lambda s: s.name)
+def test_odd_shapes_logits_and_losslessness(shape, path):
+    """Shapes whose sizes are not multiples of the tiles: logits against the oracle (16-row
+    passes), then a 45-token prompt (tensor-core prompt pass) with every loop giving the ids
+    of full greedy, which in turn follow the oracle while its margins allow."""
+    gm, om = make_pair(shape, 5, 1, 0.3, 128, page_size=16, max_draft=6, linear_path=path, amplify=6.0)
+    ids = synth.make_prompt(shape.vocab, 37, 3)
+    gex, gfi = gm.debug_logits(ids, 1)
+    oex, ofi = om.teacher_logits(ids, 1)
+    assert np.abs(ofi).max() > 0.3
+    assert_logits_close(gex, oex, "exit logits")
+    assert_logits_close(gfi, ofi, "final logits")
+    prompt = synth.make_prompt(shape.vocab, 45, 4)
+    full = gm.generate_full(prompt, 40)
+    for E, d in ((1, 1), (1, 3), (1, 6)):
+        got, acc = gm.generate(prompt, E, d, 40)
+        np.testing.assert_array_equal(got, full, err_msg=f"E={E} d={d}")
+    got, acc, drafted = gm.generate_adaptive(prompt, 1, 6, 0.05, 40)
+    np.testing.assert_array_equal(got, full)
+    np.testing.assert_array_equal(gm.generate_early(prompt, shape.n_layers, 40), full)
+    ref, margins, maxabs = om.generate_full(prompt, 40)
+    k = first_low_margin(margins, maxabs)
+    np.testing.assert_array_equal(full[:k], ref[:k])
+    print(f"{shape.name} path {path}: ids follow the oracle for {k} of 40 tokens")
+
+
 # ------------------------------------------------------------------ adaptive draft length
 @pytest.mark.parametrize("path", PATHS)
 def test_adaptive_equals_generate_full_for_every_threshold(path):
