@@ -100,10 +100,11 @@ struct ls_model {
     float* second;      // per-CTA second-largest logit beside each argmax candidate (adaptive drafting)
     int32_t* drafted;   // drafts kept per step (adaptive drafting)
     int gate;           // draft pass the launches being enqueued belong to (0: none)
+    unsigned long long next_pass;  // conditional-node handle the next draft head switches on (0: none)
     int page_shift, n_pages, chunk_cap, cand_stride;
     // loop state
     int n_prompt, last_tok, prefilled_layers, grid_chunks;
-    bool use_graphs, own_stream, pdl, big_prefill;
+    bool use_graphs, own_stream, pdl, big_prefill, cond_graphs;
     int64_t launches;  // kernels enqueued (counted while building a step)
     struct G {
         cudaGraphExec_t exec;
@@ -365,7 +366,7 @@ int run_head(ls_model* m, int M, int slot, int32_t* tok_out, float* logits, floa
     LS_CK(launch_linear(m->path, EPI_ARGMAX, a, st));
     LS_CK(launch(st, argmax_finish_kernel, dim3(M), dim3(256), 0, (const ValIdx*)m->cand,
                  n_candidates(m->path, c.vocab, c.d_model, M), m->cand_stride, tok_out, m->ctl,
-                 (const float*)a.second, min_margin, m->gate));
+                 (const float*)a.second, min_margin, m->gate, m->next_pass));
     m->launches += 2;
     return LS_OK;
 }
@@ -516,42 +517,135 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
 // once an earlier pass's head has found its two largest exit logits closer than min_margin;
 // the verify pass always runs on d + 1 rows (the rows beyond the kept drafts are stale and
 // never read by the rows that count: causal attention, one dot product per output element).
-int enqueue_step(ls_model* m, int E, int d, bool reuse, float min_margin = 0.f)
+// draft pass j of a step (j == d: the extra early pass, no head)
+int enqueue_draft_pass(ls_model* m, int E, int d, int j, bool reuse, float min_margin)
+{
+    const int D = m->c.d_model;
+    float* xr = m->x + (size_t)j * D;
+    m->gate = min_margin > 0.f ? j : 0;
+    LS_TRY(run_embed(m, j == 0 ? m->ctl + CTL_CUR_TOK : m->draft + (j - 1), 1, xr, j));
+    // the exit-layer row goes to the LM head (final gain) and, pre-scaled by layer E's
+    // gain, to the verify pass (the exit-layer cache of Sec. 4.3.3)
+    LS_TRY(run_layers(m, 0, E, 1, xr, j, j, m->h + (size_t)j * D, j < d ? m->fnorm : nullptr,
+                      reuse ? m->lw[E].attn_norm : nullptr));
+    if (j < d) LS_TRY(run_head(m, 1, j, m->draft + j, nullptr, min_margin));
+    m->gate = 0;
+    return LS_OK;
+}
+
+// verify pass + accept of a step
+int enqueue_verify(ls_model* m, int E, int d, bool reuse, float min_margin)
 {
     const int D = m->c.d_model, L = m->c.n_layers;
     const bool adaptive = min_margin > 0.f;
-    if (d == 0) {
-        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
-        LS_TRY(run_layers(m, 0, E, 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
-        LS_TRY(run_head(m, 1, 0, m->verified, nullptr));
+    if (reuse) {
+        // self-verification (Sec. 4.3.2) from the exit-layer activations
+        LS_TRY(run_layers(m, E, L, d + 1, m->x, 0, 0, m->hE, m->fnorm, nullptr));
     } else {
-        for (int j = 0; j <= (reuse ? d : d - 1); ++j) {  // self-drafting (Sec. 4.3.1) + the extra early pass
-            float* xr = m->x + (size_t)j * D;
-            m->gate = adaptive ? j : 0;
-            LS_TRY(run_embed(m, j == 0 ? m->ctl + CTL_CUR_TOK : m->draft + (j - 1), 1, xr, j));
-            // the exit-layer row goes to the LM head (final gain) and, pre-scaled by layer E's
-            // gain, to the verify pass (the exit-layer cache of Sec. 4.3.3)
-            LS_TRY(run_layers(m, 0, E, 1, xr, j, j, m->h + (size_t)j * D, j < d ? m->fnorm : nullptr,
-                              reuse ? m->lw[E].attn_norm : nullptr));
-            if (j < d) LS_TRY(run_head(m, 1, j, m->draft + j, nullptr, min_margin));
-        }
-        m->gate = 0;
-        if (reuse) {
-            // self-verification (Sec. 4.3.2) from the exit-layer activations
-            LS_TRY(run_layers(m, E, L, d + 1, m->x, 0, 0, m->hE, m->fnorm, nullptr));
-        } else {
-            // the ablation of Sec. 7 (Table 7): no exit-layer cache, verification recomputes the
-            // early layers of all d+1 rows (and rewrites their k, v with the same values)
-            LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
-            LS_TRY(run_embed(m, m->draft, d, m->x + D, 1));
-            LS_TRY(run_layers(m, 0, L, d + 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
-        }
-        LS_TRY(run_head(m, d + 1, 0, m->verified, nullptr));
+        // the ablation of Sec. 7 (Table 7): no exit-layer cache, verification recomputes the
+        // early layers of all d+1 rows (and rewrites their k, v with the same values)
+        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
+        LS_TRY(run_embed(m, m->draft, d, m->x + D, 1));
+        LS_TRY(run_layers(m, 0, L, d + 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
     }
+    LS_TRY(run_head(m, d + 1, 0, m->verified, nullptr));
     LS_CK(launch(LaunchCtx{m->st, m->pdl}, accept_kernel, dim3(1), dim3(32), 0, (const int32_t*)m->draft,
                  (const int32_t*)m->verified, d, m->ctl, m->out_ids, m->accepted, adaptive ? 1 : 0,
                  adaptive ? m->drafted : (int32_t*)nullptr));
     m->launches += 1;
+    return LS_OK;
+}
+
+int enqueue_step(ls_model* m, int E, int d, bool reuse, float min_margin = 0.f)
+{
+    if (d == 0) {
+        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
+        LS_TRY(run_layers(m, 0, E, 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
+        LS_TRY(run_head(m, 1, 0, m->verified, nullptr));
+        LS_CK(launch(LaunchCtx{m->st, m->pdl}, accept_kernel, dim3(1), dim3(32), 0, (const int32_t*)m->draft,
+                     (const int32_t*)m->verified, 0, m->ctl, m->out_ids, m->accepted, 0, (int32_t*)nullptr));
+        m->launches += 1;
+        return LS_OK;
+    }
+    for (int j = 0; j <= (reuse ? d : d - 1); ++j)  // self-drafting (Sec. 4.3.1) + the extra early pass
+        LS_TRY(enqueue_draft_pass(m, E, d, j, reuse, min_margin));
+    return enqueue_verify(m, E, d, reuse, min_margin);
+}
+
+// The adaptive step as a graph whose draft passes 1..d are conditional (IF) nodes: the head of
+// pass j - 1 switches pass j on when it keeps its draft, so a step that stops drafting early
+// launches nothing for the passes it skips (as plain kernel nodes they would each still
+// cost their ~40 launches).  The handles fall back to "off" at every launch of the graph.
+int capture_adaptive_step(ls_model* m, int E, int d, float min_margin, cudaGraph_t* out)
+{
+    cudaGraph_t graph = nullptr;
+    LS_CK(cudaGraphCreate(&graph, 0));
+    cudaStream_t side = nullptr;
+    cudaStream_t mainst = m->st;
+    auto fail = [&](int rc) {
+        m->st = mainst;
+        m->next_pass = 0;
+        if (side) cudaStreamDestroy(side);
+        cudaGraphDestroy(graph);
+        return rc;
+    };
+    std::vector<cudaGraphConditionalHandle> on(d + 1, 0);
+    for (int j = 1; j <= d; ++j)
+        if (cudaGraphConditionalHandleCreate(&on[j], graph, 0, cudaGraphCondAssignDefault) != cudaSuccess)
+            return fail(LS_ERR_CUDA);
+    if (cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking) != cudaSuccess) return fail(LS_ERR_CUDA);
+    if (cudaStreamBeginCaptureToGraph(mainst, graph, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed) != cudaSuccess)
+        return fail(LS_ERR_CUDA);
+    auto abort_capture = [&](int rc) {
+        cudaGraph_t g = nullptr;
+        cudaStreamEndCapture(mainst, &g);
+        return fail(rc);
+    };
+    m->next_pass = on[1];
+    int rc = enqueue_draft_pass(m, E, d, 0, true, min_margin);
+    if (rc != LS_OK) return abort_capture(rc);
+    for (int j = 1; j <= d; ++j) {
+        cudaStreamCaptureStatus status;
+        cudaGraph_t cg = nullptr;
+        const cudaGraphNode_t* deps = nullptr;
+        size_t n_deps = 0;
+        if (cudaStreamGetCaptureInfo(mainst, &status, nullptr, &cg, &deps, &n_deps) != cudaSuccess)
+            return abort_capture(LS_ERR_CUDA);
+        cudaGraphNodeParams p = {};
+        p.type = cudaGraphNodeTypeConditional;
+        p.conditional.handle = on[j];
+        p.conditional.type = cudaGraphCondTypeIf;
+        p.conditional.size = 1;
+        cudaGraphNode_t node;
+        if (cudaGraphAddNode(&node, graph, deps, n_deps, &p) != cudaSuccess) return abort_capture(LS_ERR_CUDA);
+        if (cudaStreamUpdateCaptureDependencies(mainst, &node, 1, cudaStreamSetCaptureDependencies) != cudaSuccess)
+            return abort_capture(LS_ERR_CUDA);
+        cudaGraph_t body = p.conditional.phGraph_out[0];
+        if (cudaStreamBeginCaptureToGraph(side, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed) != cudaSuccess)
+            return abort_capture(LS_ERR_CUDA);
+        m->st = side;
+        m->next_pass = j < d ? on[j + 1] : 0;
+        rc = enqueue_draft_pass(m, E, d, j, true, min_margin);
+        m->st = mainst;
+        cudaGraph_t captured = nullptr;
+        cudaError_t e = cudaStreamEndCapture(side, &captured);
+        if (rc != LS_OK) return abort_capture(rc);
+        if (e != cudaSuccess) {
+            g_last_cuda = (int)e;
+            return abort_capture(LS_ERR_CUDA);
+        }
+    }
+    m->next_pass = 0;
+    rc = enqueue_verify(m, E, d, true, min_margin);
+    cudaGraph_t done = nullptr;
+    cudaError_t e = cudaStreamEndCapture(mainst, &done);
+    if (rc != LS_OK) return fail(rc);
+    if (e != cudaSuccess) {
+        g_last_cuda = (int)e;
+        return fail(LS_ERR_CUDA);
+    }
+    cudaStreamDestroy(side);
+    *out = graph;
     return LS_OK;
 }
 
@@ -571,14 +665,19 @@ int get_graph(ls_model* m, int E, int d, bool reuse, float min_margin, ls_model:
     if (it == m->graphs.end()) {
         cudaGraph_t graph = nullptr;
         int64_t before = m->launches;
-        LS_CK(cudaStreamBeginCapture(m->st, cudaStreamCaptureModeRelaxed));
-        int rc = enqueue_step(m, E, d, reuse, min_margin);
-        cudaError_t e = cudaStreamEndCapture(m->st, &graph);
-        if (rc != LS_OK) {
-            if (graph) cudaGraphDestroy(graph);
-            return rc;
+        cudaError_t e = cudaSuccess;
+        if (min_margin > 0.f && reuse && d > 0 && m->cond_graphs) {
+            LS_TRY(capture_adaptive_step(m, E, d, min_margin, &graph));
+        } else {
+            LS_CK(cudaStreamBeginCapture(m->st, cudaStreamCaptureModeRelaxed));
+            int rc = enqueue_step(m, E, d, reuse, min_margin);
+            e = cudaStreamEndCapture(m->st, &graph);
+            if (rc != LS_OK) {
+                if (graph) cudaGraphDestroy(graph);
+                return rc;
+            }
+            LS_CK(e);
         }
-        LS_CK(e);
         ls_model::G g;
         g.nodes = m->launches - before;
         e = cudaGraphInstantiate(&g.exec, graph, 0);
@@ -716,6 +815,9 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
     m->grid_chunks = m->chunk_cap;
     m->use_graphs = getenv("LS_NO_GRAPH") == nullptr;
     m->pdl = getenv("LS_NO_PDL") == nullptr;
+    m->cond_graphs = getenv("LS_NO_COND") == nullptr;
+    m->gate = 0;
+    m->next_pass = 0;
     m->big_prefill = getenv("LS_SMALL_PREFILL") == nullptr && tensor_map_encoder() != nullptr;
     m->launches = 0;
     memset(&m->stats, 0, sizeof(m->stats));
@@ -1132,7 +1234,7 @@ int ls_op_lm_head_argmax(int32_t path, const void* w, const void* h, int32_t M, 
     const LaunchCtx lc = {(cudaStream_t)stream, false};
     LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
     LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, n_candidates(path, V, K, M), a.cand_stride, tok,
-                 nullptr, nullptr, 0.f, 0));
+                 nullptr, nullptr, 0.f, 0, 0ull));
     return LS_OK;
 }
 
@@ -1178,7 +1280,7 @@ int ls_op_lm_head_argmax_static(int32_t path, const void* w, const void* h, int3
     const LaunchCtx lc = {(cudaStream_t)stream, false};
     LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
     LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, n_candidates(path, V, K, M), a.cand_stride, tok,
-                 nullptr, nullptr, 0.f, 0));
+                 nullptr, nullptr, 0.f, 0, 0ull));
     return LS_OK;
 }
 

@@ -605,11 +605,13 @@ attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
 // Adaptive drafting (second != nullptr; the launch is the head of draft pass `gate`, M = 1):
 // the per-CTA second-largest logits are reduced too, and when the margin between the two
 // largest exit logits is below min_margin this draft is not kept and drafting stops:
-// CTL_D_EFF = gate, which idles every later draft pass of the step.
+// CTL_D_EFF = gate, which idles every later draft pass of the step.  Where the step is a CUDA
+// graph whose later draft passes are conditional nodes, next_pass is the handle of the next
+// pass's node (0: none): it is switched on only when this draft is kept.
 __global__ void __launch_bounds__(256)
 argmax_finish_kernel(const ValIdx* __restrict__ cand, int n_cand, int cand_stride,
                      int32_t* __restrict__ tok_out, int32_t* ctl, const float* __restrict__ second,
-                     float min_margin, int gate)
+                     float min_margin, int gate, unsigned long long next_pass)
 {
     __shared__ float sv[256];
     __shared__ float s2[256];
@@ -640,7 +642,13 @@ argmax_finish_kernel(const ValIdx* __restrict__ cand, int n_cand, int cand_strid
     }
     if (threadIdx.x == 0) {
         tok_out[m] = bi;
-        if (second && ctl && m == 0 && bv - bs < min_margin && gate < ctl[CTL_D_EFF]) ctl[CTL_D_EFF] = gate;
+        if (second && ctl && m == 0) {
+            if (bv - bs < min_margin) {
+                if (gate < ctl[CTL_D_EFF]) ctl[CTL_D_EFF] = gate;
+            } else if (next_pass) {
+                cudaGraphSetConditional((cudaGraphConditionalHandle)next_pass, 1);
+            }
+        }
     }
 }
 
