@@ -663,6 +663,7 @@ int get_graph(ls_model* m, int E, int d, bool reuse, float min_margin, ls_model:
         ((uint64_t)(reuse ? 0 : 1) << 48) | ((uint64_t)E << 32) | ((uint64_t)d << 16) | (uint64_t)m->grid_chunks, mbits);
     auto it = m->graphs.find(key);
     if (it == m->graphs.end()) {
+        if (m->graphs.size() >= 64) drop_graphs(m);  // a bound on what a long-lived handle keeps
         cudaGraph_t graph = nullptr;
         int64_t before = m->launches;
         cudaError_t e = cudaSuccess;
@@ -717,10 +718,7 @@ void set_grid_chunks(ls_model* m, int max_pos_exclusive)
     int g = (max_pos_exclusive + kAttnChunk - 1) / kAttnChunk;
     if (g > m->chunk_cap) g = m->chunk_cap;
     if (g < 1) g = 1;
-    if (g != m->grid_chunks) {
-        m->grid_chunks = g;
-        drop_graphs(m);
-    }
+    m->grid_chunks = g;  // part of the graph key: graphs captured for another chunk count stay valid
 }
 
 int decode_loop(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new, int32_t flags, float min_margin);
