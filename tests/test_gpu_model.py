@@ -336,6 +336,25 @@ def test_boundary_error_codes():
     assert e.value.status == B.LS_ERR_CAPACITY
 
 
+@pytest.mark.parametrize("path", PATHS)
+def test_exactly_at_kv_capacity(path):
+    """n_prompt + max_new + d + 1 == max_seq: the last step's rows reach the last cache
+    position (the chunked attention's last, partly filled chunk; page 3 of 4 pages of 16)."""
+    d = 3
+    gm, _ = make_pair(TINY.shape, TINY.weight_seed, 2, TINY.late_scale, 64, page_size=16, max_draft=d,
+                      linear_path=path, oracle=False)
+    prompt = synth.make_prompt(TINY.shape.vocab, 20, 6)
+    full = gm.generate_full(prompt, 40)
+    ids, acc = gm.generate(prompt, 2, d, 40)          # 20 + 40 + 3 + 1 = 64
+    np.testing.assert_array_equal(ids, full)
+    ids, acc, kept = gm.generate_adaptive(prompt, 2, d, 0.05, 40)
+    np.testing.assert_array_equal(ids, full)
+    with pytest.raises(B.LsError) as e:
+        gm.generate(prompt, 2, d, 41)
+    assert e.value.status == B.LS_ERR_CAPACITY
+    assert len(gm.generate_full(prompt, 43)) == 43    # 20 + 43 + 1 = 64 for plain greedy
+
+
 # ------------------------------------------------------------------ Llama-2-7B shape
 @pytest.fixture(scope="module")
 def llama7b():
