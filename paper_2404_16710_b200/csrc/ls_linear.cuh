@@ -595,16 +595,20 @@ inline cudaError_t launch_linear_fma(const LinArgs& a, const LaunchCtx& lc)
 
 // A row's bits depend on how K is split over the warps of its tile, and on nothing else.
 // So the warps per tile come from the matrix shape alone (never from M):
-//   few row tiles (N = 4096)  -> 16 warps, 4 stages (2 CTAs per SM, all tiles in one wave)
-//   otherwise                 -> 8 warps, 6 stages (3 CTAs per SM)
-// while the tiles per CTA may follow the pass size: with the second token tile (M > 8) and
-// many row tiles (gate-up, LM head) a CTA takes two tiles (4 stages, 2 CTAs per SM).
+//   few row tiles (N = 4096)  -> 16 warps, 4 stages (3 with two token tiles), 2 CTAs per SM,
+//                                all tiles in one wave
+//   otherwise                 -> 8 warps, 6 stages (4 with two token tiles), 3 CTAs per SM
+// while the tiles per CTA may follow the pass size: from 6 rows on, where the token rows are
+// a third or more of what a tile pulls through L1, a CTA of a matrix with many row tiles
+// (gate-up, LM head) takes two tiles with 3 stages (still 3 CTAs per SM) and uses its token
+// fragments for both.  Measured on the 7B shape: gate-up 32.5 -> 31.6 us at 7 rows,
+// 36.4 -> 33.3 us at 9 rows; below 6 rows the single tile with the deeper ring is faster.
 inline bool mma_wide(int epi, int N, int K)
 {
     const int tiles = lin_grid(epi, N), nsteps = (K + 31) / 32;
     return tiles < 600 && nsteps >= 16;
 }
-inline bool mma_pair(int epi, int N, int K, int M) { return M > 8 && !mma_wide(epi, N, K) && lin_grid(epi, N) >= 1200; }
+inline bool mma_pair(int epi, int N, int K, int M) { return M >= 6 && !mma_wide(epi, N, K) && lin_grid(epi, N) >= 1200; }
 // CTAs the MMA family launches for this matrix (also the number of argmax candidates per row)
 inline int mma_grid(int epi, int N, int K, int M)
 {
@@ -635,10 +639,11 @@ template <int EPI>
 inline cudaError_t launch_linear_mma(const LinArgs& a, const LaunchCtx& lc)
 {
     if (mma_wide(EPI, a.N, a.K))
-        return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 1, 16, 4>(a, lc) : launch_linear_mma_cfg<2, EPI, 1, 16, 4>(a, lc);
+        return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 1, 16, 4>(a, lc) : launch_linear_mma_cfg<2, EPI, 1, 16, 3>(a, lc);
+    if (mma_pair(EPI, a.N, a.K, a.M))
+        return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 2, 8, 3>(a, lc) : launch_linear_mma_cfg<2, EPI, 2, 8, 3>(a, lc);
     if (a.M <= 8) return launch_linear_mma_cfg<1, EPI, 1, 8, 6>(a, lc);
-    if (mma_pair(EPI, a.N, a.K, a.M)) return launch_linear_mma_cfg<2, EPI, 2, 8, 4>(a, lc);
-    return launch_linear_mma_cfg<2, EPI, 1, 8, 6>(a, lc);
+    return launch_linear_mma_cfg<2, EPI, 1, 8, 4>(a, lc);
 }
 
 // path: 1 = FMA, 2 = MMA
