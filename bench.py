@@ -41,7 +41,7 @@ ADAPTIVE_MARGINS = (0.02, 0.05, 0.1, 0.2, 0.4)
 # DRAM bytes (read + write) of one launch of the roofline kernel, from the ncu capture that
 # profiles/linear_mma_kernel_llama2-7b_shapes.md summarises; keyed by (workload, rows).  Set an
 # entry to None when the kernel changes until the counters have been taken again.
-ROOFLINE_TRAFFIC = {("llama2-7b", 7): 180.44e6 + 4.06e6}
+ROOFLINE_TRAFFIC = {("llama2-7b", 7): 180.45e6 + 4.05e6}
 
 
 def peaks():
