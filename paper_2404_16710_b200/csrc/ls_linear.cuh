@@ -599,16 +599,17 @@ inline cudaError_t launch_linear_fma(const LinArgs& a, const LaunchCtx& lc)
 //                                all tiles in one wave
 //   otherwise                 -> 8 warps, 6 stages (4 with two token tiles), 3 CTAs per SM
 // while the tiles per CTA may follow the pass size: from 6 rows on, where the token rows are
-// a third or more of what a tile pulls through L1, a CTA of a matrix with many row tiles
-// (gate-up, LM head) takes two tiles with 3 stages (still 3 CTAs per SM) and uses its token
-// fragments for both.  Measured on the 7B shape: gate-up 32.5 -> 31.6 us at 7 rows,
-// 36.4 -> 33.3 us at 9 rows; below 6 rows the single tile with the deeper ring is faster.
+// a third or more of what a tile pulls through L1, a CTA of a matrix with 700 or more row
+// tiles (q|k|v, gate-up, LM head on the 7B shape) takes two tiles with 3 stages (still 3 CTAs
+// per SM) and uses its token fragments for both.  Measured on the 7B shape: gate-up 32.5 ->
+// 31.6 us and q|k|v 20.8 -> 19.4 us at 7 rows, 36.4 -> 33.3 us and 22.5 -> 20.2 us at 9 rows;
+// below 6 rows the single tile with the deeper ring is faster.
 inline bool mma_wide(int epi, int N, int K)
 {
     const int tiles = lin_grid(epi, N), nsteps = (K + 31) / 32;
     return tiles < 600 && nsteps >= 16;
 }
-inline bool mma_pair(int epi, int N, int K, int M) { return M >= 6 && !mma_wide(epi, N, K) && lin_grid(epi, N) >= 1200; }
+inline bool mma_pair(int epi, int N, int K, int M) { return M >= 6 && !mma_wide(epi, N, K) && lin_grid(epi, N) >= 700; }
 // CTAs the MMA family launches for this matrix (also the number of argmax candidates per row)
 inline int mma_grid(int epi, int N, int K, int M)
 {
