@@ -428,6 +428,15 @@ int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* 
         LS_CK(cudaFuncSetAttribute(gemm_bf16_tn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes));
         if (dev >= 0 && dev < 64) allowed[dev] = true;
     }
+    // more than one tile of rows: CTA pairs share each weight tile (a CTA stages half of it)
+    static const bool pairs_allowed = getenv("LS_NO_PAIR") == nullptr;
+    const bool pair = pairs_allowed && M > kGemmBM;
+    static bool pair_allowed[64] = {false};
+    if (pair && (dev < 0 || dev >= 64 || !pair_allowed[dev])) {
+        LS_CK(cudaFuncSetAttribute(gemm_bf16_tn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)kPairSmemBytes));
+        if (dev >= 0 && dev < 64) pair_allowed[dev] = true;
+    }
     CUtensorMap ma, mb[3];
     LS_TRY(make_tile_map(&ma, A, (uint64_t)M, (uint64_t)K, kGemmBM));
     const uint16_t* bs[3] = {B0, B1 ? B1 : B0, B2 ? B2 : B0};
@@ -435,10 +444,28 @@ int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* 
     int tiles = 0;
     for (int i = 0; i < 3; ++i) {
         const int rows = segs.n[i] > 0 ? segs.n[i] : n0;  // an unused slot still gets a valid map
-        LS_TRY(make_tile_map(&mb[i], bs[i], (uint64_t)rows, (uint64_t)K, kGemmBN));
+        LS_TRY(make_tile_map(&mb[i], bs[i], (uint64_t)rows, (uint64_t)K, pair ? kGemmBN / 2 : kGemmBN));
         tiles += (segs.n[i] + kGemmBN - 1) / kGemmBN;
     }
-    dim3 grid(tiles, (M + kGemmBM - 1) / kGemmBM);
+    const int mtiles = (M + kGemmBM - 1) / kGemmBM;
+    if (pair) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((mtiles + 1) & ~1, tiles);
+        cfg.blockDim = dim3(128);
+        cfg.dynamicSmemBytes = kPairSmemBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute at;
+        at.id = cudaLaunchAttributeClusterDimension;
+        at.val.clusterDim.x = 2;
+        at.val.clusterDim.y = 1;
+        at.val.clusterDim.z = 1;
+        cfg.attrs = &at;
+        cfg.numAttrs = 1;
+        LS_CK(cudaLaunchKernelEx(&cfg, gemm_bf16_tn_pair_kernel, ma, mb[0], mb[1], mb[2], segs, M, K, C, ldc, accumulate,
+                                 status));
+        return LS_OK;
+    }
+    dim3 grid(tiles, mtiles);
     gemm_bf16_tn_kernel<<<grid, 128, kGemmSmemBytes, st>>>(ma, mb[0], mb[1], mb[2], segs, M, K, C, ldc, accumulate, status);
     LS_CK(cudaGetLastError());
     return LS_OK;

@@ -247,6 +247,194 @@ gemm_bf16_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kGemmBN) : "memory");
 }
 
+// ------------------------------------------------------------------ the same GEMM on CTA pairs
+// Two CTAs of a cluster (2 x 1 x 1: neighbours along M) compute one 256 x 256 tile with
+// tcgen05.mma.cta_group::2: each CTA stages its own 128 rows of A and HALF of the weight tile
+// (128 of the 256 rows of B), the leader CTA (cluster rank 0) issues the MMAs, which read both
+// CTAs' shared memory and write each CTA's 128 x 256 accumulator into its own tensor memory.
+// A weight byte is fetched from L2 once per 256 output rows instead of once per 128, so the
+// operand traffic per flop is two thirds of the single-CTA kernel's.
+//   - both CTAs' TMA loads signal the LEADER's full barrier (the .cta_group::2 form of the load;
+//     the barrier address with the peer bit cleared), on which the leader expects both shares;
+//   - tcgen05.commit multicasts to the barrier at the same offset in both CTAs (stage free,
+//     accumulator ready);
+//   - tensor memory is allocated and freed with the .cta_group::2 forms by warp 0 of both CTAs,
+//     and the two CTAs meet at a cluster barrier after the barrier set-up and before freeing
+//     (a CTA's shared memory must outlive the MMAs that read it).
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = (kGemmBM + kGemmBN / 2) * kGemmBK * 2;                    // 32 KB per CTA
+constexpr size_t kPairSmemBytes = (size_t)kPairStages * kPairStageBytes + 1024 + 256;
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;  // shared::cluster address of the pair's even CTA
+
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t leader_bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(leader_bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)  // arrives on `bar` in both CTAs of the pair
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+}
+
+// grid (M tiles of 128 rounded up to even, column tiles of 256 of all matrices), cluster (2, 1, 1),
+// block 128; roles as in gemm_bf16_tn_kernel, the MMA issuer only in the leader CTA.
+__global__ void __launch_bounds__(128)
+gemm_bf16_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
+                         const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
+                         const GemmSegs segs, int M, int K, float* __restrict__ C, int ldc, int accumulate,
+                         int32_t* status)
+{
+    extern __shared__ unsigned char gsm_raw[];
+    const uint32_t base = (smem_u32(gsm_raw) + 1023u) & ~1023u;
+    const uint32_t bars = base + kPairStages * kPairStageBytes;  // full[S], empty[S], accum, tmem slot
+    auto full = [&](int s) { return bars + 8u * s; };
+    auto empty = [&](int s) { return bars + 8u * (kPairStages + s); };
+    const uint32_t accum = bars + 8u * (2 * kPairStages);
+    const uint32_t tslot = accum + 8u;
+    __shared__ int failed;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint32_t rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int m0 = blockIdx.x * kGemmBM;  // the pair: blockIdx.x = 2p, 2p + 1
+    const CUtensorMap* map_b = &map_b0;
+    int N = segs.n[0], n0 = blockIdx.y * kGemmBN, col0 = 0;
+    {
+        const int t0 = (segs.n[0] + kGemmBN - 1) / kGemmBN, t1 = (segs.n[1] + kGemmBN - 1) / kGemmBN;
+        if ((int)blockIdx.y >= t0 + t1) {
+            map_b = &map_b2;
+            N = segs.n[2];
+            n0 = ((int)blockIdx.y - t0 - t1) * kGemmBN;
+            col0 = segs.n[0] + segs.n[1];
+        } else if ((int)blockIdx.y >= t0) {
+            map_b = &map_b1;
+            N = segs.n[1];
+            n0 = ((int)blockIdx.y - t0) * kGemmBN;
+            col0 = segs.n[0];
+        }
+    }
+    const int nkb = (K + kGemmBK - 1) / kGemmBK;
+    if (tid == 0) {
+        for (int s = 0; s < kPairStages; ++s) {
+            mbar_init(full(s), 1);
+            mbar_init(empty(s), 1);
+        }
+        mbar_init(accum, 1);
+        failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tslot), "r"(kGemmBN)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the peer's barriers exist before anything signals them
+    tc_fence_after();
+    uint32_t tmem;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem) : "r"(tslot));
+
+    if (warp == 0 && lane == 0) {  // TMA producer of this CTA's share
+        for (int kb = 0; kb < nkb; ++kb) {
+            const int s = kb % kPairStages;
+            if (kb >= kPairStages && !mbar_wait(empty(s), ((kb / kPairStages) - 1) & 1)) {
+                failed = 1;
+                break;
+            }
+            if (rank == 0) mbar_expect_tx(full(s), 2 * kPairStageBytes);
+            const uint32_t sa = base + s * kPairStageBytes, sb = sa + kGemmBM * kGemmBK * 2;
+            const uint32_t lead = full(s) & kPeerBitMask;
+            tma_load_2d_pair(sa, &map_a, kb * kGemmBK, m0, lead);
+            tma_load_2d_pair(sb, map_b, kb * kGemmBK, n0 + (int)rank * (kGemmBN / 2), lead);
+        }
+    } else if (rank == 0 && warp == 1 && lane == 0) {  // MMA issuer: the leader CTA only
+        // instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 256 (128 per CTA)
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kGemmBN >> 3) << 17) |
+                               ((uint32_t)((2 * kGemmBM) >> 4) << 24);
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int s = kb % kPairStages;
+            if (!mbar_wait(full(s), (kb / kPairStages) & 1)) {
+                failed = 1;
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const uint32_t sa = base + s * kPairStageBytes, sb = sa + kGemmBM * kGemmBK * 2;
+            const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sb);
+#pragma unroll
+            for (int k4 = 0; k4 < kGemmBK / 16; ++k4)
+                tc_mma_bf16_pair(tmem, da + 2 * k4, db + 2 * k4, idesc, (kb | k4) != 0);
+            tc_commit_pair(empty(s));
+        }
+        if (ok) tc_commit_pair(accum);
+    }
+    __syncwarp();
+
+    // epilogue: warp w of each CTA owns its accumulator lanes 32w..32w+31 = rows m0 + 32w + lane
+    bool have = mbar_wait(accum, 0);
+    if (!have) failed = 1;
+    tc_fence_after();
+    __syncthreads();
+    if (!failed) {
+        const int row = m0 + warp * 32 + lane;
+#pragma unroll 1
+        for (int c = 0; c < kGemmBN / 32; ++c) {
+            uint32_t v[32];
+            tc_ld32(tmem + ((uint32_t)(warp * 32) << 16) + c * 32, v);
+            if (row < M) {
+                float* dst = C + (size_t)row * ldc + col0 + n0 + c * 32;
+                if (n0 + c * 32 + 32 <= N && (((uintptr_t)dst) & 15u) == 0) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                               __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                        if (accumulate) {
+                            const float4 p = *reinterpret_cast<const float4*>(dst + j);
+                            o.x += p.x;
+                            o.y += p.y;
+                            o.z += p.z;
+                            o.w += p.w;
+                        }
+                        *reinterpret_cast<float4*>(dst + j) = o;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (n0 + c * 32 + j < N) dst[j] = accumulate ? dst[j] + __uint_as_float(v[j]) : __uint_as_float(v[j]);
+                }
+            }
+        }
+    } else if (tid == 0 && status) {
+        *status = DEV_TIMEOUT;
+        __nanosleep(1000000);  // let copies that may still be in flight land before the CTA goes away
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // both CTAs are done with tensor memory, and the MMAs with both shared memories
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kGemmBN) : "memory");
+}
+
 // ------------------------------------------------------------------ elementwise helpers of the prompt pass
 // a[m, f] = bf16(silu(gu[m, f]) * gu[m, F + f]); grid (rows), block 256; four features per
 // thread and step when F allows 16-byte accesses
