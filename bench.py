@@ -305,7 +305,7 @@ def run_own(args):
                       "num_draft": d, "late_scale": wl.late_scale, "linear_path": "mma" if path == 2 else "fma",
                       "l2": "inputs (weights) larger than L2", "replicas": world,
                       "timed_region": "decode loop from a prefilled prompt, device-resident",
-                      "kernels_per_layer": 5, "prompt_pass": "tcgen05 GEMM 128x256 tiles, blocks of 1024 rows"},
+                      "kernels_per_layer": 5, "prompt_pass": "tcgen05 cta_group::2 GEMM, 256x256 tiles on CTA pairs, blocks of 1024 rows"},
            "e2e": e2e, "gpu_launches": int(launches), "clocks": clk.summary,
            "accepted_per_step": float(acc.mean()), "acceptance_rate": float(acc.mean() / d),
            "emitted_per_step": float(NEW / len(acc)), "spec_steps": int(len(acc)), "host_syncs": int(st.host_syncs),
