@@ -187,6 +187,13 @@ int ls_read_drafted(ls_model *m, int32_t *drafted_per_step_host, int32_t *out_n_
 int ls_debug_logits(ls_model *m, const int32_t *ids_host, int32_t n, int32_t exit_layer,
                     float *exit_logits_host, float *final_logits_host);
 
+/* Logits of the next token after ls_prefill (all layers): the last prompt token is run
+ * through the model on top of the cache the prompt pass has left, g(x_L) goes to
+ * logits_host (fp32 [V]).  For parity checks of the prompt pass itself: every layer's cached
+ * k, v of every prompt position enters these logits.  The loop state is left as ls_prefill
+ * left it (ls_decode may follow). */
+int ls_debug_next_logits(ls_model *m, float *logits_host);
+
 int ls_get_stats(const ls_model *m, ls_stats *out);
 
 /* ------------------------------------------------------------------------------

@@ -24,7 +24,7 @@ LS_LINEAR_AUTO, LS_LINEAR_FMA, LS_LINEAR_MMA = 0, 1, 2
 EXPORTS = (
     "ls_strerror", "ls_last_cuda_error", "ls_workspace_bytes", "ls_model_create", "ls_model_destroy",
     "ls_set_page_table", "ls_generate", "ls_generate_adaptive", "ls_generate_full", "ls_generate_early", "ls_prefill",
-    "ls_decode", "ls_decode_flags", "ls_decode_adaptive", "ls_read_output", "ls_read_drafted", "ls_debug_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
+    "ls_decode", "ls_decode_flags", "ls_decode_adaptive", "ls_read_output", "ls_read_drafted", "ls_debug_logits", "ls_debug_next_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
     "ls_op_linear", "ls_op_gate_up_swiglu", "ls_op_lm_head_scratch_bytes", "ls_op_lm_head_argmax",
     "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_qkv_rope_append", "ls_op_attention_scratch_bytes", "ls_op_attention", "ls_op_accept",
     "ls_op_gemm", "ls_op_prefill_attention",
@@ -93,6 +93,7 @@ def lib():
             "ls_decode_adaptive": (C.c_int, [vp, i32, i32, C.c_float, i32]),
             "ls_read_drafted": (C.c_int, [vp, ip, ip]),
             "ls_debug_logits": (C.c_int, [vp, ip, i32, i32, fp, fp]),
+            "ls_debug_next_logits": (C.c_int, [vp, fp]),
             "ls_get_stats": (C.c_int, [vp, C.POINTER(ls_stats)]),
             "ls_op_embed": (C.c_int, [vp, vp, i32, i32, i32, vp, vp]),
             "ls_op_rmsnorm": (C.c_int, [vp, vp, i32, i32, C.c_float, vp, vp]),
@@ -253,6 +254,13 @@ def ls_read_output(h, max_new):
     _ck(lib().ls_read_output(h, out.ctypes.data_as(C.POINTER(C.c_int32)), C.byref(n),
                              acc.ctypes.data_as(C.POINTER(C.c_int32)), C.byref(s)), "ls_read_output")
     return out[:n.value], acc[:s.value]
+
+
+def ls_debug_next_logits(h, vocab):
+    """after ls_prefill: final logits of the last prompt token on top of the prompt pass's cache"""
+    out = np.empty(vocab, np.float32)
+    _ck(lib().ls_debug_next_logits(h, out.ctypes.data_as(C.POINTER(C.c_float))), "ls_debug_next_logits")
+    return out
 
 
 def ls_debug_logits(h, ids, exit_layer, vocab, want_exit=True, want_final=True):

@@ -1183,6 +1183,22 @@ int ls_debug_logits(ls_model* m, const int32_t* ids, int32_t n, int32_t exit_lay
     return w[CTL_STATUS] ? LS_ERR_DEVICE_STATUS : LS_OK;
 }
 
+int ls_debug_next_logits(ls_model* m, float* logits)
+{
+    if (!m || !logits || m->n_prompt < 1 || m->prefilled_layers < m->c.n_layers) return LS_ERR_INVALID_ARG;
+    const ls_config& c = m->c;
+    if (m->n_prompt + 1 > c.max_seq) return LS_ERR_CAPACITY;
+    set_grid_chunks(m, m->n_prompt + 1);
+    LS_TRY(write_ctl(m, m->n_prompt - 1, m->last_tok, 1));
+    LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
+    LS_TRY(run_layers(m, 0, c.n_layers, 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
+    LS_TRY(run_head(m, 1, 0, m->verified, m->logits));
+    LS_CK(cudaMemcpyAsync(logits, m->logits, sizeof(float) * (size_t)c.vocab, cudaMemcpyDeviceToHost, m->st));
+    int32_t w[CTL_WORDS];
+    LS_TRY(read_ctl(m, w));
+    return w[CTL_STATUS] ? LS_ERR_DEVICE_STATUS : LS_OK;
+}
+
 int ls_get_stats(const ls_model* m, ls_stats* out)
 {
     if (!m || !out) return LS_ERR_INVALID_ARG;

@@ -192,7 +192,7 @@ def test_odd_shapes_logits_and_losslessness(shape, path):
     """Shapes whose sizes are not multiples of the tiles: logits against the oracle (16-row
     passes), then a 45-token prompt (tensor-core prompt pass) with every loop giving the ids
     of full greedy, which in turn follow the oracle while its margins allow."""
-    gm, om = make_pair(shape, 5, 1, 0.3, 128, page_size=16, max_draft=6, linear_path=path, amplify=6.0)
+    gm, om = make_pair(shape, 5, 1, 0.3, 256, page_size=16, max_draft=6, linear_path=path, amplify=6.0)
     ids = synth.make_prompt(shape.vocab, 37, 3)
     gex, gfi = gm.debug_logits(ids, 1)
     oex, ofi = om.teacher_logits(ids, 1)
@@ -211,6 +211,45 @@ def test_odd_shapes_logits_and_losslessness(shape, path):
     k = first_low_margin(margins, maxabs)
     np.testing.assert_array_equal(full[:k], ref[:k])
     print(f"{shape.name} path {path}: ids follow the oracle for {k} of 40 tokens")
+    # a prompt of more than 128 rows: the prompt GEMMs run on CTA pairs (second row tile ragged),
+    # and the first token after it must be the oracle's wherever its margin allows
+    long_prompt = synth.make_prompt(shape.vocab, 150, 9)
+    full = gm.generate_full(long_prompt, 24)
+    got, acc = gm.generate(long_prompt, 1, 3, 24)
+    np.testing.assert_array_equal(got, full)
+    ref, margins, maxabs = om.generate_full(long_prompt, 24)
+    k = first_low_margin(margins, maxabs)
+    np.testing.assert_array_equal(full[:k], ref[:k])
+    print(f"{shape.name} path {path}: after a 150-token prompt the ids follow the oracle for {k} of 24 tokens")
+
+
+# ------------------------------------------------------------------ the prompt pass itself
+def _two_layers(shape, name):
+    from dataclasses import replace
+    return replace(shape, name=name, n_layers=2)
+
+
+PROMPT_CASES = [(TINY.shape, 100, None), (ODD_SHAPES[0], 150, 6.0), (ODD_SHAPES[1], 150, 6.0), (ODD_SHAPES[2], 150, 6.0),
+                (ODD_SHAPES[3], 150, 6.0), (_two_layers(synth.LLAMA2_7B, "7b-2-layers"), 300, None),
+                (_two_layers(synth.LLAMA3_8B, "8b-2-layers"), 200, None)]
+
+
+@pytest.mark.parametrize("shape,n_prompt,amp", PROMPT_CASES, ids=lambda v: getattr(v, "name", str(v)))
+def test_prompt_pass_cache_gives_the_oracle_logits(shape, n_prompt, amp):
+    """Next-token logits computed on top of the cache the prompt pass has left (tensor-core GEMMs
+    on one CTA up to 128 rows and on CTA pairs beyond, several weight matrices per launch,
+    flash-attention-style causal attention, row-wise RoPE + append) against the oracle's
+    teacher-forced final logits at the last prompt position."""
+    gm, om = make_pair(shape, 5, 1, 0.3, n_prompt + 8, page_size=64, max_draft=4, amplify=amp)
+    prompt = synth.make_prompt(shape.vocab, n_prompt, 12)
+    B.ls_prefill(gm.h, prompt)
+    got = B.ls_debug_next_logits(gm.h, shape.vocab)
+    _, ref = om.teacher_logits(prompt, 1)
+    r = assert_logits_close(got, ref[-1], "next-token logits after the prompt pass")
+    # and the 16-row passes give the same thing within the same tolerance
+    _, small = gm.debug_logits(prompt, 1, want_exit=False)
+    assert_logits_close(small[-1], ref[-1], "next-token logits through 16-row passes")
+    print(f"{shape.name} prompt {n_prompt}: max|delta|/max|logit| {r:.2e}")
 
 
 # ------------------------------------------------------------------ adaptive draft length
