@@ -284,13 +284,14 @@ int ls_op_attention(const void *q_bf16_dev, int32_t M, int32_t pos0, int32_t Hq,
 
 /* Kernels of the prompt pass (the rows that go through the model before the first draft,
  * Appendix A.4), which is a dense contraction over hundreds of rows.
- * ls_op_gemm: c[m, n] (+)= sum_k a[m, k] b[n, k] on the tcgen05 tensor cores; a bf16 [M, K],
- * b bf16 [N, K], c fp32 with leading dimension ldc >= N; accumulate != 0 adds to c (the
- * residual update of Sec. 4.1).  status_dev (device int32, may be NULL) receives 3 if one of
- * the kernel's bounded waits ran out.
+ * ls_op_gemm: c[m, n] (+)= sum_k a[m, k] b[n, k] on the tcgen05 tensor cores (up to 128 rows
+ * one CTA per 128 x 256 tile, beyond that pairs of CTAs per 256 x 256 tile); a bf16 [M, K],
+ * b bf16 [N, K], K a multiple of 8, both 16-byte aligned; c fp32 with leading dimension
+ * ldc >= N; accumulate != 0 adds to c (the residual update of Sec. 4.1).  status_dev (device
+ * int32, may be NULL) receives 3 if one of the kernel's bounded waits ran out.
  * ls_op_prefill_attention: causal attention of R rows at positions pos0 .. pos0+R-1 over the
- * paged cache (as ls_op_attention, any R, no scratch: one CTA walks the key chunks of its 16
- * rows in order with a running max / sum). */
+ * paged cache (as ls_op_attention, any R, no scratch: a CTA walks the key chunks of its rows
+ * in order with a running max / sum per row). */
 int ls_op_gemm(const void *a_bf16_dev, const void *b_bf16_dev, int32_t M, int32_t N, int32_t K,
                float *c_dev, int32_t ldc, int32_t accumulate, int32_t *status_dev, void *cuda_stream);
 int ls_op_prefill_attention(const void *q_bf16_dev, int32_t R, int32_t pos0, int32_t Hq, int32_t Hkv,
