@@ -94,6 +94,48 @@ def op_cases(shape, w, path, M, n_ctx=1030):
     }
 
 
+PROMPT_OPS = ("prompt_gemm_qkv", "prompt_gemm_gate", "prompt_gemm_down", "prompt_attention")
+
+
+def prompt_cases(shape, w, R):
+    """Kernels of the prompt pass on R rows: name -> (callable(layer index), flops per launch, distinct weights).
+    The GEMMs are the projections of one block of rows; attention is causal over the R rows themselves."""
+    D, F = shape.d_model, shape.d_ffn
+    L = len(w["wq"])
+    Hq, Hkv, hd, ps = shape.n_heads, shape.n_kv_heads, shape.head_dim, 64
+    qw, kvw = Hq * hd, Hkv * hd
+    g = torch.Generator(device="cuda").manual_seed(11)
+    h = torch.randn((R, D), device="cuda", generator=g).bfloat16()
+    a = torch.randn((R, F), device="cuda", generator=g).bfloat16()
+    wqkv = [torch.cat([w["wq"][i], w["wk"][i], w["wv"][i]]) for i in range(L)]
+    cq = torch.empty((R, qw + 2 * kvw), dtype=torch.float32, device="cuda")
+    cf = torch.empty((R, F), dtype=torch.float32, device="cuda")
+    cd = torch.zeros((R, D), dtype=torch.float32, device="cuda")
+    n_pages = -(-(R + 1) // ps)
+    kp = torch.randn((n_pages, Hkv, ps, hd), device="cuda", generator=g).bfloat16()
+    vp = torch.randn((n_pages, Hkv, ps, hd), device="cuda", generator=g).bfloat16()
+    table = torch.arange(n_pages, dtype=torch.int32, device="cuda")
+    q = (torch.randn((R, qw), device="cuda", generator=g) * 0.3).bfloat16()
+    ao = torch.empty((R, qw), dtype=torch.bfloat16, device="cuda")
+    return {
+        "prompt_gemm_qkv": (lambda i: B.ls_op_gemm(h, wqkv[i % L], cq), 2 * R * (qw + 2 * kvw) * D, L),
+        "prompt_gemm_gate": (lambda i: B.ls_op_gemm(h, w["w_gate"][i % L], cf), 2 * R * F * D, L),
+        "prompt_gemm_down": (lambda i: B.ls_op_gemm(a, w["w_down"][i % L], cd, True), 2 * R * D * F, L),
+        "prompt_attention": (lambda i: B.ls_op_prefill_attention(q, 0, Hq, Hkv, hd, ps, table, n_pages * ps, kp, vp, ao),
+                             4 * Hq * hd * R * (R + 1) // 2, 1),
+    }
+
+
+def prompt_rates(shape, w, R, ops=PROMPT_OPS, iters=20, warm=3):
+    out = {}
+    cases = prompt_cases(shape, w, R)
+    for name in ops:
+        fn, flops, rot = cases[name]
+        ms = time_op(fn, rot, iters, warm)
+        out[f"{name}@R={R}"] = {"ms": round(ms, 5), "TFLOP/s": round(flops / ms / 1e9, 1), "flops": flops}
+    return out
+
+
 def kernel_rooflines(shape, w, path, rows, peak_gbs, ops=OPS, iters=40, warm=5):
     out = {}
     for M in rows:
@@ -116,12 +158,22 @@ def main():
     ap.add_argument("--iters", type=int, default=40)
     ap.add_argument("--warm", type=int, default=5)
     ap.add_argument("--peak", type=float, default=6553.9, help="GB/s the fractions are quoted against")
+    ap.add_argument("--prompt-rows", type=int, default=0, metavar="R",
+                    help="instead: the prompt pass's GEMMs and attention on R rows (TFLOP/s); --ops picks among "
+                         + ", ".join(PROMPT_OPS))
     a = ap.parse_args()
     from dataclasses import replace
     wl = synth.WORKLOADS[a.workload]
     shape = replace(wl.shape, n_layers=a.layers)
     w = synth.make_weights(shape, wl.weight_seed, wl.exit_layer, wl.late_scale, device="cuda")
     path = B.LS_LINEAR_MMA if a.path == "mma" else B.LS_LINEAR_FMA
+    if a.prompt_rows:
+        ops = [o for o in a.ops.split(",") if o in PROMPT_OPS] or list(PROMPT_OPS)
+        res = prompt_rates(shape, w, a.prompt_rows, ops, a.iters, a.warm)
+        for k, v in res.items():
+            print(f"{k:28s} {v['ms'] * 1e3:8.2f} us  {v['TFLOP/s']:8.1f} TFLOP/s")
+        print(json.dumps(res))
+        return
     res = kernel_rooflines(shape, w, path, [int(r) for r in a.rows.split(",")], a.peak,
                            [o for o in a.ops.split(",") if o], a.iters, a.warm)
     for k, v in res.items():
