@@ -137,6 +137,12 @@ def test_eos_stops_both_loops_at_the_same_token():
     s2, _ = gm2.generate(prompt, 2, 3, 40)
     np.testing.assert_array_equal(f2, full[:first + 1])
     np.testing.assert_array_equal(s2, f2)
+    for tau in (0.02, 0.2):  # the adaptive loop (conditional draft passes) stops at the same token
+        a2, acc, kept = gm2.generate_adaptive(prompt, 2, 3, tau, 40)
+        np.testing.assert_array_equal(a2, f2)
+        assert (acc <= kept).all()
+    # and a handle that has stopped early generates normally afterwards
+    np.testing.assert_array_equal(gm2.generate_full(prompt, 40), f2)
 
 
 def test_prefill_once_decode_many():
