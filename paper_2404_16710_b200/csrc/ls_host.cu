@@ -416,10 +416,19 @@ int make_tile_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, 
 }
 
 // C[M, N] (+)= A[M, K] B[N, K]^T on the tensor cores (tcgen05), A and B bf16, C fp32
+// more than one tile of rows: CTA pairs share each weight tile (a CTA stages half of it)
+bool gemm_uses_pairs(int M)
+{
+    static const bool allowed = getenv("LS_NO_PAIR") == nullptr;
+    return allowed && M > kGemmBM;
+}
+
 // C[M, n0 + n1 + n2] (+)= A[M, K] [B0; B1; B2]^T: up to three weight matrices with the same K
-// in one launch (B1, B2 may be null)
+// in one launch (B1, B2 may be null).  swiglu_out (CTA pairs only; B0 = gate, B1 = up, n0 == n1):
+// instead of C, bf16(silu(A B0^T) * (A B1^T)) [M, n0] is written.
 int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* B1, int n1, const uint16_t* B2, int n2,
-                 int M, int K, float* C, int ldc, int accumulate, int32_t* status, cudaStream_t st)
+                 int M, int K, float* C, int ldc, int accumulate, int32_t* status, cudaStream_t st,
+                 uint16_t* swiglu_out = nullptr)
 {
     static bool allowed[64] = {false};
     int dev = 0;
@@ -428,9 +437,7 @@ int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* 
         LS_CK(cudaFuncSetAttribute(gemm_bf16_tn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes));
         if (dev >= 0 && dev < 64) allowed[dev] = true;
     }
-    // more than one tile of rows: CTA pairs share each weight tile (a CTA stages half of it)
-    static const bool pairs_allowed = getenv("LS_NO_PAIR") == nullptr;
-    const bool pair = pairs_allowed && M > kGemmBM;
+    const bool pair = gemm_uses_pairs(M);
     static bool pair_allowed[64] = {false};
     if (pair && (dev < 0 || dev >= 64 || !pair_allowed[dev])) {
         LS_CK(cudaFuncSetAttribute(gemm_bf16_tn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -448,6 +455,8 @@ int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* 
         tiles += (segs.n[i] + kGemmBN - 1) / kGemmBN;
     }
     const int mtiles = (M + kGemmBM - 1) / kGemmBM;
+    if (swiglu_out && !pair) return LS_ERR_INVALID_ARG;  // the fused epilogue exists on CTA pairs only
+    if (swiglu_out) tiles = (n0 + kGemmBN / 2 - 1) / (kGemmBN / 2);
     if (pair) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((mtiles + 1) & ~1, tiles);
@@ -462,7 +471,7 @@ int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* 
         cfg.attrs = &at;
         cfg.numAttrs = 1;
         LS_CK(cudaLaunchKernelEx(&cfg, gemm_bf16_tn_pair_kernel, ma, mb[0], mb[1], mb[2], segs, M, K, C, ldc, accumulate,
-                                 status));
+                                 status, swiglu_out));
         return LS_OK;
     }
     dim3 grid(tiles, mtiles);
@@ -530,8 +539,12 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
         LS_TRY(prefill_attn_launch(m->pq, kp, vp, m->page_table, r0, R, Hq, Hkv, hd, m->page_shift, m->po, st));
         LS_TRY(gemm_launch(m->po, w.wo, R, D, qw, m->px, D, 1, status, st));
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.ffn_norm, D, c.rms_eps, m->ph, nullptr));
-        LS_TRY(gemm_launch3(m->ph, w.wg, F, w.wu, F, nullptr, 0, R, D, m->py, 2 * F, 0, status, st));
-        swiglu_rows_kernel<<<R, 256, 0, st>>>(m->py, F, m->pa);
+        if (gemm_uses_pairs(R)) {  // gate, up and SwiGLU in one kernel
+            LS_TRY(gemm_launch3(m->ph, w.wg, F, w.wu, F, nullptr, 0, R, D, m->py, 2 * F, 0, status, st, m->pa));
+        } else {
+            LS_TRY(gemm_launch3(m->ph, w.wg, F, w.wu, F, nullptr, 0, R, D, m->py, 2 * F, 0, status, st));
+            swiglu_rows_kernel<<<R, 256, 0, st>>>(m->py, F, m->pa);
+        }
         LS_TRY(gemm_launch(m->pa, w.wd, R, D, F, m->px, D, 1, status, st));
         m->launches += 13;
     }

@@ -300,7 +300,7 @@ __global__ void __launch_bounds__(128)
 gemm_bf16_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
                          const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
                          const GemmSegs segs, int M, int K, float* __restrict__ C, int ldc, int accumulate,
-                         int32_t* status)
+                         int32_t* status, uint16_t* __restrict__ swiglu_out)
 {
     extern __shared__ unsigned char gsm_raw[];
     const uint32_t base = (smem_u32(gsm_raw) + 1023u) & ~1023u;
@@ -331,6 +331,18 @@ gemm_bf16_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             col0 = segs.n[0];
         }
     }
+    // SwiGLU mode (swiglu_out != nullptr; B0 = gate, B1 = up, both [F, K]): the pair's weight tile is
+    // 128 gate rows (staged by the leader) beside the 128 up rows of the same features (staged by
+    // its peer), so the accumulator holds gate | up of 128 features and the epilogue writes
+    // bf16(silu(gate) * up) straight into the feed-forward input: no fp32 round trip through memory
+    const bool swiglu = swiglu_out != nullptr;
+    if (swiglu) {
+        map_b = rank ? &map_b1 : &map_b0;
+        N = segs.n[0];
+        n0 = blockIdx.y * (kGemmBN / 2);
+        col0 = 0;
+    }
+    const int b_row = swiglu ? n0 : n0 + (int)rank * (kGemmBN / 2);
     const int nkb = (K + kGemmBK - 1) / kGemmBK;
     if (tid == 0) {
         for (int s = 0; s < kPairStages; ++s) {
@@ -364,7 +376,7 @@ gemm_bf16_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             const uint32_t sa = base + s * kPairStageBytes, sb = sa + kGemmBM * kGemmBK * 2;
             const uint32_t lead = full(s) & kPeerBitMask;
             tma_load_2d_pair(sa, &map_a, kb * kGemmBK, m0, lead);
-            tma_load_2d_pair(sb, map_b, kb * kGemmBK, n0 + (int)rank * (kGemmBN / 2), lead);
+            tma_load_2d_pair(sb, map_b, kb * kGemmBK, b_row, lead);
         }
     } else if (rank == 0 && warp == 1 && lane == 0) {  // MMA issuer: the leader CTA only
         // instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 256 (128 per CTA)
@@ -395,7 +407,38 @@ gemm_bf16_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
     if (!have) failed = 1;
     tc_fence_after();
     __syncthreads();
-    if (!failed) {
+    if (!failed && swiglu) {
+        const int row = m0 + warp * 32 + lane;
+#pragma unroll 1
+        for (int c = 0; c < kGemmBN / 64; ++c) {  // 32 features at a time: gate columns c*32.., up columns 128 + c*32..
+            uint32_t gt[32], up[32];
+            tc_ld32(tmem + ((uint32_t)(warp * 32) << 16) + c * 32, gt);
+            tc_ld32(tmem + ((uint32_t)(warp * 32) << 16) + kGemmBN / 2 + c * 32, up);
+            if (row < M) {
+                uint16_t* dst = swiglu_out + (size_t)row * N + n0 + c * 32;
+                if (n0 + c * 32 + 32 <= N && (((uintptr_t)dst) & 15u) == 0) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float g0 = __uint_as_float(gt[j + 2 * e]), g1 = __uint_as_float(gt[j + 2 * e + 1]);
+                            pk[e] = pack_bf16(g0 / (1.0f + expf(-g0)) * __uint_as_float(up[j + 2 * e]),
+                                              g1 / (1.0f + expf(-g1)) * __uint_as_float(up[j + 2 * e + 1]));
+                        }
+                        *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (n0 + c * 32 + j < N) {
+                            const float g0 = __uint_as_float(gt[j]);
+                            dst[j] = f2bf(g0 / (1.0f + expf(-g0)) * __uint_as_float(up[j]));
+                        }
+                }
+            }
+        }
+    } else if (!failed) {
         const int row = m0 + warp * 32 + lane;
 #pragma unroll 1
         for (int c = 0; c < kGemmBN / 32; ++c) {
