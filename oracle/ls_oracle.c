@@ -267,24 +267,34 @@ static void lm_head(const lso_model *m, const double *x, double *logits)
 }
 
 /* Teacher-forced logits: feed ids[0..n-1] at positions 0..n-1; for every
- * position write g(x_E) to exit_logits[t] and g(x_L) to final_logits[t]
- * (each [n, V], either may be NULL).  exit_layer = E counts the early layers. */
-int32_t lso_teacher_logits(lso_model *m, const int32_t *ids, int32_t n, int32_t exit_layer,
-                           double *exit_logits, double *final_logits)
+ * position t >= first write g(x_E) to exit_logits[t - first] and g(x_L) to
+ * final_logits[t - first] (each [n - first, V], either may be NULL).  Positions
+ * below `first` go through all layers exactly as the others do (they fill the
+ * cache); only their logits are not asked for.  exit_layer = E counts the
+ * early layers. */
+int32_t lso_teacher_logits_tail(lso_model *m, const int32_t *ids, int32_t n, int32_t exit_layer,
+                                int32_t first, double *exit_logits, double *final_logits)
 {
     const lso_config *c = &m->c;
-    if (n > c->max_seq || exit_layer < 1 || exit_layer > c->n_layers) return -1;
+    if (n > c->max_seq || exit_layer < 1 || exit_layer > c->n_layers || first < 0 || first > n) return -1;
     double *x = (double *)malloc(sizeof(double) * (size_t)c->d_model);
     for (int t = 0; t < n; ++t) {
         if (ids[t] < 0 || ids[t] >= c->vocab) { free(x); return -1; }
         embed(m, ids[t], x);
         layers_token(m, 0, exit_layer, x, t);
-        if (exit_logits) lm_head(m, x, exit_logits + (size_t)t * c->vocab);
+        if (exit_logits && t >= first) lm_head(m, x, exit_logits + (size_t)(t - first) * c->vocab);
         layers_token(m, exit_layer, c->n_layers, x, t);
-        if (final_logits) lm_head(m, x, final_logits + (size_t)t * c->vocab);
+        if (final_logits && t >= first) lm_head(m, x, final_logits + (size_t)(t - first) * c->vocab);
     }
     free(x);
     return 0;
+}
+
+/* the same for every position */
+int32_t lso_teacher_logits(lso_model *m, const int32_t *ids, int32_t n, int32_t exit_layer,
+                           double *exit_logits, double *final_logits)
+{
+    return lso_teacher_logits_tail(m, ids, n, exit_layer, 0, exit_logits, final_logits);
 }
 
 /* Autoregressive greedy decoding with the full model (the result every other

@@ -74,6 +74,8 @@ def lib():
         L.lso_model_free.argtypes = [C.c_void_p]
         L.lso_teacher_logits.argtypes = [C.c_void_p, ip, i32, i32, dp, dp]
         L.lso_teacher_logits.restype = i32
+        L.lso_teacher_logits_tail.argtypes = [C.c_void_p, ip, i32, i32, i32, dp, dp]
+        L.lso_teacher_logits_tail.restype = i32
         L.lso_generate_full.argtypes = [C.c_void_p, ip, i32, i32, ip, ip, dp, dp]
         L.lso_generate_full.restype = i32
         L.lso_generate_early.argtypes = [C.c_void_p, ip, i32, i32, i32, ip, ip]
@@ -222,6 +224,20 @@ class Model:
                                       _dp(fi) if want_final else None)
         if rc:
             raise ValueError("lso_teacher_logits: bad arguments")
+        return ex, fi
+
+    def teacher_logits_tail(self, ids, exit_layer, first, want_exit=True, want_final=True):
+        """Teacher-forced logits of positions first .. len(ids)-1 only ([len(ids) - first, V]); the
+        earlier positions still run through every layer (they fill the cache)."""
+        ids = np.ascontiguousarray(ids, dtype=np.int32)
+        n, V = ids.size, self.cfg.vocab
+        ex = np.empty((n - first, V)) if want_exit else None
+        fi = np.empty((n - first, V)) if want_final else None
+        rc = lib().lso_teacher_logits_tail(self._h, _ip(ids), n, exit_layer, first,
+                                           _dp(ex) if want_exit else None,
+                                           _dp(fi) if want_final else None)
+        if rc:
+            raise ValueError("lso_teacher_logits_tail: bad arguments")
         return ex, fi
 
     def generate_full(self, prompt, max_new):

@@ -55,6 +55,21 @@ def test_cached_forward_equals_no_cache_recomputation(shape, E):
     assert np.abs(fi).max() > 0.1  # the comparison is not vacuous
 
 
+@pytest.mark.parametrize("first", [0, 5, 12, 13])
+def test_teacher_logits_tail_equals_no_cache_recomputation(first):
+    """Logits asked for the last positions only: the rows of the no-cache recomputation at those
+    positions (and the earlier positions still fill the cache: the rows would differ otherwise)."""
+    shape = synth.MICRO_GQA
+    m, cfg, w = oracle_model(shape, weights=loud_weights(shape))
+    ids = synth.make_prompt(shape.vocab, 13, 5)
+    ex, fi = m.teacher_logits_tail(ids, 2, first)
+    assert ex.shape == fi.shape == (13 - first, shape.vocab)
+    np.testing.assert_allclose(ex, B.logits_at(cfg, w, ids, 2)[first:], rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(fi, B.logits_at(cfg, w, ids, shape.n_layers)[first:], rtol=1e-9, atol=1e-11)
+    with pytest.raises(ValueError):
+        m.teacher_logits_tail(ids, 2, 14)
+
+
 def test_greedy_and_early_exit_equal_no_cache_greedy():
     shape = synth.MICRO_GQA
     m, cfg, w = oracle_model(shape, weights=loud_weights(shape))
