@@ -11,9 +11,13 @@ LOGIT_TOL = 3e-2  # max|delta| <= LOGIT_TOL * max|logit| (bf16 weights/activatio
 
 
 def make_pair(shape, seed, scale_from, late_scale, max_seq, page_size=64, max_draft=8, eos_id=-1,
-              linear_path=B.LS_LINEAR_AUTO, amplify=None, oracle=True):
-    """-> (gpu Model, oracle Model or None)"""
-    w = synth.make_weights(shape, seed, scale_from, late_scale, device="cuda")
+              linear_path=B.LS_LINEAR_AUTO, amplify=None, oracle=True, draw_on="cuda"):
+    """-> (gpu Model, oracle Model or None).  draw_on="cpu": the weights are drawn by the host
+    generator (whose stream differs from the device's) and then moved to the GPU, for tests whose
+    seeds were picked with the oracle alone on a machine without a GPU."""
+    w = synth.make_weights(shape, seed, scale_from, late_scale, device=draw_on)
+    if draw_on != "cuda":
+        w = {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in w.items()}
     if amplify:
         w = synth.amplify(w, amplify)
     gm = B.Model(shape, w, max_seq, page_size, max_draft, eos_id, linear_path)

@@ -89,18 +89,6 @@ def test_generate_equals_generate_full_for_every_exit_and_draft(path):
 
 
 @pytest.mark.parametrize("path", PATHS)
-def test_accepted_per_step_matches_oracle_on_the_safe_prefix(path):
-    gm, om = make_pair(TINY.shape, TINY.weight_seed, TINY.exit_layer, TINY.late_scale, 128, linear_path=path)
-    prompt = synth.make_prompt(TINY.shape.vocab, TINY.n_prompt, TINY.prompt_seed)
-    ref_ids, ref_acc, _ = om.generate_spec(prompt, TINY.exit_layer, TINY.num_draft, TINY.max_new)
-    ids, acc = gm.generate(prompt, TINY.exit_layer, TINY.num_draft, TINY.max_new)
-    _, margins, maxabs = om.generate_full(prompt, TINY.max_new)
-    k = first_low_margin(margins, maxabs)
-    np.testing.assert_array_equal(ids[:k], ref_ids[:k])
-    print(f"path {path}: mean accepted/step gpu {acc.mean():.3f} oracle {ref_acc.mean():.3f}, safe prefix {k}")
-
-
-@pytest.mark.parametrize("path", PATHS)
 def test_zero_late_scale_accepts_every_draft(path):
     E, d = 2, 3
     gm, om = make_pair(TINY.shape, TINY.weight_seed, E, 0.0, 128, linear_path=path)
@@ -427,16 +415,21 @@ def test_llama7b_generate_equals_generate_full_at_full_size(llama7b):
 
 
 def test_llama7b_logits_against_oracle_on_a_short_prompt(llama7b):
-    """What the oracle can afford at this shape: a few teacher-forced positions."""
+    """What the oracle can afford at this shape: 17 teacher-forced positions (a 16-row pass and
+    a single-row pass through all 32 layers)."""
     from oracle import ls_oracle as O
     wl, gm, w = llama7b
     s = wl.shape
     cfg = O.Config(s.n_layers, s.d_model, s.n_heads, s.n_kv_heads, s.head_dim, s.d_ffn, s.vocab,
-                   s.rms_eps, s.rope_theta, 8)
+                   s.rms_eps, s.rope_theta, 24)
     om = O.Model(cfg, synth.as_uint16(w))
-    ids = synth.make_prompt(s.vocab, 3, 17)
+    ids = synth.make_prompt(s.vocab, 17, 17)
     oex, ofi = om.teacher_logits(ids, wl.exit_layer)
     gex, gfi = gm.debug_logits(ids, wl.exit_layer)
     r1 = assert_logits_close(gex, oex, "exit logits")
     r2 = assert_logits_close(gfi, ofi, "final logits")
+    for g, o in ((gex, oex), (gfi, ofi)):
+        part = np.partition(o, -2, axis=1)
+        safe = (part[:, -1] - part[:, -2]) > LOGIT_TOL * np.abs(o).max()
+        assert (g.argmax(1)[safe] == o.argmax(1)[safe]).all()
     print(f"7B: max|delta|/max|logit| exit {r1:.2e} final {r2:.2e}; max|logit| {np.abs(ofi).max():.3f}")
