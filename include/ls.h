@@ -271,16 +271,18 @@ int ls_op_qkv_rope_append(int32_t linear_path, const void *wq_dev, const void *w
                           void *k_pages_dev, void *v_pages_dev, void *cuda_stream);
 
 /* Causal attention of rows m at positions pos0+m over cache positions 0..pos0+m, with
- * grouped KV heads (query head i reads KV head i / (Hq/Hkv)).  q bf16 [M, Hq*hd];
- * out bf16 [M, Hq*hd].  The cache is split into fixed chunks of absolute positions
- * whose partial (max, sum, weighted values) are merged in chunk order by the
- * CTA that finishes last (a counter in the scratch area; nothing waits).
- * scratch_dev: ls_op_attention_scratch_bytes(...) bytes. */
-size_t ls_op_attention_scratch_bytes(int32_t Hq, int32_t hd, int32_t max_seq);
+ * grouped KV heads (query head i reads KV head i / (Hq/Hkv)): the one KV cache that the
+ * draft and the verify stage share (Sec. 4.3.3).  q bf16 [M, Hq*hd]; out bf16 [M, Hq*hd].
+ * One thread-block cluster per KV head; the cache is cut by absolute position into spans
+ * (a fixed number of 64-key chunks per CTA, derived from max_seq), each CTA keeps a running
+ * (max, sum, weighted values) over its span and the spans are combined in span order through
+ * distributed shared memory.  A row's result depends on its position only, never on M.
+ * No scratch memory.  max_seq: capacity of the cache in tokens (<= 16384); it fixes the span
+ * length, so calls that are to agree bit for bit must pass the same value. */
 int ls_op_attention(const void *q_bf16_dev, int32_t M, int32_t pos0, int32_t Hq, int32_t Hkv,
                     int32_t hd, int32_t page_size, const int32_t *page_table_dev, int32_t max_seq,
-                    const void *k_pages_dev, const void *v_pages_dev, void *scratch_dev,
-                    void *out_bf16_dev, void *cuda_stream);
+                    const void *k_pages_dev, const void *v_pages_dev, void *out_bf16_dev,
+                    void *cuda_stream);
 
 /* Kernels of the prompt pass (the rows that go through the model before the first draft,
  * Appendix A.4), which is a dense contraction over hundreds of rows.

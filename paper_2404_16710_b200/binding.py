@@ -26,7 +26,7 @@ EXPORTS = (
     "ls_set_page_table", "ls_generate", "ls_generate_adaptive", "ls_generate_full", "ls_generate_early", "ls_prefill",
     "ls_decode", "ls_decode_flags", "ls_decode_adaptive", "ls_read_output", "ls_read_drafted", "ls_debug_logits", "ls_debug_next_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
     "ls_op_linear", "ls_op_gate_up_swiglu", "ls_op_lm_head_scratch_bytes", "ls_op_lm_head_argmax",
-    "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_qkv_rope_append", "ls_op_attention_scratch_bytes", "ls_op_attention", "ls_op_accept",
+    "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_qkv_rope_append", "ls_op_attention", "ls_op_accept",
     "ls_op_gemm", "ls_op_prefill_attention",
 )
 
@@ -105,8 +105,7 @@ def lib():
             "ls_op_rope_append": (C.c_int, [vp, i32, i32, i32, i32, i32, C.c_float, i32, vp, i32, vp, vp, vp, vp]),
             "ls_op_qkv_rope_append": (C.c_int, [i32, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, C.c_float, i32, vp, i32,
                                                 vp, vp, vp, vp]),
-            "ls_op_attention_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
-            "ls_op_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]),
+            "ls_op_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp]),
             "ls_op_accept": (C.c_int, [vp, vp, i32, vp, vp, vp, vp]),
             "ls_op_gemm": (C.c_int, [vp, vp, i32, i32, i32, vp, i32, i32, vp, vp]),
             "ls_op_prefill_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp]),
@@ -336,13 +335,9 @@ def ls_op_qkv_rope_append(path, wq, wk, wv, h, pos0, Hq, Hkv, hd, theta, page_si
                                     _stream()), "ls_op_qkv_rope_append")
 
 
-def ls_op_attention_scratch_bytes(Hq, hd, max_seq):
-    return lib().ls_op_attention_scratch_bytes(Hq, hd, max_seq)
-
-
-def ls_op_attention(q, pos0, Hq, Hkv, hd, page_size, page_table, max_seq, k_pages, v_pages, scratch, out):
+def ls_op_attention(q, pos0, Hq, Hkv, hd, page_size, page_table, max_seq, k_pages, v_pages, out):
     _ck(lib().ls_op_attention(_dev(q), q.shape[0], pos0, Hq, Hkv, hd, page_size, _dev(page_table), max_seq,
-                              _dev(k_pages), _dev(v_pages), _dev(scratch), _dev(out), _stream()), "ls_op_attention")
+                              _dev(k_pages), _dev(v_pages), _dev(out), _stream()), "ls_op_attention")
 
 
 def ls_op_gemm(a, b, c, accumulate=False, status=None):

@@ -17,11 +17,13 @@
 #include <cstdlib>
 #include <cstring>
 #include <map>
+#include <tuple>
 #include <mutex>
 #include <new>
 #include <vector>
 
 #include "ls.h"
+#include "ls_attention.cuh"
 #include "ls_linear.cuh"
 #include "ls_prefill.cuh"
 
@@ -88,8 +90,8 @@ struct ls_model {
     // workspace
     uint16_t *kpages, *vpages;
     size_t layer_kv_elems;
-    int32_t *page_table, *ctl, *draft, *verified, *out_ids, *accepted, *ids, *attn_counters;
-    float *inv_freq, *x, *part, *logits;
+    int32_t *page_table, *ctl, *draft, *verified, *out_ids, *accepted, *ids;
+    float *inv_freq, *x, *logits;
     uint16_t *h, *q, *o, *a;
     uint16_t* hE;  // exit-layer activations, already multiplied by the gain of layer E's norm (Sec. 4.3.3)
     float *px, *py;          // prompt pass: residual rows and projection outputs of one block
@@ -101,9 +103,10 @@ struct ls_model {
     int32_t* drafted;   // drafts kept per step (adaptive drafting)
     int gate;           // draft pass the launches being enqueued belong to (0: none)
     unsigned long long next_pass;  // conditional-node handle the next draft head switches on (0: none)
-    int page_shift, n_pages, chunk_cap, cand_stride;
+    int page_shift, n_pages, cand_stride;
+    AttnPlan attn;  // cluster size and chunks per CTA of the attention kernel: constants of the model
     // loop state
-    int n_prompt, last_tok, prefilled_layers, grid_chunks;
+    int n_prompt, last_tok, prefilled_layers;
     bool use_graphs, own_stream, pdl, big_prefill, cond_graphs;
     int64_t launches;  // kernels enqueued (counted while building a step)
     struct G {
@@ -129,7 +132,6 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
         return p;
     };
     const int n_pages = (c.max_seq + c.page_size - 1) / c.page_size;
-    const int chunk_cap = (c.max_seq + kAttnChunk - 1) / kAttnChunk;
     const int cand_stride = (c.vocab + 15) / 16;
     const size_t layer_kv = (size_t)n_pages * c.n_kv_heads * c.page_size * c.head_dim;
     const size_t qw = (size_t)c.n_heads * c.head_dim, kvw = (size_t)c.n_kv_heads * c.head_dim;
@@ -144,8 +146,6 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     unsigned char* ac = take(sizeof(int32_t) * c.max_seq);
     unsigned char* ids = take(sizeof(int32_t) * c.max_seq);
     unsigned char* x = take(sizeof(float) * kMaxRows * c.d_model);
-    unsigned char* part = take(sizeof(float) * kMaxRows * c.n_heads * chunk_cap * attn_part_pitch(c.head_dim));
-    unsigned char* actr = take(sizeof(int32_t) * c.n_kv_heads);
     unsigned char* logits = take(sizeof(float) * kMaxRows * c.vocab);
     unsigned char* h = take(2 * (size_t)kMaxRows * c.d_model);
     unsigned char* q = take(2 * (size_t)kMaxRows * qw);
@@ -187,8 +187,6 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
         m->accepted = (int32_t*)ac;
         m->ids = (int32_t*)ids;
         m->x = (float*)x;
-        m->part = (float*)part;
-        m->attn_counters = (int32_t*)actr;
         m->logits = (float*)logits;
         m->h = (uint16_t*)h;
         m->q = (uint16_t*)q;
@@ -198,7 +196,6 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
         m->second = (float*)second;
         m->drafted = (int32_t*)drafted;
         m->n_pages = n_pages;
-        m->chunk_cap = chunk_cap;
         m->cand_stride = cand_stride;
         m->page_shift = log2_exact(c.page_size);
     }
@@ -206,33 +203,128 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
 }
 
 // ------------------------------------------------------------------ kernel launch helpers
-int attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
-                int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int hd, int page_shift,
-                int max_seq, int chunk_cap, int grid_chunks, float* part, int32_t* counters, uint16_t* out,
-                const LaunchCtx& lc, int gate = 0)
+template <int HD, int QT>
+int attn_launch_t(const AttnPlan& plan, const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
+                  int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift, int max_seq, uint16_t* out,
+                  const LaunchCtx& lc, int gate)
 {
-    const int Q = Hq / Hkv * M;
-    dim3 grid(grid_chunks, Hkv);
-    if (hd == 128) {
-        LS_CK(launch(lc, attn_kernel<128>, grid, dim3(kAttnThreads), attn_smem_bytes<128>(Q), q, kp, vp, pt, ctl, pos_off, M,
-                     Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out, gate));
-    } else {
-        LS_CK(launch(lc, attn_kernel<64>, grid, dim3(kAttnThreads), attn_smem_bytes<64>(Q), q, kp, vp, pt, ctl, pos_off, M,
-                     Hq, Hkv, page_shift, max_seq, chunk_cap, part, counters, out, gate));
-    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan.csize, Hkv);
+    cfg.blockDim = dim3(kAttnThreads);
+    cfg.dynamicSmemBytes = attn_smem_bytes<HD>(Hq / Hkv * M);
+    cfg.stream = lc.st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = plan.csize;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = lc.pdl ? 2 : 1;
+    LS_CK(cudaLaunchKernelEx(&cfg, attn_cluster_kernel<HD, QT>, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift,
+                             max_seq, plan.span, out, gate));
     return LS_OK;
 }
 
-int attn_allow_smem(int hd, int group)
+template <int HD>
+int attn_launch_hd(const AttnPlan& plan, const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
+                   int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift, int max_seq, uint16_t* out,
+                   const LaunchCtx& lc, int gate)
 {
-    const int Q = group * kMaxRows;
-    if (hd == 128) {
-        LS_CK(cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)attn_smem_bytes<128>(Q)));
-    } else {
-        LS_CK(cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)attn_smem_bytes<64>(Q)));
+    const int Q = Hq / Hkv * M;  // the instantiation that holds Q queries in tiles of 16
+    if (Q <= 16) return attn_launch_t<HD, 1>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
+    if (Q <= 32) return attn_launch_t<HD, 2>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
+    if (Q <= 64) return attn_launch_t<HD, 4>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
+    return attn_launch_t<HD, 8>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
+}
+
+int attn_launch(const AttnPlan& plan, const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
+                int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int hd, int page_shift, int max_seq, uint16_t* out,
+                const LaunchCtx& lc, int gate = 0)
+{
+    if (hd == 128) return attn_launch_hd<128>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
+    return attn_launch_hd<64>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
+}
+
+template <int HD, int QT>
+cudaError_t attn_prepare_t(int group, int Hkv, int csize, int* clusters)
+{
+    const int rows = 16 * QT / group;  // rows of the largest pass this instantiation serves
+    if (rows < 1) return cudaSuccess;
+    const size_t smem = attn_smem_bytes<HD>(group * (rows < kMaxRows ? rows : kMaxRows));
+    cudaError_t e = cudaFuncSetAttribute(attn_cluster_kernel<HD, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess || !clusters) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(csize, Hkv);
+    cfg.blockDim = dim3(kAttnThreads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at;
+    at.id = cudaLaunchAttributeClusterDimension;
+    at.val.clusterDim.x = csize;
+    at.val.clusterDim.y = 1;
+    at.val.clusterDim.z = 1;
+    cfg.attrs = &at;
+    cfg.numAttrs = 1;
+    return cudaOccupancyMaxActiveClusters(clusters, attn_cluster_kernel<HD, QT>, &cfg);
+}
+
+template <int HD>
+cudaError_t attn_prepare_hd(int group, int Hkv, int csize, int* clusters)
+{
+    // every instantiation gets its shared-memory allowance; the residency question is asked
+    // of the one that serves single-row passes (the bulk of the loop)
+    cudaError_t e = attn_prepare_t<HD, 1>(group, Hkv, csize, clusters);
+    if (e == cudaSuccess) e = attn_prepare_t<HD, 2>(group, Hkv, csize, nullptr);
+    if (e == cudaSuccess) e = attn_prepare_t<HD, 4>(group, Hkv, csize, nullptr);
+    if (e == cudaSuccess) e = attn_prepare_t<HD, 8>(group, Hkv, csize, nullptr);
+    return e;
+}
+
+// Cluster size and chunks per CTA for a cache of max_seq positions: the largest cluster (up to
+// 8 CTAs) with which one cluster per KV head is resident at the same time, so that no head
+// waits for another to finish; 8 if no size achieves that.  A function of the model's shape and
+// the device only -- never of a pass -- because the chunks per CTA enter a row's arithmetic.
+int attn_plan(int hd, int group, int Hkv, int max_seq, AttnPlan* out)
+{
+    struct Key {
+        int dev, hd, group, Hkv, cap;
+        bool operator<(const Key& o) const
+        {
+            return std::tie(dev, hd, group, Hkv, cap) < std::tie(o.dev, o.hd, o.group, o.Hkv, o.cap);
+        }
+    };
+    static std::map<Key, AttnPlan> plans;
+    static std::mutex mu;
+    const int cap = (max_seq + kAttnChunk - 1) / kAttnChunk;
+    int dev = 0;
+    LS_CK(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(mu);
+    const Key key = {dev, hd, group, Hkv, cap};
+    auto it = plans.find(key);
+    if (it == plans.end()) {
+        int best = 0;
+        const int cmax = cap < kAttnMaxCluster ? cap : kAttnMaxCluster;
+        for (int cs = cmax; cs >= 1 && !best; --cs) {
+            int clusters = 0;
+            cudaError_t e = hd == 128 ? attn_prepare_hd<128>(group, Hkv, cs, &clusters)
+                                      : attn_prepare_hd<64>(group, Hkv, cs, &clusters);
+            if (e != cudaSuccess) {
+                cudaGetLastError();  // a cluster size the device refuses: try the next one
+                continue;
+            }
+            if (clusters >= Hkv) best = cs;
+        }
+        if (!best) {
+            best = cmax;
+            LS_CK(hd == 128 ? attn_prepare_hd<128>(group, Hkv, best, nullptr) : attn_prepare_hd<64>(group, Hkv, best, nullptr));
+        }
+        AttnPlan p;
+        p.csize = best;
+        p.span = (cap + best - 1) / best;
+        it = plans.emplace(key, p).first;
     }
+    *out = it->second;
     return LS_OK;
 }
 
@@ -316,8 +408,8 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off, int
         a.gate = m->gate;
         norm_in(m, a, slot);
         LS_CK(launch_linear(m->path, EPI_QKV, a, st));
-        LS_TRY(attn_launch(m->q, kp, vp, m->page_table, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift,
-                           c.max_seq, m->chunk_cap, m->grid_chunks, m->part, m->attn_counters, m->o, st, m->gate));
+        LS_TRY(attn_launch(m->attn, m->q, kp, vp, m->page_table, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift,
+                           c.max_seq, m->o, st, m->gate));
         a = lin_args(w.wo, m->o, M, D, qw);
         a.out = xrow;
         a.ldo = D;
@@ -700,7 +792,7 @@ int get_graph(ls_model* m, int E, int d, bool reuse, float min_margin, ls_model:
     uint32_t mbits;
     memcpy(&mbits, &min_margin, sizeof(mbits));
     const std::pair<uint64_t, uint32_t> key(
-        ((uint64_t)(reuse ? 0 : 1) << 48) | ((uint64_t)E << 32) | ((uint64_t)d << 16) | (uint64_t)m->grid_chunks, mbits);
+        ((uint64_t)(reuse ? 0 : 1) << 48) | ((uint64_t)E << 32) | ((uint64_t)d << 16), mbits);
     auto it = m->graphs.find(key);
     if (it == m->graphs.end()) {
         if (m->graphs.size() >= 64) drop_graphs(m);  // a bound on what a long-lived handle keeps
@@ -751,14 +843,6 @@ int check_ids(const ls_model* m, const int32_t* ids, int n)
     for (int i = 0; i < n; ++i)
         if (ids[i] < 0 || ids[i] >= m->c.vocab) return LS_ERR_INVALID_ARG;
     return LS_OK;
-}
-
-void set_grid_chunks(ls_model* m, int max_pos_exclusive)
-{
-    int g = (max_pos_exclusive + kAttnChunk - 1) / kAttnChunk;
-    if (g > m->chunk_cap) g = m->chunk_cap;
-    if (g < 1) g = 1;
-    m->grid_chunks = g;  // part of the graph key: graphs captured for another chunk count stay valid
 }
 
 int decode_loop(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new, int32_t flags, float min_margin);
@@ -850,7 +934,6 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
     size_t used = carve(*cfg, (unsigned char*)workspace, m);
     m->n_prompt = 0;
     m->prefilled_layers = 0;
-    m->grid_chunks = m->chunk_cap;
     m->use_graphs = getenv("LS_NO_GRAPH") == nullptr;
     m->pdl = getenv("LS_NO_PDL") == nullptr;
     m->cond_graphs = getenv("LS_NO_COND") == nullptr;
@@ -886,7 +969,7 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
         g_last_cuda = (int)e;
         return fail(LS_ERR_CUDA);
     }
-    int rc = attn_allow_smem(cfg->head_dim, cfg->n_heads / cfg->n_kv_heads);
+    int rc = attn_plan(cfg->head_dim, cfg->n_heads / cfg->n_kv_heads, cfg->n_kv_heads, cfg->max_seq, &m->attn);
     if (rc != LS_OK) return fail(rc);
     *out = m;
     return LS_OK;
@@ -927,7 +1010,6 @@ int ls_prefill(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t lay
     if (layers < 1 || layers > L) return LS_ERR_INVALID_ARG;
     if (n_prompt > m->c.max_seq) return LS_ERR_CAPACITY;
     m->n_prompt = 0;
-    set_grid_chunks(m, n_prompt);
     LS_CK(cudaMemcpyAsync(m->ids, prompt, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, m->st));
     LS_TRY(write_ctl(m, 0, 0, 0));
     LS_CK(cudaEventRecord(m->ev0, m->st));
@@ -998,7 +1080,6 @@ int decode_loop(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_
     const int need_layers = (d > 0) ? L : E;
     if (m->prefilled_layers < need_layers) return LS_ERR_INVALID_ARG;
     if ((int64_t)m->n_prompt + max_new + d + 1 > c.max_seq) return LS_ERR_CAPACITY;
-    set_grid_chunks(m, m->n_prompt + max_new + d + 1);
 
     ls_model::G* g = nullptr;
     if (m->use_graphs) LS_TRY(get_graph(m, E, d, reuse, min_margin, &g));
@@ -1169,7 +1250,6 @@ int ls_debug_logits(ls_model* m, const int32_t* ids, int32_t n, int32_t exit_lay
     if (exit_layer < 1 || exit_layer > L) return LS_ERR_INVALID_ARG;
     if (n > m->c.max_seq) return LS_ERR_CAPACITY;
     m->n_prompt = 0;
-    set_grid_chunks(m, n);
     LS_CK(cudaMemcpyAsync(m->ids, ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, m->st));
     LS_TRY(write_ctl(m, 0, 0, 0));
     for (int r0 = 0; r0 < n; r0 += kMaxRows) {
@@ -1201,7 +1281,6 @@ int ls_debug_next_logits(ls_model* m, float* logits)
     if (!m || !logits || m->n_prompt < 1 || m->prefilled_layers < m->c.n_layers) return LS_ERR_INVALID_ARG;
     const ls_config& c = m->c;
     if (m->n_prompt + 1 > c.max_seq) return LS_ERR_CAPACITY;
-    set_grid_chunks(m, m->n_prompt + 1);
     LS_TRY(write_ctl(m, m->n_prompt - 1, m->last_tok, 1));
     LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
     LS_TRY(run_layers(m, 0, c.n_layers, 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
@@ -1386,31 +1465,15 @@ int ls_op_qkv_rope_append(int32_t path, const void* wq, const void* wk, const vo
     return LS_OK;
 }
 
-size_t ls_op_attention_scratch_bytes(int32_t Hq, int32_t hd, int32_t max_seq)
-{
-    if (Hq < 1 || hd < 1 || max_seq < 1) return 0;
-    size_t cap = (size_t)(max_seq + kAttnChunk - 1) / kAttnChunk;
-    // chunk partials, then one counter per KV head (at most Hq of them)
-    return align_up(sizeof(float) * LS_MAX_ROWS * (size_t)Hq * cap * (size_t)attn_part_pitch(hd), 256) +
-           align_up(sizeof(int32_t) * (size_t)Hq, 256);
-}
-
 int ls_op_attention(const void* q, int32_t M, int32_t pos0, int32_t Hq, int32_t Hkv, int32_t hd, int32_t page_size,
-                    const int32_t* page_table, int32_t max_seq, const void* kp, const void* vp, void* scratch,
-                    void* out, void* stream)
+                    const int32_t* page_table, int32_t max_seq, const void* kp, const void* vp, void* out, void* stream)
 {
     LS_TRY(kv_check(M, pos0, Hq, Hkv, hd, page_size, max_seq));
-    if (!aligned16(q) || !page_table || !aligned16(kp) || !aligned16(vp) || !aligned16(scratch) || !out)
-        return LS_ERR_INVALID_ARG;
-    LS_TRY(attn_allow_smem(hd, Hq / Hkv));
-    const int cap = (max_seq + kAttnChunk - 1) / kAttnChunk;
-    const int chunks = (pos0 + M + kAttnChunk - 1) / kAttnChunk;
-    const size_t part_bytes = align_up(sizeof(float) * LS_MAX_ROWS * (size_t)Hq * cap * (size_t)attn_part_pitch(hd), 256);
-    int32_t* counters = (int32_t*)((unsigned char*)scratch + part_bytes);
-    LS_CK(cudaMemsetAsync(counters, 0, sizeof(int32_t) * Hkv, (cudaStream_t)stream));
-    return attn_launch((const uint16_t*)q, (const uint16_t*)kp, (const uint16_t*)vp, page_table, nullptr, pos0, M, Hq,
-                       Hkv, hd, log2_exact(page_size), max_seq, cap, chunks, (float*)scratch, counters, (uint16_t*)out,
-                       LaunchCtx{(cudaStream_t)stream, false});
+    if (!aligned16(q) || !page_table || !aligned16(kp) || !aligned16(vp) || !out) return LS_ERR_INVALID_ARG;
+    AttnPlan plan;
+    LS_TRY(attn_plan(hd, Hq / Hkv, Hkv, max_seq, &plan));
+    return attn_launch(plan, (const uint16_t*)q, (const uint16_t*)kp, (const uint16_t*)vp, page_table, nullptr, pos0, M,
+                       Hq, Hkv, hd, log2_exact(page_size), max_seq, (uint16_t*)out, LaunchCtx{(cudaStream_t)stream, false});
 }
 
 int ls_op_gemm(const void* a, const void* b, int32_t M, int32_t N, int32_t K, float* c, int32_t ldc, int32_t accumulate,

@@ -1,6 +1,5 @@
 // Non-GEMV kernels of the decode loop: embedding, RMSNorm, rotary embedding + KV append,
-// chunked causal attention over the paged cache with its ordered merge, argmax finish,
-// accept/rollback.
+// argmax finish, accept/rollback (attention: ls_attention.cuh).
 //
 // Invariant kept by every kernel here: the instructions that produce row m's result do
 // not depend on how many rows the pass has.  The verification pass of num_draft+1 rows
@@ -170,41 +169,12 @@ __global__ void rope_append_kernel(const float* __restrict__ qkv, int Hq, int Hk
     dst[j + half] = f2bf(b);
 }
 
-// ------------------------------------------------------------------ attention
-// grid (chunks, Hkv), block 256.  CTA = keys [64*ch, 64*ch + 64) of KV head kh, all
-// G = Hq/Hkv query heads of the group, all M rows.  Row m at position pos0+m sees keys
-// <= pos0+m.  Every CTA writes, per (row, head, chunk), the un-normalised partial
-// (o[HD], max, sum); the CTA that finishes last for its KV head (a counter, no waiting)
-// merges the chunks of that head's queries IN CHUNK ORDER and writes the bf16 output.
-// Chunks are cut by absolute position, so a row's result depends on its position only.
-//
-// q.k and p.v run on the tensor cores (mma.sync.m16n8k16, fp32 accumulate) at EVERY pass size,
-// one row or sixteen: queries are the 16-row operand (tiles of 16, zero-padded), so the
-// instruction sequence behind a row does not depend on M.  q.k: warp w owns keys 8w..8w+7;
-// a thread's 16-byte pieces of its query rows and of its key row are its fragments (the
-// contraction index is permuted alike on both sides).  p.v: p is rounded to bf16, warp w owns
-// 16 (HD 128) or 8 (HD 64) output dims, V fragments come transposed out of ldmatrix.
-// Row pitches keep every access pattern free of bank conflicts: K and Q rows 64 mod 128
-// bytes, V rows 16 mod 128 bytes.
-//
-// shared memory: Ks [64][HD*2+64 B] | Vs [64][HD*2+16 B] | Qb bf16 [Qpad][HD*2+64 B]
-//                | S f32 [Qpad][72] | Pb bf16 [Qpad][72]          (Qpad = Q rounded up to 16)
+// ------------------------------------------------------------------ attention: shared constants
+// (the decode / verify kernel is in ls_attention.cuh; the two helpers below serve the FMA walk
+// of the prompt pass)
 constexpr int kAttnThreads = 256;
-constexpr int kAttnMaxChunks = 256;  // chunks the merge can hold weights for: max_seq <= 16384
-constexpr int kMergeBatch = 8;       // queries merged together (one warp each)
+constexpr int kAttnMaxChunks = 256;  // chunks of 64 keys a cache may hold: max_seq <= 16384
 constexpr int kAttnSP = 72;          // floats per row of S, bf16 per row of Pb
-template <int HD>
-__host__ __device__ constexpr size_t attn_smem_bytes(int Q)
-{
-    const size_t qpad = ((size_t)Q + 15) / 16 * 16;
-    size_t stage = (size_t)kAttnChunk * (HD * 2 + 64) + (size_t)kAttnChunk * (HD * 2 + 16) + qpad * (HD * 2 + 64) +
-                   qpad * kAttnSP * 4 + qpad * kAttnSP * 2;
-    // merge (reuses the same memory): weights and sums [8][256] each, slice sums [4][8 slices][HD]
-    size_t merge = sizeof(float) * (2 * (size_t)kMergeBatch * kAttnMaxChunks + 4 * 8 * (size_t)HD + kMergeBatch);
-    return stage > merge ? stage : merge;
-}
-// floats per (row, head, chunk) partial: o[HD], max, sum, 2 of padding (16-byte rows)
-__host__ __device__ constexpr int attn_part_pitch(int hd) { return hd + 4; }
 
 // scores of QB queries against the thread's key: its quarter of the dims
 template <int HD, int QB>
@@ -272,330 +242,6 @@ __device__ __forceinline__ void attn_pv(const unsigned char* Vs, const float* P,
             o[qq][0] += __shfl_xor_sync(0xffffffffu, o[qq][0], sh);
             o[qq][1] += __shfl_xor_sync(0xffffffffu, o[qq][1], sh);
         }
-}
-
-template <int HD>
-__global__ void __launch_bounds__(kAttnThreads)
-attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
-            const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table,
-            int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift,
-            int max_seq, int chunk_cap, float* part, int32_t* counters, uint16_t* __restrict__ out, int gate)
-{
-    constexpr int C = kAttnChunk, T = kAttnThreads;
-    constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 16;
-    constexpr int SP = kAttnSP, PBROW = kAttnSP * 2;
-    constexpr int SEGS = HD * 2 / 16;  // 16-byte segments per row
-    constexpr int PP = attn_part_pitch(HD);
-    extern __shared__ __align__(16) unsigned char smem[];
-    unsigned char* Ks = smem;
-    unsigned char* Vs = Ks + C * KROW;
-    const int ch = blockIdx.x, kh = blockIdx.y, tid = threadIdx.x;
-    const int warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
-    const int key0 = ch * C;
-    const uint32_t ks0 = (uint32_t)__cvta_generic_to_shared(Ks), vs0 = (uint32_t)__cvta_generic_to_shared(Vs);
-    const bool one_page = page_shift >= 6;
-
-    // Cache rows below the loop's cache length do not change while the loop runs, so their
-    // copies start before the producer of q (and of this pass's own k, v rows) has finished.
-    // The length is read past L1 and may be an older, smaller one: then fewer rows go early.
-    pdl_launch_dependents();
-    int c_early = 0;
-    if (ctl && !(gate > 0 && gate > __ldcg(ctl + CTL_D_EFF))) c_early = min(__ldcg(ctl + CTL_CACHE_LEN), max_seq);
-    size_t base = 0;
-    auto stage_rows = [&](int p_lo, int p_hi, int p_fill) {
-        // rows p of the chunk with p_lo <= p <= p_hi are copied; rows p_hi < p <= p_fill are zeroed
-#pragma unroll
-        for (int it = 0; it < C * SEGS / T; ++it) {
-            const int idx = tid + it * T;
-            const int r = idx / SEGS, sg = idx % SEGS;
-            const int p = key0 + r;
-            if (p < p_lo || p > p_fill) continue;
-            const bool ok = p <= p_hi;
-            const size_t off = (one_page ? base + (size_t)r * HD
-                                         : kv_row_offset(page_table, ok ? p : key0, page_shift, Hkv, kh, HD)) +
-                               (size_t)sg * 8;
-            cp_async16_cg(ks0 + r * KROW + sg * 16, kpages + off, ok ? 16 : 0);
-            cp_async16_cg(vs0 + r * VROW + sg * 16, vpages + off, ok ? 16 : 0);
-        }
-    };
-    if (key0 < c_early) {
-        if (one_page) base = kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD);
-        stage_rows(0, c_early - 1, c_early - 1);
-    }
-    pdl_wait();
-    auto leave = [&]() {  // nothing in flight may outlive the CTA's shared memory
-        cp_async_commit();
-        cp_async_wait<0>();
-    };
-    if (pass_idle(ctl, gate)) return leave();
-    const int pos0 = (ctl ? ctl[CTL_CACHE_LEN] : 0) + pos_off;
-    const int last_pos = pos0 + M - 1;
-    if (key0 > last_pos) return leave();
-    const int n_active = last_pos / C + 1;  // CTAs of this KV head that take part
-    if (last_pos >= max_seq || pos0 < 0 || n_active > chunk_cap || n_active > (int)gridDim.x) {
-        if (ctl && tid == 0) ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
-        return leave();
-    }
-    if (c_early > pos0) c_early = pos0;  // (cannot happen: the length only grows; rows >= pos0 are this pass's)
-    const int G = Hq / Hkv, Q = G * M;  // query qi = m * G + g
-    const int Qpad = (Q + 15) & ~15;
-
-    unsigned char* Qb = Vs + C * VROW;
-    float* S = reinterpret_cast<float*>(Qb + (size_t)Qpad * KROW);
-    unsigned char* Pb = reinterpret_cast<unsigned char*>(S + (size_t)Qpad * SP);
-
-    // the group's queries (bf16, 16-byte pieces): issue the global loads first, so that they
-    // travel together with the page-table lookup and the K/V copies
-    constexpr int QPT = 2;
-    const int nq = Qpad * SEGS;
-    uint4 qreg[QPT];
-#pragma unroll
-    for (int i = 0; i < QPT; ++i) {
-        const int idx = tid + i * T;
-        qreg[i] = make_uint4(0, 0, 0, 0);
-        if (idx < nq) {
-            const int qi = idx / SEGS, sg = idx % SEGS;
-            if (qi < Q) {
-                const int m = qi / G, g = qi % G;
-                qreg[i] = *reinterpret_cast<const uint4*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + sg * 8);
-            }
-        }
-    }
-    // stage the remaining K and V rows of the chunk (zeros beyond the last visible key):
-    // asynchronous copies, all in flight at once; a chunk never straddles a page of 64 tokens
-    // or more
-    if (one_page) base = kv_row_offset(page_table, key0, page_shift, Hkv, kh, HD);
-    stage_rows(c_early, last_pos, key0 + C - 1);
-    cp_async_commit();
-#pragma unroll
-    for (int i = 0; i < QPT; ++i) {
-        const int idx = tid + i * T;
-        if (idx < nq) *reinterpret_cast<uint4*>(Qb + (idx / SEGS) * KROW + (idx % SEGS) * 16) = qreg[i];
-    }
-    for (int idx = tid + QPT * T; idx < nq; idx += T) {  // more than two tiles of queries
-        const int qi = idx / SEGS, sg = idx % SEGS;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (qi < Q) {
-            const int m = qi / G, g = qi % G;
-            v = *reinterpret_cast<const uint4*>(q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + sg * 8);
-        }
-        *reinterpret_cast<uint4*>(Qb + qi * KROW + sg * 16) = v;
-    }
-    cp_async_wait<0>();
-    __syncthreads();
-
-    // phase 1: s = q.k -- warp w: keys 8w..8w+7 against every tile of 16 queries
-    for (int qt = 0; qt < Qpad; qt += 16) {
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-        const unsigned char* qa = Qb + (qt + g8) * KROW + 16 * t4;
-        const unsigned char* kb = Ks + (8 * warp + g8) * KROW + 16 * t4;
-#pragma unroll
-        for (int j = 0; j < HD / 32; ++j) {
-            const uint4 A0 = *reinterpret_cast<const uint4*>(qa + 64 * j);
-            const uint4 A1 = *reinterpret_cast<const uint4*>(qa + 8 * KROW + 64 * j);
-            const uint4 Bk = *reinterpret_cast<const uint4*>(kb + 64 * j);
-            mma_bf16_16816(c, A0.x, A1.x, A0.y, A1.y, Bk.x, Bk.y);
-            mma_bf16_16816(c, A0.z, A1.z, A0.w, A1.w, Bk.z, Bk.w);
-        }
-        float* s = S + (size_t)(qt + g8) * SP + 8 * warp + 2 * t4;
-        *reinterpret_cast<float2*>(s) = make_float2(c[0], c[1]);
-        *reinterpret_cast<float2*>(s + 8 * SP) = make_float2(c[2], c[3]);
-    }
-    __syncthreads();
-
-    // phase 2: one warp per query: scale, mask, max, exp, sum over the 64 keys of the chunk;
-    // p goes to Pb as bf16 (zeros for the padding rows of the last tile)
-    {
-        const float scale = rsqrtf((float)HD);
-        for (int qi = warp; qi < Qpad; qi += T / 32) {
-            uint16_t* pb = reinterpret_cast<uint16_t*>(Pb + (size_t)qi * PBROW);
-            if (qi >= Q) {
-                pb[lane] = 0;
-                pb[lane + 32] = 0;
-                continue;
-            }
-            const int m = qi / G, g = qi % G;
-            const int pos = pos0 + m;
-            float s0 = S[(size_t)qi * SP + lane] * scale;
-            float s1 = S[(size_t)qi * SP + lane + 32] * scale;
-            if (key0 + lane > pos) s0 = -INFINITY;
-            if (key0 + lane + 32 > pos) s1 = -INFINITY;
-            float mx = fmaxf(s0, s1);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            const float p0 = (s0 == -INFINITY) ? 0.f : expf(s0 - mx);
-            const float p1 = (s1 == -INFINITY) ? 0.f : expf(s1 - mx);
-            float l = p0 + p1;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-            pb[lane] = f2bf(p0);
-            pb[lane + 32] = f2bf(p1);
-            if (lane == 0) {
-                float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP;
-                dst[HD] = mx;
-                dst[HD + 1] = l;
-            }
-        }
-    }
-    __syncthreads();
-
-    // phase 3: o = p.v -- warp w: output dims NTW*8*w .. for every tile of 16 queries
-    {
-        constexpr int NTW = HD / 64;  // n8 tiles per warp: 2 (HD 128) or 1 (HD 64)
-        const int d0 = NTW * 8 * warp;
-        const uint32_t vs0 = (uint32_t)__cvta_generic_to_shared(Vs);
-        // ldmatrix: lane L addresses row L%8 of matrix L/8; matrices 0, 1: keys 0-7, 8-15 of
-        // the 16-key block at dims d0..d0+7; matrices 2, 3: the same keys at dims d0+8..
-        const int mi = lane >> 3, mr = lane & 7;
-        const uint32_t vlane = vs0 + (uint32_t)(((mi & 1) * 8 + mr) * VROW + (d0 + ((NTW == 2) ? (mi >> 1) * 8 : 0)) * 2);
-        for (int qt = 0; qt < Qpad; qt += 16) {
-            float c[NTW][4];
-#pragma unroll
-            for (int nt = 0; nt < NTW; ++nt)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) c[nt][i] = 0.f;
-            const unsigned char* pa = Pb + (size_t)(qt + g8) * PBROW + 4 * t4;
-#pragma unroll
-            for (int kk = 0; kk < C / 16; ++kk) {
-                const uint32_t a0 = *reinterpret_cast<const uint32_t*>(pa + 32 * kk);
-                const uint32_t a1 = *reinterpret_cast<const uint32_t*>(pa + 8 * PBROW + 32 * kk);
-                const uint32_t a2 = *reinterpret_cast<const uint32_t*>(pa + 32 * kk + 16);
-                const uint32_t a3 = *reinterpret_cast<const uint32_t*>(pa + 8 * PBROW + 32 * kk + 16);
-                uint32_t r0, r1, r2, r3;
-                ldmatrix_x4_trans(vlane + (uint32_t)(16 * kk * VROW), r0, r1, r2, r3);
-                mma_bf16_16816(c[0], a0, a1, a2, a3, r0, r1);
-                if (NTW == 2) mma_bf16_16816(c[NTW - 1], a0, a1, a2, a3, r2, r3);
-            }
-#pragma unroll
-            for (int hrow = 0; hrow < 2; ++hrow) {
-                const int qi = qt + g8 + 8 * hrow;
-                if (qi < Q) {
-                    const int m = qi / G, g = qi % G;
-                    float* dst = part + (((size_t)m * Hq + (size_t)kh * G + g) * chunk_cap + ch) * PP + d0 + 2 * t4;
-#pragma unroll
-                    for (int nt = 0; nt < NTW; ++nt)
-                        *reinterpret_cast<float2*>(dst + 8 * nt) = make_float2(c[nt][2 * hrow], c[nt][2 * hrow + 1]);
-                }
-            }
-        }
-    }
-
-    // who is last for this KV head?  (publish the partials, then count; nobody waits)
-    __shared__ int is_last;
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const int prev = atomicAdd(&counters[kh], 1);
-        is_last = (prev == n_active - 1);
-        if (is_last) counters[kh] = 0;  // ready for the next launch
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-
-    // Merge in a fixed order, in two round trips to L2 per batch of 8 queries:
-    //  A  one warp per query: all chunk (max, sum) pairs at once -> global max, weights
-    //     w_c = exp(max_c - max) and the denominator (summed in chunk order by one lane);
-    //  B  four queries at a time: warp s sums the weighted o of chunks c = s, s+8, ... of each
-    //     (lanes over the dims), then one warp per query adds the 8 slice sums in slice
-    //     order, divides and stores.
-    // The order depends on the row's position only, never on M.
-    {
-        constexpr int DPL = HD / 32;  // dims per lane: 4 or 2
-        const int warp = tid >> 5, lane = tid & 31;
-        float* Wt = reinterpret_cast<float*>(smem);                 // [8][kAttnMaxChunks] weights
-        float* Ls = Wt + kMergeBatch * kAttnMaxChunks;              // [8][kAttnMaxChunks] chunk sums
-        float* Ob = Ls + kMergeBatch * kAttnMaxChunks;              // [4 queries][8 slices][HD]
-        float* Lq = Ob + 4 * 8 * HD;                                // [8] denominators
-        for (int qb = 0; qb < Q; qb += kMergeBatch) {
-            __syncthreads();  // previous batch (and the phases before) are done with this memory
-            {
-                const int qi = qb + warp;
-                if (qi < Q) {
-                    const int m = qi / G, h = kh * G + qi % G;
-                    const int nch = (pos0 + m) / C + 1;
-                    const float* base = part + ((size_t)m * Hq + h) * chunk_cap * PP;
-                    float* wt = Wt + warp * kAttnMaxChunks;
-                    float* ls = Ls + warp * kAttnMaxChunks;
-                    float mx = -INFINITY;
-                    for (int c = lane; c < nch; c += 32) {
-                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(base + (size_t)c * PP + HD));
-                        wt[c] = ml.x;
-                        ls[c] = ml.y;
-                        mx = fmaxf(mx, ml.x);
-                    }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                    for (int c = lane; c < nch; c += 32) wt[c] = expf(wt[c] - mx);
-                    __syncwarp();
-                    if (lane == 0) {
-                        float l = 0.f;
-                        for (int c = 0; c < nch; ++c) l = fmaf(ls[c], wt[c], l);
-                        Lq[warp] = l;
-                    }
-                }
-            }
-            __syncthreads();
-            for (int w0 = 0; w0 < kMergeBatch && qb + w0 < Q; w0 += 4) {  // four queries at a time
-                float o[4][DPL];
-#pragma unroll
-                for (int ww = 0; ww < 4; ++ww) {
-#pragma unroll
-                    for (int i = 0; i < DPL; ++i) o[ww][i] = 0.f;
-                    const int qi = qb + w0 + ww;
-                    if (qi < Q) {
-                        const int m = qi / G, h = kh * G + qi % G;
-                        const int nch = (pos0 + m) / C + 1;
-                        const float* base = part + ((size_t)m * Hq + h) * chunk_cap * PP + lane * DPL;
-                        const float* wt = Wt + (w0 + ww) * kAttnMaxChunks;
-#pragma unroll 4
-                        for (int c = warp; c < nch; c += 8) {
-                            const float wc = wt[c];
-                            if (DPL == 4) {
-                                const float4 v = __ldcg(reinterpret_cast<const float4*>(base + (size_t)c * PP));
-                                o[ww][0] = fmaf(v.x, wc, o[ww][0]);
-                                o[ww][1] = fmaf(v.y, wc, o[ww][1]);
-                                o[ww][DPL - 2] = fmaf(v.z, wc, o[ww][DPL - 2]);
-                                o[ww][DPL - 1] = fmaf(v.w, wc, o[ww][DPL - 1]);
-                            } else {
-                                const float2 v = __ldcg(reinterpret_cast<const float2*>(base + (size_t)c * PP));
-                                o[ww][0] = fmaf(v.x, wc, o[ww][0]);
-                                o[ww][1] = fmaf(v.y, wc, o[ww][1]);
-                            }
-                        }
-                    }
-                }
-#pragma unroll
-                for (int ww = 0; ww < 4; ++ww)
-#pragma unroll
-                    for (int i = 0; i < DPL; ++i) Ob[(ww * 8 + warp) * HD + lane * DPL + i] = o[ww][i];
-                __syncthreads();
-                if (warp < 4 && qb + w0 + warp < Q) {  // warp ww finishes query w0 + ww
-                    const int qi = qb + w0 + warp;
-                    const int m = qi / G, h = kh * G + qi % G;
-                    const float l = Lq[w0 + warp];
-                    float r[DPL];
-#pragma unroll
-                    for (int i = 0; i < DPL; ++i) {
-                        float a = 0.f;
-#pragma unroll
-                        for (int sl = 0; sl < 8; ++sl) a += Ob[(warp * 8 + sl) * HD + lane * DPL + i];
-                        r[i] = a / l;
-                    }
-                    uint16_t* dst = out + ((size_t)m * Hq + h) * HD + lane * DPL;
-                    if (DPL == 4) {
-                        uint2 pk;
-                        pk.x = pack_bf16(r[0], r[1]);
-                        pk.y = pack_bf16(r[DPL - 2], r[DPL - 1]);
-                        *reinterpret_cast<uint2*>(dst) = pk;
-                    } else {
-                        *reinterpret_cast<uint32_t*>(dst) = pack_bf16(r[0], r[1]);
-                    }
-                }
-                __syncthreads();
-            }
-        }
-    }
 }
 
 // ------------------------------------------------------------------ argmax finish

@@ -289,10 +289,6 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
-}
 
 // grid (M tiles of 128 rounded up to even, column tiles of 256 of all matrices), cluster (2, 1, 1),
 // block 128; roles as in gemm_bf16_tn_kernel, the MMA issuer only in the leader CTA.

@@ -76,14 +76,12 @@ def op_cases(shape, w, path, M, n_ctx=1030):
     table = torch.arange(n_pages, dtype=torch.int32, device="cuda")
     q = (torch.randn((M, qw), device="cuda", generator=g) * 0.3).bfloat16()
     ao = torch.empty((M, qw), dtype=torch.bfloat16, device="cuda")
-    asc = torch.empty(B.ls_op_attention_scratch_bytes(Hq, hd, max_seq), dtype=torch.uint8, device="cuda")
     xs = torch.randn((M, D), device="cuda", generator=g)
     hn = torch.empty((M, D), dtype=torch.bfloat16, device="cuda")
     gain = w["attn_norm"][0]
     kv_bytes = 2 * 2 * Hkv * hd * (n_ctx + M)
     return {
-        "attention": (lambda i: B.ls_op_attention(q, n_ctx, Hq, Hkv, hd, ps, table, max_seq, kp[i % kvl], vp[i % kvl],
-                                                  asc, ao), kv_bytes, kvl),
+        "attention": (lambda i: B.ls_op_attention(q, n_ctx, Hq, Hkv, hd, ps, table, max_seq, kp[i % kvl], vp[i % kvl], ao), kv_bytes, kvl),
         "rmsnorm": (lambda i: B.ls_op_rmsnorm(xs, gain, 1e-5, hn), 4 * M * D, 1),
         "gate_up_swiglu": (lambda i: B.ls_op_gate_up_swiglu(path, w["w_gate"][i % L], w["w_up"][i % L], h, act),
                            4 * F * D, L),

@@ -280,9 +280,8 @@ def test_attention(Hq, Hkv, hd, M, pos0):
         kp[table[p // page_size], :, p % page_size, :] = kl[p]
         vp[table[p // page_size], :, p % page_size, :] = vl[p]
     q = rnd((M, Hq * hd), 52, 0.5).bfloat16()
-    scratch = torch.empty(B.ls_op_attention_scratch_bytes(Hq, hd, max_seq), dtype=torch.uint8, device="cuda")
     out = torch.empty((M, Hq * hd), dtype=torch.bfloat16, device="cuda")
-    B.ls_op_attention(q, pos0, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp, scratch, out)
+    B.ls_op_attention(q, pos0, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp, out)
     torch.cuda.synchronize()
     kf, vf, qf = vals(kl).reshape(n + 8, -1), vals(vl).reshape(n + 8, -1), vals(q)
     for m in range(M):
@@ -296,13 +295,12 @@ def test_attention_rows_do_not_depend_on_pass_size():
     kp.copy_(rnd(kp.shape, 60).bfloat16())
     vp.copy_(rnd(vp.shape, 61).bfloat16())
     q = rnd((16, Hq * hd), 62, 0.5).bfloat16()
-    scratch = torch.empty(B.ls_op_attention_scratch_bytes(Hq, hd, max_seq), dtype=torch.uint8, device="cuda")
     full = torch.empty((16, Hq * hd), dtype=torch.bfloat16, device="cuda")
-    B.ls_op_attention(q, pos0, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp, scratch, full)
+    B.ls_op_attention(q, pos0, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp, full)
     for m in (0, 3, 15):
         one = torch.empty((1, Hq * hd), dtype=torch.bfloat16, device="cuda")
         B.ls_op_attention(q[m:m + 1].contiguous(), pos0 + m, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp,
-                          scratch, one)
+                          one)
         torch.cuda.synchronize()
         assert torch.equal(one[0], full[m]), f"row {m}"
 
