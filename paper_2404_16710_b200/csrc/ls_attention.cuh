@@ -148,6 +148,7 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
     // chunks of the span that lie wholly below it are fetched before the producer of q (and of
     // this pass's own k, v rows) has finished.  The length is read past L1 and may be an older,
     // smaller one: then fewer chunks go early.
+    TR_T0
     pdl_launch_dependents();
     cluster_arrive_relaxed();  // "this CTA runs": waited for before the first write into another CTA's memory
     int phys0[NST];  // the page table does not change while a loop runs: look the first chunks up at once
@@ -162,6 +163,7 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
         if (early[s]) stage_chunk(chunk0 + s, s, c_early - 1, phys0[s]);
     }
     pdl_wait();
+    TR_T1
     auto leave = [&]() {  // nothing in flight may outlive the CTA's shared memory; every arrive gets its wait
         cp_async_commit();
         cp_async_wait<0>();
@@ -444,6 +446,7 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
                 pack_bf16(__fdividef(o0, l), __fdividef(o1, l));
         }
     }
+    TR_END(kpages, M > 1 ? 1 : 0)
 }
 
 }  // namespace ls

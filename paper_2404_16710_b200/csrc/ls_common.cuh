@@ -49,11 +49,14 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p)
                  : "l"(p));
     return v;
 }
-// 16-byte read of small, heavily re-used data (activations): keep in L1.
+// 16-byte read of small, heavily re-used data (activations): keep in L1.  A coherent load:
+// the rows are written by the kernel before this one, which under programmatic dependent
+// launch may still have been running when this kernel's CTAs started, so the read-only
+// (non-coherent) path is not allowed for them.
 __device__ __forceinline__ uint4 ld_reuse16(const void* p)
 {
     uint4 v;
-    asm volatile("ld.global.nc.L1::evict_last.v4.u32 {%0,%1,%2,%3}, [%4];"
+    asm volatile("ld.global.L1::evict_last.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p));
     return v;
@@ -115,6 +118,54 @@ __device__ __forceinline__ void cluster_sync_all()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+
+#ifdef LS_TRACE
+// ---- Timeline instrumentation, compiled in only with -DLS_TRACE (a separate library used by
+// paper_2404_16710_b200/timeline.py; the product build carries none of it).  The linear and
+// attention kernels stamp the global timer at CTA start, after the dependency wait and at CTA
+// end; one CTA in eight folds its stamps into the record of its launch (first / last start,
+// first / last wait release, first / last end).  A launch is identified by a pointer that is
+// unique to it within one pass (its weight matrix, its layer's K pages) plus 1 for passes of
+// more than one row; the record's slot is a hash of that key, which the host re-computes.
+struct TraceRec { unsigned long long key, s0, s1, w0, w1, e0, e1, n; };
+constexpr int kTraceSlots = 1 << 18;
+__device__ TraceRec g_trace[kTraceSlots];
+__device__ int g_trace_on;
+__device__ __forceinline__ unsigned long long gtime()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__host__ __device__ __forceinline__ unsigned trace_hash(unsigned long long k)
+{
+    return (unsigned)((k * 0x9E3779B97F4A7C15ull) >> 40) & (unsigned)(kTraceSlots - 1);
+}
+__device__ __forceinline__ void tr_commit(const void* key, int sub, unsigned long long t0, unsigned long long t1)
+{
+    if (!*(volatile int*)&g_trace_on) return;
+    const unsigned lin = blockIdx.x + blockIdx.y * gridDim.x, tot = gridDim.x * gridDim.y;
+    if ((lin % 8) != 3 && lin != tot - 1 && lin != 0) return;
+    const unsigned long long t2 = gtime();
+    const unsigned long long k = (unsigned long long)key + (unsigned long long)sub;
+    TraceRec* r = g_trace + trace_hash(k);
+    atomicMax(&r->key, k);
+    atomicMin(&r->s0, t0);
+    atomicMax(&r->s1, t0);
+    atomicMin(&r->w0, t1);
+    atomicMax(&r->w1, t1);
+    atomicMin(&r->e0, t2);
+    atomicMax(&r->e1, t2);
+    atomicAdd(&r->n, 1ull);
+}
+#define TR_T0 const unsigned long long tr0 = gtime();
+#define TR_T1 const unsigned long long tr1 = gtime();
+#define TR_END(key, sub) if (threadIdx.x == 0) tr_commit(key, sub, tr0, tr1);
+#else
+#define TR_T0
+#define TR_T1
+#define TR_END(key, sub)
+#endif
 
 struct LaunchCtx {
     cudaStream_t st;

@@ -213,15 +213,21 @@ int attn_launch_t(const AttnPlan& plan, const uint16_t* q, const uint16_t* kp, c
     cfg.blockDim = dim3(kAttnThreads);
     cfg.dynamicSmemBytes = attn_smem_bytes<HD>(Hq / Hkv * M);
     cfg.stream = lc.st;
-    cudaLaunchAttribute at[2];
+    // Load-balancing placement: the hardware may put several CTAs of a cluster on one SM.  With
+    // the default (spread) policy, clusters that arrive while the previous kernel is still
+    // draining are laid out one CTA per SM, two clusters per GPC, and the other half of the
+    // grid only starts when those have finished: attention then runs as two waves.
+    cudaLaunchAttribute at[3];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = plan.csize;
     at[0].val.clusterDim.y = 1;
     at[0].val.clusterDim.z = 1;
-    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[1].val.programmaticStreamSerializationAllowed = 1;
+    at[1].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;
+    at[1].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
+    at[2].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[2].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
-    cfg.numAttrs = lc.pdl ? 2 : 1;
+    cfg.numAttrs = lc.pdl ? 3 : 2;
     LS_CK(cudaLaunchKernelEx(&cfg, attn_cluster_kernel<HD, QT>, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift,
                              max_seq, plan.span, out, gate));
     return LS_OK;
@@ -259,13 +265,15 @@ cudaError_t attn_prepare_t(int group, int Hkv, int csize, int* clusters)
     cfg.gridDim = dim3(csize, Hkv);
     cfg.blockDim = dim3(kAttnThreads);
     cfg.dynamicSmemBytes = smem;
-    cudaLaunchAttribute at;
-    at.id = cudaLaunchAttributeClusterDimension;
-    at.val.clusterDim.x = csize;
-    at.val.clusterDim.y = 1;
-    at.val.clusterDim.z = 1;
-    cfg.attrs = &at;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = csize;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;
+    at[1].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
+    cfg.attrs = at;
+    cfg.numAttrs = 2;
     return cudaOccupancyMaxActiveClusters(clusters, attn_cluster_kernel<HD, QT>, &cfg);
 }
 
@@ -800,8 +808,16 @@ int get_graph(ls_model* m, int E, int d, bool reuse, float min_margin, ls_model:
         int64_t before = m->launches;
         cudaError_t e = cudaSuccess;
         if (min_margin > 0.f && reuse && d > 0 && m->cond_graphs) {
-            LS_TRY(capture_adaptive_step(m, E, d, min_margin, &graph));
-        } else {
+            // a driver without conditional nodes (or out of handles): from now on the adaptive
+            // step is the ordinary capture, whose skipped draft passes idle on their gate
+            if (capture_adaptive_step(m, E, d, min_margin, &graph) != LS_OK) {
+                cudaGetLastError();
+                m->cond_graphs = false;
+                m->launches = before;
+                graph = nullptr;
+            }
+        }
+        if (!graph) {
             LS_CK(cudaStreamBeginCapture(m->st, cudaStreamCaptureModeRelaxed));
             int rc = enqueue_step(m, E, d, reuse, min_margin);
             e = cudaStreamEndCapture(m->st, &graph);
@@ -1505,5 +1521,27 @@ int ls_op_accept(const int32_t* draft, const int32_t* verified, int32_t d, int32
                  out_ids, accepted, 0, nullptr));
     return LS_OK;
 }
+
+
+#ifdef LS_TRACE
+// Timeline build (-DLS_TRACE, see ls_common.cuh): clear the records and switch recording on or off ...
+int ls_trace_reset(int on)
+{
+    std::vector<TraceRec> z(kTraceSlots);
+    for (auto& r : z) { r.key = 0; r.s0 = r.w0 = r.e0 = ~0ull; r.s1 = r.w1 = r.e1 = 0; r.n = 0; }
+    LS_CK(cudaDeviceSynchronize());
+    LS_CK(cudaMemcpyToSymbol(g_trace, z.data(), sizeof(TraceRec) * kTraceSlots));
+    LS_CK(cudaMemcpyToSymbol(g_trace_on, &on, sizeof(int)));
+    LS_CK(cudaDeviceSynchronize());
+    return LS_OK;
+}
+// ... and copy the kTraceSlots records (8 x uint64 each) to the host
+int ls_trace_read(void* out)
+{
+    LS_CK(cudaDeviceSynchronize());
+    LS_CK(cudaMemcpyFromSymbol(out, g_trace, sizeof(TraceRec) * kTraceSlots));
+    return LS_OK;
+}
+#endif
 
 }  // extern "C"

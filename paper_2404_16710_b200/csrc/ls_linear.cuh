@@ -126,8 +126,10 @@ __device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.0f +
 template <int MT, int EPI>
 __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
 {
+    TR_T0
     pdl_launch_dependents();
     pdl_wait();
+    TR_T1
     if (pass_idle(a.ctl, a.gate)) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint16_t* rp[4];
@@ -295,6 +297,7 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
             if (a.second) a.second[(size_t)m * a.cand_stride + blockIdx.x] = s2;
         }
     }
+    TR_END(a.w0, a.M > 1 ? 1 : 0)
 }
 
 // =============================================================================== MMA family
@@ -324,6 +327,7 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
 {
     constexpr int T = WARPS * 32;
     extern __shared__ __align__(16) unsigned char ring[];
+    TR_T0
     pdl_launch_dependents();
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
@@ -397,6 +401,7 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
         for (int p = 0; p < STAGES - 1; ++p) issue_w(warp + p * WARPS, p);
     }
     pdl_wait();
+    TR_T1
     if (pass_idle(a.ctl, a.gate)) {
         cp_async_commit();
         cp_async_wait<0>();
@@ -577,6 +582,7 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             if (a.second) a.second[(size_t)m * a.cand_stride + blockIdx.x] = s2;
         }
     }
+    TR_END(a.w0, a.M > 1 ? 1 : 0)
 }
 
 // =============================================================================== launchers
@@ -603,13 +609,19 @@ inline cudaError_t launch_linear_fma(const LinArgs& a, const LaunchCtx& lc)
 // tiles (q|k|v, gate-up, LM head on the 7B shape) takes two tiles with 3 stages (still 3 CTAs
 // per SM) and uses its token fragments for both.  Measured on the 7B shape: gate-up 32.5 ->
 // 31.6 us and q|k|v 20.8 -> 19.4 us at 7 rows, 36.4 -> 33.3 us and 22.5 -> 20.2 us at 9 rows;
-// below 6 rows the single tile with the deeper ring is faster.
+// below 6 rows the single tile with the deeper ring is faster -- except for q|k|v, which takes two
+// tiles at every pass size: its CTAs then fit the device in one wave (384 on the 7B shape), they
+// all end together, and the attention clusters that follow on the stream are placed at once
+// instead of trickling in behind a second wave (in the loop: q|k|v 19.5 -> 17.9 us at 1 row).
 inline bool mma_wide(int epi, int N, int K)
 {
     const int tiles = lin_grid(epi, N), nsteps = (K + 31) / 32;
     return tiles < 600 && nsteps >= 16;
 }
-inline bool mma_pair(int epi, int N, int K, int M) { return M >= 6 && !mma_wide(epi, N, K) && lin_grid(epi, N) >= 700; }
+inline bool mma_pair(int epi, int N, int K, int M)
+{
+    return (M >= 6 || epi == EPI_QKV) && !mma_wide(epi, N, K) && lin_grid(epi, N) >= 700;
+}
 // CTAs the MMA family launches for this matrix (also the number of argmax candidates per row)
 inline int mma_grid(int epi, int N, int K, int M)
 {
