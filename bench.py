@@ -38,10 +38,23 @@ UNIT = "tokens/s"
 
 # thresholds on the exit-logit margin tried by the adaptive-draft-length leg (logit units)
 ADAPTIVE_MARGINS = (0.02, 0.05, 0.1, 0.2, 0.4)
-# DRAM bytes (read + write) of one launch of the roofline kernel, from the ncu capture that
-# profiles/linear_mma_kernel_llama2-7b_shapes.md summarises; keyed by (workload, rows).  Set an
-# entry to None when the kernel changes until the counters have been taken again.
-ROOFLINE_TRAFFIC = {("llama2-7b", 7): 180.45e6 + 4.05e6}
+# DRAM bytes (read + write) per launch, as ncu counted them, are kept beside the ncu summaries:
+# the table in this file has one row per (workload, op, rows) that was captured.
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.md")
+
+
+def measured_traffic(workload, op, rows):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch from the committed ncu table, or
+    None when that (workload, op, rows) has no row there."""
+    try:
+        with open(TRAFFIC_TABLE) as f:
+            for line in f:
+                c = [x.strip() for x in line.strip().strip("|").split("|")]
+                if len(c) >= 5 and c[0] == workload and c[1] == op and c[2] == str(rows):
+                    return float(c[3]) + float(c[4])
+    except OSError:
+        pass
+    return None
 
 
 def peaks():
@@ -158,9 +171,12 @@ def run_reference(args):
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * max_new / value,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": args.workload, "shape": wl.shape.name, "n_prompt": wl.n_prompt,
-                      "max_new": wl.max_new, "exit_layer": wl.exit_layer, "num_draft": wl.num_draft,
-                      "late_scale": wl.late_scale, "note": "CPU oracle (fp64, OpenMP) on a bounded sample"},
+           "config": {"workload": args.workload, "shape": wl.shape.name, "n_prompt": n_prompt,
+                      "max_new": max_new, "exit_layer": wl.exit_layer, "num_draft": wl.num_draft,
+                      "late_scale": wl.late_scale,
+                      "note": f"CPU oracle (fp64, OpenMP) on a bounded sample: the workload's prompt cut to its first "
+                              f"{n_prompt} ids and {max_new} new tokens (the workload itself: prompt {wl.n_prompt}, "
+                              f"{wl.max_new} new tokens)"},
            "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": desc},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
@@ -307,31 +323,56 @@ def run_own(args):
                       "timed_region": "decode loop from a prefilled prompt, device-resident",
                       "kernels_per_layer": 5, "prompt_pass": "tcgen05 cta_group::2 GEMM, 256x256 tiles on CTA pairs, blocks of 1024 rows"},
            "e2e": e2e, "gpu_launches": int(launches), "clocks": clk.summary,
-           "accepted_per_step": float(acc.mean()), "acceptance_rate": float(acc.mean() / d),
-           "emitted_per_step": float(NEW / len(acc)), "spec_steps": int(len(acc)), "host_syncs": int(st.host_syncs),
+           # the numbers the value is read against come first, the long tables last
            "full_greedy": {"value": full_tok_s, "unit": UNIT, "hbm_GB/s": round(full_gbs, 1),
                            "hbm_frac_measured": round(full_gbs / peak, 4), "hbm_frac_8TBs": round(full_gbs / 8000, 4)},
-           "speedup_vs_full_greedy": value / world / full_tok_s, "without_exit_cache_reuse": no_reuse, "adaptive_draft": adaptive,
-           "ids_equal_full_greedy": lossless,
+           "speedup_vs_full_greedy": value / world / full_tok_s,
            "loop_hbm": {"GB/s": round(loop_gbs, 1), "frac_measured": round(loop_gbs / peak, 4),
                         "frac_8TBs": round(loop_gbs / 8000, 4), "bytes_per_loop": int(sched_bytes)},
+           "ids_equal_full_greedy": lossless,
+           "accepted_per_step": float(acc.mean()), "acceptance_rate": float(acc.mean() / d),
+           "emitted_per_step": float(NEW / len(acc)), "spec_steps": int(len(acc)), "host_syncs": int(st.host_syncs),
            "prefill_ms": prefill_ms}
 
     if rank == 0 and world == 1:
         from paper_2404_16710_b200 import opbench
         ks = opbench.kernel_rooflines(s, w, path, (1, d + 1), peak)
-        dom = ks[f"gate_up_swiglu@M={d + 1}"]
-        out["roofline"] = {"bound": "hbm", "kernel": f"linear_{'mma' if path == 2 else 'fma'}_kernel (gate-up + SwiGLU, "
-                           f"M={d + 1}, verify pass)", "achieved": dom["GB/s"], "peak": peak, "unit": "GB/s",
-                           "frac": dom["frac"], "traffic": ROOFLINE_TRAFFIC.get((args.workload, d + 1)),
-                           "algorithmic_bytes": dom["bytes"], "peak_kind": f"of {peak_kind} (burst copy)",
-                           "how": "CUDA events around 40 launches through the C ABI, rotating over the layers' weights"}
-        out["kernels"] = ks
+        # The gate-up + SwiGLU linear is the largest kernel of a layer.  By share of the loop's time
+        # its single-row launches (draft passes) dominate, its (d+1)-row launch (verify pass) is the
+        # slower of the two per byte: the roofline object is the former, `verify_pass` the latter.
+        fam = "mma" if path == 2 else "fma"
+
+        def roof(M):
+            k = ks[f"gate_up_swiglu@M={M}"]
+            return {"rows": M, "achieved": k["GB/s"], "frac": k["frac"], "us_per_launch": round(k["ms"] * 1e3, 2),
+                    "algorithmic_bytes": k["bytes"], "traffic": measured_traffic(args.workload, "gate_up_swiglu", M)}
+        n_draft_launches = len(acc) * (d + 1) * E
+        n_verify_launches = len(acc) * (s.n_layers - E)
+        loop_ms_mean = statistics.mean(loop_ms)
+        r1, rv = roof(1), roof(d + 1)
+        out["roofline"] = {"bound": "hbm", "kernel": f"linear_{fam}_kernel, gate-up + SwiGLU, 1 row (draft passes)",
+                           "achieved": r1["achieved"], "peak": peak, "unit": "GB/s", "frac": r1["frac"],
+                           "traffic": r1["traffic"], "algorithmic_bytes": r1["algorithmic_bytes"],
+                           "us_per_launch": r1["us_per_launch"],
+                           "share_of_loop_time_est": round(n_draft_launches * r1["us_per_launch"] / 1e3 / loop_ms_mean, 3),
+                           "verify_pass": dict(rv, share_of_loop_time_est=round(
+                               n_verify_launches * rv["us_per_launch"] / 1e3 / loop_ms_mean, 3)),
+                           "peak_kind": f"of {peak_kind} (burst copy)",
+                           "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, "
+                                             "profiles/dram_traffic_per_launch.md (null: not captured for this workload)",
+                           "how": "CUDA events around a CUDA graph of 40 launches through the C ABI, rotating over the "
+                                  "layers' weights (each launch streams from HBM), launches serialised (no dependent-launch overlap)"}
         # the CPU oracle on a bounded sample of the same workload
         n_p, n_new = cpu_sample_sizes(s)
         O, om = oracle_model(wl, w, n_p + n_new + d + 2)
         v, desc = cpu_sample(wl, om, O, prompt, n_p, n_new)
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": desc}
+        out["without_exit_cache_reuse"] = no_reuse
+        out["adaptive_draft"] = adaptive
+        out["kernels"] = ks
+    else:
+        out["without_exit_cache_reuse"] = no_reuse
+        out["adaptive_draft"] = adaptive
     if rank == 0:
         print(json.dumps(out), flush=True)
     if dist:
@@ -350,6 +391,7 @@ def run_sweep(args):
     exits = [int(x) for x in args.sweep_exit.split(",")]
     drafts = [int(x) for x in args.sweep_draft.split(",")]
     scales = [float(x) for x in args.sweep_scale.split(",")]
+    points = []
     for scale in scales:
         for E in exits:
             wl = synth.sweep_workload(E, max(drafts), scale)
@@ -371,7 +413,7 @@ def run_sweep(args):
                 st = gm.stats()
                 ids, acc = B.ls_read_output(gm.h, NEW)
                 tok_s = NEW / (st.decode_ms / 1e3)
-                print(json.dumps({
+                points.append({
                     "sweep": "llama2-7b-shaped", "n_prompt": P, "max_new": NEW, "late_scale": scale, "exit_layer": E,
                     "num_draft": d, "tokens_per_s": round(tok_s, 1), "full_greedy_tokens_per_s": round(full_tok_s, 1),
                     "speedup": round(tok_s / full_tok_s, 3), "accepted_per_step": round(float(acc.mean()), 3),
@@ -379,10 +421,23 @@ def run_sweep(args):
                     "hbm_frac_measured": round((st.weight_bytes + st.kv_bytes) / (st.decode_ms / 1e3) / 1e9 / peak, 3),
                     "full_greedy_hbm_frac_measured": round(full_frac, 3),
                     "ids_equal_full_greedy": bool(np.array_equal(ids, full_ids)), "prefill_ms": round(prefill_ms, 1),
-                    "host_syncs": int(st.host_syncs)}), flush=True)
+                    "host_syncs": int(st.host_syncs)})
+                print(json.dumps(points[-1]), flush=True)
             gm.close()
             del gm, w
             torch.cuda.empty_cache()
+    best = max(points, key=lambda p: p["tokens_per_s"])
+    fracs = [p["hbm_frac_measured"] for p in points]
+    fulls = [p["full_greedy_tokens_per_s"] for p in points]
+    print(json.dumps({"sweep_summary": {
+        "points": len(points), "all_ids_equal_full_greedy": all(p["ids_equal_full_greedy"] for p in points),
+        "best": {k: best[k] for k in ("late_scale", "exit_layer", "num_draft", "tokens_per_s", "speedup",
+                                      "accepted_per_step", "hbm_frac_measured")},
+        "worst_speedup": min(p["speedup"] for p in points),
+        "full_greedy_tokens_per_s": [min(fulls), max(fulls)],
+        "full_greedy_hbm_frac_measured": [min(p["full_greedy_hbm_frac_measured"] for p in points),
+                                          max(p["full_greedy_hbm_frac_measured"] for p in points)],
+        "hbm_frac_measured": [min(fracs), max(fracs)]}}), flush=True)
 
 
 def main():
