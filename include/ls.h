@@ -158,6 +158,34 @@ int ls_generate_full(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prom
 int ls_generate_early(ls_model *m, const int32_t *prompt_ids_host, int32_t n_prompt,
                       int32_t exit_layer, int32_t max_new, int32_t *out_ids_host, int32_t *out_n);
 
+/* Several sequences through the loop together (the paper's Sec. 9 leaves batching to future
+ * work; the loop itself is Sec. 4.3 / Appendix A.4, run per sequence).  Decoding one sequence is
+ * bound by reading the weights; with B sequences every pass carries B rows (draft) or
+ * B * (num_draft + 1) rows (verify), so each weight byte read from HBM serves all of them.
+ * Each sequence drafts, verifies and accepts on its own: its own cache length, its own share
+ * of the KV pages (n_pages / B pages, i.e. a capacity of (n_pages / B) * page_size positions),
+ * its own accepted-per-step record; a sequence that reaches max_new (or EOS) stops emitting
+ * while the others go on.  Every sequence's ids are bit-identical to what ls_generate_full
+ * returns for its prompt alone on the same model.
+ *   prompts_host      the prompts one after the other, prompt_lens_host[b] ids each
+ *   exit_layer, num_draft   as in ls_generate; exit_layer == 0 and num_draft == 0: plain greedy
+ *   out_ids_host      [n_seq][max_new], out_n[b] valid ids in row b
+ *   accepted_per_step [n_seq][max_new], out_n_steps[b] valid entries in row b
+ * Errors: LS_ERR_CAPACITY if n_seq * (num_draft + 1) > LS_MAX_ROWS, num_draft > max_draft or a
+ * prompt + max_new + num_draft + 1 exceeds a sequence's share of the cache; LS_ERR_INVALID_ARG
+ * for n_seq < 1, bad ids, exit_layer outside [1, L-1] with num_draft > 0.  The single-sequence
+ * state left by ls_prefill is discarded (the sequences use its pages).
+ * ls_prefill_batch / ls_decode_batch / ls_read_output_seq are the halves, as below. */
+int ls_generate_batch(ls_model *m, int32_t n_seq, const int32_t *prompts_host,
+                      const int32_t *prompt_lens_host, int32_t exit_layer, int32_t num_draft,
+                      int32_t max_new, int32_t *out_ids_host, int32_t *out_n,
+                      int32_t *accepted_per_step_host, int32_t *out_n_steps);
+int ls_prefill_batch(ls_model *m, int32_t n_seq, const int32_t *prompts_host,
+                     const int32_t *prompt_lens_host);
+int ls_decode_batch(ls_model *m, int32_t exit_layer, int32_t num_draft, int32_t max_new);
+int ls_read_output_seq(ls_model *m, int32_t seq, int32_t *out_ids_host, int32_t *out_n,
+                       int32_t *accepted_per_step_host, int32_t *out_n_steps);
+
 /* The two halves of a generate call, for callers that keep everything on the device
  * (and for timing the decode loop alone).  ls_prefill copies the prompt, runs
  * prompt[0..n-2] through the first `layers` layers (0 = all L; early-exit decoding
@@ -273,12 +301,13 @@ int ls_op_qkv_rope_append(int32_t linear_path, const void *wq_dev, const void *w
 /* Causal attention of rows m at positions pos0+m over cache positions 0..pos0+m, with
  * grouped KV heads (query head i reads KV head i / (Hq/Hkv)): the one KV cache that the
  * draft and the verify stage share (Sec. 4.3.3).  q bf16 [M, Hq*hd]; out bf16 [M, Hq*hd].
- * One thread-block cluster per KV head; the cache is cut by absolute position into spans
- * (a fixed number of 64-key chunks per CTA, derived from max_seq), each CTA keeps a running
- * (max, sum, weighted values) over its span and the spans are combined in span order through
- * distributed shared memory.  A row's result depends on its position only, never on M.
- * No scratch memory.  max_seq: capacity of the cache in tokens (<= 16384); it fixes the span
- * length, so calls that are to agree bit for bit must pass the same value. */
+ * One thread-block cluster per KV head; the cache is cut by absolute position into chunks of
+ * 64 keys that are dealt out round-robin to the cluster's CTAs, each CTA keeps a running
+ * (max, sum, weighted values) over its chunks and the CTAs' results are combined in CTA order
+ * through distributed shared memory.  A row's result depends on its position only, never on M.
+ * No scratch memory.  max_seq: capacity of the cache in tokens (<= 16384); it bounds the
+ * positions (and, below 512, the cluster size: calls that are to agree bit for bit on caches
+ * that small must pass the same value). */
 int ls_op_attention(const void *q_bf16_dev, int32_t M, int32_t pos0, int32_t Hq, int32_t Hkv,
                     int32_t hd, int32_t page_size, const int32_t *page_table_dev, int32_t max_seq,
                     const void *k_pages_dev, const void *v_pages_dev, void *out_bf16_dev,

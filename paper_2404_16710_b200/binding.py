@@ -24,7 +24,8 @@ LS_LINEAR_AUTO, LS_LINEAR_FMA, LS_LINEAR_MMA = 0, 1, 2
 EXPORTS = (
     "ls_strerror", "ls_last_cuda_error", "ls_workspace_bytes", "ls_model_create", "ls_model_destroy",
     "ls_set_page_table", "ls_generate", "ls_generate_adaptive", "ls_generate_full", "ls_generate_early", "ls_prefill",
-    "ls_decode", "ls_decode_flags", "ls_decode_adaptive", "ls_read_output", "ls_read_drafted", "ls_debug_logits", "ls_debug_next_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
+    "ls_decode", "ls_decode_flags", "ls_decode_adaptive", "ls_read_output", "ls_read_drafted",
+    "ls_generate_batch", "ls_prefill_batch", "ls_decode_batch", "ls_read_output_seq", "ls_debug_logits", "ls_debug_next_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
     "ls_op_linear", "ls_op_gate_up_swiglu", "ls_op_lm_head_scratch_bytes", "ls_op_lm_head_argmax",
     "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_qkv_rope_append", "ls_op_attention", "ls_op_accept",
     "ls_op_gemm", "ls_op_prefill_attention",
@@ -89,6 +90,10 @@ def lib():
             "ls_decode": (C.c_int, [vp, i32, i32, i32]),
             "ls_decode_flags": (C.c_int, [vp, i32, i32, i32, i32]),
             "ls_read_output": (C.c_int, [vp, ip, ip, ip, ip]),
+            "ls_generate_batch": (C.c_int, [vp, i32, ip, ip, i32, i32, i32, ip, ip, ip, ip]),
+            "ls_prefill_batch": (C.c_int, [vp, i32, ip, ip]),
+            "ls_decode_batch": (C.c_int, [vp, i32, i32, i32]),
+            "ls_read_output_seq": (C.c_int, [vp, i32, ip, ip, ip, ip]),
             "ls_generate_adaptive": (C.c_int, [vp, ip, i32, i32, i32, C.c_float, i32, ip, ip, ip, ip, ip]),
             "ls_decode_adaptive": (C.c_int, [vp, i32, i32, C.c_float, i32]),
             "ls_read_drafted": (C.c_int, [vp, ip, ip]),
@@ -255,6 +260,44 @@ def ls_read_output(h, max_new):
     return out[:n.value], acc[:s.value]
 
 
+def _cat_prompts(prompts):
+    lens = np.asarray([len(p) for p in prompts], dtype=np.int32)
+    flat = np.ascontiguousarray(np.concatenate([np.asarray(p, dtype=np.int32) for p in prompts]))
+    return flat, lens
+
+
+def ls_prefill_batch(h, prompts):
+    flat, lens = _cat_prompts(prompts)
+    ipt = C.POINTER(C.c_int32)
+    _ck(lib().ls_prefill_batch(h, len(prompts), flat.ctypes.data_as(ipt), lens.ctypes.data_as(ipt)), "ls_prefill_batch")
+
+
+def ls_decode_batch(h, exit_layer, num_draft, max_new):
+    _ck(lib().ls_decode_batch(h, exit_layer, num_draft, max_new), "ls_decode_batch")
+
+
+def ls_read_output_seq(h, seq, max_new):
+    out, acc = np.zeros(max_new, np.int32), np.zeros(max_new, np.int32)
+    n, s = C.c_int32(), C.c_int32()
+    ipt = C.POINTER(C.c_int32)
+    _ck(lib().ls_read_output_seq(h, seq, out.ctypes.data_as(ipt), C.byref(n), acc.ctypes.data_as(ipt), C.byref(s)),
+        "ls_read_output_seq")
+    return out[:n.value], acc[:s.value]
+
+
+def ls_generate_batch(h, prompts, exit_layer, num_draft, max_new):
+    """-> [(ids, accepted_per_step)] per sequence"""
+    flat, lens = _cat_prompts(prompts)
+    B = len(prompts)
+    out, acc = np.zeros((B, max_new), np.int32), np.zeros((B, max_new), np.int32)
+    n, st = np.zeros(B, np.int32), np.zeros(B, np.int32)
+    ipt = C.POINTER(C.c_int32)
+    _ck(lib().ls_generate_batch(h, B, flat.ctypes.data_as(ipt), lens.ctypes.data_as(ipt), exit_layer, num_draft, max_new,
+                                out.ctypes.data_as(ipt), n.ctypes.data_as(ipt), acc.ctypes.data_as(ipt),
+                                st.ctypes.data_as(ipt)), "ls_generate_batch")
+    return [(out[b, :n[b]].copy(), acc[b, :st[b]].copy()) for b in range(B)]
+
+
 def ls_debug_next_logits(h, vocab):
     """after ls_prefill: final logits of the last prompt token on top of the prompt pass's cache"""
     out = np.empty(vocab, np.float32)
@@ -395,6 +438,9 @@ class Model:
 
     def generate_early(self, prompt, exit_layer, max_new):
         return ls_generate_early(self.h, prompt, exit_layer, max_new)
+
+    def generate_batch(self, prompts, exit_layer, num_draft, max_new):
+        return ls_generate_batch(self.h, prompts, exit_layer, num_draft, max_new)
 
     def debug_logits(self, ids, exit_layer, want_exit=True, want_final=True):
         return ls_debug_logits(self.h, ids, exit_layer, self.shape.vocab, want_exit, want_final)

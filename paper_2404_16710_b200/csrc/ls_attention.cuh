@@ -1,20 +1,21 @@
 // Decode / verify attention over the paged bf16 KV cache (one KV cache shared by the draft
 // and the verify stage, LayerSkip Sec. 4.3.3), for passes of up to 16 rows.
 //
-// One thread-block cluster per KV head.  The keys are cut by ABSOLUTE position into spans of
-// R chunks of 64 keys; CTA k of the cluster owns span k (keys [64 R k, 64 R (k+1))), streams its
-// chunks through a two-stage cp.async ring and keeps a running (max, sum, weighted values) per
+// One thread-block cluster of S CTAs per KV head.  The keys are cut by ABSOLUTE position into
+// chunks of 64; CTA k of the cluster owns the chunks k, k + S, k + 2S, ... (its "span"), streams
+// them through a two-stage cp.async ring and keeps a running (max, sum, weighted values) per
 // query -- the online-softmax recurrence, chunk after chunk in position order.  The spans'
 // results never go through global memory: every CTA leaves (max, sum, values) in its own shared
 // memory, the cluster meets at a barrier, and each CTA then combines a slice of the
 // (query, dim) outputs by reading all spans through distributed shared memory, in span order.
 // No counters, no fences, no second kernel.
 //
-// R = ceil(ceil(max_seq / 64) / cluster size) is a constant of the model, so what a row's
-// result depends on is its position alone: a chunk or a span that lies wholly beyond the row's
-// position leaves its running state bit for bit as it was (weights 0, scale factor exp(0)),
-// which makes the verify pass of d+1 rows (Sec. 4.3.2) reproduce single-token decoding exactly,
-// whatever the pass size and whatever later rows share the launch.
+// Which CTA takes a chunk depends on the chunk's position and on S, a constant of the model's
+// head layout, so what a row's result depends on is its position alone -- not the pass size,
+// not the cache capacity, not the other sequences of a pass: a chunk that lies wholly beyond
+// the row's position leaves its running state bit for bit as it was (weights 0, scale factor
+// exp(0)), which makes the verify pass of d+1 rows (Sec. 4.3.2) reproduce single-token decoding
+// exactly.  Dealing the chunks out round-robin also keeps the CTAs evenly loaded at any length.
 //
 // q.k and p.v run on the tensor cores (mma.sync.m16n8k16, fp32 accumulate) at every pass size:
 // the queries of the KV head's group (rows x G) are the 16-row operand in tiles of 16,
@@ -31,9 +32,9 @@ namespace ls {
 constexpr int kAttnStages = 2;       // K/V chunks in flight per CTA
 constexpr int kAttnMaxCluster = 8;   // portable cluster size
 
-// launch shape of the attention kernel for one model: CTAs per cluster, chunks of 64 keys per CTA
+// launch shape of the attention kernel for one model: CTAs per cluster
 struct AttnPlan {
-    int csize, span;
+    int csize;
 };
 
 __device__ __forceinline__ uint32_t cluster_ctarank()
@@ -81,14 +82,17 @@ __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
-// grid (cluster size, Hkv), cluster (cluster size, 1, 1), block 256.  QT: tiles of 16 queries
-// the instantiation can hold (Q = G * M <= 16 QT).  span_chunks: R above.
+// grid (cluster size, Hkv, sequences), cluster (cluster size, 1, 1), block 256.  QT: tiles of 16
+// queries the instantiation can hold (Q = G * rows per sequence <= 16 QT).
+// With several sequences per pass (gridDim.z = B; M counts all rows) the cluster of sequence b
+// takes the rows r = m B + b, that sequence's control block and its page-table entries
+// (b * pt_stride ..); max_seq is then the capacity of one sequence.
 template <int HD, int QT>
 __global__ void __launch_bounds__(kAttnThreads)
 attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ kpages,
                     const uint16_t* __restrict__ vpages, const int32_t* __restrict__ page_table,
                     int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift,
-                    int max_seq, int span_chunks, uint16_t* __restrict__ out, int gate)
+                    int max_seq, uint16_t* __restrict__ out, int gate, int pt_stride)
 {
     constexpr int C = kAttnChunk, T = kAttnThreads, NST = kAttnStages;
     constexpr int KROW = HD * 2 + 64, VROW = HD * 2 + 16;
@@ -100,9 +104,13 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
     static_assert(STAGE % 16 == 0, "stages keep 16-byte alignment");
     extern __shared__ __align__(16) unsigned char smem[];
     const int kh = blockIdx.y, tid = threadIdx.x;
+    const int nseq = (int)gridDim.z, sq = (int)blockIdx.z;
+    const int32_t* sctl = ctl ? ctl + sq * CTL_WORDS : nullptr;  // this sequence's control words
+    page_table += sq * pt_stride;
+    M /= nseq;  // rows of this sequence
     const int rank = (int)cluster_ctarank(), csize = (int)gridDim.x;
     const int warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
-    const int chunk0 = rank * span_chunks;  // first chunk of this CTA's span
+    auto chunk_of = [&](int i) { return rank + i * csize; };  // i-th chunk of this CTA's span
     const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(smem);
     const bool one_page = page_shift >= 6;  // a chunk never straddles a page of 64 tokens or more
 
@@ -153,14 +161,14 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
     cluster_arrive_relaxed();  // "this CTA runs": waited for before the first write into another CTA's memory
     int phys0[NST];  // the page table does not change while a loop runs: look the first chunks up at once
 #pragma unroll
-    for (int s = 0; s < NST; ++s) phys0[s] = (s < span_chunks && (chunk0 + s) * C < max_seq) ? chunk_page(chunk0 + s) : 0;
+    for (int s = 0; s < NST; ++s) phys0[s] = chunk_of(s) * C < max_seq ? chunk_page(chunk_of(s)) : 0;
     int c_early = 0;
-    if (ctl && !(gate > 0 && gate > __ldcg(ctl + CTL_D_EFF))) c_early = min(__ldcg(ctl + CTL_CACHE_LEN), max_seq);
+    if (ctl && !(gate > 0 && gate > __ldcg(ctl + CTL_D_EFF))) c_early = min(__ldcg(sctl + CTL_CACHE_LEN), max_seq);
     bool early[NST];
 #pragma unroll
     for (int s = 0; s < NST; ++s) {
-        early[s] = s < span_chunks && (chunk0 + s + 1) * C <= c_early;
-        if (early[s]) stage_chunk(chunk0 + s, s, c_early - 1, phys0[s]);
+        early[s] = (chunk_of(s) + 1) * C <= c_early;
+        if (early[s]) stage_chunk(chunk_of(s), s, c_early - 1, phys0[s]);
     }
     pdl_wait();
     TR_T1
@@ -172,19 +180,19 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
     // the two ways out below are taken by every CTA of the grid alike (they depend on the
     // control words and the launch arguments only), so no CTA is left waiting at a cluster barrier
     if (pass_idle(ctl, gate)) return leave();
-    const int pos0 = (ctl ? ctl[CTL_CACHE_LEN] : 0) + pos_off;
+    const int pos0 = (ctl ? sctl[CTL_CACHE_LEN] : 0) + pos_off;
     const int last_pos = pos0 + M - 1;
     const int G = Hq / Hkv, Q = G * M;  // query qi = m * G + g
     const int Qpad = (Q + 15) & ~15;
-    if (last_pos >= max_seq || pos0 < 0 || last_pos / (C * span_chunks) >= csize || Qpad > 16 * QT) {
+    if (last_pos >= max_seq || pos0 < 0 || Qpad > 16 * QT) {
         if (ctl && tid == 0) ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
         return leave();
     }
     // (an early chunk lies below a cache length that only grows: below pos0, all of it visible)
-    const int span_keys = C * span_chunks;
-    const int n_active = last_pos / span_keys + 1;  // spans with a visible key
+    const int last_chunk = last_pos / C;
+    const int n_active = min(csize, last_chunk + 1);  // spans with a visible key
     // chunks this CTA walks: its span, cut at the last visible key
-    const int nc = rank < n_active ? min(span_chunks, last_pos / C + 1 - chunk0) : 0;
+    const int nc = rank <= last_chunk ? (last_chunk - rank) / csize + 1 : 0;
 
     unsigned char* Qb = smem + NST * STAGE;
     unsigned char* Pb = Qb + (size_t)Qpad * KROW;
@@ -202,14 +210,15 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
         const uint32_t qb0 = smem0 + (uint32_t)(NST * STAGE);
         for (int qi = r0; qi < Qpad; qi += T / SEGS) {
             const int m = qi < Q ? fastdiv(qi, G, gmul) : 0, g = qi < Q ? qi - m * G : 0;
-            cp_async16_ca(qb0 + qi * KROW + seg * 16, q + ((size_t)m * Hq + (size_t)kh * G + g) * HD + seg * 8, qi < Q ? 16 : 0);
+            cp_async16_ca(qb0 + qi * KROW + seg * 16, q + ((size_t)(m * nseq + sq) * Hq + (size_t)kh * G + g) * HD + seg * 8,
+                          qi < Q ? 16 : 0);
         }
     }
     // the first chunks that did not go early (zeros beyond the last visible key), one commit
     // group per chunk slot, empty when the span has no such chunk
 #pragma unroll
     for (int s = 0; s < NST; ++s) {
-        if (s < nc && !early[s]) stage_chunk(chunk0 + s, s, last_pos, phys0[s]);
+        if (s < nc && !early[s]) stage_chunk(chunk_of(s), s, last_pos, phys0[s]);
         cp_async_commit();
     }
     for (int qi = tid; qi < Qpad; qi += T) {
@@ -245,11 +254,11 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
 
     uint4 qf0[HD / 32], qf1[HD / 32];
     for (int i = 0; i < nc; ++i) {
-        const int s = i % NST, key0 = (chunk0 + i) * C;
+        const int s = i % NST, key0 = chunk_of(i) * C;
         const unsigned char* Ks = smem + s * STAGE;
         const float* Mold = Mrun + (i & 1) * Qpad;
         float* Mnew = Mrun + ((i + 1) & 1) * Qpad;
-        const int phys_next = i + NST < nc ? chunk_page(chunk0 + i + NST) : 0;
+        const int phys_next = i + NST < nc ? chunk_page(chunk_of(i + NST)) : 0;
         cp_async_wait<NST - 1>();
         __syncthreads();
         if (QT == 1 && i == 0) {  // a single tile of queries: its fragments stay in registers
@@ -377,7 +386,7 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
         }
         if (i + NST < nc) {
             __syncthreads();  // everybody is done with stage s: refill it with the chunk NST further on
-            stage_chunk(chunk0 + i + NST, s, last_pos, phys_next);
+            stage_chunk(chunk_of(i + NST), s, last_pos, phys_next);
         }
         cp_async_commit();
     }
@@ -389,7 +398,7 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
     // every owner its (max, sum) per query -- for the rows that can see span j at all.
     const int total = Q * HP;
     const int per = (total + n_active - 1) / n_active;
-    const uint32_t pmul = fastdiv_mul((uint32_t)per), smul = fastdiv_mul((uint32_t)span_keys);
+    const uint32_t pmul = fastdiv_mul((uint32_t)per);
     cluster_wait();  // every CTA of the cluster runs: its shared memory may be written
     if (nc > 0) {
         const float* Mfin = Mrun + (nc & 1) * Qpad;
@@ -399,7 +408,7 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
 #pragma unroll
             for (int hrow = 0; hrow < 2; ++hrow) {
                 const int qi = 16 * t + g8 + 8 * hrow;
-                if (rowpos[t][hrow] >= rank * span_keys) {  // the row sees this span (padding rows: -1)
+                if (rowpos[t][hrow] >= rank * C) {  // the row sees this span's first chunk (padding rows: -1)
 #pragma unroll
                     for (int nt = 0; nt < NTW; ++nt) {
                         const int pp = qi * HP + (d0 + 8 * nt) / 2 + t4;
@@ -412,7 +421,7 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
         }
         for (int idx = tid; idx < Q * kAttnMaxCluster; idx += T) {
             const int qi = idx / kAttnMaxCluster, k = idx % kAttnMaxCluster;
-            if (k < n_active && pos0 + fastdiv(qi, G, gmul) >= rank * span_keys)
+            if (k < n_active && pos0 + fastdiv(qi, G, gmul) >= rank * C)
                 st_cluster_f2(cluster_map(rml0 + 8u * (uint32_t)(rank * Qpad + qi), k), Mfin[qi], Lrun[qi]);
         }
     }
@@ -425,7 +434,7 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
         for (int pp = rank * per + tid; pp < hi; pp += T) {
             const int qi = pp / HP, dp = pp % HP;
             const int m = fastdiv(qi, G, gmul), g = qi - m * G;
-            const int nk = fastdiv(pos0 + m, span_keys, smul) + 1;  // spans this row sees (<= n_active)
+            const int nk = min(csize, ((pos0 + m) >> 6) + 1);  // spans this row sees (<= n_active)
             float mx = -INFINITY;
 #pragma unroll
             for (int j = 0; j < kAttnMaxCluster; ++j)
@@ -442,7 +451,7 @@ attn_cluster_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
                     o1 = fmaf(o.y, w, o1);
                 }
             }
-            *reinterpret_cast<uint32_t*>(out + ((size_t)m * Hq + (size_t)kh * G + g) * HD + 2 * dp) =
+            *reinterpret_cast<uint32_t*>(out + ((size_t)(m * nseq + sq) * Hq + (size_t)kh * G + g) * HD + 2 * dp) =
                 pack_bf16(__fdividef(o0, l), __fdividef(o1, l));
         }
     }

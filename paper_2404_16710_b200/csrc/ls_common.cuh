@@ -18,8 +18,13 @@ enum Ctl : int {
     CTL_EOS = 6,
     CTL_STATUS = 7,     // non-zero: a kernel's bounds check refused an access
     CTL_D_EFF = 8,      // adaptive drafting: drafts this step keeps; kernels of draft pass j > this return at once
+    CTL_SEQ_DONE = 9,   // several sequences per pass: this sequence has finished (CTL_DONE of block 0: all have)
     CTL_WORDS = 16
 };
+// Several sequences per pass (B of them): sequence b has its own block of control words at
+// ctl + b * CTL_WORDS, its own pages (page table entries b * pt_stride ..) and its own output
+// arrays.  Row r of a pass belongs to sequence r % B and is that sequence's row r / B, so the
+// rows of one draft position are contiguous.  B = 1 is the single-sequence loop.
 constexpr int kNoStop = 0x7fffffff;  // CTL_D_EFF while no draft pass has stopped the drafting
 
 enum DevStatus : int { DEV_OK = 0, DEV_BAD_TOKEN = 1, DEV_POS_OVERFLOW = 2 };

@@ -105,6 +105,13 @@ struct ls_model {
     unsigned long long next_pass;  // conditional-node handle the next draft head switches on (0: none)
     int page_shift, n_pages, cand_stride;
     AttnPlan attn;  // cluster size and chunks per CTA of the attention kernel: constants of the model
+    // The sequences the passes being enqueued carry (ls_common.cuh): their number, the page-table
+    // entries and the cache capacity of each, and the table entry of the first.  One sequence
+    // owns the whole table; B sequences get n_pages / B pages each.
+    int nseq, pt_stride, seq_cap;
+    const int32_t* pt;
+    std::vector<int> b_n_prompt, b_last_tok;               // several sequences: prompt length and last prompt token of each
+    std::vector<std::vector<int32_t>> b_out, b_acc;        // ... and what the last ls_decode_batch produced
     // loop state
     int n_prompt, last_tok, prefilled_layers;
     bool use_graphs, own_stream, pdl, big_prefill, cond_graphs;
@@ -139,11 +146,12 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     unsigned char* vp = take(layer_kv * c.n_layers * 2);
     unsigned char* pt = take(sizeof(int32_t) * n_pages);
     unsigned char* fr = take(sizeof(float) * (c.head_dim / 2));
-    unsigned char* ctl = take(sizeof(int32_t) * CTL_WORDS);
+    unsigned char* ctl = take(sizeof(int32_t) * CTL_WORDS * kMaxRows);  // one block per sequence of a pass
     unsigned char* dr = take(sizeof(int32_t) * kMaxRows);
     unsigned char* ve = take(sizeof(int32_t) * kMaxRows);
-    unsigned char* oi = take(sizeof(int32_t) * c.max_seq);
-    unsigned char* ac = take(sizeof(int32_t) * c.max_seq);
+    // outputs: sequence b of a pass of several writes from b * (its share of the pages' positions) on
+    unsigned char* oi = take(sizeof(int32_t) * (size_t)n_pages * c.page_size);
+    unsigned char* ac = take(sizeof(int32_t) * (size_t)n_pages * c.page_size);
     unsigned char* ids = take(sizeof(int32_t) * c.max_seq);
     unsigned char* x = take(sizeof(float) * kMaxRows * c.d_model);
     unsigned char* logits = take(sizeof(float) * kMaxRows * c.vocab);
@@ -206,12 +214,12 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
 template <int HD, int QT>
 int attn_launch_t(const AttnPlan& plan, const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
                   int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift, int max_seq, uint16_t* out,
-                  const LaunchCtx& lc, int gate)
+                  const LaunchCtx& lc, int gate, int nseq, int pt_stride)
 {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(plan.csize, Hkv);
+    cfg.gridDim = dim3(plan.csize, Hkv, nseq);
     cfg.blockDim = dim3(kAttnThreads);
-    cfg.dynamicSmemBytes = attn_smem_bytes<HD>(Hq / Hkv * M);
+    cfg.dynamicSmemBytes = attn_smem_bytes<HD>(Hq / Hkv * (M / nseq));
     cfg.stream = lc.st;
     // Load-balancing placement: the hardware may put several CTAs of a cluster on one SM.  With
     // the default (spread) policy, clusters that arrive while the previous kernel is still
@@ -229,28 +237,32 @@ int attn_launch_t(const AttnPlan& plan, const uint16_t* q, const uint16_t* kp, c
     cfg.attrs = at;
     cfg.numAttrs = lc.pdl ? 3 : 2;
     LS_CK(cudaLaunchKernelEx(&cfg, attn_cluster_kernel<HD, QT>, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift,
-                             max_seq, plan.span, out, gate));
+                             max_seq, out, gate, pt_stride));
     return LS_OK;
 }
 
 template <int HD>
 int attn_launch_hd(const AttnPlan& plan, const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
                    int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int page_shift, int max_seq, uint16_t* out,
-                   const LaunchCtx& lc, int gate)
+                   const LaunchCtx& lc, int gate, int nseq, int pt_stride)
 {
-    const int Q = Hq / Hkv * M;  // the instantiation that holds Q queries in tiles of 16
-    if (Q <= 16) return attn_launch_t<HD, 1>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
-    if (Q <= 32) return attn_launch_t<HD, 2>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
-    if (Q <= 64) return attn_launch_t<HD, 4>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
-    return attn_launch_t<HD, 8>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
+    const int Q = Hq / Hkv * (M / nseq);  // the instantiation that holds a sequence's Q queries in tiles of 16
+    if (Q <= 16)
+        return attn_launch_t<HD, 1>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate, nseq, pt_stride);
+    if (Q <= 32)
+        return attn_launch_t<HD, 2>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate, nseq, pt_stride);
+    if (Q <= 64)
+        return attn_launch_t<HD, 4>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate, nseq, pt_stride);
+    return attn_launch_t<HD, 8>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate, nseq, pt_stride);
 }
 
 int attn_launch(const AttnPlan& plan, const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt,
                 int32_t* ctl, int pos_off, int M, int Hq, int Hkv, int hd, int page_shift, int max_seq, uint16_t* out,
-                const LaunchCtx& lc, int gate = 0)
+                const LaunchCtx& lc, int gate = 0, int nseq = 1, int pt_stride = 0)
 {
-    if (hd == 128) return attn_launch_hd<128>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
-    return attn_launch_hd<64>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate);
+    if (hd == 128)
+        return attn_launch_hd<128>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate, nseq, pt_stride);
+    return attn_launch_hd<64>(plan, q, kp, vp, pt, ctl, pos_off, M, Hq, Hkv, page_shift, max_seq, out, lc, gate, nseq, pt_stride);
 }
 
 template <int HD, int QT>
@@ -289,10 +301,11 @@ cudaError_t attn_prepare_hd(int group, int Hkv, int csize, int* clusters)
     return e;
 }
 
-// Cluster size and chunks per CTA for a cache of max_seq positions: the largest cluster (up to
-// 8 CTAs) with which one cluster per KV head is resident at the same time, so that no head
-// waits for another to finish; 8 if no size achieves that.  A function of the model's shape and
-// the device only -- never of a pass -- because the chunks per CTA enter a row's arithmetic.
+// Cluster size for a cache of max_seq positions: the largest cluster (up to 8 CTAs, no more
+// than the cache has chunks) with which one cluster per KV head is resident at the same time, so
+// that no head waits for another to finish; 8 if no size achieves that.  A function of the
+// model's shape and the device only -- never of a pass -- because the cluster size decides which
+// chunks a CTA folds together, which enters a row's arithmetic.
 int attn_plan(int hd, int group, int Hkv, int max_seq, AttnPlan* out)
 {
     struct Key {
@@ -329,7 +342,6 @@ int attn_plan(int hd, int group, int Hkv, int max_seq, AttnPlan* out)
         }
         AttnPlan p;
         p.csize = best;
-        p.span = (cap + best - 1) / best;
         it = plans.emplace(key, p).first;
     }
     *out = it->second;
@@ -353,6 +365,7 @@ LinArgs lin_args(const uint16_t* w, const uint16_t* h, int M, int N, int K)
     a.M = M;
     a.N = N;
     a.K = K;
+    a.nseq = 1;
     return a;
 }
 
@@ -402,7 +415,9 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off, int
         a.n1 = kvw;
         a.ctl = m->ctl;
         a.inv_freq = m->inv_freq;
-        a.page_table = m->page_table;
+        a.page_table = m->pt;
+        a.nseq = m->nseq;
+        a.pt_stride = m->pt_stride;
         a.q_out = m->q;
         a.kpages = kp;
         a.vpages = vp;
@@ -410,14 +425,14 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off, int
         a.Hkv = Hkv;
         a.hd = hd;
         a.page_shift = m->page_shift;
-        a.max_seq = c.max_seq;
+        a.max_seq = m->seq_cap;
         a.pos_off = pos_off;
         a.theta = c.rope_theta;
         a.gate = m->gate;
         norm_in(m, a, slot);
         LS_CK(launch_linear(m->path, EPI_QKV, a, st));
-        LS_TRY(attn_launch(m->attn, m->q, kp, vp, m->page_table, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift,
-                           c.max_seq, m->o, st, m->gate));
+        LS_TRY(attn_launch(m->attn, m->q, kp, vp, m->pt, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift, m->seq_cap, m->o,
+                           st, m->gate, m->nseq, m->pt_stride));
         a = lin_args(w.wo, m->o, M, D, qw);
         a.out = xrow;
         a.ldo = D;
@@ -471,11 +486,11 @@ int run_head(ls_model* m, int M, int slot, int32_t* tok_out, float* logits, floa
     return LS_OK;
 }
 
-int run_embed(ls_model* m, const int32_t* tok_dev, int M, float* xrow, int slot)
+int run_embed(ls_model* m, const int32_t* tok_dev, int M, float* xrow, int slot, int tok_stride = 1)
 {
     LS_CK(launch(LaunchCtx{m->st, m->pdl}, embed_kernel, dim3(M), dim3(256), 0, m->emb, tok_dev, m->c.d_model,
                  m->c.vocab, xrow, m->ctl, m->lw[0].attn_norm, m->h + (size_t)slot * m->c.d_model,
-                 m->ss + (size_t)slot * m->n_part, m->n_part, m->n_part, m->gate));
+                 m->ss + (size_t)slot * m->n_part, m->n_part, m->n_part, m->gate, tok_stride));
     m->launches += 1;
     return LS_OK;
 }
@@ -627,16 +642,16 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
     const LaunchCtx lc = {st, false};
     int32_t* status = m->ctl + CTL_STATUS;
     LS_CK(launch(lc, embed_kernel, dim3(R), dim3(256), 0, m->emb, m->ids + r0, D, c.vocab, m->px, m->ctl, nullptr,
-                 nullptr, nullptr, 0, 0, 0));
+                 nullptr, nullptr, 0, 0, 0, 1));
     for (int l = 0; l < layers; ++l) {
         const LayerW& w = m->lw[l];
         uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
         uint16_t* vp = m->vpages + (size_t)l * m->layer_kv_elems;
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.attn_norm, D, c.rms_eps, m->ph, nullptr));
         LS_TRY(gemm_launch3(m->ph, w.wq, qw, w.wk, kvw, w.wv, kvw, R, D, m->py, qkvw, 0, status, st));
-        rope_append_rows_kernel<<<R, 256, 0, st>>>(m->py, Hq, Hkv, hd, m->inv_freq, m->page_shift, m->page_table, c.max_seq,
-                                                  r0, m->pq, kp, vp, status);
-        LS_TRY(prefill_attn_launch(m->pq, kp, vp, m->page_table, r0, R, Hq, Hkv, hd, m->page_shift, m->po, st));
+        rope_append_rows_kernel<<<R, 256, 0, st>>>(m->py, Hq, Hkv, hd, m->inv_freq, m->page_shift, m->pt, m->seq_cap, r0,
+                                                  m->pq, kp, vp, status);
+        LS_TRY(prefill_attn_launch(m->pq, kp, vp, m->pt, r0, R, Hq, Hkv, hd, m->page_shift, m->po, st));
         LS_TRY(gemm_launch(m->po, w.wo, R, D, qw, m->px, D, 1, status, st));
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.ffn_norm, D, c.rms_eps, m->ph, nullptr));
         if (gemm_uses_pairs(R)) {  // gate, up and SwiGLU in one kernel
@@ -660,52 +675,58 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
 // draft pass j of a step (j == d: the extra early pass, no head)
 int enqueue_draft_pass(ls_model* m, int E, int d, int j, bool reuse, float min_margin)
 {
-    const int D = m->c.d_model;
-    float* xr = m->x + (size_t)j * D;
+    const int D = m->c.d_model, B = m->nseq;
+    float* xr = m->x + (size_t)j * B * D;  // rows j B .. j B + B - 1: draft position j of every sequence
     m->gate = min_margin > 0.f ? j : 0;
-    LS_TRY(run_embed(m, j == 0 ? m->ctl + CTL_CUR_TOK : m->draft + (j - 1), 1, xr, j));
+    if (j == 0) LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, B, xr, 0, CTL_WORDS));
+    else LS_TRY(run_embed(m, m->draft + (size_t)(j - 1) * B, B, xr, j * B));
     // the exit-layer row goes to the LM head (final gain) and, pre-scaled by layer E's
     // gain, to the verify pass (the exit-layer cache of Sec. 4.3.3)
-    LS_TRY(run_layers(m, 0, E, 1, xr, j, j, m->h + (size_t)j * D, j < d ? m->fnorm : nullptr,
+    LS_TRY(run_layers(m, 0, E, B, xr, j, j * B, m->h + (size_t)j * B * D, j < d ? m->fnorm : nullptr,
                       reuse ? m->lw[E].attn_norm : nullptr));
-    if (j < d) LS_TRY(run_head(m, 1, j, m->draft + j, nullptr, min_margin));
+    if (j < d) LS_TRY(run_head(m, B, j * B, m->draft + (size_t)j * B, nullptr, min_margin));
     m->gate = 0;
+    return LS_OK;
+}
+
+int enqueue_accept(ls_model* m, int d, bool adaptive)
+{
+    const LaunchCtx lc = {m->st, m->pdl};
+    if (m->nseq > 1)
+        LS_CK(launch(lc, accept_batch_kernel, dim3(1), dim3(32), 0, (const int32_t*)m->draft, (const int32_t*)m->verified, d,
+                     m->nseq, m->ctl, m->out_ids, m->accepted, m->seq_cap));
+    else
+        LS_CK(launch(lc, accept_kernel, dim3(1), dim3(32), 0, (const int32_t*)m->draft, (const int32_t*)m->verified, d,
+                     m->ctl, m->out_ids, m->accepted, adaptive ? 1 : 0, adaptive ? m->drafted : (int32_t*)nullptr));
+    m->launches += 1;
     return LS_OK;
 }
 
 // verify pass + accept of a step
 int enqueue_verify(ls_model* m, int E, int d, bool reuse, float min_margin)
 {
-    const int D = m->c.d_model, L = m->c.n_layers;
-    const bool adaptive = min_margin > 0.f;
+    const int D = m->c.d_model, L = m->c.n_layers, B = m->nseq;
     if (reuse) {
         // self-verification (Sec. 4.3.2) from the exit-layer activations
-        LS_TRY(run_layers(m, E, L, d + 1, m->x, 0, 0, m->hE, m->fnorm, nullptr));
+        LS_TRY(run_layers(m, E, L, (d + 1) * B, m->x, 0, 0, m->hE, m->fnorm, nullptr));
     } else {
         // the ablation of Sec. 7 (Table 7): no exit-layer cache, verification recomputes the
         // early layers of all d+1 rows (and rewrites their k, v with the same values)
-        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
-        LS_TRY(run_embed(m, m->draft, d, m->x + D, 1));
-        LS_TRY(run_layers(m, 0, L, d + 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
+        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, B, m->x, 0, CTL_WORDS));
+        LS_TRY(run_embed(m, m->draft, d * B, m->x + (size_t)B * D, B));
+        LS_TRY(run_layers(m, 0, L, (d + 1) * B, m->x, 0, 0, m->h, m->fnorm, nullptr));
     }
-    LS_TRY(run_head(m, d + 1, 0, m->verified, nullptr));
-    LS_CK(launch(LaunchCtx{m->st, m->pdl}, accept_kernel, dim3(1), dim3(32), 0, (const int32_t*)m->draft,
-                 (const int32_t*)m->verified, d, m->ctl, m->out_ids, m->accepted, adaptive ? 1 : 0,
-                 adaptive ? m->drafted : (int32_t*)nullptr));
-    m->launches += 1;
-    return LS_OK;
+    LS_TRY(run_head(m, (d + 1) * B, 0, m->verified, nullptr));
+    return enqueue_accept(m, d, min_margin > 0.f);
 }
 
 int enqueue_step(ls_model* m, int E, int d, bool reuse, float min_margin = 0.f)
 {
     if (d == 0) {
-        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, 1, m->x, 0));
-        LS_TRY(run_layers(m, 0, E, 1, m->x, 0, 0, m->h, m->fnorm, nullptr));
-        LS_TRY(run_head(m, 1, 0, m->verified, nullptr));
-        LS_CK(launch(LaunchCtx{m->st, m->pdl}, accept_kernel, dim3(1), dim3(32), 0, (const int32_t*)m->draft,
-                     (const int32_t*)m->verified, 0, m->ctl, m->out_ids, m->accepted, 0, (int32_t*)nullptr));
-        m->launches += 1;
-        return LS_OK;
+        LS_TRY(run_embed(m, m->ctl + CTL_CUR_TOK, m->nseq, m->x, 0, CTL_WORDS));
+        LS_TRY(run_layers(m, 0, E, m->nseq, m->x, 0, 0, m->h, m->fnorm, nullptr));
+        LS_TRY(run_head(m, m->nseq, 0, m->verified, nullptr));
+        return enqueue_accept(m, 0, false);
     }
     for (int j = 0; j <= (reuse ? d : d - 1); ++j)  // self-drafting (Sec. 4.3.1) + the extra early pass
         LS_TRY(enqueue_draft_pass(m, E, d, j, reuse, min_margin));
@@ -800,7 +821,7 @@ int get_graph(ls_model* m, int E, int d, bool reuse, float min_margin, ls_model:
     uint32_t mbits;
     memcpy(&mbits, &min_margin, sizeof(mbits));
     const std::pair<uint64_t, uint32_t> key(
-        ((uint64_t)(reuse ? 0 : 1) << 48) | ((uint64_t)E << 32) | ((uint64_t)d << 16), mbits);
+        ((uint64_t)m->nseq << 52) | ((uint64_t)(reuse ? 0 : 1) << 48) | ((uint64_t)E << 32) | ((uint64_t)d << 16), mbits);
     auto it = m->graphs.find(key);
     if (it == m->graphs.end()) {
         if (m->graphs.size() >= 64) drop_graphs(m);  // a bound on what a long-lived handle keeps
@@ -859,6 +880,83 @@ int check_ids(const ls_model* m, const int32_t* ids, int n)
     for (int i = 0; i < n; ++i)
         if (ids[i] < 0 || ids[i] >= m->c.vocab) return LS_ERR_INVALID_ARG;
     return LS_OK;
+}
+
+// rows 0 .. n_prompt-2 of one prompt through `layers` layers into the cache of the sequence the
+// model's view (pt, seq_cap) points at; the last prompt token is the first input of the loop
+int prefill_rows(ls_model* m, const int32_t* prompt, int n_prompt, int layers)
+{
+    LS_CK(cudaMemcpyAsync(m->ids, prompt, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, m->st));
+    LS_TRY(write_ctl(m, 0, 0, 0));
+    const int rows = n_prompt - 1;
+    if (rows > kMaxRows && m->big_prefill) {
+        // the prompt pass proper: blocks of up to 1024 rows on the tensor cores
+        const int pb = m->c.max_seq < kPrefillBlock ? m->c.max_seq : kPrefillBlock;
+        for (int r0 = 0; r0 < rows; r0 += pb) LS_TRY(prefill_block(m, r0, rows - r0 < pb ? rows - r0 : pb, layers));
+    } else {
+        for (int r0 = 0; r0 < rows; r0 += kMaxRows) {
+            int M = rows - r0;
+            if (M > kMaxRows) M = kMaxRows;
+            LS_TRY(run_embed(m, m->ids + r0, M, m->x, 0));
+            LS_TRY(run_layers(m, 0, layers, M, m->x, r0, 0, m->h, nullptr, nullptr));
+        }
+    }
+    return LS_OK;
+}
+
+// the model's view of its sequences for the duration of a call
+struct SeqView {
+    ls_model* m;
+    SeqView(ls_model* m_, int nseq, int pt_stride, int cap, const int32_t* pt) : m(m_)
+    {
+        m->nseq = nseq;
+        m->pt_stride = pt_stride;
+        m->seq_cap = cap;
+        m->pt = pt;
+    }
+    ~SeqView()
+    {
+        m->nseq = 1;
+        m->pt_stride = 0;
+        m->seq_cap = m->c.max_seq;
+        m->pt = m->page_table;
+    }
+};
+
+// algorithmic bytes of one sequence's schedule: weights of `steps` steps and the k, v rows read
+void schedule_bytes(const ls_config& c, int E, int d, bool reuse, int n_prompt, const int32_t* acc, const int32_t* kept,
+                    int steps, int64_t* wb_out, int64_t* kb_out, int64_t* acc_out)
+{
+    const int L = c.n_layers;
+    const int64_t qw = (int64_t)c.n_heads * c.head_dim, kvw = (int64_t)c.n_kv_heads * c.head_dim;
+    const int64_t w_layer = 2 * ((qw + 2 * kvw) * c.d_model + qw * c.d_model + 3 * (int64_t)c.d_model * c.d_ffn);
+    const int64_t w_lm = 2 * (int64_t)c.vocab * c.d_model;
+    const int64_t kvb = 2 * 2 * kvw;
+    int64_t wb = 0, kb = 0, cl = n_prompt - 1, acc_sum = 0;
+    for (int s = 0; s < steps; ++s) {
+        const int n = acc[s];
+        if (d == 0) {
+            wb += E * w_layer + w_lm;
+            kb += (int64_t)E * kvb * (cl + 1);
+        } else if (reuse) {
+            // draft passes that ran: all d + 1, or with an early stop the k + 1 up to the one
+            // whose head stopped the drafting (k drafts kept); heads: one per pass but the extra one
+            const int k = kept ? kept[s] : d;
+            const int heads = k < d ? k + 1 : d;
+            wb += (int64_t)(k + 1) * E * w_layer + (int64_t)heads * w_lm + (int64_t)(L - E) * w_layer + w_lm;
+            for (int j = 0; j <= k; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
+            kb += (int64_t)(L - E) * kvb * (cl + k + 1);
+        } else {
+            wb += (int64_t)d * (E * w_layer + w_lm) + (int64_t)L * w_layer + w_lm;
+            for (int j = 0; j < d; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
+            kb += (int64_t)L * kvb * (cl + d + 1);
+        }
+        cl += n + 1;
+        acc_sum += n;
+    }
+    *wb_out = wb;
+    *kb_out = kb;
+    *acc_out = acc_sum;
 }
 
 int decode_loop(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new, int32_t flags, float min_margin);
@@ -950,6 +1048,10 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
     size_t used = carve(*cfg, (unsigned char*)workspace, m);
     m->n_prompt = 0;
     m->prefilled_layers = 0;
+    m->nseq = 1;
+    m->pt_stride = 0;
+    m->seq_cap = cfg->max_seq;
+    m->pt = m->page_table;
     m->use_graphs = getenv("LS_NO_GRAPH") == nullptr;
     m->pdl = getenv("LS_NO_PDL") == nullptr;
     m->cond_graphs = getenv("LS_NO_COND") == nullptr;
@@ -1026,22 +1128,9 @@ int ls_prefill(ls_model* m, const int32_t* prompt, int32_t n_prompt, int32_t lay
     if (layers < 1 || layers > L) return LS_ERR_INVALID_ARG;
     if (n_prompt > m->c.max_seq) return LS_ERR_CAPACITY;
     m->n_prompt = 0;
-    LS_CK(cudaMemcpyAsync(m->ids, prompt, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, m->st));
-    LS_TRY(write_ctl(m, 0, 0, 0));
+    m->b_n_prompt.clear();
     LS_CK(cudaEventRecord(m->ev0, m->st));
-    const int rows = n_prompt - 1;
-    if (rows > kMaxRows && m->big_prefill) {
-        // the prompt pass proper: blocks of up to 1024 rows on the tensor cores
-        const int pb = m->c.max_seq < kPrefillBlock ? m->c.max_seq : kPrefillBlock;
-        for (int r0 = 0; r0 < rows; r0 += pb) LS_TRY(prefill_block(m, r0, rows - r0 < pb ? rows - r0 : pb, layers));
-    } else {
-        for (int r0 = 0; r0 < rows; r0 += kMaxRows) {
-            int M = rows - r0;
-            if (M > kMaxRows) M = kMaxRows;
-            LS_TRY(run_embed(m, m->ids + r0, M, m->x, 0));
-            LS_TRY(run_layers(m, 0, layers, M, m->x, r0, 0, m->h, nullptr, nullptr));
-        }
-    }
+    LS_TRY(prefill_rows(m, prompt, n_prompt, layers));
     LS_CK(cudaEventRecord(m->ev1, m->st));
     int32_t w[CTL_WORDS];
     LS_TRY(read_ctl(m, w));
@@ -1147,34 +1236,9 @@ int decode_loop(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_
     LS_CK(cudaStreamSynchronize(m->st));
 
     // algorithmic bytes of the schedule (matrices only; norm gains and activations are noise)
-    const int64_t qw = (int64_t)c.n_heads * c.head_dim, kvw = (int64_t)c.n_kv_heads * c.head_dim;
-    const int64_t w_layer = 2 * ((qw + 2 * kvw) * c.d_model + qw * c.d_model + 3 * (int64_t)c.d_model * c.d_ffn);
-    const int64_t w_lm = 2 * (int64_t)c.vocab * c.d_model;
-    const int64_t kvb = 2 * 2 * kvw;
-    int64_t wb = 0, kb = 0, cl = m->n_prompt - 1, acc_sum = 0;
-    for (int s = 0; s < m->h_n_steps; ++s) {
-        int n = m->h_acc[s];
-        if (d == 0) {
-            wb += E * w_layer + w_lm;
-            kb += (int64_t)E * kvb * (cl + 1);
-        } else {
-            if (reuse) {
-                // draft passes that ran: all d + 1, or with an early stop the k + 1 up to the one
-                // whose head stopped the drafting (k drafts kept); heads: one per pass but the extra one
-                const int k = m->h_drafted[s];
-                const int heads = k < d ? k + 1 : d;
-                wb += (int64_t)(k + 1) * E * w_layer + (int64_t)heads * w_lm + (int64_t)(L - E) * w_layer + w_lm;
-                for (int j = 0; j <= k; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
-                kb += (int64_t)(L - E) * kvb * (cl + k + 1);
-            } else {
-                wb += (int64_t)d * (E * w_layer + w_lm) + (int64_t)L * w_layer + w_lm;
-                for (int j = 0; j < d; ++j) kb += (int64_t)E * kvb * (cl + j + 1);
-                kb += (int64_t)L * kvb * (cl + d + 1);
-            }
-        }
-        cl += n + 1;
-        acc_sum += n;
-    }
+    int64_t wb = 0, kb = 0, acc_sum = 0;
+    schedule_bytes(c, E, d, reuse, m->n_prompt, m->h_acc.data(), adaptive ? m->h_drafted.data() : nullptr, m->h_n_steps, &wb,
+                   &kb, &acc_sum);
     m->stats.decode_ms = ms;
     m->stats.weight_bytes = wb;
     m->stats.kv_bytes = kb;
@@ -1257,6 +1321,173 @@ int ls_generate_early(ls_model* m, const int32_t* prompt, int32_t n_prompt, int3
     return ls_read_output(m, out_ids, out_n, nullptr, nullptr);
 }
 
+// ------------------------------------------------------------------ several sequences per pass
+int ls_prefill_batch(ls_model* m, int32_t n_seq, const int32_t* prompts, const int32_t* prompt_lens)
+{
+    if (!m || !prompts || !prompt_lens || n_seq < 1 || n_seq > LS_MAX_ROWS) return LS_ERR_INVALID_ARG;
+    const int pps = m->n_pages / n_seq, cap = pps * m->c.page_size;  // pages and positions per sequence
+    size_t off = 0;
+    for (int b = 0; b < n_seq; ++b) {
+        LS_TRY(check_ids(m, prompts + off, prompt_lens[b]));
+        if (prompt_lens[b] > cap) return LS_ERR_CAPACITY;
+        off += prompt_lens[b];
+    }
+    m->n_prompt = 0;  // the single-sequence state is gone: the sequences share its pages
+    m->b_n_prompt.clear();
+    m->b_last_tok.clear();
+    LS_CK(cudaEventRecord(m->ev0, m->st));
+    off = 0;
+    for (int b = 0; b < n_seq; ++b) {
+        SeqView view(m, 1, 0, cap, m->page_table + (size_t)b * pps);
+        LS_TRY(prefill_rows(m, prompts + off, prompt_lens[b], m->c.n_layers));
+        off += prompt_lens[b];
+    }
+    LS_CK(cudaEventRecord(m->ev1, m->st));
+    int32_t w[CTL_WORDS];
+    LS_TRY(read_ctl(m, w));
+    if (w[CTL_STATUS]) return LS_ERR_DEVICE_STATUS;
+    float ms = 0.f;
+    LS_CK(cudaEventElapsedTime(&ms, m->ev0, m->ev1));
+    m->stats.prefill_ms = ms;
+    off = 0;
+    for (int b = 0; b < n_seq; ++b) {
+        m->b_n_prompt.push_back(prompt_lens[b]);
+        m->b_last_tok.push_back(prompts[off + prompt_lens[b] - 1]);
+        off += prompt_lens[b];
+    }
+    m->prefilled_layers = m->c.n_layers;
+    return LS_OK;
+}
+
+int ls_decode_batch(ls_model* m, int32_t exit_layer, int32_t num_draft, int32_t max_new)
+{
+    if (!m || m->b_n_prompt.empty()) return LS_ERR_INVALID_ARG;
+    const ls_config& c = m->c;
+    const int B = (int)m->b_n_prompt.size(), L = c.n_layers;
+    int E = exit_layer, d = num_draft;
+    if (max_new < 1 || d < 0 || E < 0) return LS_ERR_INVALID_ARG;
+    if (E == 0) {
+        if (d != 0) return LS_ERR_INVALID_ARG;
+        E = L;  // plain greedy, B sequences per pass
+    } else {
+        if (d < 1 || E > L - 1) return LS_ERR_INVALID_ARG;
+        if (d > c.max_draft) return LS_ERR_CAPACITY;
+    }
+    if (B * (d + 1) > LS_MAX_ROWS) return LS_ERR_CAPACITY;
+    const int pps = m->n_pages / B, cap = pps * c.page_size;
+    for (int b = 0; b < B; ++b)
+        if ((int64_t)m->b_n_prompt[b] + max_new + d + 1 > cap) return LS_ERR_CAPACITY;
+
+    SeqView view(m, B, pps, cap, m->page_table);
+    ls_model::G* g = nullptr;
+    if (m->use_graphs) LS_TRY(get_graph(m, E, d, true, 0.f, &g));
+    std::vector<int32_t> w((size_t)B * CTL_WORDS, 0);
+    for (int b = 0; b < B; ++b) {
+        int32_t* cb = w.data() + (size_t)b * CTL_WORDS;
+        cb[CTL_CACHE_LEN] = m->b_n_prompt[b] - 1;
+        cb[CTL_CUR_TOK] = m->b_last_tok[b];
+        cb[CTL_MAX_NEW] = max_new;
+        cb[CTL_EOS] = c.eos_id;
+        cb[CTL_D_EFF] = kNoStop;
+    }
+    LS_CK(cudaMemcpyAsync(m->ctl, w.data(), sizeof(int32_t) * w.size(), cudaMemcpyHostToDevice, m->st));
+    LS_CK(cudaStreamSynchronize(m->st));
+    int64_t launched = 0;
+    int syncs = 0, n_out_min = 0, steps_done = 0;
+    LS_CK(cudaEventRecord(m->ev0, m->st));
+    for (;;) {
+        // as in the single-sequence loop, for the sequence that is furthest behind
+        const int remaining = max_new - n_out_min;
+        int steps = (remaining + d) / (d + 1);
+        if (steps_done > 0 && n_out_min > 0) {
+            const int64_t est = ((int64_t)remaining * steps_done + n_out_min - 1) / n_out_min;
+            steps = (int)(est < 1 ? 1 : est);
+        }
+        for (int i = 0; i < steps; ++i) {
+            if (g) {
+                LS_CK(cudaGraphLaunch(g->exec, m->st));
+                launched += g->nodes;
+            } else {
+                const int64_t before = m->launches;
+                LS_TRY(enqueue_step(m, E, d, true, 0.f));
+                launched += m->launches - before;
+            }
+        }
+        LS_CK(cudaMemcpyAsync(w.data(), m->ctl, sizeof(int32_t) * w.size(), cudaMemcpyDeviceToHost, m->st));
+        LS_CK(cudaStreamSynchronize(m->st));
+        ++syncs;
+        n_out_min = max_new;
+        steps_done = 0;
+        for (int b = 0; b < B; ++b) {
+            const int32_t* cb = w.data() + (size_t)b * CTL_WORDS;
+            if (cb[CTL_STATUS]) return LS_ERR_DEVICE_STATUS;
+            if (cb[CTL_N_OUT] < n_out_min) n_out_min = cb[CTL_N_OUT];
+            if (cb[CTL_N_STEPS] > steps_done) steps_done = cb[CTL_N_STEPS];
+        }
+        if (w[CTL_DONE]) break;
+    }
+    LS_CK(cudaEventRecord(m->ev1, m->st));
+    LS_CK(cudaEventSynchronize(m->ev1));
+    float ms = 0.f;
+    LS_CK(cudaEventElapsedTime(&ms, m->ev0, m->ev1));
+
+    m->b_out.assign(B, {});
+    m->b_acc.assign(B, {});
+    int64_t kb = 0, acc_sum = 0, n_gen = 0, wb_longest = 0;
+    for (int b = 0; b < B; ++b) {
+        const int32_t* cb = w.data() + (size_t)b * CTL_WORDS;
+        m->b_out[b].resize(cb[CTL_N_OUT]);
+        m->b_acc[b].resize(cb[CTL_N_STEPS]);
+        LS_CK(cudaMemcpyAsync(m->b_out[b].data(), m->out_ids + (size_t)b * cap, sizeof(int32_t) * cb[CTL_N_OUT],
+                              cudaMemcpyDeviceToHost, m->st));
+        LS_CK(cudaMemcpyAsync(m->b_acc[b].data(), m->accepted + (size_t)b * cap, sizeof(int32_t) * cb[CTL_N_STEPS],
+                              cudaMemcpyDeviceToHost, m->st));
+    }
+    LS_CK(cudaStreamSynchronize(m->st));
+    // every weight byte is read once per pass for all sequences: the weights of the longest
+    // sequence's steps; each sequence reads its own k, v rows
+    for (int b = 0; b < B; ++b) {
+        int64_t wb = 0, kbb = 0, ab = 0;
+        schedule_bytes(c, E, d, true, m->b_n_prompt[b], m->b_acc[b].data(), nullptr, (int)m->b_acc[b].size(), &wb, &kbb, &ab);
+        if (wb > wb_longest) wb_longest = wb;
+        kb += kbb;
+        acc_sum += ab;
+        n_gen += (int64_t)m->b_out[b].size();
+    }
+    m->stats.decode_ms = ms;
+    m->stats.weight_bytes = wb_longest;
+    m->stats.kv_bytes = kb;
+    m->stats.kernel_launches = launched;
+    m->stats.n_generated = (int32_t)n_gen;
+    m->stats.n_steps = steps_done;
+    m->stats.n_accepted = (int32_t)acc_sum;
+    m->stats.host_syncs = syncs;
+    return LS_OK;
+}
+
+int ls_read_output_seq(ls_model* m, int32_t seq, int32_t* out_ids, int32_t* out_n, int32_t* accepted, int32_t* out_steps)
+{
+    if (!m || seq < 0 || seq >= (int)m->b_out.size()) return LS_ERR_INVALID_ARG;
+    const std::vector<int32_t>&o = m->b_out[seq], &a = m->b_acc[seq];
+    if (out_ids && !o.empty()) memcpy(out_ids, o.data(), sizeof(int32_t) * o.size());
+    if (out_n) *out_n = (int32_t)o.size();
+    if (accepted && !a.empty()) memcpy(accepted, a.data(), sizeof(int32_t) * a.size());
+    if (out_steps) *out_steps = (int32_t)a.size();
+    return LS_OK;
+}
+
+int ls_generate_batch(ls_model* m, int32_t n_seq, const int32_t* prompts, const int32_t* prompt_lens, int32_t exit_layer,
+                      int32_t num_draft, int32_t max_new, int32_t* out_ids, int32_t* out_n, int32_t* accepted,
+                      int32_t* out_steps)
+{
+    if (!m || !out_ids || !out_n || !accepted || !out_steps || max_new < 1) return LS_ERR_INVALID_ARG;
+    LS_TRY(ls_prefill_batch(m, n_seq, prompts, prompt_lens));
+    LS_TRY(ls_decode_batch(m, exit_layer, num_draft, max_new));
+    for (int b = 0; b < n_seq; ++b)
+        LS_TRY(ls_read_output_seq(m, b, out_ids + (size_t)b * max_new, out_n + b, accepted + (size_t)b * max_new, out_steps + b));
+    return LS_OK;
+}
+
 int ls_debug_logits(ls_model* m, const int32_t* ids, int32_t n, int32_t exit_layer, float* exit_logits,
                     float* final_logits)
 {
@@ -1320,7 +1551,7 @@ int ls_op_embed(const void* emb, const int32_t* tok, int32_t M, int32_t D, int32
     if (!aligned16(emb) || !tok || !aligned16(x) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8 || V < 1)
         return LS_ERR_INVALID_ARG;
     LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, embed_kernel, dim3(M), dim3(256), 0, (const uint16_t*)emb, tok,
-                 D, V, x, nullptr, nullptr, nullptr, nullptr, 0, 0, 0));
+                 D, V, x, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 1));
     return LS_OK;
 }
 

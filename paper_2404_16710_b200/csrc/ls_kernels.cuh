@@ -36,20 +36,22 @@ __device__ __forceinline__ float block_sum_256(float v, float* red)
 }
 
 // ------------------------------------------------------------------ embedding (x_0 = Emb[id])
-// grid M, block 256.  tok[m] is read from device memory.  With gain != nullptr the kernel
+// grid M, block 256.  tok[m * tok_stride] is read from device memory (stride CTL_WORDS: the
+// current tokens in the sequences' control blocks).  With gain != nullptr the kernel
 // also leaves what the first layer's fused RMSNorm needs: hout = bf16(x * gain) and the
 // row's sum of squares in ss_out[m][0] (the other n_part - 1 partial sums are zero).
 __global__ void __launch_bounds__(256)
 embed_kernel(const uint16_t* __restrict__ emb, const int32_t* __restrict__ tok, int D, int V,
              float* __restrict__ x, int32_t* ctl, const uint16_t* __restrict__ gain,
-             uint16_t* __restrict__ hout, float* __restrict__ ss_out, int ss_stride, int n_part, int gate)
+             uint16_t* __restrict__ hout, float* __restrict__ ss_out, int ss_stride, int n_part, int gate,
+             int tok_stride)
 {
     __shared__ float red[8];
     pdl_launch_dependents();
     pdl_wait();
     if (pass_idle(ctl, gate)) return;
     int m = blockIdx.x;
-    int id = tok[m];
+    int id = tok[(size_t)m * tok_stride];
     if (id < 0 || id >= V) {
         if (ctl && threadIdx.x == 0) ctl[CTL_STATUS] = DEV_BAD_TOKEN;
         id = 0;
@@ -333,6 +335,49 @@ __global__ void accept_kernel(const int32_t* __restrict__ draft, const int32_t* 
     ctl[CTL_CUR_TOK] = verified[n];
     ctl[CTL_CACHE_LEN] += n + 1;
     if (stop || n_out >= max_new) ctl[CTL_DONE] = 1;
+}
+
+// The same bookkeeping for B sequences that share every pass (thread b: sequence b).  draft and
+// verified are laid out [position][sequence]; sequence b emits into out_ids + b * out_stride
+// and records into accepted + b * out_stride; a sequence that has finished is left alone (its
+// rows keep running through the passes, nobody reads them).  CTL_DONE of block 0 is set once
+// every sequence has finished.
+__global__ void accept_batch_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ verified,
+                                    int d, int B, int32_t* ctl, int32_t* __restrict__ out_ids,
+                                    int32_t* __restrict__ accepted, int out_stride)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    if (blockIdx.x != 0 || ctl[CTL_DONE]) return;
+    const int b = threadIdx.x;
+    bool finished = true;
+    if (b < B) {
+        int32_t* c = ctl + b * CTL_WORDS;
+        finished = c[CTL_SEQ_DONE] != 0;
+        if (!finished) {
+            int n = 0;
+            while (n < d && draft[n * B + b] == verified[n * B + b]) ++n;
+            int n_out = c[CTL_N_OUT];
+            const int max_new = c[CTL_MAX_NEW], eos = c[CTL_EOS];
+            bool stop = false;
+            for (int i = 0; i <= n && n_out < max_new && !stop; ++i) {
+                const int t = (i < n) ? draft[i * B + b] : verified[n * B + b];
+                out_ids[(size_t)b * out_stride + n_out++] = t;
+                if (eos >= 0 && t == eos) stop = true;
+            }
+            const int steps = c[CTL_N_STEPS];
+            accepted[(size_t)b * out_stride + steps] = n;
+            c[CTL_N_STEPS] = steps + 1;
+            c[CTL_N_OUT] = n_out;
+            c[CTL_CUR_TOK] = verified[n * B + b];
+            c[CTL_CACHE_LEN] += n + 1;
+            if (stop || n_out >= max_new) {
+                c[CTL_SEQ_DONE] = 1;
+                finished = true;
+            }
+        }
+    }
+    if (__syncthreads_and(finished) && threadIdx.x == 0) ctl[CTL_DONE] = 1;
 }
 
 }  // namespace ls

@@ -47,6 +47,7 @@ struct LinArgs {
     const int32_t* page_table;
     uint16_t *q_out, *kpages, *vpages;
     int Hq, Hkv, hd, page_shift, max_seq, pos_off;
+    int nseq, pt_stride;         // sequences sharing the pass (row m: sequence m % nseq) and page-table entries per sequence
     float theta;
     // RMSNorm carried across kernel boundaries.  A producer (residual epilogue, embedding)
     // leaves, beside the fp32 row x, the bf16 row x*gain of its consumer's norm and the sum
@@ -86,12 +87,21 @@ __device__ __forceinline__ void qkv_rotation(const LinArgs& a, int j, int pos, f
     sincosf((float)pos * f, &sn, &cs);
 }
 
+// position of row m of the pass: its sequence's cache length + the launch's offset + its row
+// within the sequence (one sequence: cache length + offset + m)
+__device__ __forceinline__ int row_pos(const LinArgs& a, int m)
+{
+    if (a.nseq <= 1) return (a.ctl ? a.ctl[CTL_CACHE_LEN] : 0) + a.pos_off + m;
+    const int j = m / a.nseq, b = m - j * a.nseq;
+    return a.ctl[b * CTL_WORDS + CTL_CACHE_LEN] + a.pos_off + j;
+}
+
 // rotate the pair (x_j, x_{j+hd/2}) of head `head` for token m and store it: q -> q_out,
-// k, v -> the paged cache row of position pos0 + m (v is not rotated)
-__device__ __forceinline__ void qkv_store(const LinArgs& a, int head, int j, int m, int pos0, float lo, float hi,
+// k, v -> the paged cache row of the row's position in its sequence's pages (v is not rotated)
+__device__ __forceinline__ void qkv_store(const LinArgs& a, int head, int j, int m, int pos, float lo, float hi,
                                           float sn, float cs)
 {
-    const int pos = pos0 + m;
+    const int32_t* page_table = a.page_table + (a.nseq > 1 ? (m % a.nseq) * a.pt_stride : 0);
     if (pos < 0 || pos >= a.max_seq) {
         if (a.ctl) a.ctl[CTL_STATUS] = DEV_POS_OVERFLOW;
         return;
@@ -103,8 +113,8 @@ __device__ __forceinline__ void qkv_store(const LinArgs& a, int head, int j, int
     }
     uint16_t* dst;
     if (head < a.Hq) dst = a.q_out + ((size_t)m * a.Hq + head) * a.hd;
-    else if (head < a.Hq + a.Hkv) dst = a.kpages + kv_row_offset(a.page_table, pos, a.page_shift, a.Hkv, head - a.Hq, a.hd);
-    else dst = a.vpages + kv_row_offset(a.page_table, pos, a.page_shift, a.Hkv, head - a.Hq - a.Hkv, a.hd);
+    else if (head < a.Hq + a.Hkv) dst = a.kpages + kv_row_offset(page_table, pos, a.page_shift, a.Hkv, head - a.Hq, a.hd);
+    else dst = a.vpages + kv_row_offset(page_table, pos, a.page_shift, a.Hkv, head - a.Hq - a.Hkv, a.hd);
     dst[j] = f2bf(lo);
     dst[j + (a.hd >> 1)] = f2bf(hi);
 }
@@ -251,17 +261,17 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
                         a.out_bf16[(size_t)m * a.N + nrow[r]] = f2bf(silu_mul(acc[r][m], acc[r + 2][m]));
             }
     } else if (EPI == EPI_QKV) {
-        const int pos0 = (a.ctl ? a.ctl[CTL_CACHE_LEN] : 0) + a.pos_off;
         const int tph = a.hd >> 4;
 #pragma unroll
         for (int m = 0; m < MT; ++m)
             if (lane == m && m < a.M) {
+                const int pos = row_pos(a, m);
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
                     const int j = (blockIdx.x % tph) * 8 + warp * 2 + r;
                     float sn, cs;
-                    qkv_rotation(a, j, pos0 + m, sn, cs);
-                    qkv_store(a, blockIdx.x / tph, j, m, pos0, acc[r][m], acc[r + 2][m], sn, cs);
+                    qkv_rotation(a, j, pos, sn, cs);
+                    qkv_store(a, blockIdx.x / tph, j, m, pos, acc[r][m], acc[r + 2][m], sn, cs);
                 }
             }
     } else {  // EPI_ARGMAX
@@ -427,7 +437,7 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
     // the residual values and gains (EPI_RESIDUAL), the rotation factors (EPI_QKV)
     constexpr int FRAGS = TR * NT;
     float xin[4] = {0.f, 0.f, 0.f, 0.f}, gA[2] = {0.f, 0.f}, gB[2] = {0.f, 0.f}, rsn[2] = {0.f, 0.f}, rcs[2] = {1.f, 1.f};
-    int pos0_epi = 0;
+    int pos_epi[2] = {0, 0};  // positions of the thread's two token rows (EPI_QKV)
     if (tid < 32 * FRAGS) {
         const int efr = tid >> 5, etile = blockIdx.x * TR + efr / NT, em0 = (efr % NT) * 8 + 2 * t;
         if (EPI == EPI_RESIDUAL) {
@@ -446,12 +456,13 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
                 if (a.hout_b) gB[1] = bf16f(a.gain_b[nhi]);
             }
         } else if (EPI == EPI_QKV) {
-            pos0_epi = (a.ctl ? a.ctl[CTL_CACHE_LEN] : 0) + a.pos_off;
+            pos_epi[0] = row_pos(a, min(em0, a.M - 1));
+            pos_epi[1] = row_pos(a, min(em0 + 1, a.M - 1));
             const int tph = a.hd >> 4;
             if (etile < (a.N >> 4) && etile / tph < a.Hq + a.Hkv) {
                 const int j = (etile % tph) * 8 + g;
-                qkv_rotation(a, j, pos0_epi + em0, rsn[0], rcs[0]);
-                qkv_rotation(a, j, pos0_epi + em0 + 1, rsn[1], rcs[1]);
+                qkv_rotation(a, j, pos_epi[0], rsn[0], rcs[0]);
+                qkv_rotation(a, j, pos_epi[1], rsn[1], rcs[1]);
             }
         }
     }
@@ -550,8 +561,8 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             if (tile < (a.N >> 4)) {
                 const int tph = a.hd >> 4;
                 const int head = tile / tph, j = (tile % tph) * 8 + gg;
-                if (m0 < a.M) qkv_store(a, head, j, m0, pos0_epi, r[0], r[2], rsn[0], rcs[0]);
-                if (m0 + 1 < a.M) qkv_store(a, head, j, m0 + 1, pos0_epi, r[1], r[3], rsn[1], rcs[1]);
+                if (m0 < a.M) qkv_store(a, head, j, m0, pos_epi[0], r[0], r[2], rsn[0], rcs[0]);
+                if (m0 + 1 < a.M) qkv_store(a, head, j, m0 + 1, pos_epi[1], r[1], r[3], rsn[1], rcs[1]);
             }
         } else {
             vals[tr * 16 + gg][m0] = r[0];
