@@ -267,7 +267,9 @@ int ls_op_lm_head_argmax(int32_t linear_path, const void *w_dev, const void *h_b
  * cudaFree and calls nothing that allocates.
  *   - V <= LS_OP_LM_HEAD_STATIC_MAX_VOCAB, otherwise LS_ERR_CAPACITY (nothing is launched).
  *   - The first call on each device looks up the buffer's device address (with that device
- *     current); make that first call outside any stream capture.
+ *     current); make that first call outside any stream capture.  The first call of each kernel
+ *     configuration (linear path, and the class of M, V and K) also sets a kernel attribute and
+ *     loads the kernel: warm up with the same path and sizes as the calls that follow.
  *   - All calls share the one buffer and it keeps the previous call's contents.  Nothing
  *     in it has to start at zero: every candidate the finishing kernel reads is rewritten
  *     by the same call.  Two calls that may run on the GPU at the same time (different

@@ -42,6 +42,20 @@ def test_static_scratch_entry_point_matches_the_ordinary_one_twice_in_a_row(path
         assert int(want.min()) >= 0 and int(want.max()) < V
 
 
+def test_static_scratch_entry_point_leaves_device_memory_as_it_is():
+    """After a first call of the same configuration (which loads the kernel and looks the
+    buffer's address up), a call changes neither the free device memory nor what torch has
+    reserved: the entry point and everything under it allocate nothing."""
+    w, h = _case(3, 5, 4096, 256)
+    tok = torch.empty((5,), dtype=torch.int32, device="cuda")
+    B.ls_op_lm_head_argmax_static(B.LS_LINEAR_MMA, w, h, tok)
+    torch.cuda.synchronize()
+    free0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_reserved()
+    B.ls_op_lm_head_argmax_static(B.LS_LINEAR_MMA, w, h, tok)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_reserved() == reserved0
+
+
 def test_static_scratch_entry_point_refuses_a_vocabulary_beyond_its_buffer():
     V = B.LS_OP_LM_HEAD_STATIC_MAX_VOCAB + 16
     w = torch.zeros((V, 8), dtype=torch.bfloat16, device="cuda")
