@@ -44,6 +44,42 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return (uint32_t)f2bf(lo) | ((uint32_t)f2bf(hi) << 16);
 }
 
+// Sums of squares for the RMSNorm that is carried across kernel boundaries are kept EXACT: every
+// x^2 is rounded once to a multiple of 2^-32 and the multiples are added as 64-bit integers.
+// Integer addition is associative, so the sum of a row does not depend on how the row's columns
+// are dealt out to CTAs, warps and lanes -- kernels of any tiling leave the same bits, and a
+// pass of several rows reproduces single-row decoding whatever configuration it runs in.
+// Range: x^2 < 2^31 per element (saturating), row sums below 2^31 (rms up to ~700 at D = 4096).
+__device__ __forceinline__ long long sq_fixed(float x) { return __float2ll_rn(x * x * 4294967296.0f); }
+__device__ __forceinline__ float rms_rscale(long long ss, float inv_d, float eps)
+{
+    return 1.0f / sqrtf((float)ss * (1.0f / 4294967296.0f) * inv_d + eps);
+}
+// A row's sum is spread over kSsSlots accumulators (a CTA adds to slot blockIdx.x % kSsSlots)
+// so that the hundreds of CTAs of a projection do not queue up on one address; a consumer adds
+// the slots up -- in any order, the sum is exact.
+constexpr int kSsSlots = 16;
+__device__ __forceinline__ void ss_add(long long* row, long long v)
+{
+    atomicAdd(reinterpret_cast<unsigned long long*>(row + (blockIdx.x & (kSsSlots - 1))), (unsigned long long)v);
+}
+// Consumer side, called by the first 256 (or all, if fewer) threads of a CTA, whole warps: rs[m] =
+// 1 / sqrt(mean x^2 + eps) of rows m < M (M * kSsSlots <= threads calling); with clear != nullptr
+// CTA 0 zeroes the slots of the rows its successor's producer will add to.
+__device__ __forceinline__ void rms_rscales(const long long* sums, long long* clear, int M, float inv_d, float eps,
+                                            float* rs)
+{
+    const int i = threadIdx.x;
+    long long v = 0;
+    if (i < M * kSsSlots) {
+        v = __ldcg(sums + i);
+        if (clear && blockIdx.x == 0) clear[i] = 0;
+    }
+#pragma unroll
+    for (int o = kSsSlots / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (i < M * kSsSlots && (i & (kSsSlots - 1)) == 0) rs[i / kSsSlots] = rms_rscale(v, inv_d, eps);
+}
+
 // 16-byte read of streamed-once data (weights): do not allocate in L1, so that the
 // activations, which every CTA re-reads, stay there.
 __device__ __forceinline__ uint4 ld_stream16(const void* p)

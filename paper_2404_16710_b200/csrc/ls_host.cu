@@ -96,8 +96,10 @@ struct ls_model {
     uint16_t* hE;  // exit-layer activations, already multiplied by the gain of layer E's norm (Sec. 4.3.3)
     float *px, *py;          // prompt pass: residual rows and projection outputs of one block
     uint16_t *ph, *pq, *po, *pa;
-    float* ss;     // [16][n_part] partial sums of squares of the residual rows (fused RMSNorm)
-    int n_part;
+    // exact sums of squares of the residual rows (fused RMSNorm), [16][kSsSlots] each: after the
+    // attention block (o-proj adds, gate-up reads) and after the FFN or the embedding (down-proj
+    // adds, q|k|v and the LM head read)
+    long long *ss_attn, *ss_ffn;
     ValIdx* cand;
     float* second;      // per-CTA second-largest logit beside each argmax candidate (adaptive drafting)
     int32_t* drafted;   // drafts kept per step (adaptive drafting)
@@ -162,8 +164,7 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     unsigned char* cand = take(sizeof(ValIdx) * kMaxRows * cand_stride);
     unsigned char* second = take(sizeof(float) * kMaxRows * cand_stride);
     unsigned char* drafted = take(sizeof(int32_t) * c.max_seq);
-    const int n_part = (c.d_model + 15) / 16;  // CTAs of a residual projection = partial sums per row
-    unsigned char* ss = take(sizeof(float) * kMaxRows * n_part);
+    unsigned char* ss = take(sizeof(long long) * kMaxRows * kSsSlots * 2);
     unsigned char* he = take(2 * (size_t)kMaxRows * c.d_model);
     const int pb = c.max_seq < kPrefillBlock ? c.max_seq : kPrefillBlock;  // rows per block of the prompt pass
     const size_t ywide = (qw + 2 * kvw) > 2 * (size_t)c.d_ffn ? (qw + 2 * kvw) : 2 * (size_t)c.d_ffn;
@@ -180,9 +181,9 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
         m->pq = (uint16_t*)pq;
         m->po = (uint16_t*)po;
         m->pa = (uint16_t*)pa;
-        m->ss = (float*)ss;
+        m->ss_attn = (long long*)ss;
+        m->ss_ffn = m->ss_attn + kMaxRows * kSsSlots;
         m->hE = (uint16_t*)he;
-        m->n_part = n_part;
         m->kpages = (uint16_t*)kp;
         m->vpages = (uint16_t*)vp;
         m->layer_kv_elems = layer_kv;
@@ -370,20 +371,19 @@ LinArgs lin_args(const uint16_t* w, const uint16_t* h, int M, int N, int K)
 }
 
 // layers [l0, l1) on M residual rows starting at xrow; row r sits at ctl.cache_len + pos_off + r
-// fused-RMSNorm fields of a consumer / of a residual producer
-void norm_in(const ls_model* m, LinArgs& a, int slot)
+// fused-RMSNorm fields of a consumer (sums it reads, sums it clears for the producer after
+// it) and of a residual producer (sums it adds to, rows x*gain it leaves)
+void norm_in(const ls_model* m, LinArgs& a, const long long* sums, long long* clear)
 {
-    a.ss_in = m->ss + (size_t)slot * m->n_part;
-    a.ss_stride = m->n_part;
-    a.n_part = m->n_part;
+    a.ss_in = sums;
+    a.ss_clear = clear;
     a.inv_d = 1.0f / (float)m->c.d_model;
     a.eps = m->c.rms_eps;
 }
-void norm_out(const ls_model* m, LinArgs& a, int slot, const uint16_t* gain_a, uint16_t* hout_a,
-              const uint16_t* gain_b, uint16_t* hout_b)
+void norm_out(LinArgs& a, long long* sums, const uint16_t* gain_a, uint16_t* hout_a, const uint16_t* gain_b,
+              uint16_t* hout_b)
 {
-    a.ss_out = m->ss + (size_t)slot * m->n_part;
-    a.ss_stride = m->n_part;
+    a.ss_out = sums;
     a.gain_a = gain_a;
     a.hout_a = gain_a ? hout_a : nullptr;
     a.gain_b = gain_b;
@@ -429,7 +429,7 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off, int
         a.pos_off = pos_off;
         a.theta = c.rope_theta;
         a.gate = m->gate;
-        norm_in(m, a, slot);
+        norm_in(m, a, m->ss_ffn + slot * kSsSlots, m->ss_attn + slot * kSsSlots);  // rows left by an embedding or a down projection
         LS_CK(launch_linear(m->path, EPI_QKV, a, st));
         LS_TRY(attn_launch(m->attn, m->q, kp, vp, m->pt, m->ctl, pos_off, M, Hq, Hkv, hd, m->page_shift, m->seq_cap, m->o,
                            st, m->gate, m->nseq, m->pt_stride));
@@ -438,22 +438,22 @@ int run_layers(ls_model* m, int l0, int l1, int M, float* xrow, int pos_off, int
         a.ldo = D;
         a.ctl = m->ctl;
         a.gate = m->gate;
-        norm_out(m, a, slot, w.ffn_norm, hrow, nullptr, nullptr);
+        norm_out(a, m->ss_attn + slot * kSsSlots, w.ffn_norm, hrow, nullptr, nullptr);
         LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
         a = lin_args(w.wg, hrow, M, F, D);
         a.w1 = w.wu;
         a.out_bf16 = m->a;
         a.ctl = m->ctl;
         a.gate = m->gate;
-        norm_in(m, a, slot);
+        norm_in(m, a, m->ss_attn + slot * kSsSlots, m->ss_ffn + slot * kSsSlots);
         LS_CK(launch_linear(m->path, EPI_SWIGLU, a, st));
         a = lin_args(w.wd, m->a, M, D, F);
         a.out = xrow;
         a.ldo = D;
         a.ctl = m->ctl;
         a.gate = m->gate;
-        if (l + 1 < l1) norm_out(m, a, slot, m->lw[l + 1].attn_norm, hrow, nullptr, nullptr);
-        else norm_out(m, a, slot, gain_end_a, hrow, gain_end_b, herow);
+        if (l + 1 < l1) norm_out(a, m->ss_ffn + slot * kSsSlots, m->lw[l + 1].attn_norm, hrow, nullptr, nullptr);
+        else norm_out(a, m->ss_ffn + slot * kSsSlots, gain_end_a, hrow, gain_end_b, herow);
         LS_CK(launch_linear(m->path, EPI_RESIDUAL, a, st));
         m->launches += 5;
     }
@@ -477,7 +477,7 @@ int run_head(ls_model* m, int M, int slot, int32_t* tok_out, float* logits, floa
     a.ctl = m->ctl;
     a.gate = m->gate;
     a.second = min_margin > 0.f ? m->second : nullptr;
-    norm_in(m, a, slot);
+    norm_in(m, a, m->ss_ffn + slot * kSsSlots, nullptr);
     LS_CK(launch_linear(m->path, EPI_ARGMAX, a, st));
     LS_CK(launch(st, argmax_finish_kernel, dim3(M), dim3(256), 0, (const ValIdx*)m->cand,
                  n_candidates(m->path, c.vocab, c.d_model, M), m->cand_stride, tok_out, m->ctl,
@@ -490,7 +490,7 @@ int run_embed(ls_model* m, const int32_t* tok_dev, int M, float* xrow, int slot,
 {
     LS_CK(launch(LaunchCtx{m->st, m->pdl}, embed_kernel, dim3(M), dim3(256), 0, m->emb, tok_dev, m->c.d_model,
                  m->c.vocab, xrow, m->ctl, m->lw[0].attn_norm, m->h + (size_t)slot * m->c.d_model,
-                 m->ss + (size_t)slot * m->n_part, m->n_part, m->n_part, m->gate, tok_stride));
+                 m->ss_ffn + slot * kSsSlots, m->gate, tok_stride));
     m->launches += 1;
     return LS_OK;
 }
@@ -642,7 +642,7 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
     const LaunchCtx lc = {st, false};
     int32_t* status = m->ctl + CTL_STATUS;
     LS_CK(launch(lc, embed_kernel, dim3(R), dim3(256), 0, m->emb, m->ids + r0, D, c.vocab, m->px, m->ctl, nullptr,
-                 nullptr, nullptr, 0, 0, 0, 1));
+                 nullptr, nullptr, 0, 1));
     for (int l = 0; l < layers; ++l) {
         const LayerW& w = m->lw[l];
         uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
@@ -1551,7 +1551,7 @@ int ls_op_embed(const void* emb, const int32_t* tok, int32_t M, int32_t D, int32
     if (!aligned16(emb) || !tok || !aligned16(x) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8 || V < 1)
         return LS_ERR_INVALID_ARG;
     LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, embed_kernel, dim3(M), dim3(256), 0, (const uint16_t*)emb, tok,
-                 D, V, x, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 1));
+                 D, V, x, nullptr, nullptr, nullptr, nullptr, 0, 1));
     return LS_OK;
 }
 

@@ -39,14 +39,13 @@ __device__ __forceinline__ float block_sum_256(float v, float* red)
 // grid M, block 256.  tok[m * tok_stride] is read from device memory (stride CTL_WORDS: the
 // current tokens in the sequences' control blocks).  With gain != nullptr the kernel
 // also leaves what the first layer's fused RMSNorm needs: hout = bf16(x * gain) and the
-// row's sum of squares in ss_out[m][0] (the other n_part - 1 partial sums are zero).
+// row's exact sum of squares (ls_common.cuh) in slot 0 of ss_out[m][kSsSlots] (the other slots zero).
 __global__ void __launch_bounds__(256)
 embed_kernel(const uint16_t* __restrict__ emb, const int32_t* __restrict__ tok, int D, int V,
              float* __restrict__ x, int32_t* ctl, const uint16_t* __restrict__ gain,
-             uint16_t* __restrict__ hout, float* __restrict__ ss_out, int ss_stride, int n_part, int gate,
-             int tok_stride)
+             uint16_t* __restrict__ hout, long long* __restrict__ ss_out, int gate, int tok_stride)
 {
-    __shared__ float red[8];
+    __shared__ long long red[8];
     pdl_launch_dependents();
     pdl_wait();
     if (pass_idle(ctl, gate)) return;
@@ -58,7 +57,7 @@ embed_kernel(const uint16_t* __restrict__ emb, const int32_t* __restrict__ tok, 
     }
     const uint4* src = reinterpret_cast<const uint4*>(emb + (size_t)id * D);
     float4* dst = reinterpret_cast<float4*>(x + (size_t)m * D);
-    float ss = 0.f;
+    long long ss = 0;
     for (int c = threadIdx.x; c < D / 8; c += 256) {
         uint4 v = src[c];
         const float f[8] = {bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y),
@@ -76,12 +75,22 @@ embed_kernel(const uint16_t* __restrict__ emb, const int32_t* __restrict__ tok, 
             o.w = pack_bf16(f[6] * g[6], f[7] * g[7]);
             reinterpret_cast<uint4*>(hout + (size_t)m * D)[c] = o;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+            for (int e = 0; e < 8; ++e) ss += sq_fixed(f[e]);
         }
     }
     if (gain) {
-        const float tot = block_sum_256(ss, red);
-        for (int i = threadIdx.x; i < n_part; i += 256) ss_out[(size_t)m * ss_stride + i] = (i == 0) ? tot : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        if (threadIdx.x < kSsSlots) {
+            long long tot = 0;
+            if (threadIdx.x == 0) {
+#pragma unroll
+                for (int w = 0; w < 8; ++w) tot += red[w];
+            }
+            ss_out[(size_t)m * kSsSlots + threadIdx.x] = tot;
+        }
     }
 }
 

@@ -50,27 +50,18 @@ struct LinArgs {
     int nseq, pt_stride;         // sequences sharing the pass (row m: sequence m % nseq) and page-table entries per sequence
     float theta;
     // RMSNorm carried across kernel boundaries.  A producer (residual epilogue, embedding)
-    // leaves, beside the fp32 row x, the bf16 row x*gain of its consumer's norm and the sum
-    // of x^2 over its own columns; a consumer reads those rows as h, adds the partial sums in
-    // index order and scales its accumulators by 1/sqrt(mean x^2 + eps): W (x g) r = W (x r g).
-    const float* ss_in;      // consumer: [M][ss_stride] partial sums of squares; nullptr: no scaling
-    float* ss_out;           // EPI_RESIDUAL: ss_out[m * ss_stride + cta]
-    int ss_stride, n_part;   // n_part: partial sums per row (CTAs of the producer)
+    // leaves, beside the fp32 row x, the bf16 row x*gain of its consumer's norm and adds the
+    // squares of its own columns to the row's exact sum (ls_common.cuh); a consumer reads those
+    // rows as h and scales its accumulators by 1/sqrt(mean x^2 + eps): W (x g) r = W (x r g).
+    // The sums of the two norms of a layer live in two arrays; a consumer clears the rows of
+    // the array its successor's producer will add to.
+    const long long* ss_in;  // consumer: [M][kSsSlots] sums of squares; nullptr: no scaling
+    long long* ss_out;       // EPI_RESIDUAL: [M][kSsSlots] sums this launch adds to (cleared beforehand)
+    long long* ss_clear;     // consumer: [M][kSsSlots] sums to clear for the next producer, or nullptr
     float inv_d, eps;
     const uint16_t *gain_a, *gain_b;  // EPI_RESIDUAL: hout_x[m * N + n] = bf16(x_new[m][n] * gain_x[n])
     uint16_t *hout_a, *hout_b;
 };
-
-// 1/sqrt(mean x^2 + eps) of row m from its partial sums: lanes stride over the partials,
-// then a butterfly -- a fixed order that depends on nothing but n_part
-__device__ __forceinline__ float row_rscale(const LinArgs& a, int m, int lane)
-{
-    float s = 0.f;
-    for (int i = lane; i < a.n_part; i += 32) s += __ldcg(a.ss_in + (size_t)m * a.ss_stride + i);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    return 1.0f / sqrtf(s * a.inv_d + a.eps);
-}
 
 // EPI_QKV tiles pair row j of a head with row j + hd/2, the two halves of one rotary pair:
 // tile b covers pairs j = 8 (b % (hd/16)) .. +7 of head b / (hd/16).
@@ -209,10 +200,9 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
 
     if (a.ss_in) {  // fused RMSNorm: scale row m by 1/sqrt(mean x^2 + eps)
         __shared__ float rs[kMaxRows];
-        for (int m = warp; m < a.M; m += 4) {
-            const float v = row_rscale(a, m, lane);
-            if (lane == 0) rs[m] = v;
-        }
+        for (int m0 = 0; m0 < a.M; m0 += 128 / kSsSlots)  // 128 threads: 8 rows at a time
+            rms_rscales(a.ss_in + (size_t)m0 * kSsSlots, a.ss_clear ? a.ss_clear + (size_t)m0 * kSsSlots : nullptr,
+                        min(a.M - m0, 128 / kSsSlots), a.inv_d, a.eps, rs + m0);
         __syncthreads();
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
@@ -223,11 +213,11 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
     }
 
     if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
-        __shared__ float sq[4][MT];
+        __shared__ long long sq[4][MT];
 #pragma unroll
         for (int m = 0; m < MT; ++m)
             if (lane == m) {
-                float q = 0.f;
+                long long q = 0;
                 if (m < a.M) {
 #pragma unroll
                     for (int r = 0; r < 4; ++r)
@@ -236,7 +226,7 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
                             const float xn = (EPI == EPI_RESIDUAL) ? (*o + acc[r][m]) : acc[r][m];
                             *o = xn;
                             if (EPI == EPI_RESIDUAL) {
-                                q = fmaf(xn, xn, q);
+                                q += sq_fixed(xn);
                                 if (a.hout_a) a.hout_a[(size_t)m * a.N + nrow[r]] = f2bf(xn * bf16f(a.gain_a[nrow[r]]));
                                 if (a.hout_b) a.hout_b[(size_t)m * a.N + nrow[r]] = f2bf(xn * bf16f(a.gain_b[nrow[r]]));
                             }
@@ -248,7 +238,7 @@ __global__ void __launch_bounds__(128) linear_fma_kernel(const LinArgs a)
             __syncthreads();
             if (threadIdx.x < MT && threadIdx.x < a.M) {
                 const int m = threadIdx.x;
-                a.ss_out[(size_t)m * a.ss_stride + blockIdx.x] = ((sq[0][m] + sq[1][m]) + sq[2][m]) + sq[3][m];
+                ss_add(a.ss_out + (size_t)m * kSsSlots, sq[0][m] + sq[1][m] + sq[2][m] + sq[3][m]);
             }
         }
     } else if (EPI == EPI_SWIGLU) {
@@ -331,10 +321,21 @@ __host__ __device__ constexpr size_t mma_ring_bytes()
 // SM are set by the ring depth, not by registers or occupancy, and no barrier is needed
 // (nobody else reads a thread's slots).  WARPS is chosen from (N, K) alone -- never from
 // M -- so that matrices with few row tiles (N = 4096: 256 tiles) still keep enough bytes
-// in flight; TR and STAGES do not touch the arithmetic of a row.
-template <int NT, int EPI, int TR, int WARPS, int STAGES>
+// in flight; TR and STAGES do not touch the arithmetic of a row, and the sums of squares a
+// residual epilogue leaves for the next norm are exact integer sums (ls_common.cuh).
+//
+// SHARE (plain and residual projections of the wide kind, from 9 rows on; see mma_shape): the
+// grid is one CTA per SM and CTA c takes the rows [c N / G, (c+1) N / G) -- equal shares to within
+// one row, whatever the tile size -- as its TR tiles, the last one ragged: rows beyond the share
+// copy nothing and are dropped in the epilogue.  SMs get equal shares of the memory system, so
+// equal shares of the matrix keep all of them streaming to the end (256 tiles of 16 rows on 148
+// SMs leave 40 SMs idle half of the time), and one CTA per SM has room for a ring that keeps
+// 96 KB of weights in flight where two CTAs with two token tiles keep 64.  A row's arithmetic is
+// the same in both cuts of the matrix.
+template <int NT, int EPI, int TR, int WARPS, int STAGES, bool SHARE>
 __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
 {
+    static_assert(!SHARE || EPI == EPI_STORE || EPI == EPI_RESIDUAL, "shares are cut in plain output rows");
     constexpr int T = WARPS * 32;
     extern __shared__ __align__(16) unsigned char ring[];
     TR_T0
@@ -358,6 +359,21 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             pb[tr] = weight_row(a, tile * 16 + g + 8);
         }
     }
+    // SHARE: first row of the share, one past its last, and which of the thread's rows exist
+    int u0 = 0, u1 = a.N;
+    bool va[TR], vb[TR];
+    if (SHARE) {
+        u0 = (int)((long long)blockIdx.x * a.N / gridDim.x);
+        u1 = (int)((long long)(blockIdx.x + 1) * a.N / gridDim.x);
+#pragma unroll
+        for (int tr = 0; tr < TR; ++tr) {
+            const int n = u0 + tr * 16 + g;
+            va[tr] = n < u1;
+            vb[tr] = n + 8 < u1;
+            pa[tr] = weight_row(a, n);
+            pb[tr] = weight_row(a, n + 8);
+        }
+    }
     const uint16_t* hb[NT];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) hb[nt] = a.h + (size_t)min(nt * 8 + g, a.M - 1) * a.K;
@@ -378,8 +394,8 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             const int kk = (k < a.K) ? k : 0;
 #pragma unroll
             for (int tr = 0; tr < TR; ++tr) {
-                cp_async16_cg(slot(2 * tr, s), pa[tr] + kk, nb);
-                cp_async16_cg(slot(2 * tr + 1, s), pb[tr] + kk, nb);
+                cp_async16_cg(slot(2 * tr, s), pa[tr] + kk, SHARE ? (va[tr] ? nb : 0) : nb);
+                cp_async16_cg(slot(2 * tr + 1, s), pb[tr] + kk, SHARE ? (vb[tr] ? nb : 0) : nb);
             }
         }
     };
@@ -427,12 +443,8 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
         cp_async_commit();
     }
     __shared__ float rs[kMaxRows];
-    if (a.ss_in) {  // fused RMSNorm: per-row scale, computed while the first stages travel
-        for (int m = warp; m < a.M; m += WARPS) {
-            const float v = row_rscale(a, m, lane);
-            if (lane == 0) rs[m] = v;
-        }
-    }
+    if (a.ss_in && tid < 256)  // fused RMSNorm: per-row scales, fetched while the first stages travel
+        rms_rscales(a.ss_in, a.ss_clear, a.M, a.inv_d, a.eps, rs);
     // what the epilogue will need from global memory is fetched now, while the ring fills:
     // the residual values and gains (EPI_RESIDUAL), the rotation factors (EPI_QKV)
     constexpr int FRAGS = TR * NT;
@@ -441,17 +453,17 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
     if (tid < 32 * FRAGS) {
         const int efr = tid >> 5, etile = blockIdx.x * TR + efr / NT, em0 = (efr % NT) * 8 + 2 * t;
         if (EPI == EPI_RESIDUAL) {
-            const int nlo = etile * 16 + g, nhi = nlo + 8;
+            const int nlo = SHARE ? u0 + (efr / NT) * 16 + g : etile * 16 + g, nhi = nlo + 8;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int m = em0 + (i & 1), n = (i < 2) ? nlo : nhi;
-                if (m < a.M && n < a.N) xin[i] = a.out[(size_t)m * a.ldo + n];
+                if (m < a.M && n < u1) xin[i] = a.out[(size_t)m * a.ldo + n];
             }
-            if (nlo < a.N) {
+            if (nlo < u1) {
                 if (a.hout_a) gA[0] = bf16f(a.gain_a[nlo]);
                 if (a.hout_b) gB[0] = bf16f(a.gain_b[nlo]);
             }
-            if (nhi < a.N) {
+            if (nhi < u1) {
                 if (a.hout_a) gA[1] = bf16f(a.gain_a[nhi]);
                 if (a.hout_b) gB[1] = bf16f(a.gain_b[nhi]);
             }
@@ -525,16 +537,16 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
             r[3] *= s1;
         }
         if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
-            const int nlo = tile * 16 + gg, nhi = nlo + 8;
-            float q[2] = {0.f, 0.f};
+            const int nlo = SHARE ? u0 + tr * 16 + gg : tile * 16 + gg, nhi = nlo + 8;
+            long long q[2] = {0, 0};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 int m = m0 + (i & 1), n = (i < 2) ? nlo : nhi;
-                if (m < a.M && n < a.N) {
+                if (m < a.M && n < u1) {
                     const float xn = (EPI == EPI_RESIDUAL) ? (xin[i] + r[i]) : r[i];
                     a.out[(size_t)m * a.ldo + n] = xn;
                     if (EPI == EPI_RESIDUAL) {
-                        q[i & 1] = fmaf(xn, xn, q[i & 1]);
+                        q[i & 1] += sq_fixed(xn);
                         if (a.hout_a) a.hout_a[(size_t)m * a.N + n] = f2bf(xn * gA[i >> 1]);
                         if (a.hout_b) a.hout_b[(size_t)m * a.N + n] = f2bf(xn * gB[i >> 1]);
                     }
@@ -547,8 +559,8 @@ __global__ void __launch_bounds__(WARPS * 32) linear_mma_kernel(const LinArgs a)
                     q[1] += __shfl_xor_sync(0xffffffffu, q[1], sh);
                 }
                 if (gg == 0) {
-                    if (m0 < a.M) a.ss_out[(size_t)m0 * a.ss_stride + tile] = q[0];
-                    if (m0 + 1 < a.M) a.ss_out[(size_t)(m0 + 1) * a.ss_stride + tile] = q[1];
+                    if (m0 < a.M) ss_add(a.ss_out + (size_t)m0 * kSsSlots, q[0]);
+                    if (m0 + 1 < a.M) ss_add(a.ss_out + (size_t)(m0 + 1) * kSsSlots, q[1]);
                 }
             }
         } else if (EPI == EPI_SWIGLU) {
@@ -610,12 +622,23 @@ inline cudaError_t launch_linear_fma(const LinArgs& a, const LaunchCtx& lc)
     return launch(lc, linear_fma_kernel<16, EPI>, grid, block, 0, a);
 }
 
-// A row's bits depend on how K is split over the warps of its tile, and on nothing else.
-// So the warps per tile come from the matrix shape alone (never from M):
+// SMs of the current device (a wide matrix from 9 rows on is cut into one share per SM)
+inline int device_sms()
+{
+    static int sms[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms[dev] = 0;
+    return sms[dev];
+}
+
+// A row's bits depend on how K is split over the warps of its tile, and on nothing else (the
+// sums of squares for the next norm are exact).  So the warps per tile come from the matrix
+// shape alone (never from M):
 //   few row tiles (N = 4096)  -> 16 warps, 4 stages (3 with two token tiles), 2 CTAs per SM,
 //                                all tiles in one wave
 //   otherwise                 -> 8 warps, 6 stages (4 with two token tiles), 3 CTAs per SM
-// while the tiles per CTA may follow the pass size: from 6 rows on, where the token rows are
+// while everything else may follow the pass size.  From 6 rows on, where the token rows are
 // a third or more of what a tile pulls through L1, a CTA of a matrix with 700 or more row
 // tiles (q|k|v, gate-up, LM head on the 7B shape) takes two tiles with 3 stages (still 3 CTAs
 // per SM) and uses its token fragments for both.  Measured on the 7B shape: gate-up 32.5 ->
@@ -624,6 +647,10 @@ inline cudaError_t launch_linear_fma(const LinArgs& a, const LaunchCtx& lc)
 // tiles at every pass size: its CTAs then fit the device in one wave (384 on the 7B shape), they
 // all end together, and the attention clusters that follow on the stream are placed at once
 // instead of trickling in behind a second wave (in the loop: q|k|v 19.5 -> 17.9 us at 1 row).
+// From 9 rows on (two token tiles, whose fragments take ring space) the plain and residual
+// projections of the 16-warp kind are cut into one share of rows per SM (SHARE in
+// linear_mma_kernel), 2 or 3 tiles per CTA with 4 or 3 stages: 13B shape at 9 rows, down-proj
+// 35.2 -> 27.6 us and o-proj 15.6 -> 12.9 us; 7B shape, 21.1 -> 18.9 and 10.3 -> 9.9 us.
 inline bool mma_wide(int epi, int N, int K)
 {
     const int tiles = lin_grid(epi, N), nsteps = (K + 31) / 32;
@@ -633,6 +660,15 @@ inline bool mma_pair(int epi, int N, int K, int M)
 {
     return (M >= 6 || epi == EPI_QKV) && !mma_wide(epi, N, K) && lin_grid(epi, N) >= 700;
 }
+// tiles per CTA of the one-share-per-SM cut, or 0 where it does not apply
+inline int mma_share_tiles(int epi, int N, int K, int M)
+{
+    if ((epi != EPI_STORE && epi != EPI_RESIDUAL) || M <= 8 || !mma_wide(epi, N, K)) return 0;
+    const int sms = device_sms();
+    if (sms < 1 || sms >= lin_grid(epi, N)) return 0;
+    const int per_sm = ((N + sms - 1) / sms + 15) / 16;
+    return (per_sm == 2 || per_sm == 3) ? per_sm : 0;
+}
 // CTAs the MMA family launches for this matrix (also the number of argmax candidates per row)
 inline int mma_grid(int epi, int N, int K, int M)
 {
@@ -640,7 +676,7 @@ inline int mma_grid(int epi, int N, int K, int M)
     return mma_pair(epi, N, K, M) ? (tiles + 1) / 2 : tiles;
 }
 
-template <int NT, int EPI, int TR, int WARPS, int STAGES>
+template <int NT, int EPI, int TR, int WARPS, int STAGES, bool SHARE = false>
 inline cudaError_t launch_linear_mma_cfg(const LinArgs& a, const LaunchCtx& lc)
 {
     constexpr size_t smem = mma_ring_bytes<NT, TR, WARPS, STAGES>();
@@ -649,19 +685,32 @@ inline cudaError_t launch_linear_mma_cfg(const LinArgs& a, const LaunchCtx& lc)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !allowed[dev]) {
-        e = cudaFuncSetAttribute(linear_mma_kernel<NT, EPI, TR, WARPS, STAGES>,
+        e = cudaFuncSetAttribute(linear_mma_kernel<NT, EPI, TR, WARPS, STAGES, SHARE>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) allowed[dev] = true;
     }
     const int tiles = lin_grid(EPI, a.N);
-    return launch(lc, linear_mma_kernel<NT, EPI, TR, WARPS, STAGES>, dim3((tiles + TR - 1) / TR), dim3(WARPS * 32), smem,
-                  a);
+    return launch(lc, linear_mma_kernel<NT, EPI, TR, WARPS, STAGES, SHARE>, dim3(SHARE ? device_sms() : (tiles + TR - 1) / TR),
+                  dim3(WARPS * 32), smem, a);
 }
+
+template <int EPI, bool PLAIN = (EPI == EPI_STORE || EPI == EPI_RESIDUAL)>
+struct MmaShareLaunch {
+    static cudaError_t run(const LinArgs&, const LaunchCtx&, int) { return cudaErrorInvalidValue; }
+};
+template <int EPI>
+struct MmaShareLaunch<EPI, true> {
+    static cudaError_t run(const LinArgs& a, const LaunchCtx& lc, int tr)
+    {
+        return tr == 2 ? launch_linear_mma_cfg<2, EPI, 2, 16, 4, true>(a, lc) : launch_linear_mma_cfg<2, EPI, 3, 16, 3, true>(a, lc);
+    }
+};
 
 template <int EPI>
 inline cudaError_t launch_linear_mma(const LinArgs& a, const LaunchCtx& lc)
 {
+    if (const int tr = mma_share_tiles(EPI, a.N, a.K, a.M)) return MmaShareLaunch<EPI>::run(a, lc, tr);
     if (mma_wide(EPI, a.N, a.K))
         return a.M <= 8 ? launch_linear_mma_cfg<1, EPI, 1, 16, 4>(a, lc) : launch_linear_mma_cfg<2, EPI, 1, 16, 3>(a, lc);
     if (mma_pair(EPI, a.N, a.K, a.M))

@@ -39,7 +39,7 @@ def main():
     ap.add_argument("--layers", default="4", help="layers whose launches are listed one by one")
     ap.add_argument("--prompt", type=int, default=0, help="prompt length (default: the workload's)")
     a = ap.parse_args()
-    if build.stale(build.TRACE_LIB):
+    if not build.TRACE_LIB.exists():
         raise SystemExit("run `python -m paper_2404_16710_b200.build --trace` first")
     B.LIB_PATH = build.TRACE_LIB  # before the first call into the binding
     L = B.lib()
