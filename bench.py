@@ -376,7 +376,8 @@ def run_own(args):
         def roof(M):
             k = ks[f"gate_up_swiglu@M={M}"]
             return {"rows": M, "achieved": k["GB/s"], "frac": k["frac"], "us_per_launch": round(k["ms"] * 1e3, 2),
-                    "algorithmic_bytes": k["bytes"], "traffic": measured_traffic(args.workload, "gate_up_swiglu", M)}
+                    "algorithmic_bytes": k["bytes"], "traffic": measured_traffic(args.workload, "gate_up_swiglu", M),
+                    "frac_chained": k.get("frac_chained")}
         n_draft_launches = len(acc) * (d + 1) * E
         n_verify_launches = len(acc) * (s.n_layers - E)
         loop_ms_mean = statistics.mean(loop_ms)
@@ -384,7 +385,7 @@ def run_own(args):
         out["roofline"] = {"bound": "hbm", "kernel": f"linear_{fam}_kernel, gate-up + SwiGLU, 1 row (draft passes)",
                            "achieved": r1["achieved"], "peak": peak, "unit": "GB/s", "frac": r1["frac"],
                            "traffic": r1["traffic"], "algorithmic_bytes": r1["algorithmic_bytes"],
-                           "us_per_launch": r1["us_per_launch"],
+                           "us_per_launch": r1["us_per_launch"], "frac_chained": r1["frac_chained"],
                            "share_of_loop_time_est": round(n_draft_launches * r1["us_per_launch"] / 1e3 / loop_ms_mean, 3),
                            "verify_pass": dict(rv, share_of_loop_time_est=round(
                                n_verify_launches * rv["us_per_launch"] / 1e3 / loop_ms_mean, 3)),
@@ -392,7 +393,9 @@ def run_own(args):
                            "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, "
                                              "profiles/dram_traffic_per_launch.md (null: not captured for this workload)",
                            "how": "CUDA events around a CUDA graph of 40 launches through the C ABI, rotating over the "
-                                  "layers' weights (each launch streams from HBM), launches serialised (no dependent-launch overlap)"}
+                                  "layers' weights (each launch streams from HBM), launches serialised (no dependent-launch "
+                                  "overlap); frac_chained: the same launches linked by programmatic dependent launch, as "
+                                  "inside the loop (ls_op_chain)"}
         # the CPU oracle on a bounded sample of the same workload
         n_p, n_new = cpu_sample_sizes(s)
         O, om = oracle_model(wl, w, n_p + n_new + d + 2)

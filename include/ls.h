@@ -231,6 +231,17 @@ int ls_get_stats(const ls_model *m, ls_stats *out);
  * returns without synchronising.  linear_path is LS_LINEAR_FMA or LS_LINEAR_MMA.
  * ------------------------------------------------------------------------------ */
 
+/* How the decode loop chains its kernels, for the single-operation calls below: with on != 0 every
+ * later ls_op_* launch of this process carries the programmatic-dependent-launch attribute, so
+ * consecutive operations on one stream overlap the way they do inside ls_generate (Sec. 4.3's
+ * loop is one dependency chain): a kernel's CTAs may become resident and put their first weight
+ * stages in flight while the operation before it on the stream is still running; every kernel
+ * waits for that operation to finish before it touches anything but weights and the page table.
+ * Results are unchanged.  Off by default (each operation then starts after the previous one has
+ * drained, which is what a stand-alone timing of one kernel wants).  Process-wide, not per stream;
+ * the prompt-pass kernels (ls_op_gemm, ls_op_prefill_attention) are not affected. */
+int ls_op_chain(int32_t on);
+
 /* x[m,:] = float(Emb[tok[m],:]) -- the embedding lookup x_0 of Sec. 4.1. */
 int ls_op_embed(const void *emb_bf16_dev, const int32_t *tok_dev, int32_t M, int32_t D, int32_t V,
                 float *x_dev, void *cuda_stream);

@@ -28,7 +28,7 @@ EXPORTS = (
     "ls_generate_batch", "ls_prefill_batch", "ls_decode_batch", "ls_read_output_seq", "ls_debug_logits", "ls_debug_next_logits", "ls_get_stats", "ls_op_embed", "ls_op_rmsnorm",
     "ls_op_linear", "ls_op_gate_up_swiglu", "ls_op_lm_head_scratch_bytes", "ls_op_lm_head_argmax",
     "ls_op_lm_head_argmax_static", "ls_op_rope_append", "ls_op_qkv_rope_append", "ls_op_attention", "ls_op_accept",
-    "ls_op_gemm", "ls_op_prefill_attention",
+    "ls_op_gemm", "ls_op_prefill_attention", "ls_op_chain",
 )
 
 
@@ -100,6 +100,7 @@ def lib():
             "ls_debug_logits": (C.c_int, [vp, ip, i32, i32, fp, fp]),
             "ls_debug_next_logits": (C.c_int, [vp, fp]),
             "ls_get_stats": (C.c_int, [vp, C.POINTER(ls_stats)]),
+            "ls_op_chain": (C.c_int, [i32]),
             "ls_op_embed": (C.c_int, [vp, vp, i32, i32, i32, vp, vp]),
             "ls_op_rmsnorm": (C.c_int, [vp, vp, i32, i32, C.c_float, vp, vp]),
             "ls_op_linear": (C.c_int, [i32, vp, vp, i32, i32, i32, vp, i32, vp]),
@@ -330,6 +331,10 @@ def ls_op_embed(emb, tok, x):
 def ls_op_rmsnorm(x, gain, eps, out):
     M, D = x.shape
     _ck(lib().ls_op_rmsnorm(_dev(x), _dev(gain), M, D, eps, _dev(out), _stream()), "ls_op_rmsnorm")
+
+
+def ls_op_chain(on):
+    _ck(lib().ls_op_chain(int(bool(on))), "ls_op_chain")
 
 
 def ls_op_linear(path, w, h, out, residual=False):

@@ -32,6 +32,7 @@ using namespace ls;
 namespace {
 
 thread_local int g_last_cuda = 0;
+bool g_op_chain = false;  // ls_op_* launches carry the programmatic-dependent-launch attribute (ls_op_chain)
 
 #define LS_CK(expr)                         \
     do {                                    \
@@ -1546,11 +1547,17 @@ int ls_get_stats(const ls_model* m, ls_stats* out)
 }
 
 // ------------------------------------------------------------------ single operations
+int ls_op_chain(int32_t on)
+{
+    g_op_chain = on != 0;
+    return LS_OK;
+}
+
 int ls_op_embed(const void* emb, const int32_t* tok, int32_t M, int32_t D, int32_t V, float* x, void* stream)
 {
     if (!aligned16(emb) || !tok || !aligned16(x) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8 || V < 1)
         return LS_ERR_INVALID_ARG;
-    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, embed_kernel, dim3(M), dim3(256), 0, (const uint16_t*)emb, tok,
+    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, g_op_chain}, embed_kernel, dim3(M), dim3(256), 0, (const uint16_t*)emb, tok,
                  D, V, x, nullptr, nullptr, nullptr, nullptr, 0, 1));
     return LS_OK;
 }
@@ -1559,7 +1566,7 @@ int ls_op_rmsnorm(const float* x, const void* gain, int32_t M, int32_t D, float 
 {
     if (!aligned16(x) || !aligned16(gain) || !aligned16(out) || M < 1 || M > LS_MAX_ROWS || D < 8 || D % 8)
         return LS_ERR_INVALID_ARG;
-    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, rmsnorm_kernel, dim3(M), dim3(256), 0, x,
+    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, g_op_chain}, rmsnorm_kernel, dim3(M), dim3(256), 0, x,
                  (const uint16_t*)gain, D, eps, (uint16_t*)out, nullptr));
     return LS_OK;
 }
@@ -1579,7 +1586,7 @@ int ls_op_linear(int32_t path, const void* w, const void* h, int32_t M, int32_t 
     LinArgs a = lin_args((const uint16_t*)w, (const uint16_t*)h, M, N, K);
     a.out = out;
     a.ldo = N;
-    LS_CK(launch_linear(path, residual ? EPI_RESIDUAL : EPI_STORE, a, LaunchCtx{(cudaStream_t)stream, false}));
+    LS_CK(launch_linear(path, residual ? EPI_RESIDUAL : EPI_STORE, a, LaunchCtx{(cudaStream_t)stream, g_op_chain}));
     return LS_OK;
 }
 
@@ -1591,7 +1598,7 @@ int ls_op_gate_up_swiglu(int32_t path, const void* wg, const void* wu, const voi
     LinArgs a = lin_args((const uint16_t*)wg, (const uint16_t*)h, M, F, K);
     a.w1 = (const uint16_t*)wu;
     a.out_bf16 = (uint16_t*)out;
-    LS_CK(launch_linear(path, EPI_SWIGLU, a, LaunchCtx{(cudaStream_t)stream, false}));
+    LS_CK(launch_linear(path, EPI_SWIGLU, a, LaunchCtx{(cudaStream_t)stream, g_op_chain}));
     return LS_OK;
 }
 
@@ -1611,7 +1618,7 @@ int ls_op_lm_head_argmax(int32_t path, const void* w, const void* h, int32_t M, 
     a.cand_stride = (V + 15) / 16;
     a.out = logits;
     a.ldo = V;
-    const LaunchCtx lc = {(cudaStream_t)stream, false};
+    const LaunchCtx lc = {(cudaStream_t)stream, g_op_chain};
     LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
     LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, n_candidates(path, V, K, M), a.cand_stride, tok,
                  nullptr, nullptr, 0.f, 0, 0ull));
@@ -1657,7 +1664,7 @@ int ls_op_lm_head_argmax_static(int32_t path, const void* w, const void* h, int3
     a.cand = (ValIdx*)scratch;
     a.cand_stride = (V + 15) / 16;
     a.ldo = V;
-    const LaunchCtx lc = {(cudaStream_t)stream, false};
+    const LaunchCtx lc = {(cudaStream_t)stream, g_op_chain};
     LS_CK(launch_linear(path, EPI_ARGMAX, a, lc));
     LS_CK(launch(lc, argmax_finish_kernel, dim3(M), dim3(256), 0, a.cand, n_candidates(path, V, K, M), a.cand_stride, tok,
                  nullptr, nullptr, 0.f, 0, 0ull));
@@ -1678,7 +1685,7 @@ int ls_op_rope_append(const float* qkv, int32_t M, int32_t pos0, int32_t Hq, int
 {
     LS_TRY(kv_check(M, pos0, Hq, Hkv, hd, page_size, max_seq));
     if (!qkv || !page_table || !q_out || !aligned16(kp) || !aligned16(vp) || !(theta > 0.f)) return LS_ERR_INVALID_ARG;
-    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, rope_append_kernel, dim3(M, Hq + 2 * Hkv), dim3(hd / 2), 0, qkv,
+    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, g_op_chain}, rope_append_kernel, dim3(M, Hq + 2 * Hkv), dim3(hd / 2), 0, qkv,
                  Hq, Hkv, hd, nullptr, theta, log2_exact(page_size), page_table, max_seq, (uint16_t*)q_out, (uint16_t*)kp,
                  (uint16_t*)vp, nullptr, pos0));
     return LS_OK;
@@ -1708,7 +1715,7 @@ int ls_op_qkv_rope_append(int32_t path, const void* wq, const void* wk, const vo
     a.max_seq = max_seq;
     a.pos_off = pos0;
     a.theta = theta;
-    LS_CK(launch_linear(path, EPI_QKV, a, LaunchCtx{(cudaStream_t)stream, false}));
+    LS_CK(launch_linear(path, EPI_QKV, a, LaunchCtx{(cudaStream_t)stream, g_op_chain}));
     return LS_OK;
 }
 
@@ -1720,7 +1727,7 @@ int ls_op_attention(const void* q, int32_t M, int32_t pos0, int32_t Hq, int32_t 
     AttnPlan plan;
     LS_TRY(attn_plan(hd, Hq / Hkv, Hkv, max_seq, &plan));
     return attn_launch(plan, (const uint16_t*)q, (const uint16_t*)kp, (const uint16_t*)vp, page_table, nullptr, pos0, M,
-                       Hq, Hkv, hd, log2_exact(page_size), max_seq, (uint16_t*)out, LaunchCtx{(cudaStream_t)stream, false});
+                       Hq, Hkv, hd, log2_exact(page_size), max_seq, (uint16_t*)out, LaunchCtx{(cudaStream_t)stream, g_op_chain});
 }
 
 int ls_op_gemm(const void* a, const void* b, int32_t M, int32_t N, int32_t K, float* c, int32_t ldc, int32_t accumulate,
@@ -1748,7 +1755,7 @@ int ls_op_accept(const int32_t* draft, const int32_t* verified, int32_t d, int32
                  int32_t* accepted, void* stream)
 {
     if (!draft || !verified || !state || !out_ids || !accepted || d < 0 || d >= LS_MAX_ROWS) return LS_ERR_INVALID_ARG;
-    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, false}, accept_kernel, dim3(1), dim3(32), 0, draft, verified, d, state,
+    LS_CK(launch(LaunchCtx{(cudaStream_t)stream, g_op_chain}, accept_kernel, dim3(1), dim3(32), 0, draft, verified, d, state,
                  out_ids, accepted, 0, nullptr));
     return LS_OK;
 }

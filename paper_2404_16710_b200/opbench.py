@@ -134,15 +134,28 @@ def prompt_rates(shape, w, R, ops=PROMPT_OPS, iters=20, warm=3):
     return out
 
 
-def kernel_rooflines(shape, w, path, rows, peak_gbs, ops=OPS, iters=40, warm=5):
+def kernel_rooflines(shape, w, path, rows, peak_gbs, ops=OPS, iters=40, warm=5, chained=True):
+    """Per op and pass size: one launch alone (launches serialised: each starts when the one before
+    has drained) and, with ``chained``, the same launches linked by programmatic dependent launch as
+    inside the decode loop (``ms_chained``: a launch's CTAs move in and prefetch while its
+    predecessor's last CTAs finish).  Fractions are algorithmic bytes / time / peak_gbs."""
     out = {}
     for M in rows:
         cases = op_cases(shape, w, path, M)
         for name in ops:
             fn, nbytes, rot = cases[name]
             ms = time_op(fn, rot, iters, warm)
-            out[f"{name}@M={M}"] = {"ms": round(ms, 5), "GB/s": round(nbytes / ms / 1e6, 1),
-                                    "frac": round(nbytes / ms / 1e6 / peak_gbs, 4), "bytes": nbytes}
+            e = {"ms": round(ms, 5), "GB/s": round(nbytes / ms / 1e6, 1),
+                 "frac": round(nbytes / ms / 1e6 / peak_gbs, 4), "bytes": nbytes}
+            if chained:
+                B.ls_op_chain(True)
+                try:
+                    msc = time_op(fn, rot, iters, warm)
+                finally:
+                    B.ls_op_chain(False)
+                e["ms_chained"] = round(msc, 5)
+                e["frac_chained"] = round(nbytes / msc / 1e6 / peak_gbs, 4)
+            out[f"{name}@M={M}"] = e
     return out
 
 
@@ -175,7 +188,8 @@ def main():
     res = kernel_rooflines(shape, w, path, [int(r) for r in a.rows.split(",")], a.peak,
                            [o for o in a.ops.split(",") if o], a.iters, a.warm)
     for k, v in res.items():
-        print(f"{k:28s} {v['ms'] * 1e3:8.2f} us  {v['GB/s']:8.1f} GB/s  {v['frac']:.3f} of {a.peak:.0f}")
+        print(f"{k:28s} {v['ms'] * 1e3:8.2f} us  {v['GB/s']:8.1f} GB/s  {v['frac']:.3f} of {a.peak:.0f}   chained "
+              f"{v['ms_chained'] * 1e3:8.2f} us  {v['frac_chained']:.3f}")
     print(json.dumps(res))
 
 

@@ -117,6 +117,63 @@ def test_linear_rows_do_not_depend_on_pass_size(path):
     assert torch.equal(out.flip(0), outs[9])
 
 
+def test_chained_operations_give_the_same_results():
+    """ls_op_chain(1): consecutive operations overlap as they do inside the decode loop (a kernel
+    moves in while its predecessor finishes and waits before it reads the predecessor's output).
+    A dependent sequence -- three residual updates of one buffer, then gate-up on another --
+    gives bit-identical results either way."""
+    path = B.LS_LINEAR_MMA
+    N = K = 1024
+    ws = [rnd((N, K), 40 + i, 0.05).bfloat16() for i in range(3)]
+    wg, wu = rnd((704, K), 50, 0.05).bfloat16(), rnd((704, K), 51, 0.05).bfloat16()
+    h = rnd((5, K), 44).bfloat16()
+    outs = []
+    for on in (False, True, False):
+        B.ls_op_chain(on)
+        try:
+            x = torch.zeros((5, N), dtype=torch.float32, device="cuda")
+            act = torch.empty((5, 704), dtype=torch.bfloat16, device="cuda")
+            for w in ws:
+                B.ls_op_linear(path, w, h, x, True)
+            B.ls_op_gate_up_swiglu(path, wg, wu, h, act)
+            torch.cuda.synchronize()
+        finally:
+            B.ls_op_chain(False)
+        outs.append((x, act))
+    for x, act in outs[1:]:
+        assert torch.equal(x, outs[0][0]) and torch.equal(act, outs[0][1])
+
+
+@pytest.mark.parametrize("residual", [False, True])
+@pytest.mark.parametrize("N,K", [(4096, 4096), (5120, 1024), (4100, 520)])
+def test_wide_matrices_cut_per_sm_give_the_same_rows(N, K, residual):
+    """From 9 rows on the wide matrices (o-proj and down-proj shapes) are cut into one share of
+    rows per SM instead of one 16-row tile per CTA; shares are ragged (4096 / 148 rows). Every
+    output row is bit-identical to what the single-row pass gives, at every pass size on both
+    sides of the switch, with and without the residual add; sampled rows against the oracle."""
+    path = B.LS_LINEAR_MMA
+    w = rnd((N, K), 31, 0.05).bfloat16()
+    h = rnd((16, K), 32).bfloat16()
+    x0 = rnd((16, N), 33)
+    single = torch.empty((16, N), dtype=torch.float32, device="cuda")
+    for m in range(16):
+        o = x0[m:m + 1].clone() if residual else torch.empty((1, N), dtype=torch.float32, device="cuda")
+        B.ls_op_linear(path, w, h[m:m + 1].contiguous(), o, residual)
+        single[m] = o[0]
+    for M in (8, 9, 11, 16):
+        out = x0[:M].clone() if residual else torch.empty((M, N), dtype=torch.float32, device="cuda")
+        B.ls_op_linear(path, w, h[:M].contiguous(), out, residual)
+        torch.cuda.synchronize()
+        assert torch.equal(out, single[:M]), f"M={M}"
+    rows = np.unique(np.concatenate([[0, 26, 27, 28, 55, N - 29, N - 1], np.random.default_rng(3).integers(0, N, 24)]))
+    wb, hv = bits(w[torch.from_numpy(rows).cuda()]), vals(h)
+    got = single.cpu().numpy().astype(np.float64)[:, rows]
+    base = x0.cpu().numpy().astype(np.float64)[:, rows] if residual else 0.0
+    for m in (0, 9, 15):
+        ref = O.linear(wb, hv[m]) + (base[m] if residual else 0.0)
+        np.testing.assert_allclose(got[m], ref, rtol=0, atol=2e-5 * np.abs(ref).max())
+
+
 @pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("M,F,K", [(1, 8, 32), (3, 88, 96), (7, 688, 256), (16, 100, 520), (5, 11008, 4096)])
 def test_gate_up_swiglu(path, M, F, K):
