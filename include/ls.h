@@ -329,7 +329,8 @@ int ls_op_attention(const void *q_bf16_dev, int32_t M, int32_t pos0, int32_t Hq,
 /* Kernels of the prompt pass (the rows that go through the model before the first draft,
  * Appendix A.4), which is a dense contraction over hundreds of rows.
  * ls_op_gemm: c[m, n] (+)= sum_k a[m, k] b[n, k] on the tcgen05 tensor cores (up to 128 rows
- * one CTA per 128 x 256 tile, beyond that pairs of CTAs per 256 x 256 tile); a bf16 [M, K],
+ * one CTA per 128 x 256 tile, beyond that persistent pairs of CTAs on 256 x 256 tiles with two
+ * accumulators in tensor memory, so that a tile's epilogue overlaps the next tile's MMAs); a bf16 [M, K],
  * b bf16 [N, K], K a multiple of 8, both 16-byte aligned; c fp32 with leading dimension
  * ldc >= N; accumulate != 0 adds to c (the residual update of Sec. 4.1).  status_dev (device
  * int32, may be NULL) receives 3 if one of the kernel's bounded waits ran out.

@@ -554,12 +554,6 @@ int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* 
         if (dev >= 0 && dev < 64) allowed[dev] = true;
     }
     const bool pair = gemm_uses_pairs(M);
-    static bool pair_allowed[64] = {false};
-    if (pair && (dev < 0 || dev >= 64 || !pair_allowed[dev])) {
-        LS_CK(cudaFuncSetAttribute(gemm_bf16_tn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)kPairSmemBytes));
-        if (dev >= 0 && dev < 64) pair_allowed[dev] = true;
-    }
     CUtensorMap ma, mb[3];
     LS_TRY(make_tile_map(&ma, A, (uint64_t)M, (uint64_t)K, kGemmBM));
     const uint16_t* bs[3] = {B0, B1 ? B1 : B0, B2 ? B2 : B0};
@@ -574,10 +568,9 @@ int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* 
     if (swiglu_out && !pair) return LS_ERR_INVALID_ARG;  // the fused epilogue exists on CTA pairs only
     if (swiglu_out) tiles = (n0 + kGemmBN / 2 - 1) / (kGemmBN / 2);
     if (pair) {
+        // one CTA pair per two SMs, each walking its share of the 256 x 256 tiles
+        static int max_pairs[64] = {0};
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((mtiles + 1) & ~1, tiles);
-        cfg.blockDim = dim3(128);
-        cfg.dynamicSmemBytes = kPairSmemBytes;
         cfg.stream = st;
         cudaLaunchAttribute at;
         at.id = cudaLaunchAttributeClusterDimension;
@@ -586,8 +579,24 @@ int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* 
         at.val.clusterDim.z = 1;
         cfg.attrs = &at;
         cfg.numAttrs = 1;
-        LS_CK(cudaLaunchKernelEx(&cfg, gemm_bf16_tn_pair_kernel, ma, mb[0], mb[1], mb[2], segs, M, K, C, ldc, accumulate,
-                                 status, swiglu_out));
+        cfg.dynamicSmemBytes = kPairSmemBytes;
+        cfg.blockDim = dim3(kPersistThreads);
+        if (dev < 0 || dev >= 64) return LS_ERR_UNSUPPORTED;
+        if (!max_pairs[dev]) {
+            LS_CK(cudaFuncSetAttribute(gemm_bf16_tn_pair_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kPairSmemBytes));
+            int sms = 0, n = 0;
+            LS_CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+            cfg.gridDim = dim3(sms & ~1);
+            LS_CK(cudaOccupancyMaxActiveClusters(&n, gemm_bf16_tn_pair_persistent_kernel, &cfg));
+            if (n < 1) return LS_ERR_UNSUPPORTED;
+            max_pairs[dev] = n < sms / 2 ? n : sms / 2;
+        }
+        const int n_tiles = tiles * ((mtiles + 1) / 2);
+        const int pairs = n_tiles < max_pairs[dev] ? n_tiles : max_pairs[dev];
+        cfg.gridDim = dim3(2 * pairs);
+        LS_CK(cudaLaunchKernelEx(&cfg, gemm_bf16_tn_pair_persistent_kernel, ma, mb[0], mb[1], mb[2], segs, M, K, C, ldc,
+                                 accumulate, status, swiglu_out));
         return LS_OK;
     }
     dim3 grid(tiles, mtiles);

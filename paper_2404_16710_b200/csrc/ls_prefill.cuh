@@ -290,67 +290,99 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         : "memory");
 }
 
-// grid (M tiles of 128 rounded up to even, column tiles of 256 of all matrices), cluster (2, 1, 1),
-// block 128; roles as in gemm_bf16_tn_kernel, the MMA issuer only in the leader CTA.
-__global__ void __launch_bounds__(128)
-gemm_bf16_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
-                         const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
-                         const GemmSegs segs, int M, int K, float* __restrict__ C, int ldc, int accumulate,
-                         int32_t* status, uint16_t* __restrict__ swiglu_out)
+// The kernel is persistent: grid = one CTA pair per two SMs, cluster (2, 1, 1), block 192.  Every
+// pair walks a list of tiles (pair p takes tiles p, p + P, p + 2P, ...; rows fastest, so the
+// pairs that run side by side share a weight tile in L2) and the roles live in warps of their
+// own: warps 0-3 read accumulators back and store, lane 0 of warp 4 feeds the ring with TMA,
+// lane 0 of warp 5 (leader CTA) issues the MMAs.  Tensor memory holds TWO accumulators (2 x 256 of its 512 columns): while the epilogue
+// warps drain tile i, the MMAs of tile i + 1 already fill the other one, and the operand ring
+// never drains between tiles.  Two more barrier pairs carry that: accf[b] "accumulator b is
+// complete" (tcgen05.commit, multicast to both CTAs) and acce[b] "accumulator b has been read"
+// (in the leader CTA; the eight epilogue warps of the pair arrive on it, the peer's through the
+// cluster's shared-memory window).  Every wait is bounded as in the one-tile kernels.
+constexpr int kPersistThreads = 192;
+constexpr int kPersistTmemCols = 2 * kGemmBN;
+
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+__global__ void __launch_bounds__(kPersistThreads)
+gemm_bf16_tn_pair_persistent_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
+                                    const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
+                                    const GemmSegs segs, int M, int K, float* __restrict__ C, int ldc, int accumulate,
+                                    int32_t* status, uint16_t* __restrict__ swiglu_out)
 {
     extern __shared__ unsigned char gsm_raw[];
     const uint32_t base = (smem_u32(gsm_raw) + 1023u) & ~1023u;
-    const uint32_t bars = base + kPairStages * kPairStageBytes;  // full[S], empty[S], accum, tmem slot
+    const uint32_t bars = base + kPairStages * kPairStageBytes;  // full[S], empty[S], accf[2], acce[2], tmem slot
     auto full = [&](int s) { return bars + 8u * s; };
     auto empty = [&](int s) { return bars + 8u * (kPairStages + s); };
-    const uint32_t accum = bars + 8u * (2 * kPairStages);
-    const uint32_t tslot = accum + 8u;
+    auto accf = [&](int b) { return bars + 8u * (2 * kPairStages + b); };
+    auto acce = [&](int b) { return bars + 8u * (2 * kPairStages + 2 + b); };
+    const uint32_t tslot = bars + 8u * (2 * kPairStages + 4);
     __shared__ int failed;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint32_t rank;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
-    const int m0 = blockIdx.x * kGemmBM;  // the pair: blockIdx.x = 2p, 2p + 1
-    const CUtensorMap* map_b = &map_b0;
-    int N = segs.n[0], n0 = blockIdx.y * kGemmBN, col0 = 0;
-    {
-        const int t0 = (segs.n[0] + kGemmBN - 1) / kGemmBN, t1 = (segs.n[1] + kGemmBN - 1) / kGemmBN;
-        if ((int)blockIdx.y >= t0 + t1) {
-            map_b = &map_b2;
-            N = segs.n[2];
-            n0 = ((int)blockIdx.y - t0 - t1) * kGemmBN;
-            col0 = segs.n[0] + segs.n[1];
-        } else if ((int)blockIdx.y >= t0) {
-            map_b = &map_b1;
-            N = segs.n[1];
-            n0 = ((int)blockIdx.y - t0) * kGemmBN;
-            col0 = segs.n[0];
-        }
-    }
-    // SwiGLU mode (swiglu_out != nullptr; B0 = gate, B1 = up, both [F, K]): the pair's weight tile is
-    // 128 gate rows (staged by the leader) beside the 128 up rows of the same features (staged by
-    // its peer), so the accumulator holds gate | up of 128 features and the epilogue writes
-    // bf16(silu(gate) * up) straight into the feed-forward input: no fp32 round trip through memory
     const bool swiglu = swiglu_out != nullptr;
-    if (swiglu) {
-        map_b = rank ? &map_b1 : &map_b0;
-        N = segs.n[0];
-        n0 = blockIdx.y * (kGemmBN / 2);
-        col0 = 0;
-    }
-    const int b_row = swiglu ? n0 : n0 + (int)rank * (kGemmBN / 2);
+    const int t0 = (segs.n[0] + kGemmBN - 1) / kGemmBN, t1 = (segs.n[1] + kGemmBN - 1) / kGemmBN,
+              t2 = (segs.n[2] + kGemmBN - 1) / kGemmBN;
+    const int col_tiles = swiglu ? (segs.n[0] + kGemmBN / 2 - 1) / (kGemmBN / 2) : t0 + t1 + t2;
+    const int row_pairs = ((M + kGemmBM - 1) / kGemmBM + 1) / 2;
+    const int n_tiles = col_tiles * row_pairs;
+    const int n_pairs = (int)gridDim.x / 2, pair = (int)blockIdx.x / 2;
     const int nkb = (K + kGemmBK - 1) / kGemmBK;
+
+    // column tile ny -> weight matrix, its row count, first row of the tile in it, first output column
+    struct Cols {
+        const CUtensorMap* map;
+        int N, n0, col0;
+    };
+    auto cols_of = [&](int ny) {
+        Cols c;
+        if (swiglu) {
+            // the pair's weight tile is 128 gate rows (staged by the leader) beside the 128 up rows of
+            // the same features (staged by its peer): the accumulator holds gate | up of 128 features
+            c.map = rank ? &map_b1 : &map_b0;
+            c.N = segs.n[0];
+            c.n0 = ny * (kGemmBN / 2);
+            c.col0 = 0;
+        } else if (ny >= t0 + t1) {
+            c.map = &map_b2;
+            c.N = segs.n[2];
+            c.n0 = (ny - t0 - t1) * kGemmBN;
+            c.col0 = segs.n[0] + segs.n[1];
+        } else if (ny >= t0) {
+            c.map = &map_b1;
+            c.N = segs.n[1];
+            c.n0 = (ny - t0) * kGemmBN;
+            c.col0 = segs.n[0];
+        } else {
+            c.map = &map_b0;
+            c.N = segs.n[0];
+            c.n0 = ny * kGemmBN;
+            c.col0 = 0;
+        }
+        return c;
+    };
+
     if (tid == 0) {
         for (int s = 0; s < kPairStages; ++s) {
             mbar_init(full(s), 1);
             mbar_init(empty(s), 1);
         }
-        mbar_init(accum, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(accf(b), 1);
+            mbar_init(acce(b), 8);  // four epilogue warps in each CTA of the pair
+        }
         failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tslot), "r"(kGemmBN)
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tslot), "r"(kPersistTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
@@ -361,117 +393,153 @@ gemm_bf16_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
     uint32_t tmem;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem) : "r"(tslot));
 
-    if (warp == 0 && lane == 0) {  // TMA producer of this CTA's share
-        for (int kb = 0; kb < nkb; ++kb) {
-            const int s = kb % kPairStages;
-            if (kb >= kPairStages && !mbar_wait(empty(s), ((kb / kPairStages) - 1) & 1)) {
-                failed = 1;
-                break;
+    if (warp == 4) {
+        if (lane == 0) {  // TMA producer of this CTA's share
+            int it = 0;
+            bool ok = true;
+            for (int t = pair; t < n_tiles && ok; t += n_pairs) {
+                const Cols c = cols_of(t / row_pairs);
+                const int m0 = ((t % row_pairs) * 2 + (int)rank) * kGemmBM;
+                const int b_row = swiglu ? c.n0 : c.n0 + (int)rank * (kGemmBN / 2);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % kPairStages;
+                    if (it >= kPairStages && !mbar_wait(empty(s), ((it / kPairStages) - 1) & 1)) {
+                        failed = 1;
+                        ok = false;
+                        break;
+                    }
+                    if (rank == 0) mbar_expect_tx(full(s), 2 * kPairStageBytes);
+                    const uint32_t sa = base + s * kPairStageBytes, sb = sa + kGemmBM * kGemmBK * 2;
+                    const uint32_t lead = full(s) & kPeerBitMask;
+                    tma_load_2d_pair(sa, &map_a, kb * kGemmBK, m0, lead);
+                    tma_load_2d_pair(sb, c.map, kb * kGemmBK, b_row, lead);
+                }
             }
-            if (rank == 0) mbar_expect_tx(full(s), 2 * kPairStageBytes);
-            const uint32_t sa = base + s * kPairStageBytes, sb = sa + kGemmBM * kGemmBK * 2;
-            const uint32_t lead = full(s) & kPeerBitMask;
-            tma_load_2d_pair(sa, &map_a, kb * kGemmBK, m0, lead);
-            tma_load_2d_pair(sb, map_b, kb * kGemmBK, b_row, lead);
         }
-    } else if (rank == 0 && warp == 1 && lane == 0) {  // MMA issuer: the leader CTA only
-        // instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 256 (128 per CTA)
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kGemmBN >> 3) << 17) |
-                               ((uint32_t)((2 * kGemmBM) >> 4) << 24);
-        bool ok = true;
-        for (int kb = 0; kb < nkb && ok; ++kb) {
-            const int s = kb % kPairStages;
-            if (!mbar_wait(full(s), (kb / kPairStages) & 1)) {
+    } else if (warp == 5) {
+        if (rank == 0 && lane == 0) {  // MMA issuer: the leader CTA only
+            // instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 256 (128 per CTA)
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kGemmBN >> 3) << 17) |
+                                   ((uint32_t)((2 * kGemmBM) >> 4) << 24);
+            int it = 0, i = 0;
+            bool ok = true;
+            for (int t = pair; t < n_tiles && ok; t += n_pairs, ++i) {
+                const int b = i & 1;
+                // accumulator b free: its previous tile (i - 2) has been read by all eight warps
+                if (i >= 2 && !mbar_wait(acce(b), ((i >> 1) - 1) & 1)) {
+                    failed = 1;
+                    break;
+                }
+                tc_fence_after();
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % kPairStages;
+                    if (!mbar_wait(full(s), (it / kPairStages) & 1)) {
+                        failed = 1;
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = base + s * kPairStageBytes, sb = sa + kGemmBM * kGemmBK * 2;
+                    const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sb);
+#pragma unroll
+                    for (int k4 = 0; k4 < kGemmBK / 16; ++k4)
+                        tc_mma_bf16_pair(tmem + (uint32_t)(b * kGemmBN), da + 2 * k4, db + 2 * k4, idesc, (kb | k4) != 0);
+                    tc_commit_pair(empty(s));
+                }
+                if (ok) tc_commit_pair(accf(b));
+            }
+        }
+    } else {
+        // epilogue: warp w of each CTA owns its accumulator lanes 32w..32w+31 = rows m0 + 32w + lane
+        const uint32_t acce_leader[2] = {cluster_map(acce(0), 0), cluster_map(acce(1), 0)};
+        int i = 0;
+        for (int t = pair; t < n_tiles; t += n_pairs, ++i) {
+            const int b = i & 1;
+            const Cols c = cols_of(t / row_pairs);
+            const int N = c.N, n0 = c.n0, col0 = c.col0;
+            const int row = ((t % row_pairs) * 2 + (int)rank) * kGemmBM + warp * 32 + lane;
+            if (!mbar_wait(accf(b), (i >> 1) & 1)) {
                 failed = 1;
-                ok = false;
                 break;
             }
             tc_fence_after();
-            const uint32_t sa = base + s * kPairStageBytes, sb = sa + kGemmBM * kGemmBK * 2;
-            const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sb);
+            const uint32_t tacc = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * kGemmBN);
+            if (swiglu) {
+#pragma unroll 1
+                for (int cc = 0; cc < kGemmBN / 64; ++cc) {  // 32 features at a time: gate columns cc*32.., up columns 128 + cc*32..
+                    uint32_t gt[32], up[32];
+                    tc_ld32(tacc + cc * 32, gt);
+                    tc_ld32(tacc + kGemmBN / 2 + cc * 32, up);
+                    if (row < M) {
+                        uint16_t* dst = swiglu_out + (size_t)row * N + n0 + cc * 32;
+                        if (n0 + cc * 32 + 32 <= N && (((uintptr_t)dst) & 15u) == 0) {
 #pragma unroll
-            for (int k4 = 0; k4 < kGemmBK / 16; ++k4)
-                tc_mma_bf16_pair(tmem, da + 2 * k4, db + 2 * k4, idesc, (kb | k4) != 0);
-            tc_commit_pair(empty(s));
+                            for (int j = 0; j < 32; j += 8) {
+                                uint32_t pk[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float g0 = __uint_as_float(gt[j + 2 * e]), g1 = __uint_as_float(gt[j + 2 * e + 1]);
+                                    pk[e] = pack_bf16(g0 / (1.0f + expf(-g0)) * __uint_as_float(up[j + 2 * e]),
+                                                      g1 / (1.0f + expf(-g1)) * __uint_as_float(up[j + 2 * e + 1]));
+                                }
+                                *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (n0 + cc * 32 + j < N) {
+                                    const float g0 = __uint_as_float(gt[j]);
+                                    dst[j] = f2bf(g0 / (1.0f + expf(-g0)) * __uint_as_float(up[j]));
+                                }
+                        }
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int cc = 0; cc < kGemmBN / 32; ++cc) {
+                    uint32_t v[32];
+                    tc_ld32(tacc + cc * 32, v);
+                    if (row < M) {
+                        float* dst = C + (size_t)row * ldc + col0 + n0 + cc * 32;
+                        if (n0 + cc * 32 + 32 <= N && (((uintptr_t)dst) & 15u) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                       __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                                if (accumulate) {
+                                    const float4 q = *reinterpret_cast<const float4*>(dst + j);
+                                    o.x += q.x;
+                                    o.y += q.y;
+                                    o.z += q.z;
+                                    o.w += q.w;
+                                }
+                                *reinterpret_cast<float4*>(dst + j) = o;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (n0 + cc * 32 + j < N)
+                                    dst[j] = accumulate ? dst[j] + __uint_as_float(v[j]) : __uint_as_float(v[j]);
+                        }
+                    }
+                }
+            }
+            // this warp has read its lanes of accumulator b: tell the MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acce_leader[b]);
         }
-        if (ok) tc_commit_pair(accum);
     }
     __syncwarp();
-
-    // epilogue: warp w of each CTA owns its accumulator lanes 32w..32w+31 = rows m0 + 32w + lane
-    bool have = mbar_wait(accum, 0);
-    if (!have) failed = 1;
-    tc_fence_after();
+    tc_fence_before();
     __syncthreads();
-    if (!failed && swiglu) {
-        const int row = m0 + warp * 32 + lane;
-#pragma unroll 1
-        for (int c = 0; c < kGemmBN / 64; ++c) {  // 32 features at a time: gate columns c*32.., up columns 128 + c*32..
-            uint32_t gt[32], up[32];
-            tc_ld32(tmem + ((uint32_t)(warp * 32) << 16) + c * 32, gt);
-            tc_ld32(tmem + ((uint32_t)(warp * 32) << 16) + kGemmBN / 2 + c * 32, up);
-            if (row < M) {
-                uint16_t* dst = swiglu_out + (size_t)row * N + n0 + c * 32;
-                if (n0 + c * 32 + 32 <= N && (((uintptr_t)dst) & 15u) == 0) {
-#pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float g0 = __uint_as_float(gt[j + 2 * e]), g1 = __uint_as_float(gt[j + 2 * e + 1]);
-                            pk[e] = pack_bf16(g0 / (1.0f + expf(-g0)) * __uint_as_float(up[j + 2 * e]),
-                                              g1 / (1.0f + expf(-g1)) * __uint_as_float(up[j + 2 * e + 1]));
-                        }
-                        *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (n0 + c * 32 + j < N) {
-                            const float g0 = __uint_as_float(gt[j]);
-                            dst[j] = f2bf(g0 / (1.0f + expf(-g0)) * __uint_as_float(up[j]));
-                        }
-                }
-            }
-        }
-    } else if (!failed) {
-        const int row = m0 + warp * 32 + lane;
-#pragma unroll 1
-        for (int c = 0; c < kGemmBN / 32; ++c) {
-            uint32_t v[32];
-            tc_ld32(tmem + ((uint32_t)(warp * 32) << 16) + c * 32, v);
-            if (row < M) {
-                float* dst = C + (size_t)row * ldc + col0 + n0 + c * 32;
-                if (n0 + c * 32 + 32 <= N && (((uintptr_t)dst) & 15u) == 0) {
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                               __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                        if (accumulate) {
-                            const float4 p = *reinterpret_cast<const float4*>(dst + j);
-                            o.x += p.x;
-                            o.y += p.y;
-                            o.z += p.z;
-                            o.w += p.w;
-                        }
-                        *reinterpret_cast<float4*>(dst + j) = o;
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (n0 + c * 32 + j < N) dst[j] = accumulate ? dst[j] + __uint_as_float(v[j]) : __uint_as_float(v[j]);
-                }
-            }
-        }
-    } else if (tid == 0 && status) {
+    if (failed && tid == 0 && status) {
         *status = DEV_TIMEOUT;
         __nanosleep(1000000);  // let copies that may still be in flight land before the CTA goes away
     }
-    tc_fence_before();
-    __syncthreads();
     cluster_sync_all();  // both CTAs are done with tensor memory, and the MMAs with both shared memories
     if (warp == 0)
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kGemmBN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kPersistTmemCols) : "memory");
 }
 
 // ------------------------------------------------------------------ elementwise helpers of the prompt pass
