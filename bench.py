@@ -237,43 +237,64 @@ def run_own(args):
         print(json.dumps({"profile_region": args.profile_region, "launches": int(gm.stats().kernel_launches)}))
         return
 
-    # ---- device-resident timing: prompt already prefilled in HBM, decode loop only
-    B.ls_prefill(gm.h, prompt)
-    prefill_ms = gm.stats().prefill_ms
+    # ---- device-resident timing: prompts already prefilled in HBM, decode loop only.  The timed steps
+    # rotate over a few prompts of the same recipe (each on a handle of its own, prefilled beforehand):
+    # the accepted drafts per step of a synthetic model hinge on near-ties of its exit logits and
+    # swing by +-0.4 from one prompt to the next, so one prompt repeated K times would put that draw
+    # into the headline number; full greedy decoding runs over the same prompts.
+    n_prompts = max(1, min(args.steps, 4))
+    prompts = [prompt] + [synth.make_prompt(s.vocab, P, wl.prompt_seed + rank + 7919 * i) for i in range(1, n_prompts)]
+    gms = [gm] + [B.Model(s, w, max_seq, 64, max(d, 1)) for _ in range(1, n_prompts)]
+    prefill_all = []
+    for g, pr in zip(gms, prompts):
+        B.ls_prefill(g.h, pr)
+        prefill_all.append(g.stats().prefill_ms)
+    prefill_ms = statistics.median(prefill_all)
     for _ in range(args.warmup):
         B.ls_decode(gm.h, E, d, NEW)
-    spec_ids, acc = B.ls_read_output(gm.h, NEW)
+    spec_out = []
+    for g in gms:
+        B.ls_decode(g.h, E, d, NEW)
+        spec_out.append(B.ls_read_output(g.h, NEW))
+    spec_ids = spec_out[0][0]
+    acc = np.concatenate([a for _, a in spec_out])
     launches = 0
-    loop_ms = []
+    loop_ms, loop_bytes = [], []
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clk:
         e0.record()
-        for _ in range(args.steps):
-            B.ls_decode(gm.h, E, d, NEW)
-            st = gm.stats()
+        for k in range(args.steps):
+            g = gms[k % n_prompts]
+            B.ls_decode(g.h, E, d, NEW)
+            st = g.stats()
             launches += st.kernel_launches
             loop_ms.append(st.decode_ms)
+            loop_bytes.append(st.weight_bytes + st.kv_bytes)
         e1.record()
         barrier()
     total_ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
     st = gm.stats()
     value = job_tokens_per_s(world, args.steps, NEW, total_ms)
-    sched_bytes = st.weight_bytes + st.kv_bytes
-    loop_gbs = sched_bytes / (statistics.mean(loop_ms) / 1e3) / 1e9
+    sched_bytes = statistics.mean(loop_bytes)
+    loop_gbs = sum(loop_bytes) / (sum(loop_ms) / 1e3) / 1e9
+    spec_ms_per_step = sum(loop_ms) / sum(len(spec_out[k % n_prompts][1]) for k in range(args.steps))
 
-    # ---- the same library's full-model greedy decoding, same model, same prompt
+    # ---- the same library's full-model greedy decoding, same model, same prompts
     for _ in range(min(args.warmup, 2)):
         B.ls_decode(gm.h, 0, 0, NEW)
-    full_ms = []
-    for _ in range(max(1, min(args.steps, 3))):
-        B.ls_decode(gm.h, 0, 0, NEW)
-        full_ms.append(gm.stats().decode_ms)
-    fst = gm.stats()
-    full_ids, _ = B.ls_read_output(gm.h, NEW)
-    full_tok_s = NEW / (statistics.mean(full_ms) / 1e3)
-    full_gbs = (fst.weight_bytes + fst.kv_bytes) / (statistics.mean(full_ms) / 1e3) / 1e9
-    lossless = bool(np.array_equal(full_ids, spec_ids))
+    full_ms, full_bytes, lossless = [], [], True
+    for g, (ids_g, _) in zip(gms, spec_out):
+        B.ls_decode(g.h, 0, 0, NEW)
+        fst = g.stats()
+        full_ms.append(fst.decode_ms)
+        full_bytes.append(fst.weight_bytes + fst.kv_bytes)
+        lossless = lossless and bool(np.array_equal(B.ls_read_output(g.h, NEW)[0], ids_g))
+    full_tok_s = NEW * len(full_ms) / (sum(full_ms) / 1e3)
+    full_gbs = sum(full_bytes) / (sum(full_ms) / 1e3) / 1e9
+    for g in gms[1:]:
+        g.close()
+    del gms
 
     # ---- the paper's "without KVQ reuse" ablation (Table 7): verify recomputes the early layers
     B.ls_decode_flags(gm.h, E, d, NEW, B.LS_DECODE_NO_EXIT_CACHE)
@@ -333,13 +354,13 @@ def run_own(args):
 
     # ---- end to end through the public call: host prompt in, host ids out, prefill included
     e2e_ms = []
-    for i in range(1 + max(1, min(args.steps, 3))):
+    for i in range(1 + max(1, min(args.steps, 4))):
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        ids, a2 = gm.generate(prompt, E, d, NEW)
+        ids, a2 = gm.generate(prompts[i % n_prompts], E, d, NEW)
         if i:
             e2e_ms.append((time.perf_counter() - t0) * 1e3)
-    e2e_worst = max_over_ranks(statistics.median(e2e_ms), dist, "cuda")  # median call of this rank, slowest rank
+    e2e_worst = max_over_ranks(statistics.mean(e2e_ms), dist, "cuda")  # mean call over the rotated prompts, slowest rank
     est = gm.stats()
     e2e = {"value": world * NEW / (e2e_worst / 1e3), "unit": UNIT, "h2d_bytes_per_step": 4 * P + 32 * 2,
            "d2h_bytes_per_step": 4 * len(ids) + 4 * len(a2) + 32 * (est.host_syncs + 1),
@@ -350,7 +371,7 @@ def run_own(args):
            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
            "config": {"workload": args.workload, "shape": s.name, "n_prompt": P, "max_new": NEW, "exit_layer": E,
                       "num_draft": d, "late_scale": wl.late_scale, "linear_path": "mma" if path == 2 else "fma",
-                      "l2": "inputs (weights) larger than L2", "replicas": world,
+                      "l2": "inputs (weights) larger than L2", "replicas": world, "prompts_rotated": n_prompts,
                       "timed_region": "decode loop from a prefilled prompt, device-resident",
                       "kernels_per_layer": 5, "prompt_pass": "persistent tcgen05 cta_group::2 GEMM, 256x256 tiles on CTA pairs, two TMEM accumulators, blocks of 1024 rows"},
            "e2e": e2e, "gpu_launches": int(launches), "clocks": clk.summary,
@@ -362,7 +383,8 @@ def run_own(args):
                         "frac_8TBs": round(loop_gbs / 8000, 4), "bytes_per_loop": int(sched_bytes)},
            "ids_equal_full_greedy": lossless,
            "accepted_per_step": float(acc.mean()), "acceptance_rate": float(acc.mean() / d),
-           "emitted_per_step": float(NEW / len(acc)), "spec_steps": int(len(acc)), "host_syncs": int(st.host_syncs),
+           "emitted_per_step": float(NEW * n_prompts / len(acc)), "spec_steps_per_prompt": [int(len(a)) for _, a in spec_out],
+           "ms_per_spec_step": round(spec_ms_per_step, 4), "host_syncs": int(st.host_syncs),
            "prefill_ms": prefill_ms}
 
     if rank == 0 and world == 1:
@@ -378,8 +400,8 @@ def run_own(args):
             return {"rows": M, "achieved": k["GB/s"], "frac": k["frac"], "us_per_launch": round(k["ms"] * 1e3, 2),
                     "algorithmic_bytes": k["bytes"], "traffic": measured_traffic(args.workload, "gate_up_swiglu", M),
                     "frac_chained": k.get("frac_chained")}
-        n_draft_launches = len(acc) * (d + 1) * E
-        n_verify_launches = len(acc) * (s.n_layers - E)
+        n_draft_launches = len(acc) / n_prompts * (d + 1) * E
+        n_verify_launches = len(acc) / n_prompts * (s.n_layers - E)
         loop_ms_mean = statistics.mean(loop_ms)
         r1, rv = roof(1), roof(d + 1)
         out["roofline"] = {"bound": "hbm", "kernel": f"linear_{fam}_kernel, gate-up + SwiGLU, 1 row (draft passes)",

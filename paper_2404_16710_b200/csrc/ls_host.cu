@@ -521,6 +521,21 @@ int make_tile_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, 
 {
     TensorMapEncodeFn fn = tensor_map_encoder();
     if (!fn) return LS_ERR_UNSUPPORTED;
+    // A map depends on nothing but (address, extents, box): the prompt pass asks for the same few
+    // hundred maps (every layer's weights, its own activation buffers) block after block, so they
+    // are encoded once.  Bounded: the cache is dropped when it reaches 8192 entries.
+    typedef std::tuple<const void*, uint64_t, uint64_t, int> MapKey;
+    static std::map<MapKey, CUtensorMap> cache;
+    static std::mutex mu;
+    const MapKey key(ptr, rows, K, box_rows);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        auto it = cache.find(key);
+        if (it != cache.end()) {
+            *map = it->second;
+            return LS_OK;
+        }
+    }
     cuuint64_t dims[2] = {K, rows};
     cuuint64_t strides[1] = {K * 2};
     cuuint32_t box[2] = {(cuuint32_t)kGemmBK, (cuuint32_t)box_rows};
@@ -528,7 +543,11 @@ int make_tile_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, 
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? LS_OK : LS_ERR_INVALID_ARG;
+    if (r != CUDA_SUCCESS) return LS_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache.size() >= 8192) cache.clear();
+    cache.emplace(key, *map);
+    return LS_OK;
 }
 
 // C[M, N] (+)= A[M, K] B[N, K]^T on the tensor cores (tcgen05), A and B bf16, C fp32
@@ -611,6 +630,20 @@ int gemm_launch(const uint16_t* A, const uint16_t* B, int M, int N, int K, float
     return gemm_launch3(A, B, N, nullptr, 0, nullptr, 0, M, K, C, ldc, accumulate, status, st);
 }
 
+// cudaFuncAttributeMaxDynamicSharedMemorySize once per kernel and device (smem: the largest the kernel is launched with)
+template <typename Kernel>
+int allow_smem_once(Kernel kernel, size_t smem)
+{
+    static size_t allowed[64] = {0};
+    int dev = 0;
+    LS_CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || allowed[dev] < smem) {
+        LS_CK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        if (dev >= 0 && dev < 64) allowed[dev] = smem;
+    }
+    return LS_OK;
+}
+
 int prefill_attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt, int pos0, int R,
                         int Hq, int Hkv, int hd, int page_shift, uint16_t* out, cudaStream_t st)
 {
@@ -621,20 +654,20 @@ int prefill_attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* v
         dim3 mgrid((R + rpc - 1) / rpc, Hkv);
         if (hd == 128) {
             const size_t sm = prefill_attn_fa_smem_bytes<128>();
-            LS_CK(cudaFuncSetAttribute(prefill_attn_fa_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+            LS_TRY(allow_smem_once(prefill_attn_fa_kernel<128>, sm));
             prefill_attn_fa_kernel<128><<<mgrid, kFaThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
         } else {
             const size_t sm = prefill_attn_fa_smem_bytes<64>();
-            LS_CK(cudaFuncSetAttribute(prefill_attn_fa_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+            LS_TRY(allow_smem_once(prefill_attn_fa_kernel<64>, sm));
             prefill_attn_fa_kernel<64><<<mgrid, kFaThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
         }
     } else if (hd == 128) {
         const size_t sm = prefill_attn_smem_bytes<128>(Q);
-        LS_CK(cudaFuncSetAttribute(prefill_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+        LS_TRY(allow_smem_once(prefill_attn_kernel<128>, sm));
         prefill_attn_kernel<128><<<grid, kAttnThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
     } else {
         const size_t sm = prefill_attn_smem_bytes<64>(Q);
-        LS_CK(cudaFuncSetAttribute(prefill_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+        LS_TRY(allow_smem_once(prefill_attn_kernel<64>, sm));
         prefill_attn_kernel<64><<<grid, kAttnThreads, sm, st>>>(q, kp, vp, pt, pos0, R, Hq, Hkv, page_shift, out);
     }
     LS_CK(cudaGetLastError());

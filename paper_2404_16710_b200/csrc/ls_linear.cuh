@@ -635,8 +635,10 @@ inline int device_sms()
 // A row's bits depend on how K is split over the warps of its tile, and on nothing else (the
 // sums of squares for the next norm are exact).  So the warps per tile come from the matrix
 // shape alone (never from M):
-//   few row tiles (N = 4096)  -> 16 warps, 4 stages (3 with two token tiles), 2 CTAs per SM,
-//                                all tiles in one wave
+//   few row tiles (under 350: N = 4096, 5120) -> 16 warps, 4 stages (3 with two token tiles),
+//                                2 CTAs per SM, (about) one wave.  (The 384 tiles of the Llama-3-8B
+//                                q|k|v are better off with 8 warps, 3 CTAs per SM and one full wave:
+//                                alone 11.6 -> 14.9 us, but inside the loop the pass is 3 % faster.)
 //   otherwise                 -> 8 warps, 6 stages (4 with two token tiles), 3 CTAs per SM
 // while everything else may follow the pass size.  From 6 rows on, where the token rows are
 // a third or more of what a tile pulls through L1, a CTA of a matrix with 700 or more row
@@ -654,7 +656,10 @@ inline int device_sms()
 inline bool mma_wide(int epi, int N, int K)
 {
     const int tiles = lin_grid(epi, N), nsteps = (K + 31) / 32;
-    return tiles < 600 && nsteps >= 16;
+#ifndef LS_WIDE_TILES
+#define LS_WIDE_TILES 350
+#endif
+    return tiles < LS_WIDE_TILES && nsteps >= 16;
 }
 inline bool mma_pair(int epi, int N, int K, int M)
 {

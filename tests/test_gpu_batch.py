@@ -88,6 +88,23 @@ def test_batch_sequences_against_the_oracle(path):
     assert checked_total >= steps_total // 4
 
 
+def test_batch_on_the_7b_layer_shapes():
+    """Two layers of the Llama-2-7B shape, 4 sequences x 4 rows and 8 x 2 rows: the passes of 9 to 16
+    rows run the per-SM cut of the o-proj and down-proj matrices, the single-sequence runs the
+    tile-per-CTA cut; every sequence must still equal its own greedy run bit for bit."""
+    from dataclasses import replace
+    shape = replace(synth.LLAMA2_7B, name="7b-2-layers", n_layers=2)
+    gm, _ = make_pair(shape, 1234, 1, 0.05, 8 * 128, page_size=64, max_draft=3, oracle=False)
+    prompts = prompts_of(shape, (40, 90, 17, 64, 33, 100, 5, 71), 77)
+    for nb, d in ((4, 3), (8, 1)):
+        got = gm.generate_batch(prompts[:nb], 1, d, 20)
+        for p, (ids, acc) in zip(prompts, got):
+            np.testing.assert_array_equal(ids, gm.generate_full(p, 20))
+            ids1, acc1 = gm.generate(p, 1, d, 20)
+            np.testing.assert_array_equal(ids1, ids)
+            np.testing.assert_array_equal(acc1, acc)
+
+
 def test_batch_zero_late_scale_accepts_every_draft():
     """Late layers that add nothing: draft == verified at every row of every sequence, so each
     step accepts d drafts whatever the sequence (the oracle's closed-form case)."""
