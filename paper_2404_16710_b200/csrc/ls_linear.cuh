@@ -656,10 +656,7 @@ inline int device_sms()
 inline bool mma_wide(int epi, int N, int K)
 {
     const int tiles = lin_grid(epi, N), nsteps = (K + 31) / 32;
-#ifndef LS_WIDE_TILES
-#define LS_WIDE_TILES 350
-#endif
-    return tiles < LS_WIDE_TILES && nsteps >= 16;
+    return tiles < 350 && nsteps >= 16;
 }
 inline bool mma_pair(int epi, int N, int K, int M)
 {
