@@ -93,6 +93,7 @@ struct ls_model {
     size_t layer_kv_elems;
     int32_t *page_table, *ctl, *draft, *verified, *out_ids, *accepted, *ids;
     float *inv_freq, *x, *logits;
+    float2* rope_tab;  // (cos, sin) of every position and rotary pair, for the prompt pass's q|k|v epilogue
     uint16_t *h, *q, *o, *a;
     uint16_t* hE;  // exit-layer activations, already multiplied by the gain of layer E's norm (Sec. 4.3.3)
     float *px, *py;          // prompt pass: residual rows and projection outputs of one block
@@ -149,6 +150,7 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
     unsigned char* vp = take(layer_kv * c.n_layers * 2);
     unsigned char* pt = take(sizeof(int32_t) * n_pages);
     unsigned char* fr = take(sizeof(float) * (c.head_dim / 2));
+    unsigned char* rt = take(sizeof(float2) * (size_t)c.max_seq * (c.head_dim / 2));
     unsigned char* ctl = take(sizeof(int32_t) * CTL_WORDS * kMaxRows);  // one block per sequence of a pass
     unsigned char* dr = take(sizeof(int32_t) * kMaxRows);
     unsigned char* ve = take(sizeof(int32_t) * kMaxRows);
@@ -190,6 +192,7 @@ size_t carve(const ls_config& c, unsigned char* base, ls_model* m)
         m->layer_kv_elems = layer_kv;
         m->page_table = (int32_t*)pt;
         m->inv_freq = (float*)fr;
+        m->rope_tab = (float2*)rt;
         m->ctl = (int32_t*)ctl;
         m->draft = (int32_t*)dr;
         m->verified = (int32_t*)ve;
@@ -563,7 +566,7 @@ bool gemm_uses_pairs(int M)
 // instead of C, bf16(silu(A B0^T) * (A B1^T)) [M, n0] is written.
 int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* B1, int n1, const uint16_t* B2, int n2,
                  int M, int K, float* C, int ldc, int accumulate, int32_t* status, cudaStream_t st,
-                 uint16_t* swiglu_out = nullptr)
+                 uint16_t* swiglu_out = nullptr, const RopeEpi* rope = nullptr)
 {
     static bool allowed[64] = {false};
     int dev = 0;
@@ -614,10 +617,14 @@ int gemm_launch3(const uint16_t* A, const uint16_t* B0, int n0, const uint16_t* 
         const int n_tiles = tiles * ((mtiles + 1) / 2);
         const int pairs = n_tiles < max_pairs[dev] ? n_tiles : max_pairs[dev];
         cfg.gridDim = dim3(2 * pairs);
+        RopeEpi re;
+        memset(&re, 0, sizeof(re));
+        if (rope) re = *rope;
         LS_CK(cudaLaunchKernelEx(&cfg, gemm_bf16_tn_pair_persistent_kernel, ma, mb[0], mb[1], mb[2], segs, M, K, C, ldc,
-                                 accumulate, status, swiglu_out));
+                                 accumulate, status, swiglu_out, re));
         return LS_OK;
     }
+    if (rope) return LS_ERR_INVALID_ARG;  // the fused rotary epilogue exists on CTA pairs only
     dim3 grid(tiles, mtiles);
     gemm_bf16_tn_kernel<<<grid, 128, kGemmSmemBytes, st>>>(ma, mb[0], mb[1], mb[2], segs, M, K, C, ldc, accumulate, status);
     LS_CK(cudaGetLastError());
@@ -691,9 +698,14 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
         uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
         uint16_t* vp = m->vpages + (size_t)l * m->layer_kv_elems;
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.attn_norm, D, c.rms_eps, m->ph, nullptr));
-        LS_TRY(gemm_launch3(m->ph, w.wq, qw, w.wk, kvw, w.wv, kvw, R, D, m->py, qkvw, 0, status, st));
-        rope_append_rows_kernel<<<R, 256, 0, st>>>(m->py, Hq, Hkv, hd, m->inv_freq, m->page_shift, m->pt, m->seq_cap, r0,
-                                                  m->pq, kp, vp, status);
+        if (gemm_uses_pairs(R)) {  // q|k|v, rotary embedding and cache append in one kernel
+            const RopeEpi re = {m->rope_tab, m->pt, m->pq, kp, vp, Hq, Hkv, hd, m->page_shift, m->seq_cap, r0};
+            LS_TRY(gemm_launch3(m->ph, w.wq, qw, w.wk, kvw, w.wv, kvw, R, D, m->py, qkvw, 0, status, st, nullptr, &re));
+        } else {
+            LS_TRY(gemm_launch3(m->ph, w.wq, qw, w.wk, kvw, w.wv, kvw, R, D, m->py, qkvw, 0, status, st));
+            rope_append_rows_kernel<<<R, 256, 0, st>>>(m->py, Hq, Hkv, hd, m->inv_freq, m->page_shift, m->pt, m->seq_cap, r0,
+                                                      m->pq, kp, vp, status);
+        }
         LS_TRY(prefill_attn_launch(m->pq, kp, vp, m->pt, r0, R, Hq, Hkv, hd, m->page_shift, m->po, st));
         LS_TRY(gemm_launch(m->po, w.wo, R, D, qw, m->px, D, 1, status, st));
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.ffn_norm, D, c.rms_eps, m->ph, nullptr));
@@ -704,7 +716,7 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
             swiglu_rows_kernel<<<R, 256, 0, st>>>(m->py, F, m->pa);
         }
         LS_TRY(gemm_launch(m->pa, w.wd, R, D, F, m->px, D, 1, status, st));
-        m->launches += 13;
+        m->launches += gemm_uses_pairs(R) ? 11 : 13;  // pairs: rotary epilogue and SwiGLU live in the GEMMs
     }
     LS_CK(cudaGetLastError());
     return LS_OK;
@@ -1122,6 +1134,10 @@ int ls_model_create(const ls_config* cfg, const ls_weights* w, void* workspace, 
         e = cudaMemcpyAsync(m->page_table, pt.data(), sizeof(int32_t) * pt.size(), cudaMemcpyHostToDevice, m->st);
         if (e == cudaSuccess)
             e = cudaMemcpyAsync(m->inv_freq, fr.data(), sizeof(float) * fr.size(), cudaMemcpyHostToDevice, m->st);
+        if (e == cudaSuccess) {
+            rope_table_kernel<<<cfg->max_seq, cfg->head_dim / 2, 0, m->st>>>(m->inv_freq, cfg->head_dim / 2, m->rope_tab);
+            e = cudaGetLastError();
+        }
         if (e == cudaSuccess) e = cudaStreamSynchronize(m->st);
     }
     if (e == cudaSuccess) e = cudaEventCreate(&m->ev0);

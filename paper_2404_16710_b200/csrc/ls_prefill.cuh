@@ -300,6 +300,30 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
 // complete" (tcgen05.commit, multicast to both CTAs) and acce[b] "accumulator b has been read"
 // (in the leader CTA; the eight epilogue warps of the pair arrive on it, the peer's through the
 // cluster's shared-memory window).  Every wait is bounded as in the one-tile kernels.
+// q|k|v epilogue of the prompt pass: instead of fp32 C, the rotary embedding is applied to the
+// accumulator and q goes out as bf16 [M, Hq hd], k and v into the paged cache at positions
+// pos0 + row (B0 = W_q, B1 = W_k, B2 = W_v).  A 256-column tile holds whole heads (hd 64 or 128), and
+// the two halves of a rotary pair (j, j + hd/2) are two 32-column reads of the thread's accumulator
+// row.  The angles come from a table of (cos, sin)(pos * theta^(-2j/hd)) filled once per model by
+// rope_table_kernel with the arithmetic of the decode kernels.  q_out == nullptr: not this mode.
+struct RopeEpi {
+    const float2* table;  // [max_seq][hd/2]
+    const int32_t* page_table;
+    uint16_t *q_out, *kpages, *vpages;
+    int Hq, Hkv, hd, page_shift, max_seq, pos0;
+};
+
+// grid (positions), block hd/2
+__global__ void rope_table_kernel(const float* __restrict__ inv_freq, int half, float2* __restrict__ table)
+{
+    const int pos = blockIdx.x, j = threadIdx.x;
+    if (j < half) {
+        float sn, cs;
+        sincosf((float)pos * inv_freq[j], &sn, &cs);
+        table[(size_t)pos * half + j] = make_float2(cs, sn);
+    }
+}
+
 constexpr int kPersistThreads = 192;
 constexpr int kPersistTmemCols = 2 * kGemmBN;
 
@@ -312,7 +336,7 @@ __global__ void __launch_bounds__(kPersistThreads)
 gemm_bf16_tn_pair_persistent_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
                                     const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
                                     const GemmSegs segs, int M, int K, float* __restrict__ C, int ldc, int accumulate,
-                                    int32_t* status, uint16_t* __restrict__ swiglu_out)
+                                    int32_t* status, uint16_t* __restrict__ swiglu_out, const RopeEpi rope)
 {
     extern __shared__ unsigned char gsm_raw[];
     const uint32_t base = (smem_u32(gsm_raw) + 1023u) & ~1023u;
@@ -491,6 +515,54 @@ gemm_bf16_tn_pair_persistent_kernel(const __grid_constant__ CUtensorMap map_a, c
                                     const float g0 = __uint_as_float(gt[j]);
                                     dst[j] = f2bf(g0 / (1.0f + expf(-g0)) * __uint_as_float(up[j]));
                                 }
+                        }
+                    }
+                }
+            } else if (rope.q_out) {
+                // whole heads of q, k or v (the tile's matrix says which): rotate pairs, convert, store
+                const int hd = rope.hd, half = hd >> 1, pos = rope.pos0 + row;
+                const int seg = col0 == 0 ? 0 : (col0 == segs.n[0] ? 1 : 2);  // 0: q, 1: k, 2: v
+                const bool row_ok = row < M && pos >= 0 && pos < rope.max_seq;
+                if (row < M && !row_ok && status) *status = DEV_POS_OVERFLOW;
+#pragma unroll 1
+                for (int hh = 0; hh < kGemmBN / hd; ++hh) {
+                    const int head = (n0 + hh * hd) / hd;  // head within its matrix
+                    uint16_t* dst = nullptr;
+                    if (row_ok && n0 + hh * hd < N) {
+                        if (seg == 0) dst = rope.q_out + ((size_t)row * rope.Hq + head) * hd;
+                        else
+                            dst = (seg == 1 ? rope.kpages : rope.vpages) +
+                                  kv_row_offset(rope.page_table, pos, rope.page_shift, rope.Hkv, head, hd);
+                    }
+#pragma unroll 1
+                    for (int cc = 0; cc < half / 32; ++cc) {
+                        uint32_t lo[32], hi[32];
+                        tc_ld32(tacc + hh * hd + cc * 32, lo);
+                        tc_ld32(tacc + hh * hd + half + cc * 32, hi);
+                        if (dst) {
+                            const float2* tb = rope.table + (size_t)pos * half + cc * 32;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                uint32_t pl[4], ph[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    float a0 = __uint_as_float(lo[j + 2 * e]), a1 = __uint_as_float(lo[j + 2 * e + 1]);
+                                    float b0 = __uint_as_float(hi[j + 2 * e]), b1 = __uint_as_float(hi[j + 2 * e + 1]);
+                                    if (seg != 2) {
+                                        const float4 t = *reinterpret_cast<const float4*>(tb + j + 2 * e);  // cos, sin, cos, sin
+                                        const float r0 = a0 * t.x - b0 * t.y, s0 = a0 * t.y + b0 * t.x;
+                                        const float r1 = a1 * t.z - b1 * t.w, s1 = a1 * t.w + b1 * t.z;
+                                        a0 = r0;
+                                        b0 = s0;
+                                        a1 = r1;
+                                        b1 = s1;
+                                    }
+                                    pl[e] = pack_bf16(a0, a1);
+                                    ph[e] = pack_bf16(b0, b1);
+                                }
+                                *reinterpret_cast<uint4*>(dst + cc * 32 + j) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+                                *reinterpret_cast<uint4*>(dst + half + cc * 32 + j) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+                            }
                         }
                     }
                 }
