@@ -335,14 +335,20 @@ int ls_op_attention(const void *q_bf16_dev, int32_t M, int32_t pos0, int32_t Hq,
  * ldc >= N; accumulate != 0 adds to c (the residual update of Sec. 4.1).  status_dev (device
  * int32, may be NULL) receives 3 if one of the kernel's bounded waits ran out.
  * ls_op_prefill_attention: causal attention of R rows at positions pos0 .. pos0+R-1 over the
- * paged cache (as ls_op_attention, any R, no scratch: a CTA walks the key chunks of its rows
- * in order with a running max / sum per row). */
+ * paged cache (as ls_op_attention, any R, no scratch; the pools hold ceil(max_seq / page_size)
+ * pages and every table entry is below that).  Head dim 128 and R >= 128: one CTA per (128 rows,
+ * query head) on the tcgen05 tensor cores -- q.k and p.v of 128 x 128 x 128 with the scores and
+ * the running output in tensor memory, K and V by TMA from the pages, the softmax one row per
+ * thread; status_dev (device int32, may be NULL) receives 3 if one of its bounded waits ran
+ * out.  Otherwise a CTA walks the key chunks of its rows in order with a running max / sum per
+ * row on mma.sync (status_dev is not written).  Keys at positions >= pos0 + R are never used,
+ * whatever bits the pages hold there. */
 int ls_op_gemm(const void *a_bf16_dev, const void *b_bf16_dev, int32_t M, int32_t N, int32_t K,
                float *c_dev, int32_t ldc, int32_t accumulate, int32_t *status_dev, void *cuda_stream);
 int ls_op_prefill_attention(const void *q_bf16_dev, int32_t R, int32_t pos0, int32_t Hq, int32_t Hkv,
                             int32_t hd, int32_t page_size, const int32_t *page_table_dev,
                             int32_t max_seq, const void *k_pages_dev, const void *v_pages_dev,
-                            void *out_bf16_dev, void *cuda_stream);
+                            void *out_bf16_dev, int32_t *status_dev, void *cuda_stream);
 
 /* match + crop of Appendix A.4 on device arrays: n = number of leading i < d with
  * draft[i] == verified[i]; appends draft[0..n-1], verified[n] to out_ids (truncated at

@@ -114,7 +114,7 @@ def lib():
             "ls_op_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp]),
             "ls_op_accept": (C.c_int, [vp, vp, i32, vp, vp, vp, vp]),
             "ls_op_gemm": (C.c_int, [vp, vp, i32, i32, i32, vp, i32, i32, vp, vp]),
-            "ls_op_prefill_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp]),
+            "ls_op_prefill_attention": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -395,9 +395,10 @@ def ls_op_gemm(a, b, c, accumulate=False, status=None):
         "ls_op_gemm")
 
 
-def ls_op_prefill_attention(q, pos0, Hq, Hkv, hd, page_size, page_table, max_seq, k_pages, v_pages, out):
+def ls_op_prefill_attention(q, pos0, Hq, Hkv, hd, page_size, page_table, max_seq, k_pages, v_pages, out, status=None):
     _ck(lib().ls_op_prefill_attention(_dev(q), q.shape[0], pos0, Hq, Hkv, hd, page_size, _dev(page_table), max_seq,
-                                      _dev(k_pages), _dev(v_pages), _dev(out), _stream()), "ls_op_prefill_attention")
+                                      _dev(k_pages), _dev(v_pages), _dev(out), _dev(status), _stream()),
+        "ls_op_prefill_attention")
 
 
 def ls_op_accept(draft, verified, d, state, out_ids, accepted):

@@ -26,6 +26,7 @@
 #include "ls_attention.cuh"
 #include "ls_linear.cuh"
 #include "ls_prefill.cuh"
+#include "ls_prefill_attn.cuh"
 
 using namespace ls;
 
@@ -651,9 +652,33 @@ int allow_smem_once(Kernel kernel, size_t smem)
     return LS_OK;
 }
 
-int prefill_attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt, int pos0, int R,
-                        int Hq, int Hkv, int hd, int page_shift, uint16_t* out, cudaStream_t st)
+// rows at positions pos0 .. pos0 + R - 1 over the paged cache of one layer (pool_pages pages).
+// Head dim 128 and at least one full tile of rows: the tcgen05 kernel (status: where it reports a
+// wait that ran out); otherwise the mma.sync walk (G <= 4) or the FMA walk.
+bool attn_uses_tc(int R, int hd, int pos0, int page_shift)
 {
+    static const bool allowed = getenv("LS_NO_TC_ATTN") == nullptr && tensor_map_encoder() != nullptr;
+    const int box_rows = (1 << page_shift) < kTcAttnB ? (1 << page_shift) : kTcAttnB;
+    return allowed && hd == kTcAttnB && R >= kTcAttnB && (pos0 + R + box_rows - 1) / box_rows <= kTcAttnMaxBoxes;
+}
+
+int prefill_attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* vp, const int32_t* pt, int pos0, int R,
+                        int Hq, int Hkv, int hd, int page_shift, int pool_pages, uint16_t* out, int32_t* status,
+                        cudaStream_t st)
+{
+    if (attn_uses_tc(R, hd, pos0, page_shift)) {
+        const int ps = 1 << page_shift, box_rows = ps < kTcAttnB ? ps : kTcAttnB;
+        CUtensorMap mq, mk, mv;
+        LS_TRY(make_tile_map(&mq, q, (uint64_t)R, (uint64_t)Hq * hd, kTcAttnB));
+        LS_TRY(make_tile_map(&mk, kp, (uint64_t)pool_pages * Hkv * ps, (uint64_t)hd, box_rows));
+        LS_TRY(make_tile_map(&mv, vp, (uint64_t)pool_pages * Hkv * ps, (uint64_t)hd, box_rows));
+        LS_TRY(allow_smem_once(prefill_attn_tc_kernel, kTcAttnSmemBytes));
+        dim3 tgrid(Hq, (R + kTcAttnB - 1) / kTcAttnB);
+        prefill_attn_tc_kernel<<<tgrid, kTcAttnThreads, kTcAttnSmemBytes, st>>>(mq, mk, mv, pt, pos0, R, Hq, Hkv, page_shift,
+                                                                               box_rows, out, status);
+        LS_CK(cudaGetLastError());
+        return LS_OK;
+    }
     const int G = Hq / Hkv, Q = G * kMaxRows;
     dim3 grid((R + 15) / 16, Hkv);
     if (G == 1 || G == 2 || G == 4) {  // tensor-core kernel: 64 queries per CTA, 16 per warp
@@ -706,7 +731,7 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
             rope_append_rows_kernel<<<R, 256, 0, st>>>(m->py, Hq, Hkv, hd, m->inv_freq, m->page_shift, m->pt, m->seq_cap, r0,
                                                       m->pq, kp, vp, status);
         }
-        LS_TRY(prefill_attn_launch(m->pq, kp, vp, m->pt, r0, R, Hq, Hkv, hd, m->page_shift, m->po, st));
+        LS_TRY(prefill_attn_launch(m->pq, kp, vp, m->pt, r0, R, Hq, Hkv, hd, m->page_shift, m->n_pages, m->po, status, st));
         LS_TRY(gemm_launch(m->po, w.wo, R, D, qw, m->px, D, 1, status, st));
         LS_CK(launch(lc, rmsnorm_kernel, dim3(R), dim3(256), 0, m->px, w.ffn_norm, D, c.rms_eps, m->ph, nullptr));
         if (gemm_uses_pairs(R)) {  // gate, up and SwiGLU in one kernel
@@ -1798,7 +1823,7 @@ int ls_op_gemm(const void* a, const void* b, int32_t M, int32_t N, int32_t K, fl
 
 int ls_op_prefill_attention(const void* q, int32_t R, int32_t pos0, int32_t Hq, int32_t Hkv, int32_t hd,
                             int32_t page_size, const int32_t* page_table, int32_t max_seq, const void* kp,
-                            const void* vp, void* out, void* stream)
+                            const void* vp, void* out, int32_t* status, void* stream)
 {
     if (R < 1 || pos0 < 0 || Hq < 1 || Hkv < 1 || Hq % Hkv || Hq / Hkv > 8 || (hd != 64 && hd != 128) ||
         page_size < 16 || page_size > 1024 || log2_exact(page_size) < 0)
@@ -1806,7 +1831,8 @@ int ls_op_prefill_attention(const void* q, int32_t R, int32_t pos0, int32_t Hq, 
     if ((int64_t)pos0 + R > max_seq) return LS_ERR_CAPACITY;
     if (!aligned16(q) || !page_table || !aligned16(kp) || !aligned16(vp) || !out) return LS_ERR_INVALID_ARG;
     return prefill_attn_launch((const uint16_t*)q, (const uint16_t*)kp, (const uint16_t*)vp, page_table, pos0, R, Hq,
-                               Hkv, hd, log2_exact(page_size), (uint16_t*)out, (cudaStream_t)stream);
+                               Hkv, hd, log2_exact(page_size), (max_seq + page_size - 1) / page_size, (uint16_t*)out, status,
+                               (cudaStream_t)stream);
 }
 
 int ls_op_accept(const int32_t* draft, const int32_t* verified, int32_t d, int32_t* state, int32_t* out_ids,

@@ -456,3 +456,41 @@ def test_prefill_attention(Hq, Hkv, hd, R, pos0):
     for m in sorted({0, R // 2, R - 1, min(R - 1, 15), min(R - 1, 16)}):
         ref = O.attention(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd)
         assert (np.abs(vals(out[m]) - ref) <= attention_tol(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd, ref)).all()
+
+
+# head dim 128 and at least 128 rows: the tcgen05 kernel (tiles of 128 rows, key blocks of 128).
+# Pages smaller than, equal to and larger than a key block; row counts and start positions that
+# leave ragged tiles and blocks; everything beyond the prompt holds NaN bit patterns, which must
+# not reach any output.  ramp: keys grow with their position and the queries are large, so that
+# a row's maximum keeps rising by more than the rescaling threshold from block to block.
+@pytest.mark.parametrize("Hq,Hkv", [(4, 4), (8, 2), (8, 1)])
+@pytest.mark.parametrize("R,pos0,page_size,ramp", [(128, 0, 64, False), (200, 0, 16, False), (300, 77, 32, True),
+                                                   (257, 1024, 256, False), (640, 130, 64, True), (129, 383, 128, False)])
+def test_prefill_attention_tensor_core(Hq, Hkv, R, pos0, page_size, ramp):
+    hd = 128
+    n = pos0 + R
+    max_seq = -(-(n + 130) // page_size) * page_size
+    table, table_d, kp, vp = kv_setup(Hkv, hd, page_size, max_seq, True)
+    kp.fill_(float("nan"))
+    vp.fill_(float("nan"))
+    kl = rnd((n, Hkv, hd), 60)
+    if ramp:
+        kl = kl * (1.0 + 3.0 * torch.arange(n, device="cuda").float() / n)[:, None, None]
+    kl = kl.bfloat16()
+    vl = rnd((n, Hkv, hd), 61).bfloat16()
+    phys = torch.from_numpy(table[np.arange(n) // page_size].astype(np.int64)).cuda()
+    slot = torch.arange(n, device="cuda") % page_size
+    kp[phys, :, slot, :] = kl
+    vp[phys, :, slot, :] = vl
+    q = rnd((R, Hq * hd), 62, 3.0 if ramp else 0.5).bfloat16()
+    out = torch.full((R, Hq * hd), float("nan"), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.ls_op_prefill_attention(q, pos0, Hq, Hkv, hd, page_size, table_d, max_seq, kp, vp, out, status)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0, "a bounded wait inside the attention kernel ran out"
+    assert torch.isfinite(out.float()).all()
+    kf, vf, qf = vals(kl).reshape(n, -1), vals(vl).reshape(n, -1), vals(q)
+    rows = sorted({0, 1, 127, 128 % R, R // 2, R - 1, (R - 1) // 128 * 128} | set(np.random.default_rng(4).integers(0, R, 4).tolist()))
+    for m in rows:
+        ref = O.attention(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd)
+        assert (np.abs(vals(out[m]) - ref) <= attention_tol(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd, ref)).all(), m
