@@ -3,16 +3,16 @@
 // One CTA per (tile of 128 prompt rows, query head) walks the key blocks of 128 cache positions
 // that its rows can see.  Per key block j:
 //   S_j = Q K_j^T      tcgen05.mma, 128 x 128 x 128, fp32 in tensor memory (two S buffers)
-//   P_j = exp2(S_j c - m)   four warps, one query row per thread: tcgen05.ld of the row, running
-//                      maximum m and sum l in registers, P_j rounded to bf16 into 128B-swizzled
-//                      shared memory (the K-major A operand of the next product)
+//   P_j = exp2(S_j c - m)   eight warps, two threads per query row (64 columns each): tcgen05.ld of
+//                      the row, running maximum m and sum l in registers, P_j rounded to bf16 into
+//                      128B-swizzled shared memory (the K-major A operand of the next product)
 //   O  += P_j V_j      tcgen05.mma with V as the MN-major B operand straight from the cache
 //                      layout [key][dim]; O stays in tensor memory for the whole walk
-// Roles in warps of their own: warps 0-3 softmax and epilogue (warp w owns tensor-memory lanes
-// 32w..32w+31), lane 0 of warp 4 feeds Q once and K, V through two-stage mbarrier rings by TMA (one
-// box per cache page and 64-column half), lane 0 of warp 5 issues the MMAs.  S_{j+1} is issued
-// before the MMA lane waits for P_j, so the tensor pipe works on it while the softmax warps are
-// busy with block j.
+// Roles in warps of their own: warps 0-7 softmax and epilogue (warps w and w + 4 own tensor-memory
+// lanes 32w..32w+31), lane 0 of warp 8 feeds Q once and K, lane 0
+// of warp 10 V, through two-stage mbarrier rings by TMA (one box per cache page and 64-column half),
+// lane 0 of warp 9 issues the MMAs.  S_{j+1} is issued before the MMA lane waits for P_j, so the tensor pipe
+// works on it while the softmax warps are busy with block j.
 // O is rescaled in tensor memory (tcgen05.ld / st) only when a row's maximum has grown by more
 // than 8 (in log2 units) beyond the one its p values are taken against: the softmax is the same
 // function, p stays below 2^8, and the read-modify-write of O leaves the steady state.
@@ -26,13 +26,13 @@
 
 namespace ls {
 
-constexpr int kTcAttnThreads = 192;
+constexpr int kTcAttnThreads = 352;
 constexpr int kTcAttnB = 128;                            // rows per tile, keys per block, head dim
 constexpr int kTcAttnTile = kTcAttnB * kTcAttnB * 2;     // 32 KB: 128 x 128 bf16 as two 64-column halves
 constexpr int kTcAttnHalf = kTcAttnTile / 2;
 constexpr int kTcAttnMaxBoxes = 1024;                    // page boxes of one sequence
 constexpr int kTcAttnTmemCols = 512;                     // S0 | S1 | O | (unused)
-constexpr size_t kTcAttnSmemBytes = 6 * (size_t)kTcAttnTile + kTcAttnMaxBoxes * 4 + 1024 + 256;
+constexpr size_t kTcAttnSmemBytes = 6 * (size_t)kTcAttnTile + kTcAttnMaxBoxes * 4 + 4 * kTcAttnB * 4 + 1024 + 256;
 
 __device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t* v)
 {
@@ -64,6 +64,12 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)  // both roundings (to nearest even) in one instruction
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 __device__ __forceinline__ float ex2_approx(float x)
 {
     float y;
@@ -85,7 +91,7 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t smem_addr)
     return d;
 }
 
-// grid (query heads, tiles of 128 rows), block 192.  q bf16 [R, Hq * 128] (map_q: boxes of 128 rows
+// grid (query heads, tiles of 128 rows), block 352.  q bf16 [R, Hq * 128] (map_q: boxes of 128 rows
 // x 64 columns); map_k / map_v: the cache of one layer as rows of 128 dims, row (page * Hkv + kv
 // head) * page_size + slot, boxes of box_rows = min(page_size, 128) rows x 64 columns.  Rows at
 // positions pos0 .. pos0 + R - 1; keys 0 .. pos0 + R - 1 are in the cache.  The heavy tiles (the
@@ -102,7 +108,8 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     unsigned char* gbase = tca_raw + (base - raw0);
     const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
     int32_t* rowc = reinterpret_cast<int32_t*>(gbase + 6 * TILE);  // first cache row of every page box
-    const uint32_t bars = base + 6 * TILE + kTcAttnMaxBoxes * 4;
+    float* xch = reinterpret_cast<float*>(gbase + 6 * TILE + kTcAttnMaxBoxes * 4);  // [2][2][128]: what the two threads of a row swap
+    const uint32_t bars = base + 6 * TILE + kTcAttnMaxBoxes * 4 + 4 * B * 4;
     const uint32_t q_full = bars;
     auto k_full = [&](int s) { return bars + 8u + 8u * s; };
     auto k_empty = [&](int s) { return bars + 24u + 8u * s; };
@@ -110,6 +117,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     auto v_empty = [&](int s) { return bars + 56u + 8u * s; };
     auto s_full = [&](int s) { return bars + 72u + 8u * s; };
     const uint32_t p_full = bars + 88u, pv_done = bars + 96u, tslot = bars + 104u;
+    auto pair_bar = [&](int w) { return bars + 112u + 8u * w; };
     __shared__ int failed;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -132,8 +140,9 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             mbar_init(v_empty(s), 1);
             mbar_init(s_full(s), 1);
         }
-        mbar_init(p_full, 128);
+        mbar_init(p_full, 256);
         mbar_init(pv_done, 1);
+        for (int w = 0; w < 4; ++w) mbar_init(pair_bar(w), 64);
         failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -154,37 +163,34 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem) : "r"(tslot));
     const uint32_t tO = tmem + 2 * B;
 
-    if (warp == 4 && lane == 0) {
-        // ---------------------------------------------------------------- TMA producer
-        mbar_expect_tx(q_full, TILE);
-        tma_load_2d(sQ, &map_q, head * B, q0, q_full);
-        tma_load_2d(sQ + HALF, &map_q, head * B + 64, q0, q_full);
+    if ((warp == 8 || warp == 10) && lane == 0) {
+        // ---------------------------------------------------------------- TMA producers: warp 8 Q and K, warp 10 V
+        // (one lane each, so that the next K does not queue behind a V stage that is still being read)
+        const bool isK = warp == 8;
+        if (isK) {
+            mbar_expect_tx(q_full, TILE);
+            tma_load_2d(sQ, &map_q, head * B, q0, q_full);
+            tma_load_2d(sQ + HALF, &map_q, head * B + 64, q0, q_full);
+        }
+        const CUtensorMap* map = isK ? &map_k : &map_v;
+        const uint32_t ring = isK ? sK : sV;
         for (int j = 0; j < nkb; ++j) {
             const int s = j & 1, key0 = j * B;
             const int nb = min(bpb, (min(n_valid, key0 + B) - key0 + box_rows - 1) / box_rows);
             const uint32_t bytes = (uint32_t)nb * box_rows * 256u;
-            if (j >= 2 && !mbar_wait(k_empty(s), ((j >> 1) - 1) & 1)) {
+            const uint32_t full = isK ? k_full(s) : v_full(s), empty = isK ? k_empty(s) : v_empty(s);
+            if (j >= 2 && !mbar_wait(empty, ((j >> 1) - 1) & 1)) {
                 failed = 1;
                 break;
             }
-            mbar_expect_tx(k_full(s), bytes);
+            mbar_expect_tx(full, bytes);
             for (int b = 0; b < nb; ++b) {
-                const uint32_t dst = sK + s * TILE + b * box_rows * 128;
-                tma_load_2d(dst, &map_k, 0, rowc[j * bpb + b], k_full(s));
-                tma_load_2d(dst + HALF, &map_k, 64, rowc[j * bpb + b], k_full(s));
-            }
-            if (j >= 2 && !mbar_wait(v_empty(s), ((j >> 1) - 1) & 1)) {
-                failed = 1;
-                break;
-            }
-            mbar_expect_tx(v_full(s), bytes);
-            for (int b = 0; b < nb; ++b) {
-                const uint32_t dst = sV + s * TILE + b * box_rows * 128;
-                tma_load_2d(dst, &map_v, 0, rowc[j * bpb + b], v_full(s));
-                tma_load_2d(dst + HALF, &map_v, 64, rowc[j * bpb + b], v_full(s));
+                const uint32_t dst = ring + s * TILE + b * box_rows * 128;
+                tma_load_2d(dst, map, 0, rowc[j * bpb + b], full);
+                tma_load_2d(dst + HALF, map, 64, rowc[j * bpb + b], full);
             }
         }
-    } else if (warp == 5 && lane == 0) {
+    } else if (warp == 9 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
         // instruction descriptors: D fp32, A and B bf16, N = 128, M = 128; S: both operands K-major,
         // P V: B (= V) MN-major
@@ -228,15 +234,31 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             tc_commit(pv_done);
         }
         if (!ok) failed = 1;
-    } else if (warp < 4) {
-        // ---------------------------------------------------------------- softmax, one row per thread
-        const uint32_t lane_t = tmem + ((uint32_t)(warp * 32) << 16);
-        const int qpos = min(pos0 + q0 + tid, last_pos);  // (rows beyond the prompt: masked like the last one)
+    } else if (warp < 8) {
+        // ---------------------------------------------------------------- softmax, two threads per row
+        // warps w and w + 4 own tensor-memory lanes 32 (w % 4) ..: thread (row, half) takes columns
+        // 64 half .. 64 half + 63 of its row of S (and of O); the two meet once per block to agree on
+        // the row's maximum (an mbarrier per pair of warps, so that this wait is bounded like the others)
+        const int w4 = warp & 3, half = warp >> 2, row = w4 * 32 + lane;
+        const uint32_t lane_t = tmem + ((uint32_t)(w4 * 32) << 16) + 64 * half;
+        const uint32_t lane_o = tO + ((uint32_t)(w4 * 32) << 16) + 64 * half;
+        const int qpos = min(pos0 + q0 + row, last_pos);  // (rows beyond the prompt: masked like the last one)
         const float sc = rsqrtf((float)B) * 1.4426950408889634f;
         float m_used = 0.f, l = 0.f;
         bool ok = true;
         // (a wait ends for the whole warp alike: the tensor-memory loads below want the warp converged)
         auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(bar, parity)) != 0; };
+        int n_meet = 0;
+        // hand v to the row's other thread and return what that one handed over
+        auto swap_with_partner = [&](float v, float& other) {
+            float* slot = xch + (n_meet & 1) * 2 * B;
+            slot[half * B + row] = v;
+            mbar_arrive(pair_bar(w4));
+            if (!wait_all(pair_bar(w4), n_meet & 1)) return false;
+            other = slot[(half ^ 1) * B + row];
+            ++n_meet;
+            return true;
+        };
         for (int j = 0; j < nkb; ++j) {
             const int s = j & 1, key0 = j * B;
             if (!wait_all(s_full(s), (j >> 1) & 1)) {
@@ -244,24 +266,28 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 break;
             }
             tc_fence_after();
-            uint32_t sv[B];
-#pragma unroll
-            for (int c = 0; c < B / 32; ++c) tc_ld32_nowait(lane_t + s * B + c * 32, sv + 32 * c);
+            uint32_t sv[B / 2];
+            tc_ld32_nowait(lane_t + s * B, sv);
+            tc_ld32_nowait(lane_t + s * B + 32, sv + 32);
             tc_wait_ld();
-            const int lim = qpos - key0;  // columns 0 .. lim are visible
-            float mx = -INFINITY;
-            if (lim >= B - 1) {
+            const int lim = qpos - key0 - 64 * half;  // this thread's columns 0 .. lim are visible
+            if (lim < B / 2 - 1) {
 #pragma unroll
-                for (int c = 0; c < B; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
-            } else {
-#pragma unroll
-                for (int c = 0; c < B; ++c) {
-                    const float v = c <= lim ? __uint_as_float(sv[c]) : -INFINITY;
-                    sv[c] = __float_as_uint(v);
-                    mx = fmaxf(mx, v);
-                }
+                for (int c = 0; c < B / 2; ++c)
+                    if (c > lim) sv[c] = 0xff800000u;  // -inf
             }
-            mx *= sc;
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one
+#pragma unroll
+            for (int c = 0; c < B / 2; c += 4) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) mx4[i] = fmaxf(mx4[i], __uint_as_float(sv[c + i]));
+            }
+            float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc, mx_other;
+            if (!swap_with_partner(mx, mx_other)) {
+                ok = false;
+                break;
+            }
+            mx = fmaxf(mx, mx_other);
             if (j == 0) {
                 m_used = mx;  // key 0 is visible to every row
             } else {
@@ -276,36 +302,36 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     if (need) m_used = mx;
                     l *= alpha;
 #pragma unroll 1
-                    for (int c = 0; c < B / 32; ++c) {
+                    for (int c = 0; c < 2; ++c) {
                         uint32_t ov[32];
-                        tc_ld32(tO + ((uint32_t)(warp * 32) << 16) + c * 32, ov);
+                        tc_ld32(lane_o + c * 32, ov);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                        tc_st32(tO + ((uint32_t)(warp * 32) << 16) + c * 32, ov);
+                        tc_st32(lane_o + c * 32, ov);
                     }
                 }
             }
             // p = exp2(s c - m), rounded to bf16 in place (two per word); the sum takes the unrounded values
             const float neg = -m_used;
-            float sum = 0.f;
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < B / 2; ++c) {
+            for (int c = 0; c < B / 4; ++c) {
                 const float p0 = ex2_approx(fmaf(__uint_as_float(sv[2 * c]), sc, neg));
                 const float p1 = ex2_approx(fmaf(__uint_as_float(sv[2 * c + 1]), sc, neg));
-                sum += p0 + p1;
-                sv[c] = pack_bf16(p0, p1);
+                sum4[c & 3] += p0 + p1;
+                sv[c] = pack_bf16x2(p0, p1);
             }
-            l += sum;
+            l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
             // P's buffer is free (and O at rest) once the product of block j - 1 has finished
             if (j > 0 && !wait_all(pv_done, (j - 1) & 1)) {
                 ok = false;
                 break;
             }
             {
-                const uint32_t prow = sP + tid * 128;
+                const uint32_t prow = sP + half * HALF + row * 128;
 #pragma unroll
-                for (int c16 = 0; c16 < 16; ++c16) {
-                    const uint32_t addr = prow + (c16 >> 3) * HALF + (((c16 & 7) ^ (tid & 7)) << 4);
+                for (int c16 = 0; c16 < 8; ++c16) {
+                    const uint32_t addr = prow + ((c16 ^ (row & 7)) << 4);
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(sv[4 * c16]), "r"(sv[4 * c16 + 1]),
                                  "r"(sv[4 * c16 + 2]), "r"(sv[4 * c16 + 3])
                                  : "memory");
@@ -316,36 +342,36 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     ok = false;
                     break;
                 }
-                if (tid >= n_valid - key0) {
-                    const uint32_t vrow = sV + s * TILE + tid * 128;
+                if (row >= n_valid - key0) {
+                    const uint32_t vrow = sV + s * TILE + half * HALF + row * 128;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
+                    for (int c = 0; c < 8; ++c)
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vrow + 16 * c), "r"(0u) : "memory");
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vrow + HALF + 16 * c), "r"(0u) : "memory");
-                    }
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // P (and V) as the tensor core will read them
             tc_fence_before();
             mbar_arrive(p_full);
         }
+        float l_other = 0.f;
+        if (ok && !swap_with_partner(l, l_other)) ok = false;
         if (ok && !wait_all(pv_done, (nkb - 1) & 1)) ok = false;
         tc_fence_after();
         if (ok) {
-            const float inv = 1.f / l;
-            uint16_t* dst = out + ((size_t)(q0 + tid) * Hq + head) * B;
+            const float inv = 1.f / (l + l_other);
+            uint16_t* dst = out + ((size_t)(q0 + row) * Hq + head) * B + 64 * half;
 #pragma unroll 1
-            for (int c = 0; c < B / 32; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t ov[32];
-                tc_ld32(tO + ((uint32_t)(warp * 32) << 16) + c * 32, ov);
-                if (tid < rows_here) {
+                tc_ld32(lane_o + c * 32, ov);
+                if (row < rows_here) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
                         uint4 w;
-                        w.x = pack_bf16(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv);
-                        w.y = pack_bf16(__uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
-                        w.z = pack_bf16(__uint_as_float(ov[i + 4]) * inv, __uint_as_float(ov[i + 5]) * inv);
-                        w.w = pack_bf16(__uint_as_float(ov[i + 6]) * inv, __uint_as_float(ov[i + 7]) * inv);
+                        w.x = pack_bf16x2(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv);
+                        w.y = pack_bf16x2(__uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
+                        w.z = pack_bf16x2(__uint_as_float(ov[i + 4]) * inv, __uint_as_float(ov[i + 5]) * inv);
+                        w.w = pack_bf16x2(__uint_as_float(ov[i + 6]) * inv, __uint_as_float(ov[i + 7]) * inv);
                         *reinterpret_cast<uint4*>(dst + c * 32 + i) = w;
                     }
                 }
