@@ -1,19 +1,26 @@
 // Causal attention of the prompt pass on the 5th-gen tensor cores (head dim 128).
 //
 // One CTA per (tile of 128 prompt rows, query head) walks the key blocks of 128 cache positions
-// that its rows can see.  Per key block j:
-//   S_j = Q K_j^T      tcgen05.mma, 128 x 128 x 128, fp32 in tensor memory (two S buffers)
-//   P_j = exp2(S_j c - m)   eight warps, two threads per query row (64 columns each): tcgen05.ld of
-//                      the row, running maximum m and sum l in registers, P_j rounded to bf16 into
-//                      128B-swizzled shared memory (the K-major A operand of the next product)
-//   O  += P_j V_j      tcgen05.mma with V as the MN-major B operand straight from the cache
-//                      layout [key][dim]; O stays in tensor memory for the whole walk
-// Roles in warps of their own: warps 0-7 softmax and epilogue (warps w and w + 4 own tensor-memory
-// lanes 32w..32w+31), lane 0 of warp 8 feeds Q once and K, lane 0
-// of warp 10 V, through two-stage mbarrier rings by TMA (one box per cache page and 64-column half),
-// lane 0 of warp 9 issues the MMAs.  S_{j+1} is issued before the MMA lane waits for P_j, so the tensor pipe
-// works on it while the softmax warps are busy with block j.
-// O is rescaled in tensor memory (tcgen05.ld / st) only when a row's maximum has grown by more
+// that its rows can see, as TWO independent online-softmax streams: stream A takes the even
+// blocks, stream B the odd ones, each with its own score buffer, running (max, sum) per row and
+// output accumulator; the two are merged at the end like the spans of a split cache.  While one
+// stream's four warps are in their latency chain (wait for the scores, tcgen05.ld, maximum, 128
+// exponentials per row, store) the other stream's products run on the tensor pipe, and the
+// exponentials of the two streams keep the special-function unit busy in turn.  Per block j of
+// stream g = j mod 2:
+//   S_j = Q K_j^T      tcgen05.mma, 128 x 128 x 128, fp32 into S_g (tensor memory)
+//   P_j = exp2(S_j c - m)   four warps, one query row per thread: the row of S_g by tcgen05.ld,
+//                      running maximum m and sum l in registers, P_j rounded to bf16 and written
+//                      back by tcgen05.st over the first 64 columns of S_g (two keys per word)
+//   O_g += P_j V_j     tcgen05.mma with A = P_j read from tensor memory and V as the MN-major B
+//                      operand straight from the cache layout [key][dim]
+// so P never touches shared memory.  S_{j+2} overwrites P_j: it is issued after P_j V_j and the
+// tensor pipe runs its instructions in order.
+// Roles in warps of their own: warps 0-3 stream A, warps 4-7 stream B (warp w owns tensor-memory
+// lanes 32 (w mod 4) ..), lane 0 of warp 8 feeds Q once and K, lane 0 of warp 10 V, through two-stage
+// mbarrier rings by TMA (one box per cache page and 64-column half; stage = stream), lane 0 of
+// warp 9 issues the MMAs in the order S_0, S_1, PV_0, S_2, PV_1, S_3, ...
+// O_g is rescaled in tensor memory (tcgen05.ld / st) only when a row's maximum has grown by more
 // than 8 (in log2 units) beyond the one its p values are taken against: the softmax is the same
 // function, p stays below 2^8, and the read-modify-write of O leaves the steady state.
 // Keys at positions >= pos0 + R are not part of the prompt: their pages are not fetched, their
@@ -31,8 +38,8 @@ constexpr int kTcAttnB = 128;                            // rows per tile, keys 
 constexpr int kTcAttnTile = kTcAttnB * kTcAttnB * 2;     // 32 KB: 128 x 128 bf16 as two 64-column halves
 constexpr int kTcAttnHalf = kTcAttnTile / 2;
 constexpr int kTcAttnMaxBoxes = 1024;                    // page boxes of one sequence
-constexpr int kTcAttnTmemCols = 512;                     // S0 | S1 | O | (unused)
-constexpr size_t kTcAttnSmemBytes = 6 * (size_t)kTcAttnTile + kTcAttnMaxBoxes * 4 + 4 * kTcAttnB * 4 + 1024 + 256;
+constexpr int kTcAttnTmemCols = 512;                     // S_A | S_B | O_A | O_B
+constexpr size_t kTcAttnSmemBytes = 5 * (size_t)kTcAttnTile + kTcAttnMaxBoxes * 4 + 4 * kTcAttnB * 4 + 1024 + 256;
 
 __device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t* v)
 {
@@ -59,6 +66,17 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* v)
           "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]), "r"(taddr)
         : "memory");
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+// D[tmem] (+)= A[tmem: 128 lanes x 16 bf16 in 8 columns] * B[smem desc], fp32 accumulate
+__device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
@@ -106,18 +124,18 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     const uint32_t raw0 = smem_u32(tca_raw);
     const uint32_t base = (raw0 + 1023u) & ~1023u;  // swizzled tiles want 1024-byte alignment
     unsigned char* gbase = tca_raw + (base - raw0);
-    const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
-    int32_t* rowc = reinterpret_cast<int32_t*>(gbase + 6 * TILE);  // first cache row of every page box
-    float* xch = reinterpret_cast<float*>(gbase + 6 * TILE + kTcAttnMaxBoxes * 4);  // [2][2][128]: what the two threads of a row swap
-    const uint32_t bars = base + 6 * TILE + kTcAttnMaxBoxes * 4 + 4 * B * 4;
+    const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE;
+    int32_t* rowc = reinterpret_cast<int32_t*>(gbase + 5 * TILE);  // first cache row of every page box
+    float2* ml = reinterpret_cast<float2*>(gbase + 5 * TILE + kTcAttnMaxBoxes * 4);  // [2][128]: (max, sum) of a stream's row
+    const uint32_t bars = base + 5 * TILE + kTcAttnMaxBoxes * 4 + 4 * B * 4;
     const uint32_t q_full = bars;
     auto k_full = [&](int s) { return bars + 8u + 8u * s; };
     auto k_empty = [&](int s) { return bars + 24u + 8u * s; };
     auto v_full = [&](int s) { return bars + 40u + 8u * s; };
     auto v_empty = [&](int s) { return bars + 56u + 8u * s; };
     auto s_full = [&](int s) { return bars + 72u + 8u * s; };
-    const uint32_t p_full = bars + 88u, pv_done = bars + 96u, tslot = bars + 104u;
-    auto pair_bar = [&](int w) { return bars + 112u + 8u * w; };
+    auto p_full = [&](int s) { return bars + 88u + 8u * s; };
+    const uint32_t all_done = bars + 104u, merge_bar = bars + 112u, tslot = bars + 120u;
     __shared__ int failed;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -139,10 +157,10 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             mbar_init(v_full(s), 1);
             mbar_init(v_empty(s), 1);
             mbar_init(s_full(s), 1);
+            mbar_init(p_full(s), 128);
         }
-        mbar_init(p_full, 256);
-        mbar_init(pv_done, 1);
-        for (int w = 0; w < 4; ++w) mbar_init(pair_bar(w), 64);
+        mbar_init(all_done, 1);
+        mbar_init(merge_bar, 256);
         failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -161,7 +179,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     tc_fence_after();
     uint32_t tmem;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem) : "r"(tslot));
-    const uint32_t tO = tmem + 2 * B;
+    // columns: S_A 0.., S_B 128.., O_A 256.., O_B 384..
 
     if ((warp == 8 || warp == 10) && lane == 0) {
         // ---------------------------------------------------------------- TMA producers: warp 8 Q and K, warp 10 V
@@ -192,187 +210,163 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         }
     } else if (warp == 9 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
-        // instruction descriptors: D fp32, A and B bf16, N = 128, M = 128; S: both operands K-major,
-        // P V: B (= V) MN-major
+        // instruction descriptors: D fp32, A and B bf16, N = 128, M = 128; S: both operands K-major
+        // in shared memory; P V: A (= P) in tensor memory, B (= V) MN-major
         const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(B >> 3) << 17) | ((uint32_t)(B >> 4) << 24);
         const uint32_t idesc_pv = idesc_s | (1u << 16);
         bool ok = mbar_wait(q_full, 0);
-        auto issue_s = [&](int j) {  // S_j into buffer j & 1
-            const int s = j & 1;
-            if (!mbar_wait(k_full(s), (j >> 1) & 1)) return false;
-            tc_fence_after();
+        for (int j = 0; j <= nkb && ok; ++j) {
+            if (j < nkb) {  // S_j into S_g (behind P_{j-2} V_{j-2} on the pipe, which read P from the same columns)
+                const int g = j & 1;
+                if (!mbar_wait(k_full(g), (j >> 1) & 1)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
 #pragma unroll
-            for (int ks = 0; ks < B / 16; ++ks) {
-                const uint64_t da = umma_desc_sw128(sQ + (ks >> 2) * HALF) + 2 * (ks & 3);
-                const uint64_t db = umma_desc_sw128(sK + s * TILE + (ks >> 2) * HALF) + 2 * (ks & 3);
-                tc_mma_bf16(tmem + s * B, da, db, idesc_s, ks != 0);
+                for (int ks = 0; ks < B / 16; ++ks) {
+                    const uint64_t da = umma_desc_sw128(sQ + (ks >> 2) * HALF) + 2 * (ks & 3);
+                    const uint64_t db = umma_desc_sw128(sK + g * TILE + (ks >> 2) * HALF) + 2 * (ks & 3);
+                    tc_mma_bf16(tmem + g * B, da, db, idesc_s, ks != 0);
+                }
+                tc_commit(k_empty(g));
+                tc_commit(s_full(g));
             }
-            tc_commit(k_empty(s));
-            tc_commit(s_full(s));
-            return true;
-        };
-        ok = ok && issue_s(0);
-        for (int j = 0; j < nkb && ok; ++j) {
-            // (buffer (j + 1) & 1 was last read for block j - 1, whose P has been waited for)
-            if (j + 1 < nkb && !issue_s(j + 1)) {
-                ok = false;
-                break;
-            }
-            const int s = j & 1;
-            if (!mbar_wait(v_full(s), (j >> 1) & 1) || !mbar_wait(p_full, j & 1)) {
-                ok = false;
-                break;
-            }
-            tc_fence_after();
+            if (j >= 1) {  // O_g += P_{j-1} V_{j-1}
+                const int jj = j - 1, g = jj & 1;
+                if (!mbar_wait(v_full(g), (jj >> 1) & 1) || !mbar_wait(p_full(g), (jj >> 1) & 1)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
 #pragma unroll
-            for (int kk = 0; kk < B / 16; ++kk) {  // 16 keys per MMA: 32 bytes along P's rows, 2048 bytes down V
-                const uint64_t da = umma_desc_sw128(sP + (kk >> 2) * HALF) + 2 * (kk & 3);
-                const uint64_t db = umma_desc_sw128_mn(sV + s * TILE) + (uint64_t)(kk * (2048 >> 4));
-                tc_mma_bf16(tO, da, db, idesc_pv, (j | kk) != 0);
+                for (int kk = 0; kk < B / 16; ++kk) {  // 16 keys per MMA: 8 columns of P, 2048 bytes down V
+                    const uint64_t db = umma_desc_sw128_mn(sV + g * TILE) + (uint64_t)(kk * (2048 >> 4));
+                    tc_mma_bf16_ta(tmem + (2 + g) * B, tmem + g * B + 8 * kk, db, idesc_pv, (jj >= 2) || kk != 0);
+                }
+                tc_commit(v_empty(g));
             }
-            tc_commit(v_empty(s));
-            tc_commit(pv_done);
         }
-        if (!ok) failed = 1;
+        if (ok) tc_commit(all_done);
+        else failed = 1;
     } else if (warp < 8) {
-        // ---------------------------------------------------------------- softmax, two threads per row
-        // warps w and w + 4 own tensor-memory lanes 32 (w % 4) ..: thread (row, half) takes columns
-        // 64 half .. 64 half + 63 of its row of S (and of O); the two meet once per block to agree on
-        // the row's maximum (an mbarrier per pair of warps, so that this wait is bounded like the others)
-        const int w4 = warp & 3, half = warp >> 2, row = w4 * 32 + lane;
-        const uint32_t lane_t = tmem + ((uint32_t)(w4 * 32) << 16) + 64 * half;
-        const uint32_t lane_o = tO + ((uint32_t)(w4 * 32) << 16) + 64 * half;
+        // ---------------------------------------------------------------- softmax: stream g, one row per thread
+        const int w4 = warp & 3, g = warp >> 2, row = w4 * 32 + lane;
+        const uint32_t lane_s = tmem + ((uint32_t)(w4 * 32) << 16) + g * B;        // this row of S_g (and P)
+        const uint32_t lane_o = tmem + ((uint32_t)(w4 * 32) << 16) + (2 + g) * B;  // this row of O_g
         const int qpos = min(pos0 + q0 + row, last_pos);  // (rows beyond the prompt: masked like the last one)
         const float sc = rsqrtf((float)B) * 1.4426950408889634f;
-        float m_used = 0.f, l = 0.f;
+        float m_used = -INFINITY, l = 0.f;  // (-inf: no visible key yet; every p so far was zero)
         bool ok = true;
         // (a wait ends for the whole warp alike: the tensor-memory loads below want the warp converged)
         auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(bar, parity)) != 0; };
-        int n_meet = 0;
-        // hand v to the row's other thread and return what that one handed over
-        auto swap_with_partner = [&](float v, float& other) {
-            float* slot = xch + (n_meet & 1) * 2 * B;
-            slot[half * B + row] = v;
-            mbar_arrive(pair_bar(w4));
-            if (!wait_all(pair_bar(w4), n_meet & 1)) return false;
-            other = slot[(half ^ 1) * B + row];
-            ++n_meet;
-            return true;
-        };
-        for (int j = 0; j < nkb; ++j) {
-            const int s = j & 1, key0 = j * B;
-            if (!wait_all(s_full(s), (j >> 1) & 1)) {
+        for (int j = g; j < nkb; j += 2) {
+            const int i = j >> 1, key0 = j * B;
+            // (S_j complete means P_{j-2} V_{j-2} complete: the commit covers everything issued before it)
+            if (!wait_all(s_full(g), i & 1)) {
                 ok = false;
                 break;
             }
             tc_fence_after();
-            uint32_t sv[B / 2];
-            tc_ld32_nowait(lane_t + s * B, sv);
-            tc_ld32_nowait(lane_t + s * B + 32, sv + 32);
-            tc_wait_ld();
-            const int lim = qpos - key0 - 64 * half;  // this thread's columns 0 .. lim are visible
-            if (lim < B / 2 - 1) {
+            uint32_t sv[B];
 #pragma unroll
-                for (int c = 0; c < B / 2; ++c)
+            for (int c = 0; c < B / 32; ++c) tc_ld32_nowait(lane_s + c * 32, sv + 32 * c);
+            tc_wait_ld();
+            const int lim = qpos - key0;  // columns 0 .. lim are visible
+            if (lim < B - 1) {
+#pragma unroll
+                for (int c = 0; c < B; ++c)
                     if (c > lim) sv[c] = 0xff800000u;  // -inf
             }
-            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one of 128
 #pragma unroll
-            for (int c = 0; c < B / 2; c += 4) {
+            for (int c = 0; c < B; c += 4) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) mx4[i] = fmaxf(mx4[i], __uint_as_float(sv[c + i]));
+                for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(sv[c + k]));
             }
-            float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc, mx_other;
-            if (!swap_with_partner(mx, mx_other)) {
-                ok = false;
-                break;
-            }
-            mx = fmaxf(mx, mx_other);
-            if (j == 0) {
-                m_used = mx;  // key 0 is visible to every row
-            } else {
-                const bool need = mx > m_used + 8.f;
-                if (__any_sync(0xffffffffu, need)) {  // the warp's 32 rows of O, each by its own factor
-                    if (!wait_all(pv_done, (j - 1) & 1)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after();
-                    const float alpha = need ? ex2_approx(m_used - mx) : 1.f;
-                    if (need) m_used = mx;
-                    l *= alpha;
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
+            const bool first = m_used == -INFINITY;  // nothing accumulated for this row yet: O_g's row is zero (or unwritten)
+            const bool need = !first && mx > m_used + 8.f;
+            if (__any_sync(0xffffffffu, need)) {  // the warp's 32 rows of O_g, each by its own factor
+                const float alpha = need ? ex2_approx(m_used - mx) : 1.f;
+                l *= alpha;
 #pragma unroll 1
-                    for (int c = 0; c < 2; ++c) {
-                        uint32_t ov[32];
-                        tc_ld32(lane_o + c * 32, ov);
+                for (int c = 0; c < B / 32; ++c) {
+                    uint32_t ov[32];
+                    tc_ld32(lane_o + c * 32, ov);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                        tc_st32(lane_o + c * 32, ov);
-                    }
+                    for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * alpha);
+                    tc_st32(lane_o + c * 32, ov);
                 }
             }
+            if (first || need) m_used = mx;
             // p = exp2(s c - m), rounded to bf16 in place (two per word); the sum takes the unrounded values
-            const float neg = -m_used;
+            const float neg = m_used == -INFINITY ? 0.f : -m_used;
             float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < B / 4; ++c) {
+            for (int c = 0; c < B / 2; ++c) {
                 const float p0 = ex2_approx(fmaf(__uint_as_float(sv[2 * c]), sc, neg));
                 const float p1 = ex2_approx(fmaf(__uint_as_float(sv[2 * c + 1]), sc, neg));
                 sum4[c & 3] += p0 + p1;
                 sv[c] = pack_bf16x2(p0, p1);
             }
             l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-            // P's buffer is free (and O at rest) once the product of block j - 1 has finished
-            if (j > 0 && !wait_all(pv_done, (j - 1) & 1)) {
-                ok = false;
-                break;
-            }
-            {
-                const uint32_t prow = sP + half * HALF + row * 128;
-#pragma unroll
-                for (int c16 = 0; c16 < 8; ++c16) {
-                    const uint32_t addr = prow + ((c16 ^ (row & 7)) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(sv[4 * c16]), "r"(sv[4 * c16 + 1]),
-                                 "r"(sv[4 * c16 + 2]), "r"(sv[4 * c16 + 3])
-                                 : "memory");
-                }
-            }
+            tc_st32(lane_s, sv);
+            tc_st32(lane_s + 32, sv + 32);
             if (key0 + B > n_valid) {  // the block reaches beyond the prompt: its V rows there become zeros
-                if (!wait_all(v_full(s), (j >> 1) & 1)) {
+                if (!wait_all(v_full(g), i & 1)) {
                     ok = false;
                     break;
                 }
                 if (row >= n_valid - key0) {
-                    const uint32_t vrow = sV + s * TILE + half * HALF + row * 128;
+                    const uint32_t vrow = sV + g * TILE + row * 128;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c)
+                    for (int c = 0; c < 8; ++c) {
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vrow + 16 * c), "r"(0u) : "memory");
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vrow + HALF + 16 * c), "r"(0u) : "memory");
+                    }
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // V as the tensor core will read it
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // P (and V) as the tensor core will read them
             tc_fence_before();
-            mbar_arrive(p_full);
+            mbar_arrive(p_full(g));
         }
-        float l_other = 0.f;
-        if (ok && !swap_with_partner(l, l_other)) ok = false;
-        if (ok && !wait_all(pv_done, (nkb - 1) & 1)) ok = false;
+        // merge the two streams: each thread its row's (max, sum), then columns 64 g .. 64 g + 63 of both outputs
+        ml[g * B + row] = make_float2(m_used, l);
+        mbar_arrive(merge_bar);
+        if (ok && !wait_all(merge_bar, 0)) ok = false;
+        if (ok && !wait_all(all_done, 0)) ok = false;
         tc_fence_after();
         if (ok) {
-            const float inv = 1.f / (l + l_other);
-            uint16_t* dst = out + ((size_t)(q0 + row) * Hq + head) * B + 64 * half;
+            const float2 a = ml[row], b = ml[B + row];  // (stream A has seen key 0: its maximum is finite)
+            const bool hasB = nkb > 1 && b.x != -INFINITY;
+            const float m = hasB ? fmaxf(a.x, b.x) : a.x;
+            const float wa = ex2_approx(a.x - m), wb = hasB ? ex2_approx(b.x - m) : 0.f;
+            const float inv = 1.f / (a.y * wa + b.y * wb);
+            const float fa = wa * inv, fb = wb * inv;
+            const uint32_t oa = tmem + ((uint32_t)(w4 * 32) << 16) + 2 * B + 64 * g, ob = oa + B;
+            uint16_t* dst = out + ((size_t)(q0 + row) * Hq + head) * B + 64 * g;
 #pragma unroll 1
             for (int c = 0; c < 2; ++c) {
-                uint32_t ov[32];
-                tc_ld32(lane_o + c * 32, ov);
+                uint32_t va[32], vb[32];
+                tc_ld32_nowait(oa + c * 32, va);
+                if (nkb > 1) tc_ld32_nowait(ob + c * 32, vb);
+                tc_wait_ld();
                 if (row < rows_here) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
+                    for (int k = 0; k < 32; k += 8) {
+                        float o[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            o[e] = __uint_as_float(va[k + e]) * fa;
+                            if (hasB) o[e] = fmaf(__uint_as_float(vb[k + e]), fb, o[e]);
+                        }
                         uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv);
-                        w.y = pack_bf16x2(__uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
-                        w.z = pack_bf16x2(__uint_as_float(ov[i + 4]) * inv, __uint_as_float(ov[i + 5]) * inv);
-                        w.w = pack_bf16x2(__uint_as_float(ov[i + 6]) * inv, __uint_as_float(ov[i + 7]) * inv);
-                        *reinterpret_cast<uint4*>(dst + c * 32 + i) = w;
+                        w.x = pack_bf16x2(o[0], o[1]);
+                        w.y = pack_bf16x2(o[2], o[3]);
+                        w.z = pack_bf16x2(o[4], o[5]);
+                        w.w = pack_bf16x2(o[6], o[7]);
+                        *reinterpret_cast<uint4*>(dst + c * 32 + k) = w;
                     }
                 }
             }
