@@ -718,6 +718,7 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
     int32_t* status = m->ctl + CTL_STATUS;
     LS_CK(launch(lc, embed_kernel, dim3(R), dim3(256), 0, m->emb, m->ids + r0, D, c.vocab, m->px, m->ctl, nullptr,
                  nullptr, nullptr, 0, 1));
+    m->launches += 1;
     for (int l = 0; l < layers; ++l) {
         const LayerW& w = m->lw[l];
         uint16_t* kp = m->kpages + (size_t)l * m->layer_kv_elems;
@@ -741,7 +742,7 @@ int prefill_block(ls_model* m, int r0, int R, int layers)
             swiglu_rows_kernel<<<R, 256, 0, st>>>(m->py, F, m->pa);
         }
         LS_TRY(gemm_launch(m->pa, w.wd, R, D, F, m->px, D, 1, status, st));
-        m->launches += gemm_uses_pairs(R) ? 11 : 13;  // pairs: rotary epilogue and SwiGLU live in the GEMMs
+        m->launches += gemm_uses_pairs(R) ? 7 : 9;  // pairs: rotary epilogue and SwiGLU live in the GEMMs
     }
     LS_CK(cudaGetLastError());
     return LS_OK;

@@ -677,6 +677,8 @@ rope_append_rows_kernel(const float* __restrict__ qkv, int Hq, int Hkv, int hd, 
 }
 
 // ------------------------------------------------------------------ causal attention of the prompt pass
+// (The two kernels below serve head dim 64, blocks of fewer than 128 rows and group sizes beyond 4;
+// head dim 128 with at least 128 rows runs on tcgen05, see ls_prefill_attn.cuh.)
 // grid (ceil(R/16), Hkv), block 256.  CTA = 16 consecutive rows (positions pos0 + 16 b ..),
 // KV head kh, its G query heads; it walks the key chunks 0 .. last visible in order with a
 // running (max, sum, o) per query in shared memory -- no partials, no merge.

@@ -42,7 +42,11 @@ def rel_margins(z):
 
 # ------------------------------------------------------------------ prompt pass of several blocks
 LONG_PROMPTS = [(TINY.shape, 1025, None), (TINY.shape, 2100, None), (TINY.shape, 3001, None),
-                (ODD_G2, 1100, 6.0), (ODD_G2, 2100, 6.0), (two_layers(synth.LLAMA2_7B, "7b-2-layers"), 1100, None)]
+                (ODD_G2, 1100, 6.0), (ODD_G2, 2100, 6.0), (two_layers(synth.LLAMA2_7B, "7b-2-layers"), 1100, None),
+                # head dim 128: the second block (299 rows at position 1024) also runs the tcgen05 attention kernel,
+                # over the first block's cache; the 8B shape with four query heads per KV head
+                (two_layers(synth.LLAMA2_7B, "7b-2-layers"), 1324, None),
+                (two_layers(synth.LLAMA3_8B, "8b-2-layers"), 1324, None)]
 
 
 @pytest.mark.parametrize("shape,n_prompt,amp", LONG_PROMPTS, ids=lambda v: getattr(v, "name", str(v)))
