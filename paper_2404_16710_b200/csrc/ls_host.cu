@@ -658,7 +658,7 @@ int allow_smem_once(Kernel kernel, size_t smem)
 bool attn_uses_tc(int R, int hd, int pos0, int page_shift)
 {
     static const bool allowed = getenv("LS_NO_TC_ATTN") == nullptr && tensor_map_encoder() != nullptr;
-    const int box_rows = (1 << page_shift) < kTcAttnB ? (1 << page_shift) : kTcAttnB;
+    const int box_rows = (1 << page_shift) < kTcAttnKB ? (1 << page_shift) : kTcAttnKB;
     return allowed && hd == kTcAttnB && R >= kTcAttnB && (pos0 + R + box_rows - 1) / box_rows <= kTcAttnMaxBoxes;
 }
 
@@ -667,7 +667,7 @@ int prefill_attn_launch(const uint16_t* q, const uint16_t* kp, const uint16_t* v
                         cudaStream_t st)
 {
     if (attn_uses_tc(R, hd, pos0, page_shift)) {
-        const int ps = 1 << page_shift, box_rows = ps < kTcAttnB ? ps : kTcAttnB;
+        const int ps = 1 << page_shift, box_rows = ps < kTcAttnKB ? ps : kTcAttnKB;
         CUtensorMap mq, mk, mv;
         LS_TRY(make_tile_map(&mq, q, (uint64_t)R, (uint64_t)Hq * hd, kTcAttnB));
         LS_TRY(make_tile_map(&mk, kp, (uint64_t)pool_pages * Hkv * ps, (uint64_t)hd, box_rows));
