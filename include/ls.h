@@ -337,9 +337,9 @@ int ls_op_attention(const void *q_bf16_dev, int32_t M, int32_t pos0, int32_t Hq,
  * ls_op_prefill_attention: causal attention of R rows at positions pos0 .. pos0+R-1 over the
  * paged cache (as ls_op_attention, any R, no scratch; the pools hold ceil(max_seq / page_size)
  * pages and every table entry is below that).  Head dim 128 and R >= 128: one CTA per (128 rows,
- * query head) on the tcgen05 tensor cores -- q.k and p.v of 128 x 128 x 128 with the scores and
- * the running output in tensor memory, K and V by TMA from the pages, the softmax one row per
- * thread; status_dev (device int32, may be NULL) receives 3 if one of its bounded waits ran
+ * query head) on the tcgen05 tensor cores -- key blocks of 64, the scores, the softmax weights
+ * and the running output in tensor memory, K and V by TMA from the pages, the softmax one row
+ * per thread; status_dev (device int32, may be NULL) receives 3 if one of its bounded waits ran
  * out.  Otherwise a CTA walks the key chunks of its rows in order with a running max / sum per
  * row on mma.sync (status_dev is not written).  Keys at positions >= pos0 + R are never used,
  * whatever bits the pages hold there. */
