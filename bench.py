@@ -280,6 +280,22 @@ def run_own(args):
     loop_gbs = sum(loop_bytes) / (sum(loop_ms) / 1e3) / 1e9
     spec_ms_per_step = sum(loop_ms) / sum(len(spec_out[k % n_prompts][1]) for k in range(args.steps))
 
+    # ---- end to end through the public call: host prompt in, host ids out, prefill included.  Taken right
+    # after the timed region, in the same power and clock state (the later legs run hotter).
+    e2e_ms = []
+    for i in range(1 + max(1, min(args.steps, 4))):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ids, a2 = gm.generate(prompts[i % n_prompts], E, d, NEW)
+        if i:
+            e2e_ms.append((time.perf_counter() - t0) * 1e3)
+    e2e_worst = max_over_ranks(statistics.mean(e2e_ms), dist, "cuda")  # mean call over the rotated prompts, slowest rank
+    est = gm.stats()
+    e2e = {"value": world * NEW / (e2e_worst / 1e3), "unit": UNIT, "h2d_bytes_per_step": 4 * P + 32 * 2,
+           "d2h_bytes_per_step": 4 * len(ids) + 4 * len(a2) + 32 * (est.host_syncs + 1),
+           "includes": "prompt H2D, prefill of the prompt, decode loop, ids D2H", "prefill_ms": est.prefill_ms}
+    B.ls_prefill(gm.h, prompts[0])  # the later legs start from the first prompt's cache again
+
     # ---- the same library's full-model greedy decoding, same model, same prompts
     for _ in range(min(args.warmup, 2)):
         B.ls_decode(gm.h, 0, 0, NEW)
@@ -351,20 +367,6 @@ def run_own(args):
             torch.cuda.empty_cache()
         if batch["points"]:
             batch["best"] = max(batch["points"], key=lambda q: q["value"])
-
-    # ---- end to end through the public call: host prompt in, host ids out, prefill included
-    e2e_ms = []
-    for i in range(1 + max(1, min(args.steps, 4))):
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        ids, a2 = gm.generate(prompts[i % n_prompts], E, d, NEW)
-        if i:
-            e2e_ms.append((time.perf_counter() - t0) * 1e3)
-    e2e_worst = max_over_ranks(statistics.mean(e2e_ms), dist, "cuda")  # mean call over the rotated prompts, slowest rank
-    est = gm.stats()
-    e2e = {"value": world * NEW / (e2e_worst / 1e3), "unit": UNIT, "h2d_bytes_per_step": 4 * P + 32 * 2,
-           "d2h_bytes_per_step": 4 * len(ids) + 4 * len(a2) + 32 * (est.host_syncs + 1),
-           "includes": "prompt H2D, prefill of the prompt, decode loop, ids D2H", "prefill_ms": est.prefill_ms}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
