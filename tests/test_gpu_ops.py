@@ -494,3 +494,42 @@ def test_prefill_attention_tensor_core(Hq, Hkv, R, pos0, page_size, ramp):
     for m in rows:
         ref = O.attention(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd)
         assert (np.abs(vals(out[m]) - ref) <= attention_tol(qf[m], kf[:pos0 + m + 1], vf[:pos0 + m + 1], Hq, Hkv, hd, ref)).all(), m
+
+
+
+def _tc_attention(q, kl, vl, pos0, Hq, Hkv, page_size, shuffle_seed):
+    """ls_op_prefill_attention (head dim 128) of rows q at pos0 over the logical cache kl, vl laid out
+    in pages of page_size tokens, permuted by shuffle_seed"""
+    hd, n = 128, kl.shape[0]
+    n_pages = -(-(n + 130) // page_size)
+    table = np.random.default_rng(shuffle_seed).permutation(n_pages).astype(np.int32)
+    kp = torch.full((n_pages, Hkv, page_size, hd), float("nan"), dtype=torch.bfloat16, device="cuda")
+    vp = torch.full_like(kp, float("nan"))
+    phys = torch.from_numpy(table[np.arange(n) // page_size].astype(np.int64)).cuda()
+    slot = torch.arange(n, device="cuda") % page_size
+    kp[phys, :, slot, :] = kl
+    vp[phys, :, slot, :] = vl
+    out = torch.full((q.shape[0], Hq * hd), float("nan"), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.ls_op_prefill_attention(q, pos0, Hq, Hkv, hd, page_size, torch.from_numpy(table).cuda(), n_pages * page_size, kp, vp,
+                              out, status)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    return out
+
+
+def test_prefill_attention_tensor_core_depends_on_positions_only():
+    """The tcgen05 kernel walks the cache by absolute position: the same logical cache in pages of 16,
+    64 or 256 tokens, in any page order, gives the same bits; and rows 256.. of a prompt come out the
+    same whether they are the tail of one call or a call of their own that starts at position 256
+    (tiles of 128 rows and key blocks of 64 fall on the same positions)."""
+    Hq, Hkv, hd, R = 8, 2, 128, 600
+    kl = rnd((R, Hkv, hd), 70).bfloat16()
+    vl = rnd((R, Hkv, hd), 71).bfloat16()
+    q = rnd((R, Hq * hd), 72, 1.5).bfloat16()
+    ref = _tc_attention(q, kl, vl, 0, Hq, Hkv, 64, 1)
+    assert torch.isfinite(ref.float()).all()
+    for page_size, seed in ((16, 2), (256, 3), (64, 4)):
+        assert torch.equal(_tc_attention(q, kl, vl, 0, Hq, Hkv, page_size, seed), ref), page_size
+    tail = _tc_attention(q[256:].contiguous(), kl, vl, 256, Hq, Hkv, 32, 5)
+    assert torch.equal(tail, ref[256:])
