@@ -43,3 +43,18 @@ def test_host_only_calls_work_without_a_gpu():
     cfg.head_dim = 48  # not a shape the kernels cover
     assert binding.ls_workspace_bytes(cfg) == 0
     assert binding.ls_op_lm_head_scratch_bytes(32000) == 8 * 16 * 2000
+
+
+def test_prompt_pass_ops_check_their_arguments_before_any_launch():
+    """Argument errors of the prompt-pass entry points come back as codes, on the host (no GPU touched):
+    this also pins the argument lists the binding declares for them."""
+    L = binding.lib()
+    bad = binding.LS_ERR_INVALID_ARG
+    # q, R, pos0, Hq, Hkv, hd, page_size, page_table, max_seq, k_pages, v_pages, out, status, stream
+    assert L.ls_op_prefill_attention(None, 0, 0, 8, 2, 128, 64, None, 4096, None, None, None, None, None) == bad
+    assert L.ls_op_prefill_attention(None, 128, 0, 8, 3, 128, 64, None, 4096, None, None, None, None, None) == bad
+    assert L.ls_op_prefill_attention(None, 128, 0, 8, 2, 96, 64, None, 4096, None, None, None, None, None) == bad
+    assert L.ls_op_prefill_attention(None, 128, 0, 8, 2, 128, 48, None, 4096, None, None, None, None, None) == bad
+    assert L.ls_op_prefill_attention(None, 128, 4000, 8, 2, 128, 64, None, 4096, None, None, None, None,
+                                     None) == binding.LS_ERR_CAPACITY
+    assert L.ls_op_prefill_attention(None, 128, 0, 8, 2, 128, 64, None, 4096, None, None, None, None, None) == bad  # null table
